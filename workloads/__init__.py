@@ -1,0 +1,7 @@
+"""Seeded synthetic workloads (shapes and value distributions only).
+
+This package holds none of the method's arithmetic: it only draws the random
+key / value / query tensors that both the CUDA path and the CPU oracle are fed.
+"""
+from .synth import (CONFIGS, WorkloadConfig, make_layer_kv, make_saliency,  # noqa: F401
+                    make_step_inputs)
