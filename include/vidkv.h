@@ -1,0 +1,213 @@
+/*
+ * vidkv.h -- C ABI of libvidkv: the VidKV 1.x-bit KV-cache hot path on B200 (sm_100a).
+ *
+ * What the library computes (notation of the paper, arXiv 2503.16257):
+ *   - keys    : MixQuant (Algorithm 3): per-chunk range-based channel split,
+ *               2-bit GQuant (Eq. 4) on the anomalous half of the channels,
+ *               FFT + 1-bit sign/mean-abs code (Eq. 5) on the normal half;
+ *   - values  : 1.58Quant (Eq. 6, ternary, gamma) and STPQuant (Algorithm 2):
+ *               the top n = floor(p * l_v) visual tokens by saliency (Eq. 7)
+ *               are kept at 2 bits (Eq. 4), the rest ternary;
+ *   - packing : codes, scales and zero points in one flat caller-owned buffer;
+ *   - decode  : Algorithm 1 "Decoding" -- append the new token to the FP16
+ *               residual, Softmax(q K^T / sqrt(D)) V over the packed cache plus
+ *               the residual (Eq. 3) without materialising K or V, and the
+ *               residual flush once it holds R = 128 tokens.
+ *
+ * Conventions
+ *   - Every function returns a vidkv_status_t (0 = OK, negative = error); the
+ *     library never throws, aborts or prints.
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless the
+ *     argument is documented as a host pointer.  The library allocates no
+ *     device memory: the caller asks vidkv_cache_bytes() for sizes, allocates,
+ *     and passes the buffers in.  The handle is a small host object.
+ *   - All device work is enqueued on the caller's stream (a cudaStream_t passed
+ *     as void*) and is asynchronous.  Argument errors are detected on the host
+ *     before anything is launched.
+ *   - Fixed by this build: D = 128, G = 32, R = 128, k = 0.5 (64 two-bit and 64
+ *     one-bit channels), H_q a multiple of H_kv with H_q / H_kv <= 8.  Other
+ *     shapes return VIDKV_ERR_UNSUPPORTED.
+ *   - Element types: VIDKV_F16 / VIDKV_BF16 for K, V, q, k_new, v_new (in_dtype);
+ *     VIDKV_F16 / VIDKV_BF16 / VIDKV_F32 for the attention output (out_dtype).
+ *     Input values must be finite and representable in binary16.
+ *   - One handle must not be used from two host threads at once, and calls on
+ *     one handle must be issued on one stream (or on streams the caller orders).
+ *
+ * Packed cache layout (little endian; all offsets are given by vidkv_layout_t)
+ *   per slab = (layer, batch element, KV head):
+ *     chunk table  : per chunk 128 bytes: 64 ascending anomalous channel ids,
+ *                    then 64 ascending normal channel ids (uint8).  Chunk 0 is
+ *                    the prefill; every residual flush appends a 128-token chunk.
+ *     key groups   : per 32 tokens 1152 bytes:
+ *                    [0,512)    2-bit codes, token t at 16*t, anomalous slot j in
+ *                               32-bit word j/16 at bits 2*(j%16);
+ *                    [512,768)  1-bit codes, token t at 512+8*t, spectrum column
+ *                               f in word f/32 at bit f%32 (1 = coefficient >= 0);
+ *                    [768,896)  s  (binary16) of the 64 two-bit slots;
+ *                    [896,1024) z  (binary16) of the 64 two-bit slots;
+ *                    [1024,1152) s (binary16) of the 64 spectrum columns.
+ *                    Spectrum columns of the orthonormal 64-point DFT of the
+ *                    normal channels (ascending channel order), Hermitian half:
+ *                    column 0 = Re X[0], 1 = Re X[32], 2k = Re X[k],
+ *                    2k+1 = Im X[k] for k = 1..31.
+ *     ternary supergroups : per 5 groups (160 stream tokens) 5376 bytes:
+ *                    [0,4096)   byte (j, c) at 128*j + c holds the trits of
+ *                               channel c at token j of each of the 5 groups:
+ *                               digit d_g = trit + 1, b = sum_g d_g * 3^(4-g),
+ *                               stored byte = (256*b + 242) / 243;
+ *                    [4096,5376) s (binary16) [5][128].
+ *     protected groups (STP) : per 32 protected tokens 1536 bytes:
+ *                    [0,1024) 2-bit codes, token j at 32*j, channel c in word
+ *                    c/16 at bits 2*(c%16); [1024,1280) s; [1280,1536) z.
+ *     residual     : K_r and V_r, 128 x 128 elements each, in in_dtype.
+ *   per batch element: the protection mask E as bit words plus, per word, the
+ *   number of protected tokens before it.
+ */
+#ifndef VIDKV_H_
+#define VIDKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t vidkv_status_t;
+
+enum {
+  VIDKV_OK = 0,
+  VIDKV_ERR_INVALID_ARG = -1,   /* null pointer, negative size, bad enum value, p outside [0,1] ... */
+  VIDKV_ERR_UNSUPPORTED = -2,   /* a shape or mode this build does not implement */
+  VIDKV_ERR_ALIGNMENT = -3,     /* a pointer or stride that is not 16-byte aligned */
+  VIDKV_ERR_CAPACITY = -4,      /* more tokens than the cache was sized for, buffer too small */
+  VIDKV_ERR_STATE = -5,         /* call order: decode before quantize, quantize twice, ... */
+  VIDKV_ERR_CUDA = -6,          /* a CUDA runtime call or launch failed */
+  VIDKV_ERR_TIMEOUT = -7        /* a bounded device-side wait ran out (reported via vidkv_cache_status) */
+};
+
+enum { VIDKV_F16 = 0, VIDKV_BF16 = 1, VIDKV_F32 = 2 };
+enum { VIDKV_KEY1BIT_FFT_SIGN = 0 };
+
+/* Problem description (Algorithm 1 parameters G, R, p, k; Algorithm 2 gamma). */
+typedef struct {
+  int32_t B;                  /* batch elements */
+  int32_t L;                  /* layers held by this cache */
+  int32_t H_kv;               /* KV heads */
+  int32_t H_q;                /* query heads (GQA: head h_q reads KV head h_q / (H_q/H_kv)) */
+  int32_t D;                  /* head dimension (128) */
+  int32_t G;                  /* group size (32) */
+  int32_t R;                  /* residual length (128) */
+  float k_ratio;              /* fraction of key channels kept at 2 bits (0.5) */
+  float p_ratio;              /* fraction of visual tokens protected at 2 bits, in [0, 1] */
+  float gamma;                /* ternary threshold factor (0.7) */
+  int32_t in_dtype;           /* VIDKV_F16 | VIDKV_BF16 */
+  int32_t out_dtype;          /* VIDKV_F16 | VIDKV_BF16 | VIDKV_F32 */
+  int32_t key_1bit_mode;      /* VIDKV_KEY1BIT_FFT_SIGN */
+  int32_t reserved;           /* must be 0 */
+  int64_t max_prefill_tokens; /* largest T passed to vidkv_quantize_* */
+  int64_t max_new_tokens;     /* decode steps the cache must be able to absorb */
+} vidkv_config_t;
+
+/* Byte offsets and strides of the packed cache (host struct; filled by vidkv_cache_layout). */
+typedef struct {
+  int64_t header_bytes;
+  int64_t sel_offset;         /* start of the per-batch token-selection region */
+  int64_t sel_stride_b;       /* bytes per batch element: E words, then prefix words */
+  int64_t sel_words;          /* 32-bit words per batch element in each of the two arrays */
+  int64_t slab_offset;        /* start of slab 0 */
+  int64_t slab_stride;        /* bytes per slab; slab index = (layer*B + b)*H_kv + h */
+  int64_t chunk_table_offset; /* within a slab */
+  int64_t max_chunks;
+  int64_t kgroup_offset;      /* within a slab */
+  int64_t max_kgroups;
+  int64_t tern_offset;        /* within a slab */
+  int64_t max_supergroups;
+  int64_t prot_offset;        /* within a slab */
+  int64_t max_pgroups;
+  int64_t kres_offset;        /* within a slab */
+  int64_t vres_offset;        /* within a slab */
+  int64_t total_bytes;
+} vidkv_layout_t;
+
+typedef struct vidkv_cache vidkv_cache_t;
+
+/* Sizes (host only).  cache_bytes / workspace_bytes are what vidkv_cache_init wants.
+ * The workspace holds split-KV partial results, channel ranges and the gather
+ * lists of the token selection; it carries no state between calls except the
+ * gather lists, which vidkv_quantize_values reads. */
+vidkv_status_t vidkv_cache_bytes(const vidkv_config_t* cfg, size_t* cache_bytes, size_t* workspace_bytes);
+
+/* Offsets of every region of the packed cache for this configuration (host only). */
+vidkv_status_t vidkv_cache_layout(const vidkv_config_t* cfg, vidkv_layout_t* layout);
+
+/* Create a handle over caller-owned device buffers (256-byte aligned) and zero the
+ * cache on `stream`.  The handle stays valid until vidkv_cache_destroy; the buffers
+ * must outlive it.  Returns CAPACITY if a buffer is smaller than vidkv_cache_bytes says. */
+vidkv_status_t vidkv_cache_init(const vidkv_config_t* cfg, void* cache, size_t cache_bytes,
+                                void* workspace, size_t workspace_bytes, void* stream,
+                                vidkv_cache_t** handle);
+vidkv_status_t vidkv_cache_destroy(vidkv_cache_t* handle);
+
+/* Forget all tokens (host state only; the next quantize calls overwrite the buffers). */
+vidkv_status_t vidkv_cache_reset(vidkv_cache_t* handle, void* stream);
+
+/* Sec. 3.3(2) / Eq. 7: choose the protected tokens.  saliency [B, l_v] float32 scores
+ * the visual tokens vis_begin .. vis_begin + l_v - 1 of a prompt of T tokens; the top
+ * n = floor(p_ratio * l_v) (ties: lower token index) are protected in every layer and
+ * head.  Must precede vidkv_quantize_values when p_ratio > 0; with p_ratio == 0 or
+ * saliency == NULL no token is protected.  Only tokens below T - T % G can be
+ * protected (the rest stay FP16 in the residual). */
+vidkv_status_t vidkv_select_tokens(vidkv_cache_t* handle, const float* saliency, int64_t vis_begin,
+                                   int64_t l_v, int64_t T, void* stream);
+
+/* Algorithm 2 takes the mask E as a parameter: the same, from a ready mask
+ * E [B, T] (uint8, nonzero = protected; every batch element must protect the same
+ * number of tokens, all below T - T % G). */
+vidkv_status_t vidkv_set_token_mask(vidkv_cache_t* handle, const uint8_t* E, int64_t T, void* stream);
+
+/* Algorithm 1 "Prefill", key half, for one layer: K [B, H_kv, T, D] (in_dtype) with
+ * element strides stride_b / stride_h / stride_t (channel stride 1; strides multiples
+ * of 8 elements).  The first T - T % G tokens are MixQuant-ed (Algorithm 3) into chunk
+ * 0; the last T % G tokens are copied to the FP16 residual.  Once per layer per reset. */
+vidkv_status_t vidkv_quantize_keys(vidkv_cache_t* handle, int32_t layer, const void* K, int64_t T,
+                                   int64_t stride_b, int64_t stride_h, int64_t stride_t, void* stream);
+
+/* Algorithm 1 "Prefill", value half: STPQuant (Algorithm 2) when tokens were selected,
+ * else 1.58Quant (Eq. 6).  Same argument meaning as vidkv_quantize_keys; T must equal
+ * the T given for the keys of this layer if those came first. */
+vidkv_status_t vidkv_quantize_values(vidkv_cache_t* handle, int32_t layer, const void* V, int64_t T,
+                                     int64_t stride_b, int64_t stride_h, int64_t stride_t, void* stream);
+
+/* Algorithm 1 "Decoding" for n_layers independent layers in one call:
+ *   q      [n_layers, B, H_q,  D]  (in_dtype)
+ *   k_new  [n_layers, B, H_kv, D]  (in_dtype)    appended to the residual first
+ *   v_new  [n_layers, B, H_kv, D]  (in_dtype)
+ *   out    [n_layers, B, H_q,  D]  (out_dtype)   Softmax(q K^T * softmax_scale) V
+ * softmax_scale <= 0 selects 1 / sqrt(D).  When a layer's residual reaches R tokens it
+ * is quantized into a new 128-token chunk (own channel split; values by 1.58Quant) and
+ * emptied.  All contiguous.  Returns CAPACITY when max_new_tokens would be exceeded. */
+vidkv_status_t vidkv_decode_attention(vidkv_cache_t* handle, int32_t layer_begin, int32_t n_layers,
+                                      const void* q, const void* k_new, const void* v_new, void* out,
+                                      float softmax_scale, void* stream);
+
+/* Host view of a layer's token counts (any pointer may be NULL). */
+vidkv_status_t vidkv_layer_state(const vidkv_cache_t* handle, int32_t layer, int64_t* n_quantized,
+                                 int64_t* n_residual, int64_t* n_chunks, int64_t* n_protected);
+
+/* Device status word of the cache (synchronises `stream`): VIDKV_OK or the first
+ * device-detected error. */
+vidkv_status_t vidkv_cache_status(vidkv_cache_t* handle, void* stream);
+
+/* Test and inspection only (never on the decode path): dequantize the quantized part of
+ * one layer to float32, out [B, H_kv, n_quantized, D] contiguous.  DeQuant of Algorithm 1. */
+vidkv_status_t vidkv_dequantize_keys(vidkv_cache_t* handle, int32_t layer, float* out, void* stream);
+vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* handle, int32_t layer, float* out, void* stream);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int32_t vidkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VIDKV_H_ */

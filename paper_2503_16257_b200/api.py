@@ -1,0 +1,231 @@
+"""ctypes binding of libvidkv.so: same names and argument order as include/vidkv.h."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+VIDKV_F16, VIDKV_BF16, VIDKV_F32 = 0, 1, 2
+STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "ALIGNMENT", -4: "CAPACITY",
+                -5: "STATE", -6: "CUDA", -7: "TIMEOUT"}
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+
+class VidKVError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        super().__init__(f"{fn} failed: {STATUS_NAMES.get(status, status)} ({status})")
+
+
+class _Config(C.Structure):
+    _fields_ = [("B", C.c_int32), ("L", C.c_int32), ("H_kv", C.c_int32), ("H_q", C.c_int32),
+                ("D", C.c_int32), ("G", C.c_int32), ("R", C.c_int32),
+                ("k_ratio", C.c_float), ("p_ratio", C.c_float), ("gamma", C.c_float),
+                ("in_dtype", C.c_int32), ("out_dtype", C.c_int32), ("key_1bit_mode", C.c_int32),
+                ("reserved", C.c_int32),
+                ("max_prefill_tokens", C.c_int64), ("max_new_tokens", C.c_int64)]
+
+
+class _Layout(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "header_bytes", "sel_offset", "sel_stride_b", "sel_words", "slab_offset", "slab_stride",
+        "chunk_table_offset", "max_chunks", "kgroup_offset", "max_kgroups", "tern_offset",
+        "max_supergroups", "prot_offset", "max_pgroups", "kres_offset", "vres_offset", "total_bytes")]
+
+
+@dataclass
+class VidKVConfig:
+    B: int
+    L: int
+    max_prefill_tokens: int
+    max_new_tokens: int
+    H_kv: int = 4
+    H_q: int = 28
+    D: int = 128
+    G: int = 32
+    R: int = 128
+    k_ratio: float = 0.5
+    p_ratio: float = 0.0
+    gamma: float = 0.7
+    in_dtype: int = VIDKV_F16
+    out_dtype: int = VIDKV_F32
+    key_1bit_mode: int = 0
+
+    def to_c(self) -> _Config:
+        return _Config(self.B, self.L, self.H_kv, self.H_q, self.D, self.G, self.R, self.k_ratio,
+                       self.p_ratio, self.gamma, self.in_dtype, self.out_dtype, self.key_1bit_mode, 0,
+                       self.max_prefill_tokens, self.max_new_tokens)
+
+
+_SIGNATURES = {
+    "vidkv_version": (C.c_int32, []),
+    "vidkv_cache_bytes": (C.c_int32, [C.POINTER(_Config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "vidkv_cache_layout": (C.c_int32, [C.POINTER(_Config), C.POINTER(_Layout)]),
+    "vidkv_cache_init": (C.c_int32, [C.POINTER(_Config), C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t,
+                                     C.c_void_p, C.POINTER(C.c_void_p)]),
+    "vidkv_cache_destroy": (C.c_int32, [C.c_void_p]),
+    "vidkv_cache_reset": (C.c_int32, [C.c_void_p, C.c_void_p]),
+    "vidkv_select_tokens": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p]),
+    "vidkv_set_token_mask": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
+    "vidkv_quantize_keys": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                        C.c_int64, C.c_void_p]),
+    "vidkv_quantize_values": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                          C.c_int64, C.c_void_p]),
+    "vidkv_decode_attention": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_float, C.c_void_p]),
+    "vidkv_layer_state": (C.c_int32, [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                                      C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
+    "vidkv_cache_status": (C.c_int32, [C.c_void_p, C.c_void_p]),
+    "vidkv_dequantize_keys": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
+    "vidkv_dequantize_values": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
+}
+
+
+def exported_symbols():
+    """Names the binding expects libvidkv.so to export (all of include/vidkv.h)."""
+    return sorted(_SIGNATURES)
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, "libvidkv.so")
+
+
+def load_library():
+    """Load libvidkv.so (built in-tree by ``python -m paper_2503_16257_b200.build``).
+    Fails loudly when the library is missing: there is no fallback path."""
+    global _LIB
+    if _LIB is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} not found: build it with `python -m paper_2503_16257_b200.build`")
+        lib = C.CDLL(path)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _LIB = lib
+    return _LIB
+
+
+def _check(fn: str, status: int):
+    if status != 0:
+        raise VidKVError(fn, status)
+
+
+def vidkv_version() -> int:
+    return load_library().vidkv_version()
+
+
+def vidkv_cache_bytes(cfg: VidKVConfig):
+    cb, wb = C.c_size_t(0), C.c_size_t(0)
+    c = cfg.to_c()
+    _check("vidkv_cache_bytes", load_library().vidkv_cache_bytes(C.byref(c), C.byref(cb), C.byref(wb)))
+    return cb.value, wb.value
+
+
+def vidkv_cache_layout(cfg: VidKVConfig) -> dict:
+    lay = _Layout()
+    c = cfg.to_c()
+    _check("vidkv_cache_layout", load_library().vidkv_cache_layout(C.byref(c), C.byref(lay)))
+    return {n: getattr(lay, n) for n, _ in _Layout._fields_}
+
+
+def _stream_ptr(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _strides_bht(x):
+    assert x.dim() == 4 and x.stride(3) == 1, "expected [B, H, T, D] with unit channel stride"
+    return x.stride(0), x.stride(1), x.stride(2)
+
+
+class VidKVCache:
+    """Owns the two device buffers (torch uint8 tensors) and the library handle.  Methods carry
+    the C ABI's names; tensors are passed as device pointers, work goes to the current stream."""
+
+    def __init__(self, cfg: VidKVConfig, device="cuda"):
+        import torch
+        self.cfg = cfg
+        self.lib = load_library()
+        self.cache_bytes, self.workspace_bytes = vidkv_cache_bytes(cfg)
+        self.layout = vidkv_cache_layout(cfg)
+        self.cache = torch.empty(self.cache_bytes, dtype=torch.uint8, device=device)
+        self.workspace = torch.empty(max(self.workspace_bytes, 256), dtype=torch.uint8, device=device)
+        self._c = cfg.to_c()
+        h = C.c_void_p()
+        _check("vidkv_cache_init", self.lib.vidkv_cache_init(
+            C.byref(self._c), C.c_void_p(self.cache.data_ptr()), self.cache_bytes,
+            C.c_void_p(self.workspace.data_ptr()), self.workspace.numel(), _stream_ptr(), C.byref(h)))
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.vidkv_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reset(self):
+        _check("vidkv_cache_reset", self.lib.vidkv_cache_reset(self.handle, _stream_ptr()))
+
+    def select_tokens(self, saliency, vis_begin: int, l_v: int, T: int):
+        ptr = C.c_void_p(saliency.data_ptr()) if saliency is not None else C.c_void_p(0)
+        if saliency is not None:
+            assert saliency.is_contiguous() and saliency.dtype.is_floating_point and saliency.element_size() == 4
+        _check("vidkv_select_tokens", self.lib.vidkv_select_tokens(self.handle, ptr, vis_begin, l_v, T, _stream_ptr()))
+
+    def set_token_mask(self, E, T: int):
+        assert E.is_contiguous() and E.element_size() == 1
+        _check("vidkv_set_token_mask", self.lib.vidkv_set_token_mask(self.handle, C.c_void_p(E.data_ptr()), T,
+                                                                     _stream_ptr()))
+
+    def quantize_keys(self, layer: int, K):
+        sb, sh, st = _strides_bht(K)
+        _check("vidkv_quantize_keys", self.lib.vidkv_quantize_keys(
+            self.handle, layer, C.c_void_p(K.data_ptr()), K.shape[2], sb, sh, st, _stream_ptr()))
+
+    def quantize_values(self, layer: int, V):
+        sb, sh, st = _strides_bht(V)
+        _check("vidkv_quantize_values", self.lib.vidkv_quantize_values(
+            self.handle, layer, C.c_void_p(V.data_ptr()), V.shape[2], sb, sh, st, _stream_ptr()))
+
+    def decode_attention(self, layer_begin: int, n_layers: int, q, k_new, v_new, out, softmax_scale: float = 0.0):
+        for t in (q, k_new, v_new, out):
+            assert t.is_contiguous()
+        _check("vidkv_decode_attention", self.lib.vidkv_decode_attention(
+            self.handle, layer_begin, n_layers, C.c_void_p(q.data_ptr()), C.c_void_p(k_new.data_ptr()),
+            C.c_void_p(v_new.data_ptr()), C.c_void_p(out.data_ptr()), softmax_scale, _stream_ptr()))
+
+    def layer_state(self, layer: int) -> dict:
+        a, b, c, d = C.c_int64(), C.c_int64(), C.c_int64(), C.c_int64()
+        _check("vidkv_layer_state", self.lib.vidkv_layer_state(self.handle, layer, C.byref(a), C.byref(b),
+                                                              C.byref(c), C.byref(d)))
+        return dict(n_quantized=a.value, n_residual=b.value, n_chunks=c.value, n_protected=d.value)
+
+    def status(self) -> int:
+        return self.lib.vidkv_cache_status(self.handle, _stream_ptr())
+
+    def dequantize_keys(self, layer: int):
+        import torch
+        st = self.layer_state(layer)
+        out = torch.empty((self.cfg.B, self.cfg.H_kv, st["n_quantized"], self.cfg.D), dtype=torch.float32,
+                          device=self.cache.device)
+        _check("vidkv_dequantize_keys", self.lib.vidkv_dequantize_keys(self.handle, layer, C.c_void_p(out.data_ptr()),
+                                                                       _stream_ptr()))
+        return out
+
+    def dequantize_values(self, layer: int):
+        import torch
+        st = self.layer_state(layer)
+        out = torch.empty((self.cfg.B, self.cfg.H_kv, st["n_quantized"], self.cfg.D), dtype=torch.float32,
+                          device=self.cache.device)
+        _check("vidkv_dequantize_values", self.lib.vidkv_dequantize_values(self.handle, layer,
+                                                                           C.c_void_p(out.data_ptr()), _stream_ptr()))
+        return out

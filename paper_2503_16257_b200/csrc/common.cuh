@@ -1,0 +1,93 @@
+// Shared constants and small device helpers of libvidkv (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/vidkv.h"
+
+namespace vidkv {
+
+constexpr int kD = 128;            // head dimension
+constexpr int kG = 32;             // group size (tokens per scale group)
+constexpr int kR = 128;            // residual length
+constexpr int kNA = 64;            // anomalous (2-bit) channels at k = 0.5
+constexpr int kNF = 64;            // normal channels = spectrum columns (1-bit)
+constexpr int kMaxRep = 8;         // query heads per KV head handled by one CTA
+
+constexpr int kChunkBytes = 128;   // channel permutation of one chunk
+constexpr int kKGroupBytes = 1152; // one 32-token key group
+constexpr int kKG_Codes2 = 0, kKG_Bits1 = 512, kKG_S2 = 768, kKG_Z2 = 896, kKG_S1 = 1024;
+constexpr int kSGGroups = 5;       // groups per ternary supergroup (5 trits per byte)
+constexpr int kSGBytes = 5376;
+constexpr int kSG_Scales = 4096;
+constexpr int kPGBytes = 1536;     // one 32-token protected (2-bit) value group
+constexpr int kPG_S = 1024, kPG_Z = 1280;
+constexpr int kResBytes = kR * kD * 2;
+constexpr int kHeaderBytes = 256;
+constexpr int kHdrStatus = 8;      // byte offset of the device status word
+
+constexpr uint32_t kMagic = 0x564b4456u;  // "VDKV"
+
+// Device-side view of one cache: everything a kernel needs to find a slab region.
+struct CacheView {
+  uint8_t* base;
+  int64_t sel_offset, sel_stride_b, sel_words;
+  int64_t slab_offset, slab_stride;
+  int64_t chunk_table_offset, kgroup_offset, tern_offset, prot_offset, kres_offset, vres_offset;
+  int32_t B, H_kv, H_q, rep;
+
+  __host__ __device__ uint8_t* slab(int64_t layer, int64_t b, int64_t h) const {
+    return base + slab_offset + ((layer * B + b) * H_kv + h) * slab_stride;
+  }
+  __host__ __device__ const uint32_t* e_words(int64_t b) const {
+    return reinterpret_cast<const uint32_t*>(base + sel_offset + b * sel_stride_b);
+  }
+  __host__ __device__ const uint32_t* e_prefix(int64_t b) const {
+    return e_words(b) + sel_words;
+  }
+};
+
+template <typename T> struct Elem;
+template <> struct Elem<__half> {
+  static __device__ __forceinline__ float to_float(__half v) { return __half2float(v); }
+  static __device__ __forceinline__ float2 to_float2(uint32_t v) {
+    return __half22float2(*reinterpret_cast<__half2*>(&v));
+  }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+  static __device__ __forceinline__ float2 to_float2(uint32_t v) {
+    return __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v));
+  }
+};
+
+__device__ __forceinline__ float h2f(uint16_t bits) {
+  return __half2float(__ushort_as_half(bits));
+}
+__device__ __forceinline__ uint16_t f2h_bits(float v) {
+  return __half_as_ushort(__float2half_rn(v));
+}
+
+// Monotone map float -> uint32 (for atomic min / max on floats).
+__device__ __forceinline__ uint32_t float_ordered(float f) {
+  uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_float(uint32_t u) {
+  return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+
+// Ternary byte code: five digits d in {0,1,2} (d = trit + 1), most significant first,
+// b = sum d_g * 3^(4-g); the stored byte is ceil(256 * b / 243), which lets a decoder
+// peel digits with multiply / shift and no division.
+__host__ __device__ __forceinline__ uint32_t trit_byte_encode(uint32_t b) { return (256u * b + 242u) / 243u; }
+__host__ __device__ __forceinline__ uint32_t trit_byte_decode(uint32_t q) { return (q * 243u) >> 8; }
+__host__ __device__ __forceinline__ int trit_digit(uint32_t b, int slot) {
+  const uint32_t p3[5] = {81u, 27u, 9u, 3u, 1u};
+  return static_cast<int>((b / p3[slot]) % 3u);
+}
+
+}  // namespace vidkv

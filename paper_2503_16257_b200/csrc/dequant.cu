@@ -1,0 +1,115 @@
+// Test and inspection kernels: DeQuant of Algorithm 1 for a whole layer, to float32.
+// Never used by the decode path (which reads the packed cache directly).
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace vidkv {
+
+// grid = (key groups, slabs of one layer); block = 128 threads.
+__global__ void __launch_bounds__(128) dequant_keys_kernel(CacheView cv, int layer, int64_t T_q0, int64_t T_qt,
+                                                           float* __restrict__ out) {
+  __shared__ __align__(16) uint8_t kg[kKGroupBytes];
+  __shared__ uint8_t perm[kD];
+  __shared__ float cs[64], sn[64];
+  const int tid = threadIdx.x;
+  const int slab = blockIdx.y;
+  const int b = slab / cv.H_kv, h = slab % cv.H_kv;
+  const int64_t gidx = blockIdx.x;
+  const int64_t g0n = T_q0 / kG;
+  const int chunk = gidx < g0n ? 0 : 1 + static_cast<int>((gidx - g0n) / (kR / kG));
+  const uint8_t* sp = cv.slab(layer, b, h);
+  perm[tid] = sp[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
+  if (tid < kKGroupBytes / 16)
+    reinterpret_cast<uint4*>(kg)[tid] = reinterpret_cast<const uint4*>(sp + cv.kgroup_offset + gidx * kKGroupBytes)[tid];
+  if (tid < 64) {
+    float s, c;
+    sincospif(static_cast<float>(tid) / 32.0f, &s, &c);
+    cs[tid] = c; sn[tid] = s;
+  }
+  __syncthreads();
+  float* o = out + ((static_cast<int64_t>(slab) * T_qt) + gidx * kG) * kD;
+  if (tid < 64) {
+    const int j = tid, c = perm[j];
+    const float s = h2f(reinterpret_cast<const uint16_t*>(kg + kKG_S2)[j]);
+    const float z = h2f(reinterpret_cast<const uint16_t*>(kg + kKG_Z2)[j]);
+    for (int t = 0; t < kG; ++t) {
+      const uint32_t word = reinterpret_cast<const uint32_t*>(kg + kKG_Codes2)[t * 4 + (j >> 4)];
+      o[t * kD + c] = static_cast<float>((word >> (2 * (j & 15))) & 3u) * s + z;
+    }
+  } else {
+    const int i = tid - 64, c = perm[64 + i];
+    const uint16_t* s1 = reinterpret_cast<const uint16_t*>(kg + kKG_S1);
+    for (int t = 0; t < kG; ++t) {
+      const uint32_t w0 = reinterpret_cast<const uint32_t*>(kg + kKG_Bits1)[t * 2];
+      const uint32_t w1 = reinterpret_cast<const uint32_t*>(kg + kKG_Bits1)[t * 2 + 1];
+      auto val = [&](int f) -> float {
+        const uint32_t bit = f < 32 ? (w0 >> f) & 1u : (w1 >> (f - 32)) & 1u;
+        const float s = h2f(s1[f]);
+        return bit ? s : -s;
+      };
+      float acc = val(0) + ((i & 1) ? -val(1) : val(1));
+      float acc2 = 0.0f;
+      for (int k = 1; k < 32; ++k) {
+        const int m = (k * i) & 63;
+        acc2 += val(2 * k) * cs[m] - val(2 * k + 1) * sn[m];
+      }
+      o[t * kD + c] = 0.125f * acc + 0.25f * acc2;
+    }
+  }
+}
+
+// grid = (32-token blocks of the quantized part, slabs of one layer); block = 128 threads.
+__global__ void __launch_bounds__(128) dequant_values_kernel(CacheView cv, int layer, int64_t T_q0, int64_t T_qt,
+                                                             int64_t n_prot, float* __restrict__ out) {
+  const int c = threadIdx.x;
+  const int slab = blockIdx.y;
+  const int b = slab / cv.H_kv, h = slab % cv.H_kv;
+  const uint8_t* sp = cv.slab(layer, b, h);
+  float* o = out + (static_cast<int64_t>(slab) * T_qt + static_cast<int64_t>(blockIdx.x) * kG) * kD;
+  for (int tt = 0; tt < kG; ++tt) {
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kG + tt;
+    bool prot = false;
+    int64_t pb = 0;
+    if (n_prot > 0 && t < T_q0) {
+      const uint32_t word = cv.e_words(b)[t / kG];
+      pb = cv.e_prefix(b)[t / kG] + __popc(word & ((1u << (t & 31)) - 1u));
+      prot = (word >> (t & 31)) & 1u;
+    }
+    float v;
+    if (prot) {
+      const uint8_t* pg = sp + cv.prot_offset + (pb / kG) * kPGBytes;
+      const int j = static_cast<int>(pb % kG);
+      const uint32_t word = reinterpret_cast<const uint32_t*>(pg)[j * 8 + (c >> 4)];
+      v = static_cast<float>((word >> (2 * (c & 15))) & 3u) * h2f(reinterpret_cast<const uint16_t*>(pg + kPG_S)[c]) +
+          h2f(reinterpret_cast<const uint16_t*>(pg + kPG_Z)[c]);
+    } else {
+      const int64_t n_rest = T_q0 - n_prot;
+      const int64_t u = t < T_q0 ? t - pb : (n_rest + kG - 1) / kG * kG + (t - T_q0);
+      const int64_t gi = u / kG;
+      const uint8_t* sg = sp + cv.tern_offset + (gi / kSGGroups) * kSGBytes;
+      const int slot = static_cast<int>(gi % kSGGroups);
+      const int tr = trit_digit(trit_byte_decode(sg[(u % kG) * kD + c]), slot) - 1;
+      v = static_cast<float>(tr) * h2f(reinterpret_cast<const uint16_t*>(sg + kSG_Scales)[slot * kD + c]);
+    }
+    o[tt * kD + c] = v;
+  }
+}
+
+cudaError_t launch_dequant_keys(const CacheView& cv, int layer, int64_t T_q0, int64_t n_flush, float* out,
+                                cudaStream_t stream) {
+  const int64_t T_qt = T_q0 + n_flush * kR;
+  if (T_qt == 0) return cudaSuccess;
+  dequant_keys_kernel<<<dim3(static_cast<unsigned>(T_qt / kG), cv.B * cv.H_kv), 128, 0, stream>>>(cv, layer, T_q0, T_qt, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dequant_values(const CacheView& cv, int layer, int64_t T_q0, int64_t n_flush, int64_t n_prot,
+                                  float* out, cudaStream_t stream) {
+  const int64_t T_qt = T_q0 + n_flush * kR;
+  if (T_qt == 0) return cudaSuccess;
+  dequant_values_kernel<<<dim3(static_cast<unsigned>(T_qt / kG), cv.B * cv.H_kv), 128, 0, stream>>>(cv, layer, T_q0, T_qt,
+                                                                                                     n_prot, out);
+  return cudaGetLastError();
+}
+
+}  // namespace vidkv

@@ -1,0 +1,415 @@
+// Host side of libvidkv: argument validation, sizing, per-layer token bookkeeping and the
+// launch sequences of the C ABI declared in include/vidkv.h.
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "kernels.cuh"
+
+using namespace vidkv;
+
+namespace {
+
+constexpr int64_t kAlign = 256;
+inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+  vidkv_layout_t lay;
+  int64_t max_prot;          // protected tokens the cache can hold per slab
+  int64_t max_total_tokens;  // prefill + new
+};
+
+vidkv_status_t check_config(const vidkv_config_t* c) {
+  if (!c) return VIDKV_ERR_INVALID_ARG;
+  if (c->B < 1 || c->L < 1 || c->H_kv < 1 || c->H_q < 1) return VIDKV_ERR_INVALID_ARG;
+  if (c->max_prefill_tokens < 0 || c->max_new_tokens < 0) return VIDKV_ERR_INVALID_ARG;
+  if (!(c->p_ratio >= 0.0f && c->p_ratio <= 1.0f)) return VIDKV_ERR_INVALID_ARG;
+  if (!(c->gamma >= 0.0f) || !std::isfinite(c->gamma)) return VIDKV_ERR_INVALID_ARG;
+  if (c->in_dtype != VIDKV_F16 && c->in_dtype != VIDKV_BF16) return VIDKV_ERR_INVALID_ARG;
+  if (c->out_dtype != VIDKV_F16 && c->out_dtype != VIDKV_BF16 && c->out_dtype != VIDKV_F32) return VIDKV_ERR_INVALID_ARG;
+  if (c->reserved != 0) return VIDKV_ERR_INVALID_ARG;
+  if (c->D != kD || c->G != kG || c->R != kR) return VIDKV_ERR_UNSUPPORTED;
+  if (c->k_ratio != 0.5f) return VIDKV_ERR_UNSUPPORTED;
+  if (c->key_1bit_mode != VIDKV_KEY1BIT_FFT_SIGN) return VIDKV_ERR_UNSUPPORTED;
+  if (c->H_q % c->H_kv != 0 || c->H_q / c->H_kv > kMaxRep) return VIDKV_ERR_UNSUPPORTED;
+  if (static_cast<int64_t>(c->L) * c->B * c->H_kv > 65535) return VIDKV_ERR_UNSUPPORTED;
+  return VIDKV_OK;
+}
+
+void compute_layout(const vidkv_config_t& c, Layout* out) {
+  vidkv_layout_t& l = out->lay;
+  const int64_t Tp = c.max_prefill_tokens, Nn = c.max_new_tokens;
+  const int64_t g0 = Tp / kG;
+  const int64_t max_flush = (kG - 1 + Nn) / kR;
+  out->max_prot = c.p_ratio > 0.0f ? static_cast<int64_t>(std::floor(static_cast<double>(c.p_ratio) * Tp)) : 0;
+  out->max_total_tokens = Tp + Nn;
+  l.header_bytes = kHeaderBytes;
+  l.sel_offset = kHeaderBytes;
+  l.sel_words = g0 + 1;
+  l.sel_stride_b = round_up(2 * l.sel_words * 4, kAlign);
+  l.slab_offset = round_up(l.sel_offset + l.sel_stride_b * c.B, kAlign);
+  l.max_chunks = 1 + max_flush;
+  l.max_kgroups = g0 + (kR / kG) * max_flush;
+  l.max_supergroups = (g0 + 1 + (kR / kG) * max_flush + kSGGroups - 1) / kSGGroups;
+  l.max_pgroups = (out->max_prot + kG - 1) / kG;
+  int64_t off = 0;
+  l.chunk_table_offset = off; off = round_up(off + l.max_chunks * kChunkBytes, kAlign);
+  l.kgroup_offset = off;      off = round_up(off + l.max_kgroups * kKGroupBytes, kAlign);
+  l.tern_offset = off;        off = round_up(off + l.max_supergroups * kSGBytes, kAlign);
+  l.prot_offset = off;        off = round_up(off + l.max_pgroups * kPGBytes, kAlign);
+  l.kres_offset = off;        off += kResBytes;
+  l.vres_offset = off;        off += kResBytes;
+  l.slab_stride = round_up(off, kAlign);
+  l.total_bytes = l.slab_offset + l.slab_stride * c.L * c.B * c.H_kv;
+}
+
+// Tokens per split: the largest of {640, 320, 160} that still gives >= 4 CTAs per SM on a
+// 148-SM part, else 160.
+int choose_split_tokens(int64_t T_tot, int64_t n_slabs) {
+  const int cand[3] = {640, 320, 160};
+  for (int s : cand)
+    if (n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
+  return 160;
+}
+
+int64_t max_partial_entries(const vidkv_config_t& c, int64_t T_max) {
+  int64_t best = 0;
+  if (T_max < 1) T_max = 1;
+  for (int n = 1; n <= c.L; ++n) {
+    const int64_t slabs = static_cast<int64_t>(n) * c.B * c.H_kv;
+    const int st = choose_split_tokens(T_max, slabs);
+    const int64_t e = static_cast<int64_t>(n) * c.B * c.H_q * ((T_max + st - 1) / st);
+    if (e > best) best = e;
+  }
+  return best;
+}
+
+struct WsPlan {
+  int64_t minmax_off, partials_off, idx_prot_off, idx_rest_off, counts_off, total;
+  int64_t partial_entries;
+};
+
+void plan_workspace(const vidkv_config_t& c, const Layout& L, WsPlan* w) {
+  int64_t off = 0;
+  w->minmax_off = off;
+  off = round_up(off + static_cast<int64_t>(c.L) * c.B * c.H_kv * 2 * kD * 4, kAlign);
+  w->partial_entries = max_partial_entries(c, L.max_total_tokens);
+  w->partials_off = off;
+  off = round_up(off + w->partial_entries * 130 * 4, kAlign);
+  w->idx_prot_off = off;
+  off = round_up(off + static_cast<int64_t>(c.B) * L.max_prot * 4, kAlign);
+  w->idx_rest_off = off;
+  off = round_up(off + (L.max_prot > 0 ? static_cast<int64_t>(c.B) * c.max_prefill_tokens * 4 : 0), kAlign);
+  w->counts_off = off;
+  off = round_up(off + static_cast<int64_t>(c.B) * 4, kAlign);
+  w->total = off;
+}
+
+struct LayerInfo {
+  bool k_done = false, v_done = false;
+  int64_t T = 0, T_q0 = 0, n_flush = 0, new_tokens = 0;
+  int n_res = 0;
+};
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+struct vidkv_cache {
+  vidkv_config_t cfg;
+  Layout L;
+  WsPlan ws;
+  CacheView cv;
+  uint8_t* cache;
+  uint8_t* workspace;
+  bool sel_set;
+  int64_t sel_T, n_prot;
+  std::vector<LayerInfo> layers;
+};
+
+extern "C" {
+
+int32_t vidkv_version(void) { return 100; }
+
+vidkv_status_t vidkv_cache_layout(const vidkv_config_t* cfg, vidkv_layout_t* layout) {
+  if (!layout) return VIDKV_ERR_INVALID_ARG;
+  const vidkv_status_t st = check_config(cfg);
+  if (st != VIDKV_OK) return st;
+  Layout L;
+  compute_layout(*cfg, &L);
+  *layout = L.lay;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_cache_bytes(const vidkv_config_t* cfg, size_t* cache_bytes, size_t* workspace_bytes) {
+  if (!cache_bytes || !workspace_bytes) return VIDKV_ERR_INVALID_ARG;
+  const vidkv_status_t st = check_config(cfg);
+  if (st != VIDKV_OK) return st;
+  Layout L;
+  compute_layout(*cfg, &L);
+  WsPlan w;
+  plan_workspace(*cfg, L, &w);
+  *cache_bytes = static_cast<size_t>(L.lay.total_bytes);
+  *workspace_bytes = static_cast<size_t>(w.total);
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_cache_init(const vidkv_config_t* cfg, void* cache, size_t cache_bytes, void* workspace,
+                                size_t workspace_bytes, void* stream, vidkv_cache_t** handle) {
+  if (!handle) return VIDKV_ERR_INVALID_ARG;
+  *handle = nullptr;
+  const vidkv_status_t st = check_config(cfg);
+  if (st != VIDKV_OK) return st;
+  if (!cache || !workspace) return VIDKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(cache) % kAlign) || (reinterpret_cast<uintptr_t>(workspace) % kAlign))
+    return VIDKV_ERR_ALIGNMENT;
+  vidkv_cache* h = new (std::nothrow) vidkv_cache();
+  if (!h) return VIDKV_ERR_INVALID_ARG;
+  h->cfg = *cfg;
+  compute_layout(*cfg, &h->L);
+  plan_workspace(*cfg, h->L, &h->ws);
+  if (cache_bytes < static_cast<size_t>(h->L.lay.total_bytes) || workspace_bytes < static_cast<size_t>(h->ws.total)) {
+    delete h;
+    return VIDKV_ERR_CAPACITY;
+  }
+  h->cache = static_cast<uint8_t*>(cache);
+  h->workspace = static_cast<uint8_t*>(workspace);
+  const vidkv_layout_t& l = h->L.lay;
+  CacheView& cv = h->cv;
+  cv.base = h->cache;
+  cv.sel_offset = l.sel_offset; cv.sel_stride_b = l.sel_stride_b; cv.sel_words = l.sel_words;
+  cv.slab_offset = l.slab_offset; cv.slab_stride = l.slab_stride;
+  cv.chunk_table_offset = l.chunk_table_offset; cv.kgroup_offset = l.kgroup_offset;
+  cv.tern_offset = l.tern_offset; cv.prot_offset = l.prot_offset;
+  cv.kres_offset = l.kres_offset; cv.vres_offset = l.vres_offset;
+  cv.B = cfg->B; cv.H_kv = cfg->H_kv; cv.H_q = cfg->H_q; cv.rep = cfg->H_q / cfg->H_kv;
+  h->sel_set = false; h->sel_T = 0; h->n_prot = 0;
+  h->layers.assign(cfg->L, LayerInfo());
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(h->cache, 0, static_cast<size_t>(l.total_bytes), s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }
+  const uint32_t hdr[3] = {kMagic, static_cast<uint32_t>(vidkv_version()), 0u};
+  if (cudaMemcpyAsync(h->cache, hdr, sizeof(hdr), cudaMemcpyHostToDevice, s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }
+  if (cudaStreamSynchronize(s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }   // hdr is a stack buffer
+  *handle = h;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_cache_destroy(vidkv_cache_t* h) {
+  if (!h) return VIDKV_ERR_INVALID_ARG;
+  delete h;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_cache_reset(vidkv_cache_t* h, void* stream) {
+  (void)stream;
+  if (!h) return VIDKV_ERR_INVALID_ARG;
+  h->sel_set = false; h->sel_T = 0; h->n_prot = 0;
+  h->layers.assign(h->cfg.L, LayerInfo());
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_select_tokens(vidkv_cache_t* h, const float* saliency, int64_t vis_begin, int64_t l_v, int64_t T,
+                                   void* stream) {
+  if (!h || T < 0) return VIDKV_ERR_INVALID_ARG;
+  if (T > h->cfg.max_prefill_tokens) return VIDKV_ERR_CAPACITY;
+  for (const LayerInfo& li : h->layers)
+    if (li.v_done) return VIDKV_ERR_STATE;
+  const int64_t T_q = T - T % kG;
+  if (!saliency || h->cfg.p_ratio == 0.0f) {
+    h->sel_set = true; h->sel_T = T; h->n_prot = 0;
+    return VIDKV_OK;
+  }
+  if (vis_begin < 0 || l_v < 1 || vis_begin + l_v > T_q) return VIDKV_ERR_INVALID_ARG;
+  if (!aligned16(saliency)) return VIDKV_ERR_ALIGNMENT;
+  const int64_t n = static_cast<int64_t>(std::floor(static_cast<double>(h->cfg.p_ratio) * static_cast<double>(l_v)));
+  if (n > h->L.max_prot) return VIDKV_ERR_CAPACITY;
+  if (n > 0) {
+    int32_t* ip = reinterpret_cast<int32_t*>(h->workspace + h->ws.idx_prot_off);
+    int32_t* ir = reinterpret_cast<int32_t*>(h->workspace + h->ws.idx_rest_off);
+    if (launch_select_tokens(saliency, vis_begin, l_v, n, T_q, h->cv, ip, ir, h->L.max_prot, h->cfg.max_prefill_tokens,
+                             static_cast<cudaStream_t>(stream)) != cudaSuccess)
+      return VIDKV_ERR_CUDA;
+  }
+  h->sel_set = true; h->sel_T = T; h->n_prot = n;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_set_token_mask(vidkv_cache_t* h, const uint8_t* E, int64_t T, void* stream) {
+  if (!h || !E || T < 0) return VIDKV_ERR_INVALID_ARG;
+  if (T > h->cfg.max_prefill_tokens) return VIDKV_ERR_CAPACITY;
+  for (const LayerInfo& li : h->layers)
+    if (li.v_done) return VIDKV_ERR_STATE;
+  if (h->L.max_prot == 0) return VIDKV_ERR_CAPACITY;
+  const int64_t T_q = T - T % kG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t* ip = reinterpret_cast<int32_t*>(h->workspace + h->ws.idx_prot_off);
+  int32_t* ir = reinterpret_cast<int32_t*>(h->workspace + h->ws.idx_rest_off);
+  int32_t* dc = reinterpret_cast<int32_t*>(h->workspace + h->ws.counts_off);
+  if (launch_mask_to_selection(E, T, T_q, h->cv, ip, ir, h->L.max_prot, h->cfg.max_prefill_tokens, dc, s) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  std::vector<int32_t> counts(h->cfg.B);
+  if (cudaMemcpyAsync(counts.data(), dc, sizeof(int32_t) * h->cfg.B, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  for (int b = 1; b < h->cfg.B; ++b)
+    if (counts[b] != counts[0]) return VIDKV_ERR_INVALID_ARG;
+  if (counts[0] > h->L.max_prot) return VIDKV_ERR_CAPACITY;
+  h->sel_set = true; h->sel_T = T; h->n_prot = counts[0];
+  return VIDKV_OK;
+}
+
+static vidkv_status_t check_kv_args(vidkv_cache_t* h, int32_t layer, const void* X, int64_t T, int64_t sb, int64_t sh,
+                                    int64_t st) {
+  if (!h || !X || T < 0) return VIDKV_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  if (sb < 0 || sh < 0 || st < kD) return VIDKV_ERR_INVALID_ARG;
+  if (!aligned16(X) || (sb % 8) || (sh % 8) || (st % 8)) return VIDKV_ERR_ALIGNMENT;
+  if (T > h->cfg.max_prefill_tokens) return VIDKV_ERR_CAPACITY;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_quantize_keys(vidkv_cache_t* h, int32_t layer, const void* K, int64_t T, int64_t stride_b,
+                                   int64_t stride_h, int64_t stride_t, void* stream) {
+  vidkv_status_t st = check_kv_args(h, layer, K, T, stride_b, stride_h, stride_t);
+  if (st != VIDKV_OK) return st;
+  LayerInfo& li = h->layers[layer];
+  if (li.k_done) return VIDKV_ERR_STATE;
+  if (li.v_done && li.T != T) return VIDKV_ERR_STATE;
+  const int64_t T_q = T - T % kG;
+  const int r = static_cast<int>(T % kG);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  KSrc src{K, stride_b, stride_h, stride_t, h->cfg.H_kv};
+  uint32_t* minmax = reinterpret_cast<uint32_t*>(h->workspace + h->ws.minmax_off);
+  if (launch_quantize_keys(h->cfg.in_dtype, src, T_q, h->cv, layer, 1, 0, 0, minmax, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  if (launch_copy_to_residual(h->cfg.in_dtype, src, T_q, r, h->cv, layer, false, 0, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  li.k_done = true; li.T = T; li.T_q0 = T_q; li.n_res = r; li.n_flush = 0;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_quantize_values(vidkv_cache_t* h, int32_t layer, const void* V, int64_t T, int64_t stride_b,
+                                     int64_t stride_h, int64_t stride_t, void* stream) {
+  vidkv_status_t st = check_kv_args(h, layer, V, T, stride_b, stride_h, stride_t);
+  if (st != VIDKV_OK) return st;
+  LayerInfo& li = h->layers[layer];
+  if (li.v_done) return VIDKV_ERR_STATE;
+  if (li.k_done && li.T != T) return VIDKV_ERR_STATE;
+  if (h->cfg.p_ratio > 0.0f && !h->sel_set) return VIDKV_ERR_STATE;
+  if (h->sel_set && h->n_prot > 0 && h->sel_T != T) return VIDKV_ERR_STATE;
+  const int64_t T_q = T - T % kG;
+  const int r = static_cast<int>(T % kG);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  KSrc src{V, stride_b, stride_h, stride_t, h->cfg.H_kv};
+  SelView sel{nullptr, nullptr, 0, 0, 0};
+  if (h->sel_set && h->n_prot > 0) {
+    sel.idx_prot = reinterpret_cast<int32_t*>(h->workspace + h->ws.idx_prot_off);
+    sel.idx_rest = reinterpret_cast<int32_t*>(h->workspace + h->ws.idx_rest_off);
+    sel.stride_prot = h->L.max_prot;
+    sel.stride_rest = h->cfg.max_prefill_tokens;
+    sel.n_prot = h->n_prot;
+  }
+  if (T_q > 0 && launch_quantize_values(h->cfg.in_dtype, src, T_q, h->cv, layer, sel, h->cfg.gamma, s) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  if (launch_copy_to_residual(h->cfg.in_dtype, src, T_q, r, h->cv, layer, true, 0, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  li.v_done = true; li.T = T; li.T_q0 = T_q; li.n_res = r; li.n_flush = 0;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int32_t n_layers, const void* q,
+                                      const void* k_new, const void* v_new, void* out, float softmax_scale,
+                                      void* stream) {
+  if (!h || !q || !k_new || !v_new || !out) return VIDKV_ERR_INVALID_ARG;
+  if (layer_begin < 0 || n_layers < 1 || layer_begin + n_layers > h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return VIDKV_ERR_ALIGNMENT;
+  if (!std::isfinite(softmax_scale)) return VIDKV_ERR_INVALID_ARG;
+  const LayerInfo& first = h->layers[layer_begin];
+  for (int l = layer_begin; l < layer_begin + n_layers; ++l) {
+    const LayerInfo& li = h->layers[l];
+    if (!li.k_done || !li.v_done) return VIDKV_ERR_STATE;
+    if (li.T_q0 != first.T_q0 || li.n_flush != first.n_flush || li.n_res != first.n_res) return VIDKV_ERR_STATE;
+    if (li.new_tokens + 1 > h->cfg.max_new_tokens) return VIDKV_ERR_CAPACITY;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int dt = h->cfg.in_dtype;
+  if (launch_append(dt, k_new, v_new, h->cv, layer_begin, n_layers, first.n_res, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  DecodeArgs a;
+  a.cv = h->cv;
+  a.q = q; a.k_new = k_new; a.v_new = v_new; a.out = out;
+  a.partials = reinterpret_cast<float*>(h->workspace + h->ws.partials_off);
+  a.layer0 = layer_begin; a.n_layers = n_layers;
+  a.in_dtype = dt; a.out_dtype = h->cfg.out_dtype;
+  a.n_prot = h->n_prot;
+  a.scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / std::sqrt(static_cast<float>(kD));
+  a.st.T_q0 = first.T_q0; a.st.n_flush = first.n_flush; a.st.n_res = first.n_res + 1;
+  const int64_t T_tot = first.T_q0 + first.n_flush * kR + a.st.n_res;
+  const int64_t n_slabs = static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv;
+  a.split_tokens = choose_split_tokens(T_tot, n_slabs);
+  a.n_splits = static_cast<int32_t>((T_tot + a.split_tokens - 1) / a.split_tokens);
+  if (static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_q * a.n_splits > h->ws.partial_entries) return VIDKV_ERR_CAPACITY;
+  if (launch_decode(a, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  const bool flush = a.st.n_res == kR;
+  if (flush) {
+    const int64_t es = h->cv.slab_stride / 2;    // slab stride in 16-bit elements
+    const uint8_t* slab0 = h->cache + h->cv.slab_offset + static_cast<int64_t>(layer_begin) * h->cfg.B * h->cfg.H_kv * h->cv.slab_stride;
+    KSrc ksrc{slab0 + h->cv.kres_offset, es * h->cfg.H_kv, es, kD, h->cfg.H_kv};
+    KSrc vsrc{slab0 + h->cv.vres_offset, es * h->cfg.H_kv, es, kD, h->cfg.H_kv};
+    uint32_t* minmax = reinterpret_cast<uint32_t*>(h->workspace + h->ws.minmax_off);
+    const int chunk = 1 + static_cast<int>(first.n_flush);
+    const int64_t kgroup0 = first.T_q0 / kG + (kR / kG) * first.n_flush;
+    if (launch_quantize_keys(dt, ksrc, kR, h->cv, layer_begin, n_layers, chunk, kgroup0, minmax, s) != cudaSuccess)
+      return VIDKV_ERR_CUDA;
+    const int64_t n_rest = first.T_q0 - h->n_prot;
+    const int64_t tgroup0 = (n_rest + kG - 1) / kG + (kR / kG) * first.n_flush;
+    if (launch_flush_values(dt, vsrc, h->cv, layer_begin, n_layers, tgroup0, h->cfg.gamma, s) != cudaSuccess)
+      return VIDKV_ERR_CUDA;
+  }
+  for (int l = layer_begin; l < layer_begin + n_layers; ++l) {
+    LayerInfo& li = h->layers[l];
+    li.new_tokens += 1;
+    if (flush) { li.n_flush += 1; li.n_res = 0; }
+    else li.n_res += 1;
+  }
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_layer_state(const vidkv_cache_t* h, int32_t layer, int64_t* n_quantized, int64_t* n_residual,
+                                 int64_t* n_chunks, int64_t* n_protected) {
+  if (!h || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  const LayerInfo& li = h->layers[layer];
+  if (n_quantized) *n_quantized = li.T_q0 + li.n_flush * kR;
+  if (n_residual) *n_residual = li.n_res;
+  if (n_chunks) *n_chunks = (li.T_q0 > 0 ? 1 : 0) + li.n_flush;
+  if (n_protected) *n_protected = h->n_prot;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_cache_status(vidkv_cache_t* h, void* stream) {
+  if (!h) return VIDKV_ERR_INVALID_ARG;
+  int32_t word = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&word, h->cache + kHdrStatus, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  return word;
+}
+
+vidkv_status_t vidkv_dequantize_keys(vidkv_cache_t* h, int32_t layer, float* out, void* stream) {
+  if (!h || !out || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  const LayerInfo& li = h->layers[layer];
+  if (!li.k_done) return VIDKV_ERR_STATE;
+  if (launch_dequant_keys(h->cv, layer, li.T_q0, li.n_flush, out, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* h, int32_t layer, float* out, void* stream) {
+  if (!h || !out || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  const LayerInfo& li = h->layers[layer];
+  if (!li.v_done) return VIDKV_ERR_STATE;
+  if (launch_dequant_values(h->cv, layer, li.T_q0, li.n_flush, h->n_prot, out, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  return VIDKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,91 @@
+// Internal launcher interface between the host API and the kernel files.
+#pragma once
+
+#include "common.cuh"
+
+namespace vidkv {
+
+// A [slabs, tokens, 128] source of keys or values.  Source slab i (= b * H + h, running
+// over layers first when several layers are processed) starts at
+// ptr + (i / H) * stride_b + (i % H) * stride_h elements; token t at + t * stride_t.
+struct KSrc {
+  const void* ptr;
+  int64_t stride_b, stride_h, stride_t;
+  int32_t H;
+};
+
+// Token-selection data handed to the value quantizer (NULL lists = no protection).
+struct SelView {
+  const int32_t* idx_prot;   // [B][n_prot]       ascending protected token ids
+  const int32_t* idx_rest;   // [B][T - n_prot]   ascending unprotected token ids
+  int64_t stride_prot, stride_rest;
+  int64_t n_prot;
+};
+
+__global__ void init_min_kernel(uint32_t* minmax, int n_slabs);
+
+// Algorithm 3 on `T_tokens` tokens (a multiple of 32) of every slab of layers
+// [layer0, layer0 + n_layers): writes chunk `chunk` of the chunk table and the key groups
+// starting at group index kgroup0.  minmax: scratch, 256 uint32 per slab.
+cudaError_t launch_quantize_keys(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0,
+                                 int n_layers, int chunk, int64_t kgroup0, uint32_t* minmax, cudaStream_t stream);
+
+// Algorithm 2 on the prefill tokens of one layer.  T_q (multiple of 32) tokens; the
+// unprotected ones go to ternary stream positions 0.., the protected ones to 2-bit groups.
+cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer,
+                                   const SelView& sel, float gamma, cudaStream_t stream);
+
+// 1.58Quant of a full 128-token residual of every slab of the given layers, appended at
+// ternary stream group index tgroup0 (read-modify-write of shared supergroup bytes).
+cudaError_t launch_flush_values(int dtype, const KSrc& src, const CacheView& cv, int layer0, int n_layers,
+                                int64_t tgroup0, float gamma, cudaStream_t stream);
+
+// Copy `n_tok` tokens starting at token t_begin of every slab of one layer into the
+// residual rings (rows r0 .. r0 + n_tok - 1).
+cudaError_t launch_copy_to_residual(int dtype, const KSrc& src, int64_t t_begin, int n_tok, const CacheView& cv,
+                                    int layer, bool is_value, int r0, cudaStream_t stream);
+
+// Token selection (Sec. 3.3(2)): top-n by saliency, E words + prefix counts into the cache,
+// gather lists into the workspace.
+cudaError_t launch_select_tokens(const float* saliency, int64_t vis_begin, int64_t l_v, int64_t n_prot, int64_t T_q,
+                                 const CacheView& cv, int32_t* idx_prot, int32_t* idx_rest, int64_t stride_prot,
+                                 int64_t stride_rest, cudaStream_t stream);
+cudaError_t launch_mask_to_selection(const uint8_t* E, int64_t T, int64_t T_q, const CacheView& cv, int32_t* idx_prot,
+                                     int32_t* idx_rest, int64_t stride_prot, int64_t stride_rest, int32_t* counts,
+                                     cudaStream_t stream);
+
+// Token counts the decode kernels need (the same for every layer of one call).
+struct LayerState {
+  int64_t T_q0;        // prefill tokens quantized (multiple of 32)
+  int64_t n_flush;     // flushed 128-token chunks
+  int32_t n_res;       // residual tokens (after the append of this step)
+};
+
+struct DecodeArgs {
+  CacheView cv;
+  const void* q;
+  const void* k_new;
+  const void* v_new;
+  void* out;
+  float* partials;     // [n_layers * B * H_q * n_splits][130]
+  int32_t layer0, n_layers;
+  int32_t in_dtype, out_dtype;
+  int32_t split_tokens, n_splits;
+  int64_t n_prot;      // protected tokens per batch element (0 = no STP)
+  float scale;
+  LayerState st;
+};
+
+// Split-KV attention over the packed cache + residual, then the merge of the partials.
+cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
+// Write k_new / v_new [n_layers, B, H_kv, D] into row `row` of the residual rings.
+cudaError_t launch_append(int dtype, const void* k_new, const void* v_new, const CacheView& cv, int layer0,
+                          int n_layers, int row, cudaStream_t stream);
+
+// Test-only dequantizers (float32 [B, H_kv, n_quantized, D]).
+cudaError_t launch_dequant_keys(const CacheView& cv, int layer, int64_t T_q0, int64_t n_flush, float* out,
+                                cudaStream_t stream);
+cudaError_t launch_dequant_values(const CacheView& cv, int layer, int64_t T_q0, int64_t n_flush, int64_t n_prot,
+                                  float* out, cudaStream_t stream);
+
+}  // namespace vidkv

@@ -1,0 +1,377 @@
+// Value quantizer kernels: Algorithm 2 of the paper (1.58Quant, STPQuant), the token
+// selection of Sec. 3.3(2), and the residual copies of Algorithm 1.
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace vidkv {
+
+// ---------------------------------------------------------------------------------
+// 1.58Quant (Eq. 6) of one supergroup = 5 groups x 32 stream tokens x 128 channels.
+// grid = (supergroups, slabs of one layer); block = 256 threads.
+// Stream position u of the unprotected tokens maps to token idx_rest[u] (identity when
+// no token is protected).  Byte (j, c) collects the digits of token j of each group.
+// ---------------------------------------------------------------------------------
+constexpr int kSGTokens = kSGGroups * kG;   // 160
+
+template <typename T>
+__global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest, CacheView cv, int layer,
+                                                        SelView sel, float gamma) {
+  __shared__ __align__(16) uint16_t tile[kSGTokens * kD];      // raw 16-bit elements, 40 KB
+  __shared__ float s_alpha[kSGGroups * kD];
+  const int slab = blockIdx.y;
+  const int b = slab / cv.H_kv, h = slab % cv.H_kv;
+  const T* base = reinterpret_cast<const T*>(src.ptr) + b * src.stride_b + h * src.stride_h;
+  const int64_t u0 = static_cast<int64_t>(blockIdx.x) * kSGTokens;
+  const int n_rows = static_cast<int>(min(static_cast<int64_t>(kSGTokens), n_rest - u0));
+  const int32_t* idx = sel.idx_rest ? sel.idx_rest + b * sel.stride_rest : nullptr;
+  {
+    const int lane16 = threadIdx.x & 15, row = threadIdx.x >> 4;
+    for (int r = row; r < kSGTokens; r += 16) {
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (r < n_rows) {
+        const int64_t t = idx ? idx[u0 + r] : (u0 + r);
+        v = __ldg(reinterpret_cast<const uint4*>(base + t * src.stride_t) + lane16);
+      }
+      reinterpret_cast<uint4*>(tile + r * kD)[lane16] = v;
+    }
+  }
+  __syncthreads();
+  uint8_t* sg = cv.slab(layer, b, h) + cv.tern_offset + static_cast<int64_t>(blockIdx.x) * kSGBytes;
+  // pass 1: s = Mean |v| per (group, channel), sequential over the tokens present
+  for (int item = threadIdx.x; item < kSGGroups * kD; item += 256) {
+    const int c = item & (kD - 1), g = item >> 7;
+    const int n = max(0, min(kG, n_rows - g * kG));
+    float sum = 0.0f;
+    for (int j = 0; j < n; ++j) sum += fabsf(Elem<T>::to_float(reinterpret_cast<const T*>(tile)[(g * kG + j) * kD + c]));
+    float alpha = 0.0f;
+    if (n > 0) {
+      const uint16_t sh = f2h_bits(__fdiv_rn(sum, static_cast<float>(n)));
+      reinterpret_cast<uint16_t*>(sg + kSG_Scales)[g * kD + c] = sh;
+      alpha = __fmul_rn(gamma, h2f(sh));
+    }
+    s_alpha[item] = alpha;
+  }
+  __syncthreads();
+  // pass 2: digits and bytes
+  for (int item = threadIdx.x; item < kG * kD; item += 256) {
+    const int c = item & (kD - 1), j = item >> 7;
+    uint32_t bval = 0;
+#pragma unroll
+    for (int g = 0; g < kSGGroups; ++g) {
+      const float v = Elem<T>::to_float(reinterpret_cast<const T*>(tile)[(g * kG + j) * kD + c]);
+      const float a = s_alpha[g * kD + c];
+      const uint32_t d = (g * kG + j < n_rows) ? (v > a ? 2u : (v < -a ? 0u : 1u)) : 1u;
+      bval = bval * 3u + d;
+    }
+    sg[item] = static_cast<uint8_t>(trit_byte_encode(bval));
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// 2-bit GQuant (Eq. 4) of one group of up to 32 protected tokens.  grid = (groups, slabs).
+// ---------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(128) v_protect_kernel(KSrc src, CacheView cv, int layer, SelView sel) {
+  __shared__ __align__(16) uint16_t tile[kG * kD];
+  __shared__ uint16_t s_s[kD], s_z[kD];
+  const int slab = blockIdx.y;
+  const int b = slab / cv.H_kv, h = slab % cv.H_kv;
+  const T* base = reinterpret_cast<const T*>(src.ptr) + b * src.stride_b + h * src.stride_h;
+  const int64_t p0 = static_cast<int64_t>(blockIdx.x) * kG;
+  const int n_rows = static_cast<int>(min(static_cast<int64_t>(kG), sel.n_prot - p0));
+  const int32_t* idx = sel.idx_prot + b * sel.stride_prot;
+  {
+    const int lane16 = threadIdx.x & 15, row = threadIdx.x >> 4;
+    for (int r = row; r < kG; r += 8) {
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (r < n_rows) v = __ldg(reinterpret_cast<const uint4*>(base + static_cast<int64_t>(idx[p0 + r]) * src.stride_t) + lane16);
+      reinterpret_cast<uint4*>(tile + r * kD)[lane16] = v;
+    }
+  }
+  __syncthreads();
+  uint8_t* pg = cv.slab(layer, b, h) + cv.prot_offset + static_cast<int64_t>(blockIdx.x) * kPGBytes;
+  {
+    const int c = threadIdx.x;
+    float mn = INFINITY, mx = -INFINITY;
+    for (int j = 0; j < n_rows; ++j) {
+      const float v = Elem<T>::to_float(reinterpret_cast<const T*>(tile)[j * kD + c]);
+      mn = fminf(mn, v); mx = fmaxf(mx, v);
+    }
+    const uint16_t sh = f2h_bits(__fdiv_rn(__fsub_rn(mx, mn), 3.0f)), zh = f2h_bits(mn);
+    s_s[c] = sh; s_z[c] = zh;
+    reinterpret_cast<uint16_t*>(pg + kPG_S)[c] = sh;
+    reinterpret_cast<uint16_t*>(pg + kPG_Z)[c] = zh;
+  }
+  __syncthreads();
+  for (int item = threadIdx.x; item < kG * 8; item += 128) {
+    const int j = item >> 3, wi = item & 7;
+    uint32_t word = 0;
+    if (j < n_rows) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int c = wi * 16 + i;
+        const float s = h2f(s_s[c]), z = h2f(s_z[c]);
+        const float v = Elem<T>::to_float(reinterpret_cast<const T*>(tile)[j * kD + c]);
+        float q = rintf(__fdiv_rn(__fsub_rn(v, z), s));
+        q = fminf(fmaxf(q, 0.0f), 3.0f);
+        word |= ((s == 0.0f) ? 0u : static_cast<uint32_t>(q)) << (2 * i);
+      }
+    }
+    reinterpret_cast<uint32_t*>(pg)[item] = word;
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// Residual flush, value half (Algorithm 1, Decoding): 1.58Quant of the 128 residual tokens
+// of every slab, appended as 4 groups at ternary stream group index tgroup0.  The groups
+// may land in a supergroup that already holds earlier groups, so bytes are updated digit
+// by digit.  grid = slabs (over layers); block = 128 threads (thread = channel).
+// ---------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kD) v_flush_kernel(KSrc src, CacheView cv, int layer0, int slabs_per_layer,
+                                                     int64_t tgroup0, float gamma) {
+  const int slab = blockIdx.x;
+  const int layer = layer0 + slab / slabs_per_layer;
+  const int bh = slab % slabs_per_layer;
+  const T* base = reinterpret_cast<const T*>(src.ptr) + (slab / src.H) * src.stride_b + (slab % src.H) * src.stride_h;
+  uint8_t* tern = cv.slab(layer, bh / cv.H_kv, bh % cv.H_kv) + cv.tern_offset;
+  const int c = threadIdx.x;
+  const uint32_t p3[5] = {81u, 27u, 9u, 3u, 1u};
+  for (int g4 = 0; g4 < kR / kG; ++g4) {
+    const int64_t gi = tgroup0 + g4;
+    uint8_t* sg = tern + (gi / kSGGroups) * kSGBytes;
+    const int slot = static_cast<int>(gi % kSGGroups);
+    float sum = 0.0f;
+    for (int j = 0; j < kG; ++j) sum += fabsf(Elem<T>::to_float(base[(g4 * kG + j) * src.stride_t + c]));
+    const uint16_t sh = f2h_bits(__fdiv_rn(sum, static_cast<float>(kG)));
+    reinterpret_cast<uint16_t*>(sg + kSG_Scales)[slot * kD + c] = sh;
+    const float a = __fmul_rn(gamma, h2f(sh));
+    for (int j = 0; j < kG; ++j) {
+      const float v = Elem<T>::to_float(base[(g4 * kG + j) * src.stride_t + c]);
+      const uint32_t d = v > a ? 2u : (v < -a ? 0u : 1u);
+      const uint32_t bold = trit_byte_decode(sg[j * kD + c]);
+      const uint32_t dold = (bold / p3[slot]) % 3u;
+      sg[j * kD + c] = static_cast<uint8_t>(trit_byte_encode(bold - dold * p3[slot] + d * p3[slot]));
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// Residual copies (Algorithm 1: X_r = X[l - r:], and the per-step append).
+// ---------------------------------------------------------------------------------
+template <typename T>
+__global__ void copy_to_residual_kernel(KSrc src, int64_t t_begin, int n_tok, CacheView cv, int layer,
+                                        int64_t res_offset, int r0) {
+  const int slab = blockIdx.x;
+  const int b = slab / cv.H_kv, h = slab % cv.H_kv;
+  const T* base = reinterpret_cast<const T*>(src.ptr) + b * src.stride_b + h * src.stride_h;
+  uint4* dst = reinterpret_cast<uint4*>(cv.slab(layer, b, h) + res_offset);
+  for (int i = threadIdx.x; i < n_tok * 16; i += blockDim.x) {
+    const int r = i >> 4, l = i & 15;
+    dst[(r0 + r) * 16 + l] = __ldg(reinterpret_cast<const uint4*>(base + (t_begin + r) * src.stride_t) + l);
+  }
+}
+
+// One block of 32 threads per (layer, b, h): lanes 0-15 copy the key row, 16-31 the value row.
+__global__ void append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, CacheView cv,
+                              int layer0, int slabs_per_layer, int row) {
+  const int slab = blockIdx.x;
+  const int layer = layer0 + slab / slabs_per_layer;
+  const int bh = slab % slabs_per_layer;
+  uint8_t* sp = cv.slab(layer, bh / cv.H_kv, bh % cv.H_kv);
+  const int l = threadIdx.x & 15;
+  if (threadIdx.x < 16)
+    reinterpret_cast<uint4*>(sp + cv.kres_offset)[row * 16 + l] = __ldg(k_new + static_cast<int64_t>(slab) * 16 + l);
+  else
+    reinterpret_cast<uint4*>(sp + cv.vres_offset)[row * 16 + l] = __ldg(v_new + static_cast<int64_t>(slab) * 16 + l);
+}
+
+// ---------------------------------------------------------------------------------
+// Token selection: top n of l_v saliency scores per batch element (ties: lower index).
+// One block of 1024 threads per batch element.  Phase 1: 4-pass radix select of the n-th
+// largest key.  Phase 2: E words, per-word prefix counts and the two gather lists.
+// ---------------------------------------------------------------------------------
+__device__ __forceinline__ int block_exclusive_scan_1024(int v, int* s_warp, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) s_warp[warp] = x;
+  __syncthreads();
+  if (warp == 0) {
+    int w = s_warp[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, w, o);
+      if (lane >= o) w += y;
+    }
+    s_warp[lane] = w;
+  }
+  __syncthreads();
+  const int warp_off = warp ? s_warp[warp - 1] : 0;
+  *total = s_warp[31];
+  __syncthreads();
+  return warp_off + x - v;
+}
+
+// mode 0: from saliency (radix select); mode 1: from a byte mask E [B][T].
+__global__ void __launch_bounds__(1024) select_tokens_kernel(const float* __restrict__ saliency,
+                                                             const uint8_t* __restrict__ mask, int64_t mask_stride,
+                                                             int64_t vis_begin, int64_t l_v, int64_t n_prot,
+                                                             int64_t T_q, CacheView cv, int32_t* idx_prot,
+                                                             int32_t* idx_rest, int64_t stride_prot,
+                                                             int64_t stride_rest, int32_t* counts) {
+  __shared__ int hist[256];
+  __shared__ int s_warp[32];
+  __shared__ uint32_t s_prefix, s_need;
+  const int b = blockIdx.x;
+  const float* sal = saliency ? saliency + b * l_v : nullptr;
+  uint32_t thr = 0, need = 0;
+  if (sal && n_prot > 0) {
+    uint32_t prefix = 0, pmask = 0;
+    need = static_cast<uint32_t>(n_prot);
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+      __syncthreads();
+      for (int64_t i = threadIdx.x; i < l_v; i += 1024) {
+        const uint32_t key = float_ordered(sal[i]);
+        if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        uint32_t cum = 0;
+        int d = 255;
+        for (; d > 0; --d) {
+          if (cum + hist[d] >= need) break;
+          cum += hist[d];
+        }
+        s_prefix = prefix | (static_cast<uint32_t>(d) << shift);
+        s_need = need - cum;
+      }
+      __syncthreads();
+      prefix = s_prefix; need = s_need;
+      pmask |= 255u << shift;
+      __syncthreads();
+    }
+    thr = prefix;       // key of the n-th largest; `need` of the keys equal to it are taken
+  }
+  uint32_t* e_words = const_cast<uint32_t*>(cv.e_words(b));
+  uint32_t* e_prefix = const_cast<uint32_t*>(cv.e_prefix(b));
+  const int64_t W = T_q / kG;
+  int eq_carry = 0, prot_carry = 0;
+  for (int64_t wbase = 0; wbase < W; wbase += 1024) {
+    const int64_t w = wbase + threadIdx.x;
+    uint32_t word_gt = 0, word_eq = 0;
+    if (w < W) {
+      for (int i = 0; i < 32; ++i) {
+        const int64_t t = w * 32 + i;
+        if (mask) {
+          if (mask[b * mask_stride + t]) word_gt |= 1u << i;
+        } else if (sal && n_prot > 0 && t >= vis_begin && t < vis_begin + l_v) {
+          const uint32_t key = float_ordered(sal[t - vis_begin]);
+          if (key > thr) word_gt |= 1u << i;
+          else if (key == thr) word_eq |= 1u << i;
+        }
+      }
+    }
+    int total;
+    int eq_before = block_exclusive_scan_1024(__popc(word_eq), s_warp, &total) + eq_carry;
+    eq_carry += total;
+    uint32_t word = word_gt;
+    int take = static_cast<int>(need) - eq_before;
+    for (uint32_t rem = word_eq; rem && take > 0; rem &= rem - 1, --take) word |= rem & (0u - rem);
+    int prot_before = block_exclusive_scan_1024(__popc(word), s_warp, &total) + prot_carry;
+    prot_carry += total;
+    if (w < W) {
+      e_words[w] = word;
+      e_prefix[w] = static_cast<uint32_t>(prot_before);
+      int pk = prot_before;
+      for (int i = 0; i < 32; ++i) {
+        const int64_t t = w * 32 + i;
+        if (word & (1u << i)) { if (idx_prot && pk < stride_prot) idx_prot[b * stride_prot + pk] = static_cast<int32_t>(t); ++pk; }
+        else if (idx_rest) idx_rest[b * stride_rest + (t - pk)] = static_cast<int32_t>(t);
+      }
+    }
+  }
+  if (threadIdx.x == 0) {
+    e_prefix[W] = static_cast<uint32_t>(prot_carry);
+    e_words[W] = 0;
+    if (counts) counts[b] = prot_carry;
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// Host launchers
+// ---------------------------------------------------------------------------------
+template <typename T>
+static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheView& cv, int layer, const SelView& sel,
+                                     float gamma, cudaStream_t stream) {
+  const int n_slabs = cv.B * cv.H_kv;
+  const int64_t n_rest = T_q - sel.n_prot;
+  if (n_rest > 0) {
+    const int64_t sgs = (n_rest + kSGTokens - 1) / kSGTokens;
+    v_ternary_kernel<T><<<dim3(static_cast<unsigned>(sgs), n_slabs), 256, 0, stream>>>(src, n_rest, cv, layer, sel, gamma);
+  }
+  if (sel.n_prot > 0) {
+    const int64_t pgs = (sel.n_prot + kG - 1) / kG;
+    v_protect_kernel<T><<<dim3(static_cast<unsigned>(pgs), n_slabs), 128, 0, stream>>>(src, cv, layer, sel);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer,
+                                   const SelView& sel, float gamma, cudaStream_t stream) {
+  if (dtype == VIDKV_F16) return quantize_values_t<__half>(src, T_q, cv, layer, sel, gamma, stream);
+  return quantize_values_t<__nv_bfloat16>(src, T_q, cv, layer, sel, gamma, stream);
+}
+
+cudaError_t launch_flush_values(int dtype, const KSrc& src, const CacheView& cv, int layer0, int n_layers,
+                                int64_t tgroup0, float gamma, cudaStream_t stream) {
+  const int spl = cv.B * cv.H_kv;
+  if (dtype == VIDKV_F16)
+    v_flush_kernel<__half><<<spl * n_layers, kD, 0, stream>>>(src, cv, layer0, spl, tgroup0, gamma);
+  else
+    v_flush_kernel<__nv_bfloat16><<<spl * n_layers, kD, 0, stream>>>(src, cv, layer0, spl, tgroup0, gamma);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_copy_to_residual(int dtype, const KSrc& src, int64_t t_begin, int n_tok, const CacheView& cv,
+                                    int layer, bool is_value, int r0, cudaStream_t stream) {
+  if (n_tok <= 0) return cudaSuccess;
+  const int64_t off = is_value ? cv.vres_offset : cv.kres_offset;
+  // 16-bit elements either way: the copy is type-agnostic
+  (void)dtype;
+  copy_to_residual_kernel<__half><<<cv.B * cv.H_kv, 256, 0, stream>>>(src, t_begin, n_tok, cv, layer, off, r0);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append(int dtype, const void* k_new, const void* v_new, const CacheView& cv, int layer0,
+                          int n_layers, int row, cudaStream_t stream) {
+  (void)dtype;
+  const int spl = cv.B * cv.H_kv;
+  append_kernel<<<spl * n_layers, 32, 0, stream>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
+                                                   cv, layer0, spl, row);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select_tokens(const float* saliency, int64_t vis_begin, int64_t l_v, int64_t n_prot, int64_t T_q,
+                                 const CacheView& cv, int32_t* idx_prot, int32_t* idx_rest, int64_t stride_prot,
+                                 int64_t stride_rest, cudaStream_t stream) {
+  select_tokens_kernel<<<cv.B, 1024, 0, stream>>>(saliency, nullptr, 0, vis_begin, l_v, n_prot, T_q, cv, idx_prot,
+                                                  idx_rest, stride_prot, stride_rest, nullptr);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_mask_to_selection(const uint8_t* E, int64_t T, int64_t T_q, const CacheView& cv, int32_t* idx_prot,
+                                     int32_t* idx_rest, int64_t stride_prot, int64_t stride_rest, int32_t* counts,
+                                     cudaStream_t stream) {
+  select_tokens_kernel<<<cv.B, 1024, 0, stream>>>(nullptr, E, T, 0, 0, 0, T_q, cv, idx_prot, idx_rest, stride_prot,
+                                                  stride_rest, counts);
+  return cudaGetLastError();
+}
+
+}  // namespace vidkv

@@ -1,0 +1,267 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on seeded inputs that span several tiles and a ragged tail."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import vidkv_oracle as O
+from tests import unpack as U
+from tests.helpers import (Pair, TOL_ABS, check_stats, compare_key_chunk, compare_ternary, f16_ulp_distance,
+                           new_stats, to_np)
+from workloads import CONFIGS
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare_prefill(pair: Pair):
+    cache = pair.cache_bytes()
+    stats = new_stats()
+    Tq = pair.T - pair.T % 32
+    r = pair.T % 32
+    for (layer, b, h), sc in pair.slabs.items():
+        slab = U.slab_bytes(cache, pair.lay, pair.cfg, layer, b, h)
+        k = to_np(pair.K[layer][b, h])
+        v = to_np(pair.V[layer][b, h])
+        if Tq:
+            compare_key_chunk(slab, pair.lay, 0, 0, sc.k_chunks[0], k[:Tq], stats)
+        sq = sc.v_prefill
+        n_rest = len(sq["rest_idx"])
+        if n_rest:
+            ng = (n_rest + 31) // 32
+            trits, s = U.ternary_groups(slab, pair.lay, 0, ng)
+            compare_ternary(trits, s, sq["trits"], sq["st"], v[sq["rest_idx"]], stats)
+        n_prot = len(sq["prot_idx"])
+        if n_prot:
+            E, prefix = U.selection_mask(cache, pair.lay, b, Tq)
+            assert (np.nonzero(E)[0] == sq["prot_idx"]).all(), "protected token set differs"
+            assert prefix[Tq // 32] == n_prot
+            npg = (n_prot + 31) // 32
+            codes, s, z = U.protected_groups(slab, pair.lay, npg)
+            assert (codes[:n_prot] == sq["codes2"]).all()
+            assert (s.view(np.int16) == sq["s2"].view(np.int16)).all()
+            assert (z.view(np.int16) == sq["z2"].view(np.int16)).all()
+        if r:
+            assert (U.residual(slab, pair.lay, "k", r, pair.wl.torch_dtype) == k[Tq:]).all()
+            assert (U.residual(slab, pair.lay, "v", r, pair.wl.torch_dtype) == v[Tq:]).all()
+    check_stats(stats)
+    return stats
+
+
+def _scale_tol(sc_values):
+    """2e-3 absolute, or one binary16 step of the largest scale in play where that is larger."""
+    return max(TOL_ABS, float(np.max(np.abs(sc_values))) * 2.0 ** -10 * 1.01)
+
+
+def _compare_dequant(pair: Pair):
+    for layer in range(pair.L):
+        Kd = pair.cache.dequantize_keys(layer).cpu().numpy().astype(np.float64)
+        Vd = pair.cache.dequantize_values(layer).cpu().numpy().astype(np.float64)
+        for b in range(pair.B):
+            for h in range(pair.cfg.H_kv):
+                sc = pair.slabs[(layer, b, h)]
+                ok, ov = sc.dequant_k(), sc.dequant_v()
+                assert Kd[b, h].shape == ok.shape and Vd[b, h].shape == ov.shape
+                s1max = max([float(c["s1"].astype(np.float64).max()) for c in sc.k_chunks] + [0.0])
+                assert np.abs(Kd[b, h] - ok).max() <= _scale_tol([s1max])
+                stmax = float(sc.v_prefill["st"].astype(np.float64).max()) if sc.v_prefill["st"].size else 0.0
+                for (_, s) in sc.v_flush:
+                    stmax = max(stmax, float(s.astype(np.float64).max()))
+                assert np.abs(Vd[b, h] - ov).max() <= _scale_tol([stmax])
+
+
+@pytest.mark.parametrize("name,T,B,p", [
+    ("tiny", 1632, 1, 0.0),        # the named config: 51 groups, 10.2 supergroups, 12.75 encode tiles
+    ("tiny", 1632, 1, 0.2),        # with semantic token protection (313 protected tokens)
+    ("tiny", 77, 2, 0.0),          # ragged: 64 quantized tokens + 13 residual tokens
+    ("tiny", 31, 1, 0.0),          # nothing quantized, everything in the residual
+    ("llava", 352, 1, 0.2),        # heavy-tailed values, +-5 outlier offsets
+    ("qwen", 480, 2, 0.2),         # bf16 inputs, rotary-structured keys
+])
+def test_prefill_codes_and_dequant(name, T, B, p):
+    pair = Pair(CONFIGS[name], T, B=B, L=1, p=p).prefill()
+    _compare_prefill(pair)
+    _compare_dequant(pair)
+    assert pair.cache.status() == 0
+
+
+def test_prefill_is_deterministic_and_leaves_other_regions_alone():
+    a = Pair(CONFIGS["tiny"], 1632, L=1, p=0.2).prefill()
+    b = Pair(CONFIGS["tiny"], 1632, L=1, p=0.2).prefill()
+    ca, cb = a.cache_bytes(), b.cache_bytes()
+    assert (ca == cb).all()
+    # header magic and a clean status word
+    assert ca[:4].view("<u4")[0] == 0x564B4456 and ca[8:12].view("<i4")[0] == 0
+
+
+def _decode_steps(pair: Pair, n_steps, tol=TOL_ABS):
+    worst = 0.0
+    for _ in range(n_steps):
+        out, ref = pair.decode()
+        err = np.abs(out - ref).max()
+        worst = max(worst, err)
+        assert err <= tol, f"step {pair.step - 1}: max abs error {err}"
+    return worst
+
+
+@pytest.mark.parametrize("name,T,B,p,steps", [
+    ("tiny", 1632, 1, 0.0, 16),    # the named config
+    ("tiny", 1632, 1, 0.2, 16),
+    ("tiny", 77, 2, 0.0, 5),
+    ("tiny", 31, 1, 0.0, 3),
+    ("qwen", 480, 2, 0.2, 4),
+])
+def test_decode_attention_parity(name, T, B, p, steps):
+    pair = Pair(CONFIGS[name], T, B=B, L=1, p=p, max_new=steps).prefill()
+    _decode_steps(pair, steps)
+    assert pair.cache.status() == 0
+
+
+def test_decode_parity_heavy_tailed():
+    # Student-t inputs: outputs are large, so the tolerance scales with their magnitude
+    pair = Pair(CONFIGS["llava"], 352, B=1, L=2, p=0.2, max_new=4).prefill()
+    for _ in range(4):
+        out, ref = pair.decode()
+        assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
+
+
+def test_residual_flush_parity():
+    # 64 quantized + 5 residual tokens; the residual fills at step 123 and is flushed
+    wl = CONFIGS["tiny"]
+    pair = Pair(wl, 69, B=1, L=2, p=0.0, max_new=140).prefill()
+    _decode_steps(pair, 123)
+    st = pair.cache.layer_state(0)
+    assert st == dict(n_quantized=192, n_residual=0, n_chunks=2, n_protected=0)
+    cache = pair.cache_bytes()
+    stats = new_stats()
+    for (layer, b, h), sc in pair.slabs.items():
+        assert len(sc.k_chunks) == 2 and sc.k_res.shape[0] == 0
+        slab = U.slab_bytes(cache, pair.lay, pair.cfg, layer, b, h)
+        kin, vin = pair.flushed_in[(layer, b, h)]
+        compare_key_chunk(slab, pair.lay, 1, 2, sc.k_chunks[1], kin, stats)
+        trits, s = U.ternary_groups(slab, pair.lay, 2, 4)
+        o_t, o_s = sc.v_flush[0]
+        compare_ternary(trits, s, o_t, o_s, vin, stats)
+    check_stats(stats)
+    _compare_dequant(pair)
+    _decode_steps(pair, 10)          # attention over two chunks + a fresh residual
+    assert pair.cache.layer_state(1)["n_residual"] == 10
+
+
+def test_flush_with_protected_tokens_keeps_streams_apart():
+    wl = CONFIGS["tiny"]
+    pair = Pair(wl, 256, B=1, L=1, p=0.2, max_new=135).prefill()     # 51 protected, 205 ternary (6.4 groups)
+    _decode_steps(pair, 130)
+    assert pair.cache.layer_state(0) == dict(n_quantized=384, n_residual=2, n_chunks=2, n_protected=51)
+    _compare_dequant(pair)
+
+
+def test_multi_layer_call_equals_per_layer_calls():
+    wl = CONFIGS["tiny"]
+    a = Pair(wl, 320, B=2, L=3, p=0.0, max_new=2).prefill()
+    out_all, ref = a.decode()
+    assert np.abs(out_all - ref).max() <= TOL_ABS
+    b = Pair(wl, 320, B=2, L=3, p=0.0, max_new=2).prefill()
+    from workloads import make_step_inputs
+    for layer in range(3):
+        q, k, v = make_step_inputs(wl, layer, 0, "cpu", T=320, B=2)
+        out = torch.empty((1, 2, 28, 128), dtype=torch.float32, device="cuda")
+        b.cache.decode_attention(layer, 1, q[None].cuda(), k[None].cuda(), v[None].cuda(), out)
+        assert np.array_equal(out.cpu().numpy()[0].astype(np.float64), out_all[layer])
+
+
+def test_output_dtypes():
+    import paper_2503_16257_b200 as P
+    wl = CONFIGS["tiny"]
+    from workloads import make_layer_kv, make_step_inputs
+    K, V = make_layer_kv(wl, 0, "cpu", T=160)
+    q, k, v = make_step_inputs(wl, 0, 0, "cpu", T=160)
+    outs = {}
+    for od, tdt in [(P.VIDKV_F32, torch.float32), (P.VIDKV_F16, torch.float16), (P.VIDKV_BF16, torch.bfloat16)]:
+        cfg = P.VidKVConfig(B=1, L=1, max_prefill_tokens=160, max_new_tokens=1, out_dtype=od)
+        c = P.VidKVCache(cfg)
+        c.quantize_keys(0, K.cuda()); c.quantize_values(0, V.cuda())
+        out = torch.empty((1, 1, 28, 128), dtype=tdt, device="cuda")
+        c.decode_attention(0, 1, q[None].cuda(), k[None].cuda(), v[None].cuda(), out)
+        outs[od] = out.float().cpu()
+    assert torch.equal(outs[P.VIDKV_F32].half().float(), outs[P.VIDKV_F16])
+    assert torch.equal(outs[P.VIDKV_F32].bfloat16().float(), outs[P.VIDKV_BF16])
+
+
+def test_call_order_and_capacity_errors():
+    import paper_2503_16257_b200 as P
+    wl = CONFIGS["tiny"]
+    from workloads import make_layer_kv, make_step_inputs
+    K, V = make_layer_kv(wl, 0, "cpu", T=96)
+    q, k, v = make_step_inputs(wl, 0, 0, "cpu", T=96)
+    cfg = P.VidKVConfig(B=1, L=1, max_prefill_tokens=96, max_new_tokens=1, p_ratio=0.2)
+    c = P.VidKVCache(cfg)
+    out = torch.empty((1, 1, 28, 128), dtype=torch.float32, device="cuda")
+    args = (0, 1, q[None].cuda(), k[None].cuda(), v[None].cuda(), out)
+    with pytest.raises(P.VidKVError) as e:
+        c.decode_attention(*args)                       # nothing quantized yet
+    assert e.value.status == -5
+    c.quantize_keys(0, K.cuda())
+    with pytest.raises(P.VidKVError) as e:
+        c.quantize_keys(0, K.cuda())                    # twice
+    assert e.value.status == -5
+    with pytest.raises(P.VidKVError) as e:
+        c.quantize_values(0, V.cuda())                  # p > 0 but no token selection yet
+    assert e.value.status == -5
+    c.select_tokens(None, 0, 0, 96)
+    with pytest.raises(P.VidKVError) as e:
+        c.quantize_values(0, V[:, :, :64].contiguous().cuda())     # T differs from the keys'
+    assert e.value.status == -5
+    big = torch.zeros((1, 4, 128, 128), dtype=torch.float16, device="cuda")
+    c2 = P.VidKVCache(cfg)
+    with pytest.raises(P.VidKVError) as e:
+        c2.quantize_keys(0, big)                        # more tokens than the cache was sized for
+    assert e.value.status == -4
+    with pytest.raises(P.VidKVError) as e:
+        c2.quantize_keys(0, K.cuda()[:, :, :, 1:])      # misaligned view
+    assert e.value.status in (-3, -1)
+    c.quantize_values(0, V.cuda())
+    c.decode_attention(*args)
+    with pytest.raises(P.VidKVError) as e:
+        c.decode_attention(*args)                       # max_new_tokens = 1
+    assert e.value.status == -4
+    assert c.status() == 0
+
+
+def test_token_mask_entry_point_matches_saliency_selection():
+    import paper_2503_16257_b200 as P
+    from workloads import make_layer_kv, make_saliency
+    wl = CONFIGS["tiny"]
+    T = 320
+    K, V = make_layer_kv(wl, 0, "cpu", T=T, B=2)
+    sal = make_saliency(wl, "cpu", l_v=256, B=2)
+    cfg = P.VidKVConfig(B=2, L=1, max_prefill_tokens=T, max_new_tokens=1, p_ratio=0.2)
+    a = P.VidKVCache(cfg)
+    a.select_tokens(sal.cuda(), 32, 256, T)
+    a.quantize_values(0, V.cuda())
+    E = np.stack([O.select_tokens(sal[b].numpy(), 0.2, 32, T) for b in range(2)]).astype(np.uint8)
+    b = P.VidKVCache(cfg)
+    b.set_token_mask(torch.from_numpy(E).cuda(), T)
+    b.quantize_values(0, V.cuda())
+    torch.cuda.synchronize()
+    assert torch.equal(a.cache, b.cache)
+    assert a.layer_state(0)["n_protected"] == 51
+    # a mask whose rows protect different numbers of tokens is rejected
+    E[1, 40] ^= 1
+    c = P.VidKVCache(cfg)
+    with pytest.raises(P.VidKVError):
+        c.set_token_mask(torch.from_numpy(E).cuda(), T)
+
+
+def test_saliency_ties_take_lower_index():
+    import paper_2503_16257_b200 as P
+    T = 64
+    sal = torch.zeros((1, 64), dtype=torch.float32)
+    sal[0, 10] = 2.0
+    sal[0, 20:30] = 1.0                 # ten-way tie for the remaining 11 places of n = 12
+    cfg = P.VidKVConfig(B=1, L=1, max_prefill_tokens=T, max_new_tokens=1, p_ratio=0.1875)
+    c = P.VidKVCache(cfg)
+    c.select_tokens(sal.cuda(), 0, 64, T)
+    torch.cuda.synchronize()
+    E, _ = U.selection_mask(c.cache.cpu().numpy(), c.layout, 0, T)
+    ref = O.select_tokens(sal[0].numpy(), 0.1875, 0, T)
+    assert (E == ref).all() and E.sum() == 12 and E[0] and not E[2]

@@ -1,0 +1,117 @@
+"""CPU-side checks of libvidkv.so: it loads, exports every function the header declares,
+and its host-only entry points (sizing, layout, argument validation) behave."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2503_16257_b200 as P
+from paper_2503_16257_b200 import build as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    B.build()
+    return P.load_library()
+
+
+def _header_functions():
+    text = open(os.path.join(ROOT, "include", "vidkv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(vidkv_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _header_functions()
+    assert len(names) >= 14
+    raw = ctypes.CDLL(P.library_path())
+    for n in names:
+        assert hasattr(raw, n), f"{n} declared in include/vidkv.h but not exported"
+    assert set(names) == set(P.exported_symbols())
+
+
+def test_version(lib):
+    assert P.vidkv_version() >= 100
+
+
+def test_bytes_per_token_accounting(lib):
+    # one 32-token key group: 64 ch x 2 bit + 64 ch x 1 bit + (s, z, s) binary16 x 64
+    assert 32 * (64 * 2 + 64 * 1) // 8 + 3 * 64 * 2 == 1152          # 36 B / token / head -> 1.5 bit + metadata
+    assert (64 * 2 + 64 * 1) / 128 == 1.5
+    # one ternary supergroup: 160 tokens x 128 ch x 1.6 bit + 5 x 128 binary16 scales
+    assert 160 * 128 // 5 + 5 * 128 * 2 == 5376                      # 33.6 B / token / head
+    assert 8 / 5 == 1.6 and 3 ** 5 <= 256
+    # one protected group: 32 tokens x 128 ch x 2 bit + (s, z) binary16 x 128
+    assert 32 * 128 * 2 // 8 + 2 * 128 * 2 == 1536                   # 48 B / token / head
+    cfg = P.VidKVConfig(B=4, L=28, max_prefill_tokens=196000, max_new_tokens=64)
+    lay = P.vidkv_cache_layout(cfg)
+    assert lay["max_kgroups"] == 6125 and lay["max_chunks"] == 1
+    packed = lay["max_kgroups"] * 1152 + lay["max_supergroups"] * 5376
+    fp16 = 196000 * 128 * 2 * 2
+    assert 0.13 < packed / fp16 < 0.14                               # ~86 % smaller than FP16 K+V
+    cache_bytes, ws_bytes = P.vidkv_cache_bytes(cfg)
+    assert cache_bytes == lay["total_bytes"] and cache_bytes < 0.15 * fp16 * 4 * 4 * 28
+    assert ws_bytes > 0
+
+
+def test_layout_regions_do_not_overlap(lib):
+    for p in (0.0, 0.2):
+        cfg = P.VidKVConfig(B=2, L=3, max_prefill_tokens=1000, max_new_tokens=300, p_ratio=p)
+        lay = P.vidkv_cache_layout(cfg)
+        regions = [
+            (lay["chunk_table_offset"], lay["max_chunks"] * 128),
+            (lay["kgroup_offset"], lay["max_kgroups"] * 1152),
+            (lay["tern_offset"], lay["max_supergroups"] * 5376),
+            (lay["prot_offset"], lay["max_pgroups"] * 1536),
+            (lay["kres_offset"], 128 * 128 * 2),
+            (lay["vres_offset"], 128 * 128 * 2),
+        ]
+        end = 0
+        for off, size in regions:
+            assert off >= end and off % 128 == 0
+            end = off + size
+        assert end <= lay["slab_stride"] and lay["slab_stride"] % 256 == 0
+        assert lay["slab_offset"] >= lay["sel_offset"] + 2 * lay["sel_stride_b"]
+        assert lay["total_bytes"] == lay["slab_offset"] + lay["slab_stride"] * 3 * 2 * 4
+        # 1000 prefill tokens -> 31 groups; (31 + 300) // 128 = 2 flushes possible
+        assert lay["max_chunks"] == 3 and lay["max_kgroups"] == 31 + 8
+        assert lay["max_pgroups"] == (0 if p == 0 else (200 + 31) // 32)
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(D=64), -2), (dict(G=64), -2), (dict(R=64), -2), (dict(k_ratio=0.75), -2),
+    (dict(H_q=30), -2), (dict(H_q=64), -2), (dict(key_1bit_mode=1), -2),
+    (dict(B=0), -1), (dict(p_ratio=1.5), -1), (dict(p_ratio=-0.1), -1), (dict(in_dtype=2), -1),
+    (dict(out_dtype=7), -1), (dict(max_new_tokens=-1), -1), (dict(gamma=float("nan")), -1),
+])
+def test_config_validation(lib, kw, status):
+    base = dict(B=1, L=1, max_prefill_tokens=64, max_new_tokens=4)
+    base.update(kw)
+    with pytest.raises(P.VidKVError) as e:
+        P.vidkv_cache_bytes(P.VidKVConfig(**base))
+    assert e.value.status == status
+
+
+def test_null_arguments_are_rejected_without_a_device(lib):
+    cfg = P.VidKVConfig(B=1, L=1, max_prefill_tokens=64, max_new_tokens=4).to_c()
+    assert lib.vidkv_cache_bytes(ctypes.byref(cfg), None, None) == -1
+    assert lib.vidkv_cache_layout(None, None) == -1
+    h = ctypes.c_void_p()
+    assert lib.vidkv_cache_init(ctypes.byref(cfg), None, 0, None, 0, None, ctypes.byref(h)) == -1
+    assert lib.vidkv_cache_init(ctypes.byref(cfg), ctypes.c_void_p(0x1001), 1 << 30, ctypes.c_void_p(0x1000), 1 << 30,
+                                None, ctypes.byref(h)) == -3
+    assert lib.vidkv_cache_init(ctypes.byref(cfg), ctypes.c_void_p(0x1000), 16, ctypes.c_void_p(0x1000), 16,
+                                None, ctypes.byref(h)) == -4
+    assert lib.vidkv_cache_destroy(None) == -1
+    assert lib.vidkv_decode_attention(None, 0, 1, None, None, None, None, 0.0, None) == -1
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    import paper_2503_16257_b200.api as api
+    monkeypatch.setattr(api, "_LIB", None)
+    monkeypatch.setattr(api, "library_path", lambda: "/nonexistent/libvidkv.so")
+    with pytest.raises(RuntimeError):
+        api.load_library()

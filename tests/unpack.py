@@ -1,0 +1,88 @@
+"""Test-side reader of the packed cache format documented in include/vidkv.h.
+
+Written from the format description only: it turns the bytes of one slab back into
+plain integer codes and binary16 metadata so that they can be compared with the
+oracle's unpacked codes.  It contains no quantizer arithmetic."""
+from __future__ import annotations
+
+import numpy as np
+
+G, R, D = 32, 128, 128
+KG_BYTES, SG_BYTES, PG_BYTES, CHUNK_BYTES = 1152, 5376, 1536, 128
+
+
+def slab_bytes(cache: np.ndarray, lay: dict, cfg, layer: int, b: int, h: int) -> np.ndarray:
+    idx = (layer * cfg.B + b) * cfg.H_kv + h
+    off = lay["slab_offset"] + idx * lay["slab_stride"]
+    return cache[off: off + lay["slab_stride"]]
+
+
+def chunk_perm(slab: np.ndarray, lay: dict, chunk: int):
+    e = slab[lay["chunk_table_offset"] + chunk * CHUNK_BYTES:][:CHUNK_BYTES]
+    return e[:64].astype(np.int64), e[64:].astype(np.int64)
+
+
+def key_groups(slab: np.ndarray, lay: dict, g_begin: int, n_groups: int):
+    """-> codes2 [32*n, 64] int8, bits1 [32*n, 64] uint8, s2, z2, s1 [n, 64] float16."""
+    codes2 = np.zeros((n_groups * G, 64), np.int8)
+    bits1 = np.zeros((n_groups * G, 64), np.uint8)
+    s2 = np.zeros((n_groups, 64), np.float16)
+    z2 = np.zeros((n_groups, 64), np.float16)
+    s1 = np.zeros((n_groups, 64), np.float16)
+    sh2 = 2 * (np.arange(64) % 16)
+    for g in range(n_groups):
+        rec = slab[lay["kgroup_offset"] + (g_begin + g) * KG_BYTES:][:KG_BYTES]
+        w2 = rec[0:512].view("<u4").reshape(G, 4)
+        codes2[g * G:(g + 1) * G] = (w2[:, np.arange(64) // 16] >> sh2) & 3
+        w1 = rec[512:768].view("<u4").reshape(G, 2)
+        bits1[g * G:(g + 1) * G] = (w1[:, np.arange(64) // 32] >> (np.arange(64) % 32)) & 1
+        s2[g] = rec[768:896].view("<f2")
+        z2[g] = rec[896:1024].view("<f2")
+        s1[g] = rec[1024:1152].view("<f2")
+    return codes2, bits1, s2, z2, s1
+
+
+def ternary_groups(slab: np.ndarray, lay: dict, g_begin: int, n_groups: int):
+    """-> trits [32*n, 128] int8, s [n, 128] float16 for ternary stream groups g_begin.."""
+    trits = np.zeros((n_groups * G, D), np.int8)
+    s = np.zeros((n_groups, D), np.float16)
+    for k in range(n_groups):
+        gi = g_begin + k
+        rec = slab[lay["tern_offset"] + (gi // 5) * SG_BYTES:][:SG_BYTES]
+        slot = gi % 5
+        q = rec[:4096].astype(np.int64).reshape(G, D)
+        bval = (q * 243) >> 8
+        digit = (bval // 3 ** (4 - slot)) % 3
+        trits[k * G:(k + 1) * G] = digit - 1
+        s[k] = rec[4096 + slot * 256: 4096 + (slot + 1) * 256].view("<f2")
+    return trits, s
+
+
+def protected_groups(slab: np.ndarray, lay: dict, n_groups: int):
+    codes = np.zeros((n_groups * G, D), np.int8)
+    s = np.zeros((n_groups, D), np.float16)
+    z = np.zeros((n_groups, D), np.float16)
+    sh = 2 * (np.arange(D) % 16)
+    for g in range(n_groups):
+        rec = slab[lay["prot_offset"] + g * PG_BYTES:][:PG_BYTES]
+        w = rec[:1024].view("<u4").reshape(G, 8)
+        codes[g * G:(g + 1) * G] = (w[:, np.arange(D) // 16] >> sh) & 3
+        s[g] = rec[1024:1280].view("<f2")
+        z[g] = rec[1280:1536].view("<f2")
+    return codes, s, z
+
+
+def residual(slab: np.ndarray, lay: dict, which: str, n: int, torch_dtype):
+    import torch
+    off = lay["kres_offset"] if which == "k" else lay["vres_offset"]
+    raw = slab[off: off + n * D * 2].copy()
+    return torch.from_numpy(raw).view(torch_dtype).reshape(n, D).float().numpy()
+
+
+def selection_mask(cache: np.ndarray, lay: dict, b: int, T_q: int):
+    off = lay["sel_offset"] + b * lay["sel_stride_b"]
+    words = cache[off: off + 4 * lay["sel_words"]].view("<u4")
+    prefix = cache[off + 4 * lay["sel_words"]: off + 8 * lay["sel_words"]].view("<u4")
+    t = np.arange(T_q)
+    E = ((words[t // 32] >> (t % 32)) & 1).astype(bool)
+    return E, prefix
