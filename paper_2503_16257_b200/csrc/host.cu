@@ -395,18 +395,22 @@ vidkv_status_t vidkv_cache_status(vidkv_cache_t* h, void* stream) {
 }
 
 vidkv_status_t vidkv_dequantize_keys(vidkv_cache_t* h, int32_t layer, float* out, void* stream) {
-  if (!h || !out || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  if (!h || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
   const LayerInfo& li = h->layers[layer];
   if (!li.k_done) return VIDKV_ERR_STATE;
+  if (li.T_q0 + li.n_flush * kR == 0) return VIDKV_OK;
+  if (!out) return VIDKV_ERR_INVALID_ARG;
   if (launch_dequant_keys(h->cv, layer, li.T_q0, li.n_flush, out, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return VIDKV_ERR_CUDA;
   return VIDKV_OK;
 }
 
 vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* h, int32_t layer, float* out, void* stream) {
-  if (!h || !out || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  if (!h || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
   const LayerInfo& li = h->layers[layer];
   if (!li.v_done) return VIDKV_ERR_STATE;
+  if (li.T_q0 + li.n_flush * kR == 0) return VIDKV_OK;
+  if (!out) return VIDKV_ERR_INVALID_ARG;
   if (launch_dequant_values(h->cv, layer, li.T_q0, li.n_flush, h->n_prot, out, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return VIDKV_ERR_CUDA;
   return VIDKV_OK;
