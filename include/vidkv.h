@@ -204,6 +204,14 @@ vidkv_status_t vidkv_cache_status(vidkv_cache_t* handle, void* stream);
 vidkv_status_t vidkv_dequantize_keys(vidkv_cache_t* handle, int32_t layer, float* out, void* stream);
 vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* handle, int32_t layer, float* out, void* stream);
 
+/* Profiling aid: record the two CUDA events (cudaEvent_t passed as void*) immediately before
+ * and after the split-KV attention kernel of every later vidkv_decode_attention call on this
+ * handle; NULL, NULL switches it off.  The events are the caller's. */
+vidkv_status_t vidkv_set_profile_events(vidkv_cache_t* handle, void* ev_begin, void* ev_end);
+
+/* Number of CUDA kernels this library has launched in this process (host counter). */
+uint64_t vidkv_launch_count(void);
+
 /* Library version: major * 10000 + minor * 100 + patch. */
 int32_t vidkv_version(void);
 

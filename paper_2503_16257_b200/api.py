@@ -61,6 +61,8 @@ class VidKVConfig:
 
 _SIGNATURES = {
     "vidkv_version": (C.c_int32, []),
+    "vidkv_launch_count": (C.c_uint64, []),
+    "vidkv_set_profile_events": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "vidkv_cache_bytes": (C.c_int32, [C.POINTER(_Config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "vidkv_cache_layout": (C.c_int32, [C.POINTER(_Config), C.POINTER(_Layout)]),
     "vidkv_cache_init": (C.c_int32, [C.POINTER(_Config), C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t,
@@ -115,6 +117,10 @@ def _check(fn: str, status: int):
 
 def vidkv_version() -> int:
     return load_library().vidkv_version()
+
+
+def vidkv_launch_count() -> int:
+    return load_library().vidkv_launch_count()
 
 
 def vidkv_cache_bytes(cfg: VidKVConfig):
@@ -208,6 +214,12 @@ class VidKVCache:
         _check("vidkv_layer_state", self.lib.vidkv_layer_state(self.handle, layer, C.byref(a), C.byref(b),
                                                               C.byref(c), C.byref(d)))
         return dict(n_quantized=a.value, n_residual=b.value, n_chunks=c.value, n_protected=d.value)
+
+    def set_profile_events(self, ev_begin=None, ev_end=None):
+        """torch.cuda.Event pair (created with enable_timing=True and recorded once) or None."""
+        a = C.c_void_p(ev_begin.cuda_event) if ev_begin is not None else C.c_void_p(0)
+        b = C.c_void_p(ev_end.cuda_event) if ev_end is not None else C.c_void_p(0)
+        _check("vidkv_set_profile_events", self.lib.vidkv_set_profile_events(self.handle, a, b))
 
     def status(self) -> int:
         return self.lib.vidkv_cache_status(self.handle, _stream_ptr())

@@ -346,8 +346,11 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
     attr_smem = smem;
   }
   const dim3 grid(a.n_splits, n_slabs);
+  if (a.ev_begin) cudaEventRecord(a.ev_begin, stream);
   if (a.in_dtype == VIDKV_F16) decode_split_kernel<__half><<<grid, 256, smem, stream>>>(a);
   else decode_split_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(a);
+  if (a.ev_end) cudaEventRecord(a.ev_end, stream);
+  count_launches(2);
   decode_merge_kernel<<<a.n_layers * a.cv.B * a.cv.H_q, kD, 0, stream>>>(a.partials, a.n_splits, a.out, a.out_dtype);
   return cudaGetLastError();
 }

@@ -100,6 +100,7 @@ cudaError_t launch_dequant_keys(const CacheView& cv, int layer, int64_t T_q0, in
   const int64_t T_qt = T_q0 + n_flush * kR;
   if (T_qt == 0) return cudaSuccess;
   dequant_keys_kernel<<<dim3(static_cast<unsigned>(T_qt / kG), cv.B * cv.H_kv), 128, 0, stream>>>(cv, layer, T_q0, T_qt, out);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -109,6 +110,7 @@ cudaError_t launch_dequant_values(const CacheView& cv, int layer, int64_t T_q0, 
   if (T_qt == 0) return cudaSuccess;
   dequant_values_kernel<<<dim3(static_cast<unsigned>(T_qt / kG), cv.B * cv.H_kv), 128, 0, stream>>>(cv, layer, T_q0, T_qt,
                                                                                                      n_prot, out);
+  count_launches(1);
   return cudaGetLastError();
 }
 

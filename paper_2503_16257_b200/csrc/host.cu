@@ -117,7 +117,10 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 }  // namespace
 
+namespace vidkv { unsigned long long g_launch_count = 0; }
+
 struct vidkv_cache {
+  cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
   vidkv_config_t cfg;
   Layout L;
   WsPlan ws;
@@ -132,6 +135,15 @@ struct vidkv_cache {
 extern "C" {
 
 int32_t vidkv_version(void) { return 100; }
+
+uint64_t vidkv_launch_count(void) { return g_launch_count; }
+
+vidkv_status_t vidkv_set_profile_events(vidkv_cache_t* h, void* ev_begin, void* ev_end) {
+  if (!h || ((ev_begin == nullptr) != (ev_end == nullptr))) return VIDKV_ERR_INVALID_ARG;
+  h->ev_begin = static_cast<cudaEvent_t>(ev_begin);
+  h->ev_end = static_cast<cudaEvent_t>(ev_end);
+  return VIDKV_OK;
+}
 
 vidkv_status_t vidkv_cache_layout(const vidkv_config_t* cfg, vidkv_layout_t* layout) {
   if (!layout) return VIDKV_ERR_INVALID_ARG;
@@ -341,6 +353,7 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   a.in_dtype = dt; a.out_dtype = h->cfg.out_dtype;
   a.n_prot = h->n_prot;
   a.scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / std::sqrt(static_cast<float>(kD));
+  a.ev_begin = h->ev_begin; a.ev_end = h->ev_end;
   a.st.T_q0 = first.T_q0; a.st.n_flush = first.n_flush; a.st.n_res = first.n_res + 1;
   const int64_t T_tot = first.T_q0 + first.n_flush * kR + a.st.n_res;
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv;

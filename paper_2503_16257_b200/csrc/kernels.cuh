@@ -74,7 +74,12 @@ struct DecodeArgs {
   int64_t n_prot;      // protected tokens per batch element (0 = no STP)
   float scale;
   LayerState st;
+  cudaEvent_t ev_begin, ev_end;   // optional: recorded around the split-KV kernel (profiling)
 };
+
+// Number of kernels launched by this library since it was loaded (host counter).
+extern unsigned long long g_launch_count;
+inline void count_launches(int n) { g_launch_count += static_cast<unsigned long long>(n); }
 
 // Split-KV attention over the packed cache + residual, then the merge of the partials.
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);

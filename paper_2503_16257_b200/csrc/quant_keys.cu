@@ -311,6 +311,7 @@ static cudaError_t launch_keys_t(const KSrc& src, int64_t T_tokens, const CacheV
   const int64_t blocks = (T_tokens + kEncTokens - 1) / kEncTokens;
   k_encode_kernel<T><<<dim3(static_cast<unsigned>(blocks), n_slabs), 256, smem, stream>>>(
       src, T_tokens, cv, layer0, slabs_per_layer, chunk, kgroup0);
+  count_launches(4);
   return cudaGetLastError();
 }
 

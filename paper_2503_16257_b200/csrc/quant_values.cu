@@ -315,10 +315,12 @@ static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheVi
   if (n_rest > 0) {
     const int64_t sgs = (n_rest + kSGTokens - 1) / kSGTokens;
     v_ternary_kernel<T><<<dim3(static_cast<unsigned>(sgs), n_slabs), 256, 0, stream>>>(src, n_rest, cv, layer, sel, gamma);
+    count_launches(1);
   }
   if (sel.n_prot > 0) {
     const int64_t pgs = (sel.n_prot + kG - 1) / kG;
     v_protect_kernel<T><<<dim3(static_cast<unsigned>(pgs), n_slabs), 128, 0, stream>>>(src, cv, layer, sel);
+    count_launches(1);
   }
   return cudaGetLastError();
 }
@@ -336,6 +338,7 @@ cudaError_t launch_flush_values(int dtype, const KSrc& src, const CacheView& cv,
     v_flush_kernel<__half><<<spl * n_layers, kD, 0, stream>>>(src, cv, layer0, spl, tgroup0, gamma);
   else
     v_flush_kernel<__nv_bfloat16><<<spl * n_layers, kD, 0, stream>>>(src, cv, layer0, spl, tgroup0, gamma);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -346,6 +349,7 @@ cudaError_t launch_copy_to_residual(int dtype, const KSrc& src, int64_t t_begin,
   // 16-bit elements either way: the copy is type-agnostic
   (void)dtype;
   copy_to_residual_kernel<__half><<<cv.B * cv.H_kv, 256, 0, stream>>>(src, t_begin, n_tok, cv, layer, off, r0);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -355,6 +359,7 @@ cudaError_t launch_append(int dtype, const void* k_new, const void* v_new, const
   const int spl = cv.B * cv.H_kv;
   append_kernel<<<spl * n_layers, 32, 0, stream>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
                                                    cv, layer0, spl, row);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -363,6 +368,7 @@ cudaError_t launch_select_tokens(const float* saliency, int64_t vis_begin, int64
                                  int64_t stride_rest, cudaStream_t stream) {
   select_tokens_kernel<<<cv.B, 1024, 0, stream>>>(saliency, nullptr, 0, vis_begin, l_v, n_prot, T_q, cv, idx_prot,
                                                   idx_rest, stride_prot, stride_rest, nullptr);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -371,6 +377,7 @@ cudaError_t launch_mask_to_selection(const uint8_t* E, int64_t T, int64_t T_q, c
                                      cudaStream_t stream) {
   select_tokens_kernel<<<cv.B, 1024, 0, stream>>>(nullptr, E, T, 0, 0, 0, T_q, cv, idx_prot, idx_rest, stride_prot,
                                                   stride_rest, counts);
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -13,6 +13,7 @@ Tokens are ordered visual first, then text.  Layout is ``[B, H, T, D]``.
 """
 from __future__ import annotations
 
+import functools
 from dataclasses import dataclass
 
 import torch
@@ -85,19 +86,29 @@ def _outlier_channels(cfg: WorkloadConfig, layer: int):
     return ids, sign
 
 
+@functools.lru_cache(maxsize=256)
+def _outlier_affine(cfg: WorkloadConfig, layer: int):
+    """Per-head channel-wise (scale, offset) [H_KV, D] that plants the outlier channels."""
+    ids, sign = _outlier_channels(cfg, layer)
+    scale = torch.ones((H_KV, D), dtype=torch.float32)
+    offset = torch.zeros((H_KV, D), dtype=torch.float32)
+    for h in range(H_KV):
+        for c, sg in zip(ids[h].tolist(), sign[h].tolist()):
+            scale[h, c] = 10.0
+            if cfg.outlier_sign == "plus":
+                offset[h, c] = 5.0
+            elif cfg.outlier_sign == "pm":
+                offset[h, c] = 5.0 * sg
+    return scale, offset
+
+
 def _plant_outliers(cfg: WorkloadConfig, layer: int, x: torch.Tensor, head_of_dim1):
     """x [B, n_heads, T_or_1, D]: scale/shift the planted channels of each head."""
-    ids, sign = _outlier_channels(cfg, layer)
-    for j, h in enumerate(head_of_dim1):
-        for c, sg in zip(ids[h].tolist(), sign[h].tolist()):
-            col = x[:, j, :, c]
-            if cfg.outlier_sign == "plus":
-                x[:, j, :, c] = col * 10.0 + 5.0
-            elif cfg.outlier_sign == "pm":
-                x[:, j, :, c] = col * 10.0 + 5.0 * sg
-            else:
-                x[:, j, :, c] = col * 10.0
-    return x
+    scale, offset = _outlier_affine(cfg, layer)
+    idx = torch.tensor(list(head_of_dim1), dtype=torch.long)
+    sc = scale[idx].to(x.device).view(1, len(idx), 1, D)
+    of = offset[idx].to(x.device).view(1, len(idx), 1, D)
+    return x.mul_(sc).add_(of)
 
 
 def _rope_params(cfg: WorkloadConfig, layer: int, device):
