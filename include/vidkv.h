@@ -204,6 +204,32 @@ vidkv_status_t vidkv_cache_status(vidkv_cache_t* handle, void* stream);
 vidkv_status_t vidkv_dequantize_keys(vidkv_cache_t* handle, int32_t layer, float* out, void* stream);
 vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* handle, int32_t layer, float* out, void* stream);
 
+/* For callers that cannot obtain device memory.  (The paper has no counterpart to this
+ * entry point; it exists for deployment reasons only.)  Some callers are handed their
+ * device tensors by a host framework and cannot allocate more where attention runs -- a
+ * plugin restricted to the buffers it was given, code running while the framework's memory
+ * pool is frozen, a runtime without cudaMalloc -- so they cannot supply the workspace that
+ * vidkv_cache_init wants.  This call needs no handle and no workspace: it computes
+ *   out [n_layers, B, H_q, D] (out_dtype) = Softmax(q K^T * softmax_scale) V
+ * for q [n_layers, B, H_q, D] (in_dtype) over the packed cache `cache` exactly as it stands
+ * (no append, no flush), the cache having been filled through a handle built on the same
+ * `cfg`.  The caller states the token counts that vidkv_layer_state reports for the layers:
+ * n_prefill_quantized (a multiple of G), n_flushed_chunks, n_residual (0..R) and n_protected.
+ * The split-KV partial results live in a 16 MiB array inside the library, which every GPU
+ * that loads the library keeps until the process exits; at most 32263 (query head, split)
+ * records fit, i.e. n_layers * B * H_q * ceil(tokens / split) <= 32263 with split = 160, 320
+ * or 640 tokens -- larger problems return VIDKV_ERR_CAPACITY (use fewer layers per call).
+ * Nothing is allocated or freed.  The first call on each device looks up the array's device
+ * address, so make that first call outside any stream capture.  All calls share the array:
+ * two calls whose kernels may overlap on the GPU (different streams, no ordering) race on it;
+ * calls ordered on one stream are fine, and nothing needs clearing between calls.
+ * Errors as elsewhere: INVALID_ARG, UNSUPPORTED, ALIGNMENT (cache 256-byte, q/out 16-byte
+ * aligned), CAPACITY, STATE (no tokens at all), CUDA. */
+vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const void* cache, int64_t n_prefill_quantized,
+                                    int64_t n_flushed_chunks, int32_t n_residual, int64_t n_protected,
+                                    int32_t layer_begin, int32_t n_layers, const void* q, void* out,
+                                    float softmax_scale, void* stream);
+
 /* Profiling aid: record the two CUDA events (cudaEvent_t passed as void*) immediately before
  * and after the split-KV attention kernel of every later vidkv_decode_attention call on this
  * handle; NULL, NULL switches it off.  The events are the caller's. */

@@ -62,6 +62,8 @@ class VidKVConfig:
 _SIGNATURES = {
     "vidkv_version": (C.c_int32, []),
     "vidkv_launch_count": (C.c_uint64, []),
+    "vidkv_attend_noalloc": (C.c_int32, [C.POINTER(_Config), C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int64,
+                                         C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
     "vidkv_set_profile_events": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "vidkv_cache_bytes": (C.c_int32, [C.POINTER(_Config), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "vidkv_cache_layout": (C.c_int32, [C.POINTER(_Config), C.POINTER(_Layout)]),
@@ -121,6 +123,18 @@ def vidkv_version() -> int:
 
 def vidkv_launch_count() -> int:
     return load_library().vidkv_launch_count()
+
+
+def vidkv_attend_noalloc(cfg: VidKVConfig, cache, n_prefill_quantized: int, n_flushed_chunks: int, n_residual: int,
+                         n_protected: int, layer_begin: int, n_layers: int, q, out, softmax_scale: float = 0.0):
+    """Attention of q over the packed cache tensor `cache` as it stands, for callers that cannot
+    provide workspace memory: the split-KV scratch is a fixed array inside the library.  Same
+    arguments as the C function; raises VidKVError (CAPACITY when the problem needs more than the
+    array holds)."""
+    c = cfg.to_c()
+    _check("vidkv_attend_noalloc", load_library().vidkv_attend_noalloc(
+        C.byref(c), C.c_void_p(cache.data_ptr()), n_prefill_quantized, n_flushed_chunks, n_residual, n_protected,
+        layer_begin, n_layers, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()), softmax_scale, _stream_ptr()))
 
 
 def vidkv_cache_bytes(cfg: VidKVConfig):
