@@ -51,7 +51,7 @@
  *                    column 0 = Re X[0], 1 = Re X[32], 2k = Re X[k],
  *                    2k+1 = Im X[k] for k = 1..31.
  *     ternary supergroups : per 5 groups (160 stream tokens) 5376 bytes:
- *                    [0,4096)   byte (j, c) at 128*j + c holds the trits of
+ *                    [0,4096)   byte (j, c) at 256*(j/2) + 2*c + j%2 holds the trits of
  *                               channel c at token j of each of the 5 groups:
  *                               digit d_g = trit + 1, b = sum_g d_g * 3^(4-g),
  *                               stored byte = (256*b + 242) / 243;

@@ -85,6 +85,9 @@ __device__ __forceinline__ float ordered_float(uint32_t u) {
 // peel digits with multiply / shift and no division.
 __host__ __device__ __forceinline__ uint32_t trit_byte_encode(uint32_t b) { return (256u * b + 242u) / 243u; }
 __host__ __device__ __forceinline__ uint32_t trit_byte_decode(uint32_t q) { return (q * 243u) >> 8; }
+// Byte plane of a ternary supergroup: token pairs are interleaved so that one 32-bit word
+// holds (token 2m, token 2m+1) of two neighbouring channels.
+__host__ __device__ __forceinline__ int tern_byte_offset(int j, int c) { return (j >> 1) * 256 + c * 2 + (j & 1); }
 __host__ __device__ __forceinline__ int trit_digit(uint32_t b, int slot) {
   const uint32_t p3[5] = {81u, 27u, 9u, 3u, 1u};
   return static_cast<int>((b / p3[slot]) % 3u);

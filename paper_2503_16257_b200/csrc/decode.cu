@@ -258,7 +258,7 @@ __global__ void __launch_bounds__(256) decode_split_kernel(DecodeArgs a) {
         const int j1 = static_cast<int>(min(gi * kG + kG, u1) - gi * kG);
         float g0 = 0.f, g1 = 0.f, g2 = 0.f, g3 = 0.f;
         for (int j = j0; j < j1; ++j) {
-          const float tr = static_cast<float>(trit_digit(trit_byte_decode(sg[j * kD + c]), slot) - 1);
+          const float tr = static_cast<float>(trit_digit(trit_byte_decode(sg[tern_byte_offset(j, c)]), slot) - 1);
           const int64_t u = gi * kG + j;
           const int li = mode == 1 ? static_cast<int>(u - u_fl0 + T_q0 - t0)
                                    : (stp ? static_cast<int>(sm.tern_map[u - ua0]) : static_cast<int>(u - t0));

@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(128) dequant_values_kernel(CacheView cv, int l
       const int64_t gi = u / kG;
       const uint8_t* sg = sp + cv.tern_offset + (gi / kSGGroups) * kSGBytes;
       const int slot = static_cast<int>(gi % kSGGroups);
-      const int tr = trit_digit(trit_byte_decode(sg[(u % kG) * kD + c]), slot) - 1;
+      const int tr = trit_digit(trit_byte_decode(sg[tern_byte_offset(static_cast<int>(u % kG), c)]), slot) - 1;
       v = static_cast<float>(tr) * h2f(reinterpret_cast<const uint16_t*>(sg + kSG_Scales)[slot * kD + c]);
     }
     o[tt * kD + c] = v;

@@ -54,7 +54,8 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
   __syncthreads();
   // pass 2: digits and bytes
   for (int item = threadIdx.x; item < kG * kD; item += 256) {
-    const int c = item & (kD - 1), j = item >> 7;
+    // item enumerates bytes in storage order: (token pair, channel, parity)
+    const int j = ((item >> 8) << 1) | (item & 1), c = (item >> 1) & (kD - 1);
     uint32_t bval = 0;
 #pragma unroll
     for (int g = 0; g < kSGGroups; ++g) {
@@ -63,7 +64,7 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
       const uint32_t d = (g * kG + j < n_rows) ? (v > a ? 2u : (v < -a ? 0u : 1u)) : 1u;
       bval = bval * 3u + d;
     }
-    sg[item] = static_cast<uint8_t>(trit_byte_encode(bval));
+    sg[tern_byte_offset(j, c)] = static_cast<uint8_t>(trit_byte_encode(bval));
   }
 }
 
@@ -149,9 +150,9 @@ __global__ void __launch_bounds__(kD) v_flush_kernel(KSrc src, CacheView cv, int
     for (int j = 0; j < kG; ++j) {
       const float v = Elem<T>::to_float(base[(g4 * kG + j) * src.stride_t + c]);
       const uint32_t d = v > a ? 2u : (v < -a ? 0u : 1u);
-      const uint32_t bold = trit_byte_decode(sg[j * kD + c]);
+      const uint32_t bold = trit_byte_decode(sg[tern_byte_offset(j, c)]);
       const uint32_t dold = (bold / p3[slot]) % 3u;
-      sg[j * kD + c] = static_cast<uint8_t>(trit_byte_encode(bold - dold * p3[slot] + d * p3[slot]));
+      sg[tern_byte_offset(j, c)] = static_cast<uint8_t>(trit_byte_encode(bold - dold * p3[slot] + d * p3[slot]));
     }
   }
 }

@@ -50,7 +50,7 @@ def ternary_groups(slab: np.ndarray, lay: dict, g_begin: int, n_groups: int):
         gi = g_begin + k
         rec = slab[lay["tern_offset"] + (gi // 5) * SG_BYTES:][:SG_BYTES]
         slot = gi % 5
-        q = rec[:4096].astype(np.int64).reshape(G, D)
+        q = rec[:4096].astype(np.int64).reshape(G // 2, D, 2).transpose(0, 2, 1).reshape(G, D)
         bval = (q * 243) >> 8
         digit = (bval // 3 ** (4 - slot)) % 3
         trits[k * G:(k + 1) * G] = digit - 1
