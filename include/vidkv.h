@@ -38,11 +38,14 @@
  *     chunk table  : per chunk 128 bytes: 64 ascending anomalous channel ids,
  *                    then 64 ascending normal channel ids (uint8).  Chunk 0 is
  *                    the prefill; every residual flush appends a 128-token chunk.
- *     key groups   : per 32 tokens 1152 bytes:
- *                    [0,512)    2-bit codes, token t at 16*t, anomalous slot j in
- *                               32-bit word j/16 at bits 2*(j%16);
- *                    [512,768)  1-bit codes, token t at 512+8*t, spectrum column
- *                               f in word f/32 at bit f%32 (1 = coefficient >= 0);
+ *     key groups   : per 32 tokens 1152 bytes (token t = 8 nt + tl of the group):
+ *                    [0,512)    2-bit codes as 128 32-bit words: anomalous slot
+ *                               j = 16 r + e of token t is in word ((4 tl + r) * 4 + nt)
+ *                               at bits 2 (e / 2) + 16 (e % 2)  (even slots in the low
+ *                               half-word, odd slots in the high one);
+ *                    [512,768)  1-bit codes as 128 16-bit half-words: spectrum column
+ *                               f = 16 r + e of token t is in half-word ((4 tl + r) * 4 + nt)
+ *                               at bit 15 - e (1 = coefficient >= 0);
  *                    [768,896)  s  (binary16) of the 64 two-bit slots;
  *                    [896,1024) z  (binary16) of the 64 two-bit slots;
  *                    [1024,1152) s (binary16) of the 64 spectrum columns.
@@ -51,10 +54,12 @@
  *                    column 0 = Re X[0], 1 = Re X[32], 2k = Re X[k],
  *                    2k+1 = Im X[k] for k = 1..31.
  *     ternary supergroups : per 5 groups (160 stream tokens) 5376 bytes:
- *                    [0,4096)   byte (j, c) at 256*(j/2) + 2*c + j%2 holds the trits of
- *                               channel c at token j of each of the 5 groups:
+ *                    [0,4096)   one byte per (token j of the group, channel c), holding the
+ *                               trits of channel c at token j of each of the 5 groups:
  *                               digit d_g = trit + 1, b = sum_g d_g * 3^(4-g),
- *                               stored byte = (256*b + 242) / 243;
+ *                               stored byte = (256*b + 242) / 243.  With j = 2 m + parity,
+ *                               m = 8 kt + 4 u + r and c = 32 w + 4 rho + e the byte is at
+ *                               ((((kt*2 + u)*4 + w)*4 + r)*8 + rho)*8 + 2 e + parity;
  *                    [4096,5376) s (binary16) [5][128].
  *     protected groups (STP) : per 32 protected tokens 1536 bytes:
  *                    [0,1024) 2-bit codes, token j at 32*j, channel c in word
@@ -215,10 +220,11 @@ vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* handle, int32_t layer, flo
  * (no append, no flush), the cache having been filled through a handle built on the same
  * `cfg`.  The caller states the token counts that vidkv_layer_state reports for the layers:
  * n_prefill_quantized (a multiple of G), n_flushed_chunks, n_residual (0..R) and n_protected.
- * The split-KV partial results live in a 16 MiB array inside the library, which every GPU
- * that loads the library keeps until the process exits; at most 32263 (query head, split)
- * records fit, i.e. n_layers * B * H_q * ceil(tokens / split) <= 32263 with split = 160, 320
- * or 640 tokens -- larger problems return VIDKV_ERR_CAPACITY (use fewer layers per call).
+ * The split-KV scratch lives in a 16 MiB array inside the library, which every GPU that
+ * loads the library keeps until the process exits.  It must hold 520 bytes per (query head,
+ * split) record, n_layers * B * H_q * ceil(tokens / split) of them with split = 160, 320 or
+ * 640 tokens, plus, when n_protected is 0, 3072 bytes per (layer, batch element, KV head,
+ * chunk) -- larger problems return VIDKV_ERR_CAPACITY (use fewer layers per call).
  * Nothing is allocated or freed.  The first call on each device looks up the array's device
  * address, so make that first call outside any stream capture.  All calls share the array:
  * two calls whose kernels may overlap on the GPU (different streams, no ordering) race on it;

@@ -85,9 +85,26 @@ __device__ __forceinline__ float ordered_float(uint32_t u) {
 // peel digits with multiply / shift and no division.
 __host__ __device__ __forceinline__ uint32_t trit_byte_encode(uint32_t b) { return (256u * b + 242u) / 243u; }
 __host__ __device__ __forceinline__ uint32_t trit_byte_decode(uint32_t q) { return (q * 243u) >> 8; }
-// Byte plane of a ternary supergroup: token pairs are interleaved so that one 32-bit word
-// holds (token 2m, token 2m+1) of two neighbouring channels.
-__host__ __device__ __forceinline__ int tern_byte_offset(int j, int c) { return (j >> 1) * 256 + c * 2 + (j & 1); }
+// Byte plane of a ternary supergroup (4096 bytes = 32 stream tokens x 128 channels), laid out
+// for the tensor-core decoder: token j = 2 m + parity, pair m = 8 kt + 4 u + r; channel
+// c = 32 w + 4 rho + e.  The 8 bytes (e, parity) of one (m, w, rho) are contiguous, and the
+// 32 (r, rho) combinations of one (kt, u, w) form one 256-byte run, so that a warp reads the
+// operands of one 16-token MMA step with one conflict-free 64-bit load per lane.
+__host__ __device__ __forceinline__ int tern_byte_offset(int j, int c) {
+  const int m = j >> 1, kt = m >> 3, u = (m >> 2) & 1, r = m & 3;
+  const int w = c >> 5, rho = (c >> 2) & 7, e = c & 3;
+  return (((((kt * 2 + u) * 4 + w) * 4 + r) * 8 + rho) * 8) + 2 * e + (j & 1);
+}
+// 2-bit key codes of one 32-token group (512 bytes): token t = 8 nt + tl, anomalous slot
+// j = 16 r + e.  Lane l = 4 tl + r of a warp owns the four 32-bit words 4 l .. 4 l + 3 (one per
+// nt); inside a word, slot e sits at bit 2 (e / 2) + 16 (e % 2), i.e. even slots fill the low
+// half-word and odd slots the high one (a binary16 pair comes out of one mask).
+__host__ __device__ __forceinline__ int k2_word_index(int t, int j) { return ((t & 7) * 4 + (j >> 4)) * 4 + (t >> 3); }
+__host__ __device__ __forceinline__ int k2_bit(int j) { return 2 * ((j & 15) >> 1) + 16 * (j & 1); }
+// 1-bit key codes of one group (256 bytes): spectrum column f = 16 r + e of token t lives in
+// the 16-bit half-word with the same index as the 2-bit word above, at bit 15 - e.
+__host__ __device__ __forceinline__ int k1_half_index(int t, int f) { return ((t & 7) * 4 + (f >> 4)) * 4 + (t >> 3); }
+__host__ __device__ __forceinline__ int k1_bit(int f) { return 15 - (f & 15); }
 __host__ __device__ __forceinline__ int trit_digit(uint32_t b, int slot) {
   const uint32_t p3[5] = {81u, 27u, 9u, 3u, 1u};
   return static_cast<int>((b / p3[slot]) % 3u);

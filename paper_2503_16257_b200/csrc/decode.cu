@@ -149,21 +149,18 @@ __global__ void __launch_bounds__(256) decode_split_kernel(DecodeArgs a) {
       const float* qs2 = sm.qs2 + warp * 64;
       const float* qs1 = sm.qs1 + warp * 64;
       float acc = sm.qz[warp];
-      const uint4 c2 = reinterpret_cast<const uint4*>(sm.kg + kKG_Codes2)[lane];
-      const uint32_t w2[4] = {c2.x, c2.y, c2.z, c2.w};
+      // token = lane
 #pragma unroll
-      for (int w = 0; w < 4; ++w)
+      for (int w = 0; w < 4; ++w) {
+        const uint32_t w2 = reinterpret_cast<const uint32_t*>(sm.kg + kKG_Codes2)[k2_word_index(lane, 16 * w)];
+        const uint32_t w1 = reinterpret_cast<const uint16_t*>(sm.kg + kKG_Bits1)[k1_half_index(lane, 16 * w)];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) acc += qs2[w * 16 + i] * static_cast<float>((w2[w] >> (2 * i)) & 3u);
-      const uint2 c1 = reinterpret_cast<const uint2*>(sm.kg + kKG_Bits1)[lane];
-      const uint32_t w1[2] = {c1.x, c1.y};
-#pragma unroll
-      for (int w = 0; w < 2; ++w)
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float v = qs1[w * 32 + i];
-          acc += ((w1[w] >> i) & 1u) ? v : -v;
+        for (int i = 0; i < 16; ++i) {
+          acc += qs2[w * 16 + i] * static_cast<float>((w2 >> k2_bit(i)) & 3u);
+          const float v = qs1[w * 16 + i];
+          acc += ((w1 >> k1_bit(i)) & 1u) ? v : -v;
         }
+      }
       sm.S[warp * ST + static_cast<int>(t - t0) + lane] = acc * a.scale;
     }
     __syncthreads();
@@ -335,7 +332,7 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(const float* __restric
   else reinterpret_cast<__nv_bfloat16*>(out)[qh * kD + c] = __float2bfloat16_rn(o);
 }
 
-cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
+static cudaError_t launch_decode_cc(const DecodeArgs& a, cudaStream_t stream) {
   const int n_slabs = a.n_layers * a.cv.B * a.cv.H_kv;
   const size_t smem = split_smem_bytes(a.split_tokens);
   static size_t attr_smem = 0;
@@ -350,7 +347,15 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
   if (a.in_dtype == VIDKV_F16) decode_split_kernel<__half><<<grid, 256, smem, stream>>>(a);
   else decode_split_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(a);
   if (a.ev_end) cudaEventRecord(a.ev_end, stream);
-  count_launches(2);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
+  // Protected tokens permute the value streams: those caches take the CUDA-core kernel.
+  const cudaError_t e = a.n_prot > 0 ? launch_decode_cc(a, stream) : launch_decode_mma(a, stream);
+  if (e != cudaSuccess) return e;
+  count_launches(1);
   decode_merge_kernel<<<a.n_layers * a.cv.B * a.cv.H_q, kD, 0, stream>>>(a.partials, a.n_splits, a.out, a.out_dtype);
   return cudaGetLastError();
 }

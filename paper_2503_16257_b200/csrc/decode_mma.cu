@@ -1,0 +1,512 @@
+// Decode attention over the packed cache on the tensor cores (Algorithm 1 "Decoding",
+// Eq. 3), split-KV, for caches without protected tokens (p = 0).
+//
+// The packed codes never become FP16 K or V in memory.  They are expanded in registers to
+// small exact binary16 numbers and fed to mma.sync.m16n8k16 as one operand; everything that
+// depends on the query or on the per-group metadata goes into the other operand:
+//
+//   scores (transposed: rows = query heads, columns = tokens)
+//     anomalous channels  sum_j q_j (s_j code_j + z_j)
+//                         = sum_j (q_j s_j) (4 + code_j) + sum_j q_j z_j - 4 sum_j q_j s_j
+//       codes come out of the 2-bit words with one shift and one mask as 4 + code in binary16;
+//       q_j s_j is formed per 32-token group as an exact pair hi + lo of binary16 numbers
+//       (rows 0-7 of the A operand carry hi, rows 8-15 lo, the two halves of the accumulator
+//       are added afterwards); the two constants come from one more MMA whose B operand is the
+//       raw z and s metadata;
+//     normal channels     K' = IDFT(+-s), so q . K'_t = sum_f Q_f s_f (+-1) with Q the
+//       weighted forward transform of the permuted query (decode_prep_kernel, once per chunk);
+//       the sign bits become +-1.0 with one shift and one mask.
+//   P V (rows = channels, columns = query heads)
+//     each byte of the ternary plane holds the digits of five groups; they are peeled with a
+//     multiply by 3 per digit on two bytes at a time (16-bit lanes) and leave 4 + digit =
+//     5 + trit in binary16; the 5 is removed through the accumulator's initial value
+//     -5 sum_t p_t, and the per-(group, channel) scale multiplies the group's accumulator.
+//
+// One CTA (4 warps) = one split of the token axis of one (layer, batch element, KV head).
+// The split's key groups and ternary supergroups are copied to shared memory with cp.async;
+// phase 1 (warps split the 32-token groups) writes scores, a softmax pass turns them into
+// binary16 probabilities in place, phase 2 (warps split the channels) accumulates P V.
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace vidkv {
+
+namespace {
+
+constexpr int kPrepWords = 24;     // 32-bit words per lane per (slab, chunk)
+constexpr int kThreads = 128;
+
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// q . k with the operands in the cache's element type (rows 8-15 of A unused)
+template <typename T> __device__ __forceinline__ void mma_in(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1);
+template <> __device__ __forceinline__ void mma_in<__half>(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  mma_f16(d, a0, 0u, a2, 0u, b0, b1);
+}
+template <> __device__ __forceinline__ void mma_in<__nv_bfloat16>(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0,
+                                                                  uint32_t b1) {
+  mma_bf16(d, a0, 0u, a2, 0u, b0, b1);
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ uint32_t hmul2_u(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+// a * b + c on two binary16 lanes (one rounding)
+__device__ __forceinline__ uint32_t hfma2_u(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+
+}  // namespace
+
+size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks) {
+  return static_cast<size_t>(n_slabs) * n_chunks * kPrepWords * 32 * sizeof(uint32_t);
+}
+
+// ---------------------------------------------------------------------------------
+// Query preparation: one block per (chunk, slab).  Writes, per lane of a warp, the 24
+// register images the attention kernel needs for this chunk's channel split:
+//   words  0.. 7  binary16 pairs of q at the anomalous slots (16 r + 2 i, 16 r + 2 i + 1)
+//   words  8..15  leading binary16 part of the transformed query Q at the spectrum
+//                 columns (16 r + 2 i, 16 r + 2 i + 1)
+//   words 16..23  binary16 remainder Q - leading part
+// for head lane / 4 (zero when that head does not exist) and r = lane % 4.
+// ---------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int n_chunks) {
+  __shared__ float q_raw[kMaxRep][kD];
+  __shared__ float q_hat[kMaxRep][kNF];
+  __shared__ float cs[64], sn[64];
+  __shared__ uint8_t perm[kD];
+  const CacheView& cv = a.cv;
+  const int tid = threadIdx.x;
+  const int chunk = blockIdx.x, slab = blockIdx.y;
+  const int h = slab % cv.H_kv, lb = slab / cv.H_kv;
+  const int b = lb % cv.B, layer_idx = lb / cv.B;
+  const int rep = cv.rep;
+  const uint8_t* slab_ptr = cv.slab(a.layer0 + layer_idx, b, h);
+  perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
+  const T* qp = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(lb) * cv.H_q + h * rep) * kD;
+  for (int i = tid; i < kMaxRep * kD; i += kThreads) {
+    const int r = i >> 7, c = i & 127;
+    q_raw[r][c] = r < rep ? Elem<T>::to_float(qp[r * kD + c]) : 0.0f;
+  }
+  if (tid < 64) {
+    float s, c;
+    sincospif(static_cast<float>(tid) / 32.0f, &s, &c);
+    cs[tid] = c; sn[tid] = s;
+  }
+  __syncthreads();
+  // Q_f = sum_c q_c W[c, f]: the weights with which spectrum column f enters channel c of
+  // the inverse orthonormal 64-point transform of a Hermitian half spectrum.
+  for (int i = tid; i < kMaxRep * kNF; i += kThreads) {
+    const int r = i >> 6, f = i & 63;
+    float acc = 0.0f;
+    if (f < 2) {
+      for (int c = 0; c < 64; ++c) {
+        const float qv = q_raw[r][perm[64 + c]];
+        acc += (f == 1 && (c & 1)) ? -qv : qv;
+      }
+      acc *= 0.125f;
+    } else {
+      const int k = f >> 1;
+      const bool im = f & 1;
+      for (int c = 0; c < 64; ++c) {
+        const float qv = q_raw[r][perm[64 + c]];
+        const int m = (k * c) & 63;
+        acc += qv * (im ? -sn[m] : cs[m]);
+      }
+      acc *= 0.25f;
+    }
+    q_hat[r][f] = acc;
+  }
+  __syncthreads();
+  uint32_t* out = a.prep + (static_cast<int64_t>(slab) * n_chunks + chunk) * (kPrepWords * 32);
+  for (int i = tid; i < kPrepWords * 32; i += kThreads) {
+    const int word = i >> 5, lane = i & 31;
+    const int hd = lane >> 2, r = lane & 3;
+    const int kind = word >> 3, pi = word & 7;
+    const int e0 = 16 * r + 2 * pi;
+    uint32_t v;
+    if (kind == 0) {
+      v = pack_half2(q_raw[hd][perm[e0]], q_raw[hd][perm[e0 + 1]]);
+    } else {
+      const float x0 = q_hat[hd][e0], x1 = q_hat[hd][e0 + 1];
+      const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
+      if (kind == 1) v = pack_half2(__half2float(h0), __half2float(h1));
+      else v = pack_half2(x0 - __half2float(h0), x1 - __half2float(h1));
+    }
+    out[i] = v;
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// Shared memory of the attention kernel, for a split of ST tokens (a multiple of 160):
+//   kbuf  ST/32 key groups           (reused for the output staging after phase 1)
+//   vbuf  ST/160 ternary supergroups
+//   S     8 rows of ST + 4 floats: scores, then binary16 probabilities in place
+//   psum  [ST/32][8]  -5 * (sum of the rounded probabilities of the group)
+//   red   [16]        row maxima and sums
+// ---------------------------------------------------------------------------------
+size_t decode_mma_smem_bytes(int ST) {
+  return static_cast<size_t>(ST / 32) * kKGroupBytes + static_cast<size_t>(ST / 160) * kSGBytes +
+         sizeof(float) * (8 * (ST + 4) + 8 * (ST / 32) + 16);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, int n_chunks) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  const int ST = a.split_tokens;
+  const int SS = ST + 4;                                  // row stride of S in floats
+  uint8_t* kbuf = smem_raw;
+  uint8_t* vbuf = kbuf + (ST / 32) * kKGroupBytes;
+  float* S = reinterpret_cast<float*>(vbuf + (ST / 160) * kSGBytes);
+  float* psum = S + 8 * SS;
+  float* red = psum + 8 * (ST / 32);
+
+  const CacheView& cv = a.cv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int hd = lane >> 2, r = lane & 3;
+  const int split = blockIdx.x, slab = blockIdx.y;
+  const int h = slab % cv.H_kv, lb = slab / cv.H_kv;
+  const int b = lb % cv.B, layer_idx = lb / cv.B;
+  const int rep = cv.rep;
+  const uint8_t* slab_ptr = cv.slab(a.layer0 + layer_idx, b, h);
+
+  const int64_t T_q0 = a.st.T_q0;
+  const int64_t T_qt = T_q0 + a.st.n_flush * kR;          // quantized tokens (multiple of 32)
+  const int64_t T_tot = T_qt + a.st.n_res;
+  const int64_t t0 = static_cast<int64_t>(split) * ST;
+  const int64_t t1 = min(t0 + ST, T_tot);
+  const int64_t tq1 = max(min(t1, T_qt), t0);             // end of the quantized part of this split
+  const int n_loc = static_cast<int>(t1 - t0);
+  const int nq = static_cast<int>(tq1 - t0);              // quantized tokens here (multiple of 32)
+  const int n_kg = nq / kG;                               // key groups = ternary groups (p = 0)
+  const int n_sg = (n_kg + kSGGroups - 1) / kSGGroups;
+  const int64_t gk0 = t0 / kG;
+
+  // ---- stage the packed split
+  {
+    const uint8_t* ksrc = slab_ptr + cv.kgroup_offset + gk0 * kKGroupBytes;
+    for (int i = tid; i < n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
+    cp_async_commit();
+    const uint8_t* vsrc = slab_ptr + cv.tern_offset + (t0 / (kG * kSGGroups)) * kSGBytes;
+    for (int i = tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
+    cp_async_commit();
+  }
+
+  // ================= phase 1: scores =================
+  cp_async_wait<1>();
+  __syncthreads();
+  {
+    const int64_t g0n = T_q0 / kG;                        // key groups of the prefill chunk
+    int cur_chunk = -1;
+    uint32_t qa[8], qha[8], qhb[8];
+    for (int g = warp; g < n_kg; g += 4) {
+      const int64_t gidx = gk0 + g;
+      const int chunk = gidx < g0n ? 0 : 1 + static_cast<int>((gidx - g0n) / (kR / kG));
+      if (chunk != cur_chunk) {
+        cur_chunk = chunk;
+        const uint32_t* pp = a.prep + (static_cast<int64_t>(slab) * n_chunks + chunk) * (kPrepWords * 32) + lane;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          qa[i] = __ldg(pp + i * 32);
+          qha[i] = __ldg(pp + (8 + i) * 32);
+          qhb[i] = __ldg(pp + (16 + i) * 32);
+        }
+      }
+      const uint8_t* kg = kbuf + g * kKGroupBytes;
+      uint32_t s2[8], z2[8], s1[8];
+      {
+        const uint4 x0 = *reinterpret_cast<const uint4*>(kg + kKG_S2 + 32 * r);
+        const uint4 x1 = *reinterpret_cast<const uint4*>(kg + kKG_S2 + 32 * r + 16);
+        s2[0] = x0.x; s2[1] = x0.y; s2[2] = x0.z; s2[3] = x0.w; s2[4] = x1.x; s2[5] = x1.y; s2[6] = x1.z; s2[7] = x1.w;
+        const uint4 y0 = *reinterpret_cast<const uint4*>(kg + kKG_Z2 + 32 * r);
+        const uint4 y1 = *reinterpret_cast<const uint4*>(kg + kKG_Z2 + 32 * r + 16);
+        z2[0] = y0.x; z2[1] = y0.y; z2[2] = y0.z; z2[3] = y0.w; z2[4] = y1.x; z2[5] = y1.y; z2[6] = y1.z; z2[7] = y1.w;
+        const uint4 w0 = *reinterpret_cast<const uint4*>(kg + kKG_S1 + 32 * r);
+        const uint4 w1 = *reinterpret_cast<const uint4*>(kg + kKG_S1 + 32 * r + 16);
+        s1[0] = w0.x; s1[1] = w0.y; s1[2] = w0.z; s1[3] = w0.w; s1[4] = w1.x; s1[5] = w1.y; s1[6] = w1.z; s1[7] = w1.w;
+      }
+      // constants of the group: column 2 r of the result = sum q z, column 2 r + 1 = sum q s
+      float cst;
+      {
+        float cz[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        const bool odd = hd & 1;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          mma_f16(cz, qa[2 * ks], 0u, qa[2 * ks + 1], 0u, odd ? s2[2 * ks] : z2[2 * ks], odd ? s2[2 * ks + 1] : z2[2 * ks + 1]);
+        cst = cz[0] - 4.0f * cz[1];
+      }
+      // q s as exact binary16 pairs hi + lo
+      uint32_t hi2[8], lo2[8], hi1[8], lo1[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        hi2[i] = hmul2_u(qa[i], s2[i]);
+        lo2[i] = hfma2_u(qa[i], s2[i], hi2[i] ^ 0x80008000u);
+        hi1[i] = hmul2_u(qha[i], s1[i]);
+        lo1[i] = hfma2_u(qhb[i], s1[i], hfma2_u(qha[i], s1[i], hi1[i] ^ 0x80008000u));
+      }
+      const uint4 c2 = *reinterpret_cast<const uint4*>(kg + kKG_Codes2 + lane * 16);
+      const uint2 c1 = *reinterpret_cast<const uint2*>(kg + kKG_Bits1 + lane * 8);
+      const uint32_t w2[4] = {c2.x, c2.y, c2.z, c2.w};
+      const uint32_t h1[4] = {c1.x & 0xffffu, c1.x >> 16, c1.y & 0xffffu, c1.y >> 16};
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        float acc[4] = {cst, cst, 0.0f, 0.0f};
+        const uint32_t w = w2[nt];
+        uint32_t x[8];
+        x[0] = ((w << 8) & 0x03000300u) | 0x44004400u;
+        x[1] = ((w << 6) & 0x03000300u) | 0x44004400u;
+        x[2] = ((w << 4) & 0x03000300u) | 0x44004400u;
+        x[3] = ((w << 2) & 0x03000300u) | 0x44004400u;
+        x[4] = (w & 0x03000300u) | 0x44004400u;
+        x[5] = ((w >> 2) & 0x03000300u) | 0x44004400u;
+        x[6] = ((w >> 4) & 0x03000300u) | 0x44004400u;
+        x[7] = ((w >> 6) & 0x03000300u) | 0x44004400u;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          mma_f16(acc, hi2[2 * ks], lo2[2 * ks], hi2[2 * ks + 1], lo2[2 * ks + 1], x[2 * ks], x[2 * ks + 1]);
+        // sign bits: low lane <- bit 15 - 2 m, high lane <- bit 14 - 2 m of the half-word
+        const uint32_t X = h1[nt] * 0x00020001u;
+        uint32_t y[8];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) y[m] = ((X << (2 * m)) & 0x80008000u) ^ 0xbc00bc00u;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          mma_f16(acc, hi1[2 * ks], lo1[2 * ks], hi1[2 * ks + 1], lo1[2 * ks + 1], y[2 * ks], y[2 * ks + 1]);
+        *reinterpret_cast<float2*>(S + hd * SS + g * kG + nt * 8 + 2 * r) = make_float2(acc[0] + acc[2], acc[1] + acc[3]);
+      }
+    }
+  }
+  // residual tokens of this split: q . k on the tensor cores straight from the FP16 / BF16 rows
+  if (t1 > T_qt) {
+    const int r_begin = static_cast<int>(max(t0, T_qt) - T_qt), r_end = static_cast<int>(t1 - T_qt);
+    const T* kres = reinterpret_cast<const T*>(slab_ptr + cv.kres_offset);
+    const T* qp = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(lb) * cv.H_q + h * rep) * kD;
+    uint32_t qn[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      qn[i] = hd < rep ? __ldg(reinterpret_cast<const uint32_t*>(qp + hd * kD + 8 * i + 2 * r)) : 0u;
+    const int n_tiles = (r_end - r_begin + 7) / 8;
+    for (int tile = warp; tile < n_tiles; tile += 4) {
+      const int row = min(r_begin + tile * 8 + hd, r_end - 1);          // clamped: extra columns are dropped
+      const uint32_t* kr = reinterpret_cast<const uint32_t*>(kres + static_cast<int64_t>(row) * kD) + r;
+      float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) mma_in<T>(acc, qn[2 * ks], qn[2 * ks + 1], kr[ks * 8], kr[ks * 8 + 4]);
+      const int c0 = r_begin + tile * 8 + 2 * r;
+      float* srow = S + hd * SS + static_cast<int>(T_qt - t0);
+      if (c0 < r_end) srow[c0] = acc[0];
+      if (c0 + 1 < r_end) srow[c0 + 1] = acc[1];
+    }
+  }
+  __syncthreads();
+
+  // ================= softmax numerators, in place as binary16 =================
+  {
+    const float sl2 = a.scale * 1.4426950408889634f;
+    const int n_pad = max(n_sg * kSGGroups * kG, (n_loc + 1) & ~1);      // entries the P V loops may read
+    constexpr int kMaxPerLane = 20;                                        // ST <= 640
+#pragma unroll 1
+    for (int hh = 0; hh < 2; ++hh) {
+      const int row_h = warp * 2 + hh;
+      float* row = S + row_h * SS;
+      float v[kMaxPerLane];
+      float m = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < kMaxPerLane; ++k) {
+        const int i = lane + 32 * k;
+        v[k] = i < n_loc ? row[i] : -INFINITY;
+        m = fmaxf(m, v[k]);
+      }
+#pragma unroll
+      for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      __syncwarp();
+      float l = 0.0f;
+      __half* prow = reinterpret_cast<__half*>(row);
+#pragma unroll
+      for (int k = 0; k < kMaxPerLane; ++k) {
+        const int i = lane + 32 * k;
+        const float p = i < n_loc ? exp2f((v[k] - m) * sl2) : 0.0f;
+        l += p;
+        if (i < n_pad) prow[i] = __float2half_rn(p);
+      }
+#pragma unroll
+      for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+      if (lane == 0) { red[row_h] = m * a.scale; red[8 + row_h] = l; }
+    }
+  }
+  __syncthreads();
+  // -5 * sum of the rounded probabilities of every (group, head)
+  for (int i = tid; i < n_kg * 8; i += kThreads) {
+    const int g = i >> 3, hh = i & 7;
+    const __half2* pr = reinterpret_cast<const __half2*>(reinterpret_cast<const __half*>(S + hh * SS) + g * kG);
+    float s = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const float2 f = __half22float2(pr[k]);
+      s += f.x + f.y;
+    }
+    psum[g * 8 + hh] = -5.0f * s;
+  }
+
+  // ================= phase 2: P V =================
+  cp_async_wait<0>();
+  __syncthreads();
+  float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
+  {
+    const uint8_t* prow = reinterpret_cast<const uint8_t*>(S + hd * SS);
+    for (int sg = 0; sg < n_sg; ++sg) {
+      const uint8_t* sgp = vbuf + sg * kSGBytes;
+      const int n_valid = min(kSGGroups, n_kg - sg * kSGGroups);
+      float acc[kSGGroups][2][4];
+#pragma unroll
+      for (int g = 0; g < kSGGroups; ++g) {
+        float2 ps = make_float2(0.0f, 0.0f);
+        if (g < n_valid) ps = *reinterpret_cast<const float2*>(psum + (sg * kSGGroups + g) * 8 + 2 * r);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) { acc[g][i][0] = ps.x; acc[g][i][1] = ps.y; acc[g][i][2] = ps.x; acc[g][i][3] = ps.y; }
+      }
+#pragma unroll
+      for (int kt = 0; kt < 2; ++kt) {
+        const uint2 wa = *reinterpret_cast<const uint2*>(sgp + ((((kt * 2 + 0) * 4 + warp) * 4 + r) * 8 + hd) * 8);
+        const uint2 wb = *reinterpret_cast<const uint2*>(sgp + ((((kt * 2 + 1) * 4 + warp) * 4 + r) * 8 + hd) * 8);
+        uint32_t W[8];
+        W[0] = prmt(wa.x, 0u, 0x4140u); W[1] = prmt(wa.x, 0u, 0x4342u);
+        W[2] = prmt(wb.x, 0u, 0x4140u); W[3] = prmt(wb.x, 0u, 0x4342u);
+        W[4] = prmt(wa.y, 0u, 0x4140u); W[5] = prmt(wa.y, 0u, 0x4342u);
+        W[6] = prmt(wb.y, 0u, 0x4140u); W[7] = prmt(wb.y, 0u, 0x4342u);
+#pragma unroll
+        for (int g = 0; g < kSGGroups; ++g) {
+          uint32_t A[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t t3 = W[k] * 3u;
+            A[k] = (t3 & 0x03000300u) | 0x44004400u;
+            W[k] = t3 & 0x00ff00ffu;
+          }
+          if (g < n_valid) {
+            const uint8_t* pb = prow + (sg * (kSGGroups * kG) + g * kG + kt * 16 + 2 * r) * 2;
+            const uint32_t b0 = *reinterpret_cast<const uint32_t*>(pb);
+            const uint32_t b1 = *reinterpret_cast<const uint32_t*>(pb + 16);
+            mma_f16(acc[g][0], A[0], A[1], A[2], A[3], b0, b1);
+            mma_f16(acc[g][1], A[4], A[5], A[6], A[7], b0, b1);
+          }
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < kSGGroups; ++g) {
+        if (g < n_valid) {
+          const uint2 sc = *reinterpret_cast<const uint2*>(sgp + kSG_Scales + g * (kD * 2) + (32 * warp + 4 * hd) * 2);
+          const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));
+          const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));
+          tot[0][0] += sa.x * acc[g][0][0]; tot[0][1] += sa.x * acc[g][0][1];
+          tot[0][2] += sa.y * acc[g][0][2]; tot[0][3] += sa.y * acc[g][0][3];
+          tot[1][0] += sb.x * acc[g][1][0]; tot[1][1] += sb.x * acc[g][1][1];
+          tot[1][2] += sb.y * acc[g][1][2]; tot[1][3] += sb.y * acc[g][1][3];
+        }
+      }
+    }
+  }
+  // ---- output staging: O[head][channel] (reuses the key buffer, free since phase 1; the
+  // smallest split, 160 tokens, has 5 x 1152 bytes there, more than the 4096 needed)
+  float* O = reinterpret_cast<float*>(kbuf);
+  {
+    const int c0 = 32 * warp + 4 * hd;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      O[(2 * r) * kD + c0 + 2 * i] = tot[i][0];
+      O[(2 * r + 1) * kD + c0 + 2 * i] = tot[i][1];
+      O[(2 * r) * kD + c0 + 2 * i + 1] = tot[i][2];
+      O[(2 * r + 1) * kD + c0 + 2 * i + 1] = tot[i][3];
+    }
+  }
+  __syncthreads();
+  {
+    const int c = tid;
+    float o[kMaxRep];
+#pragma unroll
+    for (int k = 0; k < kMaxRep; ++k) o[k] = O[k * kD + c];
+    if (t1 > T_qt) {
+      const int r_begin = static_cast<int>(max(t0, T_qt) - T_qt), r_end = static_cast<int>(t1 - T_qt);
+      const T* vres = reinterpret_cast<const T*>(slab_ptr + cv.vres_offset);
+      const int off = static_cast<int>(T_qt - t0);
+      for (int rr = r_begin; rr < r_end; ++rr) {
+        const float v = Elem<T>::to_float(vres[rr * kD + c]);
+#pragma unroll
+        for (int k = 0; k < kMaxRep; ++k)
+          o[k] += __half2float(reinterpret_cast<const __half*>(S + k * SS)[off + rr]) * v;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < kMaxRep; ++k) {
+      if (k < rep) {
+        const int64_t qh = static_cast<int64_t>(lb) * cv.H_q + h * rep + k;
+        float* pr = a.partials + (qh * a.n_splits + split) * 130;
+        pr[2 + c] = o[k];
+        if (c == 0) { pr[0] = red[k]; pr[1] = red[8 + k]; }
+      }
+    }
+  }
+}
+
+cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t stream) {
+  const int n_slabs = a.n_layers * a.cv.B * a.cv.H_kv;
+  const int n_chunks = static_cast<int>((a.st.T_q0 > 0 ? 1 : 0) + a.st.n_flush);
+  const size_t smem = decode_mma_smem_bytes(a.split_tokens);
+  static size_t attr_smem = 0;
+  if (smem > attr_smem) {
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(decode_mma_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    if ((e = cudaFuncSetAttribute(decode_mma_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    attr_smem = smem;
+  }
+  const int chunk_stride = n_chunks > 0 ? n_chunks : 1;
+  if (n_chunks > 0) {
+    const dim3 pgrid(n_chunks, n_slabs);
+    if (a.in_dtype == VIDKV_F16) decode_prep_kernel<__half><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride);
+    else decode_prep_kernel<__nv_bfloat16><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride);
+    count_launches(1);
+  }
+  const dim3 grid(a.n_splits, n_slabs);
+  if (a.ev_begin) cudaEventRecord(a.ev_begin, stream);
+  if (a.in_dtype == VIDKV_F16) decode_mma_kernel<__half><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
+  else decode_mma_kernel<__nv_bfloat16><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
+  if (a.ev_end) cudaEventRecord(a.ev_end, stream);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+}  // namespace vidkv

@@ -33,17 +33,16 @@ __global__ void __launch_bounds__(128) dequant_keys_kernel(CacheView cv, int lay
     const float s = h2f(reinterpret_cast<const uint16_t*>(kg + kKG_S2)[j]);
     const float z = h2f(reinterpret_cast<const uint16_t*>(kg + kKG_Z2)[j]);
     for (int t = 0; t < kG; ++t) {
-      const uint32_t word = reinterpret_cast<const uint32_t*>(kg + kKG_Codes2)[t * 4 + (j >> 4)];
-      o[t * kD + c] = static_cast<float>((word >> (2 * (j & 15))) & 3u) * s + z;
+      const uint32_t word = reinterpret_cast<const uint32_t*>(kg + kKG_Codes2)[k2_word_index(t, j)];
+      o[t * kD + c] = static_cast<float>((word >> k2_bit(j)) & 3u) * s + z;
     }
   } else {
     const int i = tid - 64, c = perm[64 + i];
     const uint16_t* s1 = reinterpret_cast<const uint16_t*>(kg + kKG_S1);
     for (int t = 0; t < kG; ++t) {
-      const uint32_t w0 = reinterpret_cast<const uint32_t*>(kg + kKG_Bits1)[t * 2];
-      const uint32_t w1 = reinterpret_cast<const uint32_t*>(kg + kKG_Bits1)[t * 2 + 1];
+      const uint16_t* hw = reinterpret_cast<const uint16_t*>(kg + kKG_Bits1);
       auto val = [&](int f) -> float {
-        const uint32_t bit = f < 32 ? (w0 >> f) & 1u : (w1 >> (f - 32)) & 1u;
+        const uint32_t bit = (hw[k1_half_index(t, f)] >> k1_bit(f)) & 1u;
         const float s = h2f(s1[f]);
         return bit ? s : -s;
       };

@@ -87,7 +87,7 @@ int64_t max_partial_entries(const vidkv_config_t& c, int64_t T_max) {
 }
 
 struct WsPlan {
-  int64_t minmax_off, partials_off, idx_prot_off, idx_rest_off, counts_off, total;
+  int64_t minmax_off, partials_off, prep_off, idx_prot_off, idx_rest_off, counts_off, total;
   int64_t partial_entries;
 };
 
@@ -98,6 +98,9 @@ void plan_workspace(const vidkv_config_t& c, const Layout& L, WsPlan* w) {
   w->partial_entries = max_partial_entries(c, L.max_total_tokens);
   w->partials_off = off;
   off = round_up(off + w->partial_entries * 130 * 4, kAlign);
+  w->prep_off = off;
+  off = round_up(off + static_cast<int64_t>(decode_prep_bytes(static_cast<int64_t>(c.L) * c.B * c.H_kv, L.lay.max_chunks)),
+                 kAlign);
   w->idx_prot_off = off;
   off = round_up(off + static_cast<int64_t>(c.B) * L.max_prot * 4, kAlign);
   w->idx_rest_off = off;
@@ -349,6 +352,7 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   a.cv = h->cv;
   a.q = q; a.k_new = k_new; a.v_new = v_new; a.out = out;
   a.partials = reinterpret_cast<float*>(h->workspace + h->ws.partials_off);
+  a.prep = reinterpret_cast<uint32_t*>(h->workspace + h->ws.prep_off);
   a.layer0 = layer_begin; a.n_layers = n_layers;
   a.in_dtype = dt; a.out_dtype = h->cfg.out_dtype;
   a.n_prot = h->n_prot;

@@ -68,6 +68,7 @@ struct DecodeArgs {
   const void* v_new;
   void* out;
   float* partials;     // [n_layers * B * H_q * n_splits][130]
+  uint32_t* prep;      // per (slab, chunk) query images of the tensor-core path (decode_prep_bytes)
   int32_t layer0, n_layers;
   int32_t in_dtype, out_dtype;
   int32_t split_tokens, n_splits;
@@ -83,6 +84,10 @@ inline void count_launches(int n) { g_launch_count += static_cast<unsigned long 
 
 // Split-KV attention over the packed cache + residual, then the merge of the partials.
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
+// The tensor-core split kernel (caches without protected tokens) and its query preparation;
+// scratch for `n_slabs` slabs of `n_chunks` chunks each.
+cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t stream);
+size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks);
 // Write k_new / v_new [n_layers, B, H_kv, D] into row `row` of the residual rings.
 cudaError_t launch_append(int dtype, const void* k_new, const void* v_new, const CacheView& cv, int layer0,
                           int n_layers, int row, cudaStream_t stream);

@@ -14,7 +14,8 @@
 
 namespace {
 
-// 16 MiB of split-KV partials: 32263 (query head, split) records of 130 floats.  Every GPU
+// 16 MiB of scratch: the split-KV partials ((query head, split) records of 130 floats) and,
+// for caches without protected tokens, 3 KiB of prepared query per (slab, chunk).  Every GPU
 // that loads this library holds the array until the process exits.
 constexpr size_t kStaticPartialFloats = 4u * 1024u * 1024u;
 static __device__ __align__(256) float g_static_partials[kStaticPartialFloats];
@@ -90,9 +91,14 @@ extern "C" vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const 
   a.split_tokens = split_tokens_for(T_tot, n_slabs);
   a.n_splits = static_cast<int32_t>((T_tot + a.split_tokens - 1) / a.split_tokens);
   const int64_t records = static_cast<int64_t>(n_layers) * cfg->B * cfg->H_q * a.n_splits;
-  if (records * 130 > static_cast<int64_t>(kStaticPartialFloats)) return VIDKV_ERR_CAPACITY;
+  // the array holds the partial records, then (256-byte aligned) the per-chunk query images
+  const int64_t prep_at = (records * 130 * 4 + 255) / 256 * 256;
+  const int64_t n_chunks = (n_prefill_quantized > 0 ? 1 : 0) + n_flushed_chunks;
+  const int64_t prep_bytes = n_protected > 0 ? 0 : static_cast<int64_t>(decode_prep_bytes(n_slabs, n_chunks));
+  if (prep_at + prep_bytes > static_cast<int64_t>(kStaticPartialFloats * sizeof(float))) return VIDKV_ERR_CAPACITY;
   const vidkv_status_t sp = static_partials(&a.partials);
   if (sp != VIDKV_OK) return sp;
+  a.prep = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(a.partials) + prep_at);
   // Every record the merge reads is written by the attention kernel of this same call, so
   // nothing in the array has to be cleared between calls.
   if (launch_decode(a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return VIDKV_ERR_CUDA;

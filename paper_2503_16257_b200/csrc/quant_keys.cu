@@ -212,7 +212,14 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
         w1 |= (x[32 + i] >= 0.0f ? 1u : 0u) << i;
       }
       uint8_t* kg = kg_base + g * kKGroupBytes;
-      reinterpret_cast<uint2*>(kg + kKG_Bits1)[lane] = make_uint2(w0, w1);
+      {
+        // half-word r holds columns 16 r .. 16 r + 15, column e at bit 15 - e
+        uint16_t* hw = reinterpret_cast<uint16_t*>(kg + kKG_Bits1);
+        hw[k1_half_index(lane, 0)] = static_cast<uint16_t>(__brev(w0 & 0xffffu) >> 16);
+        hw[k1_half_index(lane, 16)] = static_cast<uint16_t>(__brev(w0 >> 16) >> 16);
+        hw[k1_half_index(lane, 32)] = static_cast<uint16_t>(__brev(w1 & 0xffffu) >> 16);
+        hw[k1_half_index(lane, 48)] = static_cast<uint16_t>(__brev(w1 >> 16) >> 16);
+      }
       // column sums of |x| over the 32 tokens (lanes): reduce-scatter by halves
 #pragma unroll
       for (int i = 0; i < 64; ++i) x[i] = fabsf(x[i]);
@@ -271,10 +278,10 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
         float q = rintf(__fdiv_rn(__fsub_rn(v, z), s));
         q = fminf(fmaxf(q, 0.0f), 3.0f);
         const uint32_t code = (s == 0.0f) ? 0u : static_cast<uint32_t>(q);
-        word |= code << (2 * i);
+        word |= code << k2_bit(i);
       }
       uint8_t* kg = kg_base + g * kKGroupBytes;
-      reinterpret_cast<uint32_t*>(kg + kKG_Codes2)[(t & 31) * 4 + wi] = word;
+      reinterpret_cast<uint32_t*>(kg + kKG_Codes2)[k2_word_index(t & 31, wi * 16)] = word;
     }
   }
 }

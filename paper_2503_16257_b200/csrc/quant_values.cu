@@ -54,8 +54,9 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
   __syncthreads();
   // pass 2: digits and bytes
   for (int item = threadIdx.x; item < kG * kD; item += 256) {
-    // item enumerates bytes in storage order: (token pair, channel, parity)
-    const int j = ((item >> 8) << 1) | (item & 1), c = (item >> 1) & (kD - 1);
+    // item enumerates the bytes of the plane in storage order (the inverse of tern_byte_offset)
+    const int j = 2 * (8 * ((item >> 11) & 1) + 4 * ((item >> 10) & 1) + ((item >> 6) & 3)) + (item & 1);
+    const int c = 32 * ((item >> 8) & 3) + 4 * ((item >> 3) & 7) + ((item >> 1) & 3);
     uint32_t bval = 0;
 #pragma unroll
     for (int g = 0; g < kSGGroups; ++g) {
@@ -64,7 +65,7 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
       const uint32_t d = (g * kG + j < n_rows) ? (v > a ? 2u : (v < -a ? 0u : 1u)) : 1u;
       bval = bval * 3u + d;
     }
-    sg[tern_byte_offset(j, c)] = static_cast<uint8_t>(trit_byte_encode(bval));
+    sg[item] = static_cast<uint8_t>(trit_byte_encode(bval));
   }
 }
 

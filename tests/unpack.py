@@ -11,6 +11,19 @@ G, R, D = 32, 128, 128
 KG_BYTES, SG_BYTES, PG_BYTES, CHUNK_BYTES = 1152, 5376, 1536, 128
 
 
+def _tern_offsets():
+    """Byte offset of (stream token j, channel c) inside the 4096-byte plane of a supergroup."""
+    j = np.arange(G)[:, None]
+    c = np.arange(D)[None, :]
+    m = j // 2
+    kt, u, r = m // 8, (m // 4) % 2, m % 4
+    w, rho, e = c // 32, (c // 4) % 8, c % 4
+    return (((((kt * 2 + u) * 4 + w) * 4 + r) * 8 + rho) * 8) + 2 * e + j % 2
+
+
+TERN_OFF = _tern_offsets()
+
+
 def slab_bytes(cache: np.ndarray, lay: dict, cfg, layer: int, b: int, h: int) -> np.ndarray:
     idx = (layer * cfg.B + b) * cfg.H_kv + h
     off = lay["slab_offset"] + idx * lay["slab_stride"]
@@ -29,13 +42,18 @@ def key_groups(slab: np.ndarray, lay: dict, g_begin: int, n_groups: int):
     s2 = np.zeros((n_groups, 64), np.float16)
     z2 = np.zeros((n_groups, 64), np.float16)
     s1 = np.zeros((n_groups, 64), np.float16)
-    sh2 = 2 * (np.arange(64) % 16)
+    j = np.arange(64)
+    t = np.arange(G)
+    # word / half-word index of (token t, slot or column j): ((t % 8) * 4 + j // 16) * 4 + t // 8
+    idx = ((t[:, None] % 8) * 4 + j[None, :] // 16) * 4 + t[:, None] // 8
+    bit2 = 2 * ((j % 16) // 2) + 16 * (j % 2)
+    bit1 = 15 - j % 16
     for g in range(n_groups):
         rec = slab[lay["kgroup_offset"] + (g_begin + g) * KG_BYTES:][:KG_BYTES]
-        w2 = rec[0:512].view("<u4").reshape(G, 4)
-        codes2[g * G:(g + 1) * G] = (w2[:, np.arange(64) // 16] >> sh2) & 3
-        w1 = rec[512:768].view("<u4").reshape(G, 2)
-        bits1[g * G:(g + 1) * G] = (w1[:, np.arange(64) // 32] >> (np.arange(64) % 32)) & 1
+        w2 = rec[0:512].view("<u4")
+        codes2[g * G:(g + 1) * G] = (w2[idx] >> bit2[None, :]) & 3
+        w1 = rec[512:768].view("<u2")
+        bits1[g * G:(g + 1) * G] = (w1[idx] >> bit1[None, :]) & 1
         s2[g] = rec[768:896].view("<f2")
         z2[g] = rec[896:1024].view("<f2")
         s1[g] = rec[1024:1152].view("<f2")
@@ -50,7 +68,7 @@ def ternary_groups(slab: np.ndarray, lay: dict, g_begin: int, n_groups: int):
         gi = g_begin + k
         rec = slab[lay["tern_offset"] + (gi // 5) * SG_BYTES:][:SG_BYTES]
         slot = gi % 5
-        q = rec[:4096].astype(np.int64).reshape(G // 2, D, 2).transpose(0, 2, 1).reshape(G, D)
+        q = rec[:4096].astype(np.int64)[TERN_OFF]
         bval = (q * 243) >> 8
         digit = (bval // 3 ** (4 - slot)) % 3
         trits[k * G:(k + 1) * G] = digit - 1
