@@ -78,10 +78,45 @@ __device__ __forceinline__ uint32_t hfma2_u(uint32_t a, uint32_t b, uint32_t c) 
   asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
   return d;
 }
+// a * b - c on two binary16 lanes (one rounding)
+__device__ __forceinline__ uint32_t hfms2_u(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("{ .reg .b32 n; neg.f16x2 n, %3; fma.rn.f16x2 %0, %1, %2, n; }" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   const __half2 h = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&h);
 }
+// (x & m) | c and (x & m) ^ c as one three-input logic instruction
+__device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t m, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "r"(m), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t and_xor(uint32_t x, uint32_t m, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(x), "r"(m), "r"(c));
+  return d;
+}
+// Bit patterns of the code expansion.  They live in constant memory rather than in the
+// instruction stream so that mask and pattern both reach the logic instruction as register
+// operands (an instruction encodes one immediate at most).
+__constant__ uint32_t kExpand[4] = {0x03000300u,   // two-bit field at mantissa bits 8-9 of each binary16 lane
+                                    0x44004400u,   // 4.0 in each lane
+                                    0x80008000u,   // the sign bits
+                                    0xbc00bc00u};  // -1.0 in each lane
+
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
   uint32_t d;
   asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
@@ -198,6 +233,7 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
   const CacheView& cv = a.cv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int hd = lane >> 2, r = lane & 3;
+  const uint32_t m_field = kExpand[0], c_four = kExpand[1], m_sign = kExpand[2], c_neg1 = kExpand[3];
   const int split = blockIdx.x, slab = blockIdx.y;
   const int h = slab % cv.H_kv, lb = slab / cv.H_kv;
   const int b = lb % cv.B, layer_idx = lb / cv.B;
@@ -274,9 +310,9 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         hi2[i] = hmul2_u(qa[i], s2[i]);
-        lo2[i] = hfma2_u(qa[i], s2[i], hi2[i] ^ 0x80008000u);
+        lo2[i] = hfms2_u(qa[i], s2[i], hi2[i]);
         hi1[i] = hmul2_u(qha[i], s1[i]);
-        lo1[i] = hfma2_u(qhb[i], s1[i], hfma2_u(qha[i], s1[i], hi1[i] ^ 0x80008000u));
+        lo1[i] = hfma2_u(qhb[i], s1[i], hfms2_u(qha[i], s1[i], hi1[i]));
       }
       const uint4 c2 = *reinterpret_cast<const uint4*>(kg + kKG_Codes2 + lane * 16);
       const uint2 c1 = *reinterpret_cast<const uint2*>(kg + kKG_Bits1 + lane * 8);
@@ -287,14 +323,14 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
         float acc[4] = {cst, cst, 0.0f, 0.0f};
         const uint32_t w = w2[nt];
         uint32_t x[8];
-        x[0] = ((w << 8) & 0x03000300u) | 0x44004400u;
-        x[1] = ((w << 6) & 0x03000300u) | 0x44004400u;
-        x[2] = ((w << 4) & 0x03000300u) | 0x44004400u;
-        x[3] = ((w << 2) & 0x03000300u) | 0x44004400u;
-        x[4] = (w & 0x03000300u) | 0x44004400u;
-        x[5] = ((w >> 2) & 0x03000300u) | 0x44004400u;
-        x[6] = ((w >> 4) & 0x03000300u) | 0x44004400u;
-        x[7] = ((w >> 6) & 0x03000300u) | 0x44004400u;
+        x[0] = and_or(w << 8, m_field, c_four);
+        x[1] = and_or(w << 6, m_field, c_four);
+        x[2] = and_or(w << 4, m_field, c_four);
+        x[3] = and_or(w << 2, m_field, c_four);
+        x[4] = and_or(w, m_field, c_four);
+        x[5] = and_or(w >> 2, m_field, c_four);
+        x[6] = and_or(w >> 4, m_field, c_four);
+        x[7] = and_or(w >> 6, m_field, c_four);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
           mma_f16(acc, hi2[2 * ks], lo2[2 * ks], hi2[2 * ks + 1], lo2[2 * ks + 1], x[2 * ks], x[2 * ks + 1]);
@@ -302,7 +338,7 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
         const uint32_t X = h1[nt] * 0x00020001u;
         uint32_t y[8];
 #pragma unroll
-        for (int m = 0; m < 8; ++m) y[m] = ((X << (2 * m)) & 0x80008000u) ^ 0xbc00bc00u;
+        for (int m = 0; m < 8; ++m) y[m] = and_xor(X << (2 * m), m_sign, c_neg1);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
           mma_f16(acc, hi1[2 * ks], lo1[2 * ks], hi1[2 * ks + 1], lo1[2 * ks + 1], y[2 * ks], y[2 * ks + 1]);
@@ -338,30 +374,32 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
   {
     const float sl2 = a.scale * 1.4426950408889634f;
     const int n_pad = max(n_sg * kSGGroups * kG, (n_loc + 1) & ~1);      // entries the P V loops may read
-    constexpr int kMaxPerLane = 20;                                        // ST <= 640
+    constexpr int kMaxPairs = 10;                                          // ST <= 640: 320 pairs per row
 #pragma unroll 1
     for (int hh = 0; hh < 2; ++hh) {
       const int row_h = warp * 2 + hh;
       float* row = S + row_h * SS;
-      float v[kMaxPerLane];
+      float2 v[kMaxPairs];
       float m = -INFINITY;
 #pragma unroll
-      for (int k = 0; k < kMaxPerLane; ++k) {
-        const int i = lane + 32 * k;
-        v[k] = i < n_loc ? row[i] : -INFINITY;
-        m = fmaxf(m, v[k]);
+      for (int k = 0; k < kMaxPairs; ++k) {
+        const int i = 2 * lane + 64 * k;
+        v[k] = i < n_loc ? *reinterpret_cast<const float2*>(row + i) : make_float2(-INFINITY, -INFINITY);
+        if (i + 1 >= n_loc) v[k].y = -INFINITY;
+        m = fmaxf(m, fmaxf(v[k].x, v[k].y));
       }
 #pragma unroll
       for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
       __syncwarp();
+      const float ms = m * sl2;
       float l = 0.0f;
-      __half* prow = reinterpret_cast<__half*>(row);
+      uint32_t* prow = reinterpret_cast<uint32_t*>(row);
 #pragma unroll
-      for (int k = 0; k < kMaxPerLane; ++k) {
-        const int i = lane + 32 * k;
-        const float p = i < n_loc ? exp2f((v[k] - m) * sl2) : 0.0f;
-        l += p;
-        if (i < n_pad) prow[i] = __float2half_rn(p);
+      for (int k = 0; k < kMaxPairs; ++k) {
+        const int i = 2 * lane + 64 * k;
+        const float p0 = ex2_approx(fmaf(v[k].x, sl2, -ms)), p1 = ex2_approx(fmaf(v[k].y, sl2, -ms));
+        l += p0 + p1;
+        if (i < n_pad) prow[i >> 1] = pack_half2(p0, p1);
       }
 #pragma unroll
       for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
@@ -409,13 +447,16 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
         W[4] = prmt(wa.y, 0u, 0x4140u); W[5] = prmt(wa.y, 0u, 0x4342u);
         W[6] = prmt(wb.y, 0u, 0x4140u); W[7] = prmt(wb.y, 0u, 0x4342u);
 #pragma unroll
+        for (int k = 0; k < 8; ++k) W[k] = mad_u32(W[k], 3u, 0u);          // 3 * byte per 16-bit lane
+#pragma unroll
         for (int g = 0; g < kSGGroups; ++g) {
           uint32_t A[8];
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
-            const uint32_t t3 = W[k] * 3u;
-            A[k] = (t3 & 0x03000300u) | 0x44004400u;
-            W[k] = t3 & 0x00ff00ffu;
+            // W holds 3 * (remaining byte) per 16-bit lane; the digit sits at bits 8-9.
+            // Next W = 3 * (W - digit << 8) = 3 W - 3 A + 3 * 0x4400 (no lane ever borrows).
+            A[k] = and_or(W[k], m_field, c_four);
+            W[k] = mad_u32(A[k], 0xfffffffdu, mad_u32(W[k], 3u, 0xcc00cc00u));
           }
           if (g < n_valid) {
             const uint8_t* pb = prow + (sg * (kSGGroups * kG) + g * kG + kt * 16 + 2 * r) * 2;
