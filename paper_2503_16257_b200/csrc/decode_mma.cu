@@ -43,6 +43,14 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// d = a b + c with c given separately (no copy into the accumulator beforehand)
+__device__ __forceinline__ void mma_f16_c(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1, float c0, float c1, float c2, float c3) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c0), "f"(c1), "f"(c2), "f"(c3));
+}
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
   asm volatile(
@@ -320,7 +328,7 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
       const uint32_t h1[4] = {c1.x & 0xffffu, c1.x >> 16, c1.y & 0xffffu, c1.y >> 16};
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
-        float acc[4] = {cst, cst, 0.0f, 0.0f};
+        float acc[4];
         const uint32_t w = w2[nt];
         uint32_t x[8];
         x[0] = and_or(w << 8, m_field, c_four);
@@ -331,8 +339,9 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
         x[5] = and_or(w >> 2, m_field, c_four);
         x[6] = and_or(w >> 4, m_field, c_four);
         x[7] = and_or(w >> 6, m_field, c_four);
+        mma_f16_c(acc, hi2[0], lo2[0], hi2[1], lo2[1], x[0], x[1], cst, cst, 0.0f, 0.0f);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
+        for (int ks = 1; ks < 4; ++ks)
           mma_f16(acc, hi2[2 * ks], lo2[2 * ks], hi2[2 * ks + 1], lo2[2 * ks + 1], x[2 * ks], x[2 * ks + 1]);
         // sign bits: low lane <- bit 15 - 2 m, high lane <- bit 14 - 2 m of the half-word
         const uint32_t X = h1[nt] * 0x00020001u;
@@ -408,7 +417,7 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
   }
   __syncthreads();
   // -5 * sum of the rounded probabilities of every (group, head)
-  for (int i = tid; i < n_kg * 8; i += kThreads) {
+  for (int i = tid; i < n_sg * kSGGroups * 8; i += kThreads) {
     const int g = i >> 3, hh = i & 7;
     const __half2* pr = reinterpret_cast<const __half2*>(reinterpret_cast<const __half*>(S + hh * SS) + g * kG);
     float s = 0.0f;
@@ -430,13 +439,10 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
       const uint8_t* sgp = vbuf + sg * kSGBytes;
       const int n_valid = min(kSGGroups, n_kg - sg * kSGGroups);
       float acc[kSGGroups][2][4];
+      float2 ps[kSGGroups];
 #pragma unroll
-      for (int g = 0; g < kSGGroups; ++g) {
-        float2 ps = make_float2(0.0f, 0.0f);
-        if (g < n_valid) ps = *reinterpret_cast<const float2*>(psum + (sg * kSGGroups + g) * 8 + 2 * r);
-#pragma unroll
-        for (int i = 0; i < 2; ++i) { acc[g][i][0] = ps.x; acc[g][i][1] = ps.y; acc[g][i][2] = ps.x; acc[g][i][3] = ps.y; }
-      }
+      for (int g = 0; g < kSGGroups; ++g)
+        ps[g] = *reinterpret_cast<const float2*>(psum + (sg * kSGGroups + g) * 8 + 2 * r);
 #pragma unroll
       for (int kt = 0; kt < 2; ++kt) {
         const uint2 wa = *reinterpret_cast<const uint2*>(sgp + ((((kt * 2 + 0) * 4 + warp) * 4 + r) * 8 + hd) * 8);
@@ -458,10 +464,14 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
             A[k] = and_or(W[k], m_field, c_four);
             W[k] = mad_u32(A[k], 0xfffffffdu, mad_u32(W[k], 3u, 0xcc00cc00u));
           }
-          if (g < n_valid) {
-            const uint8_t* pb = prow + (sg * (kSGGroups * kG) + g * kG + kt * 16 + 2 * r) * 2;
-            const uint32_t b0 = *reinterpret_cast<const uint32_t*>(pb);
-            const uint32_t b1 = *reinterpret_cast<const uint32_t*>(pb + 16);
+          // groups past the end of the cache meet zero probabilities (and a zero scale below)
+          const uint8_t* pb = prow + (sg * (kSGGroups * kG) + g * kG + kt * 16 + 2 * r) * 2;
+          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(pb);
+          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(pb + 16);
+          if (kt == 0) {
+            mma_f16_c(acc[g][0], A[0], A[1], A[2], A[3], b0, b1, ps[g].x, ps[g].y, ps[g].x, ps[g].y);
+            mma_f16_c(acc[g][1], A[4], A[5], A[6], A[7], b0, b1, ps[g].x, ps[g].y, ps[g].x, ps[g].y);
+          } else {
             mma_f16(acc[g][0], A[0], A[1], A[2], A[3], b0, b1);
             mma_f16(acc[g][1], A[4], A[5], A[6], A[7], b0, b1);
           }
@@ -469,8 +479,9 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
       }
 #pragma unroll
       for (int g = 0; g < kSGGroups; ++g) {
-        if (g < n_valid) {
-          const uint2 sc = *reinterpret_cast<const uint2*>(sgp + kSG_Scales + g * (kD * 2) + (32 * warp + 4 * hd) * 2);
+        {
+          uint2 sc = *reinterpret_cast<const uint2*>(sgp + kSG_Scales + g * (kD * 2) + (32 * warp + 4 * hd) * 2);
+          if (g >= n_valid) sc = make_uint2(0u, 0u);
           const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));
           const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));
           tot[0][0] += sa.x * acc[g][0][0]; tot[0][1] += sa.x * acc[g][0][1];
