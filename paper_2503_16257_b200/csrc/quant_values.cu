@@ -5,67 +5,152 @@
 
 namespace vidkv {
 
+__device__ __forceinline__ __half2 as_half2(uint32_t v) { return *reinterpret_cast<const __half2*>(&v); }
+
 // ---------------------------------------------------------------------------------
 // 1.58Quant (Eq. 6) of one supergroup = 5 groups x 32 stream tokens x 128 channels.
 // grid = (supergroups, slabs of one layer); block = 256 threads.
 // Stream position u of the unprotected tokens maps to token idx_rest[u] (identity when
-// no token is protected).  Byte (j, c) collects the digits of token j of each group.
+// no token is protected).
+//   stage   the 160 x 128 tile is copied to shared memory as it is (cp.async, 16 bytes a piece);
+//   pass 1  s = Mean |v| per (group, channel): thread = (channel pair, quarter of the group's
+//           tokens), float32 partial sums combined in a fixed order;
+//   pass 2  thread = one 32-bit word of the byte plane = (token pair, channel pair): the
+//           comparisons |v| > alpha run on two channels at a time against the smallest
+//           representable number above alpha = gamma * s, the five digits of a byte are
+//           chained in binary16 (exact, <= 242), and the byte code comes from a 243-entry table.
 // ---------------------------------------------------------------------------------
 constexpr int kSGTokens = kSGGroups * kG;   // 160
+constexpr int kVRowBytes = 288;             // 256 bytes of data + padding: rows two apart land 16 banks apart
+
+template <typename T> struct Simd2;
+template <> struct Simd2<__half> {
+  // 1.0 / 0.0 in binary16 per lane
+  static __device__ __forceinline__ uint32_t ge(uint32_t a, uint32_t b) {
+    const __half2 r = __hge2(*reinterpret_cast<const __half2*>(&a), *reinterpret_cast<const __half2*>(&b));
+    return *reinterpret_cast<const uint32_t*>(&r);
+  }
+  static __device__ __forceinline__ uint32_t le(uint32_t a, uint32_t b) {
+    const __half2 r = __hle2(*reinterpret_cast<const __half2*>(&a), *reinterpret_cast<const __half2*>(&b));
+    return *reinterpret_cast<const uint32_t*>(&r);
+  }
+  // smallest element value strictly above x >= 0
+  static __device__ __forceinline__ uint16_t above(float x) {
+    return static_cast<uint16_t>(__half_as_ushort(__float2half_rd(x)) + 1u);
+  }
+};
+template <> struct Simd2<__nv_bfloat16> {
+  // the comparison yields 1.0 in bfloat16 (0x3f80); keeping bits 10-13 turns it into binary16 1.0
+  static __device__ __forceinline__ uint32_t ge(uint32_t a, uint32_t b) {
+    const __nv_bfloat162 r = __hge2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+    return *reinterpret_cast<const uint32_t*>(&r) & 0x3c003c00u;
+  }
+  static __device__ __forceinline__ uint32_t le(uint32_t a, uint32_t b) {
+    const __nv_bfloat162 r = __hle2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+    return *reinterpret_cast<const uint32_t*>(&r) & 0x3c003c00u;
+  }
+  static __device__ __forceinline__ uint16_t above(float x) {
+    return static_cast<uint16_t>(__bfloat16_as_ushort(__float2bfloat16_rd(x)) + 1u);
+  }
+};
+
+__device__ __forceinline__ void cp_async16_v(void* smem_dst, const void* gmem_src) {
+  const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
 
 template <typename T>
 __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest, CacheView cv, int layer,
                                                         SelView sel, float gamma) {
-  __shared__ __align__(16) uint16_t tile[kSGTokens * kD];      // raw 16-bit elements, 40 KB
-  __shared__ float s_alpha[kSGGroups * kD];
+  extern __shared__ __align__(16) uint8_t vsm[];
+  uint8_t* tile = vsm;                                                         // [160][288]
+  float* part = reinterpret_cast<float*>(tile + kSGTokens * kVRowBytes);       // [5][4][128]
+  uint32_t* thr = reinterpret_cast<uint32_t*>(part + kSGGroups * 4 * kD);      // [5][64] threshold pairs
+  uint8_t* lut = reinterpret_cast<uint8_t*>(thr + kSGGroups * 64);             // [256]
+  const int tid = threadIdx.x;
   const int slab = blockIdx.y;
   const int b = slab / cv.H_kv, h = slab % cv.H_kv;
   const T* base = reinterpret_cast<const T*>(src.ptr) + b * src.stride_b + h * src.stride_h;
   const int64_t u0 = static_cast<int64_t>(blockIdx.x) * kSGTokens;
   const int n_rows = static_cast<int>(min(static_cast<int64_t>(kSGTokens), n_rest - u0));
   const int32_t* idx = sel.idx_rest ? sel.idx_rest + b * sel.stride_rest : nullptr;
-  {
-    const int lane16 = threadIdx.x & 15, row = threadIdx.x >> 4;
-    for (int r = row; r < kSGTokens; r += 16) {
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (r < n_rows) {
-        const int64_t t = idx ? idx[u0 + r] : (u0 + r);
-        v = __ldg(reinterpret_cast<const uint4*>(base + t * src.stride_t) + lane16);
-      }
-      reinterpret_cast<uint4*>(tile + r * kD)[lane16] = v;
+  // ---- stage (rows past the end of the stream are zero: their trits come out 0)
+  for (int i = tid; i < kSGTokens * 16; i += 256) {
+    const int row = i >> 4, piece = i & 15;
+    uint8_t* dst = tile + row * kVRowBytes + piece * 16;
+    if (row < n_rows) {
+      const int64_t t = idx ? idx[u0 + row] : (u0 + row);
+      cp_async16_v(dst, reinterpret_cast<const uint8_t*>(base + t * src.stride_t) + piece * 16);
+    } else {
+      *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
     }
   }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  if (tid < 243) lut[tid] = static_cast<uint8_t>(trit_byte_encode(tid));
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
   uint8_t* sg = cv.slab(layer, b, h) + cv.tern_offset + static_cast<int64_t>(blockIdx.x) * kSGBytes;
-  // pass 1: s = Mean |v| per (group, channel), sequential over the tokens present
-  for (int item = threadIdx.x; item < kSGGroups * kD; item += 256) {
-    const int c = item & (kD - 1), g = item >> 7;
-    const int n = max(0, min(kG, n_rows - g * kG));
-    float sum = 0.0f;
-    for (int j = 0; j < n; ++j) sum += fabsf(Elem<T>::to_float(reinterpret_cast<const T*>(tile)[(g * kG + j) * kD + c]));
-    float alpha = 0.0f;
-    if (n > 0) {
-      const uint16_t sh = f2h_bits(__fdiv_rn(sum, static_cast<float>(n)));
-      reinterpret_cast<uint16_t*>(sg + kSG_Scales)[g * kD + c] = sh;
-      alpha = __fmul_rn(gamma, h2f(sh));
-    }
-    s_alpha[item] = alpha;
-  }
-  __syncthreads();
-  // pass 2: digits and bytes
-  for (int item = threadIdx.x; item < kG * kD; item += 256) {
-    // item enumerates the bytes of the plane in storage order (the inverse of tern_byte_offset)
-    const int j = 2 * (8 * ((item >> 11) & 1) + 4 * ((item >> 10) & 1) + ((item >> 6) & 3)) + (item & 1);
-    const int c = 32 * ((item >> 8) & 3) + 4 * ((item >> 3) & 7) + ((item >> 1) & 3);
-    uint32_t bval = 0;
+  // ---- pass 1: partial sums of |v| over 8 tokens
+  {
+    const int cp = tid & 63, q = tid >> 6;
 #pragma unroll
     for (int g = 0; g < kSGGroups; ++g) {
-      const float v = Elem<T>::to_float(reinterpret_cast<const T*>(tile)[(g * kG + j) * kD + c]);
-      const float a = s_alpha[g * kD + c];
-      const uint32_t d = (g * kG + j < n_rows) ? (v > a ? 2u : (v < -a ? 0u : 1u)) : 1u;
-      bval = bval * 3u + d;
+      float a0 = 0.0f, a1 = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(tile + (g * kG + q * 8 + j) * kVRowBytes + cp * 4);
+        const float2 f = Elem<T>::to_float2(w);
+        a0 += fabsf(f.x); a1 += fabsf(f.y);
+      }
+      *reinterpret_cast<float2*>(part + (g * 4 + q) * kD + 2 * cp) = make_float2(a0, a1);
     }
-    sg[item] = static_cast<uint8_t>(trit_byte_encode(bval));
+  }
+  __syncthreads();
+  for (int item = tid; item < kSGGroups * kD; item += 256) {
+    const int c = item & (kD - 1), g = item >> 7;
+    const int n = max(0, min(kG, n_rows - g * kG));
+    uint16_t a = 1u;                                   // empty group: every v is 0, nothing exceeds it
+    if (n > 0) {
+      const float* pp = part + g * 4 * kD + c;
+      const float sum = ((pp[0] + pp[kD]) + pp[2 * kD]) + pp[3 * kD];
+      const uint16_t sh = f2h_bits(__fdiv_rn(sum, static_cast<float>(n)));
+      reinterpret_cast<uint16_t*>(sg + kSG_Scales)[g * kD + c] = sh;
+      a = Simd2<T>::above(__fmul_rn(gamma, h2f(sh)));
+    }
+    reinterpret_cast<uint16_t*>(thr)[item] = a;
+  }
+  __syncthreads();
+  // ---- pass 2: one word of the plane per thread and step
+#pragma unroll 1
+  for (int wd = tid; wd < kG * kD / 4; wd += 256) {
+    const int cp = 16 * ((wd >> 6) & 3) + 2 * ((wd >> 1) & 7) + (wd & 1);
+    const int m = 8 * ((wd >> 9) & 1) + 4 * ((wd >> 8) & 1) + ((wd >> 4) & 3);
+    uint32_t b0 = 0u, b1 = 0u;                        // binary16 pairs (even channel, odd channel) of tokens 2m, 2m+1
+    const uint32_t three = 0x42004200u, one = 0x3c003c00u;
+#pragma unroll
+    for (int g = 0; g < kSGGroups; ++g) {
+      const uint32_t A = thr[g * 64 + cp], nA = A ^ 0x80008000u;
+      const uint8_t* rp = tile + (g * kG + 2 * m) * kVRowBytes + cp * 4;
+      const uint32_t v0 = *reinterpret_cast<const uint32_t*>(rp);
+      const uint32_t v1 = *reinterpret_cast<const uint32_t*>(rp + kVRowBytes);
+      // digit = 1 + [v > alpha] - [v < -alpha]
+      __half2 d0 = __hsub2(__hadd2(*reinterpret_cast<const __half2*>(&one), as_half2(Simd2<T>::ge(v0, A))), as_half2(Simd2<T>::le(v0, nA)));
+      __half2 d1 = __hsub2(__hadd2(*reinterpret_cast<const __half2*>(&one), as_half2(Simd2<T>::ge(v1, A))), as_half2(Simd2<T>::le(v1, nA)));
+      const __half2 t0 = __hfma2(as_half2(b0), *reinterpret_cast<const __half2*>(&three), d0);
+      const __half2 t1 = __hfma2(as_half2(b1), *reinterpret_cast<const __half2*>(&three), d1);
+      b0 = *reinterpret_cast<const uint32_t*>(&t0);
+      b1 = *reinterpret_cast<const uint32_t*>(&t1);
+    }
+    // 1024 + b puts the integer b into the low mantissa bits
+    const uint32_t k1024 = 0x64006400u;
+    const __half2 e0 = __hadd2(as_half2(b0), *reinterpret_cast<const __half2*>(&k1024));
+    const __half2 e1 = __hadd2(as_half2(b1), *reinterpret_cast<const __half2*>(&k1024));
+    const uint32_t x0 = *reinterpret_cast<const uint32_t*>(&e0), x1 = *reinterpret_cast<const uint32_t*>(&e1);
+    // word bytes: (even ch, tok 2m), (even ch, tok 2m+1), (odd ch, tok 2m), (odd ch, tok 2m+1)
+    const uint32_t word = static_cast<uint32_t>(lut[x0 & 0xffu]) | (static_cast<uint32_t>(lut[x1 & 0xffu]) << 8) |
+                          (static_cast<uint32_t>(lut[(x0 >> 16) & 0xffu]) << 16) |
+                          (static_cast<uint32_t>(lut[(x1 >> 16) & 0xffu]) << 24);
+    reinterpret_cast<uint32_t*>(sg)[wd] = word;
   }
 }
 
@@ -316,7 +401,15 @@ static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheVi
   const int64_t n_rest = T_q - sel.n_prot;
   if (n_rest > 0) {
     const int64_t sgs = (n_rest + kSGTokens - 1) / kSGTokens;
-    v_ternary_kernel<T><<<dim3(static_cast<unsigned>(sgs), n_slabs), 256, 0, stream>>>(src, n_rest, cv, layer, sel, gamma);
+    const size_t smem = kSGTokens * kVRowBytes + sizeof(float) * kSGGroups * 4 * kD + sizeof(uint32_t) * kSGGroups * 64 + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+      cudaError_t e;
+      if ((e = cudaFuncSetAttribute(v_ternary_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+      if ((e = cudaFuncSetAttribute(v_ternary_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+      attr_set = true;
+    }
+    v_ternary_kernel<T><<<dim3(static_cast<unsigned>(sgs), n_slabs), 256, smem, stream>>>(src, n_rest, cv, layer, sel, gamma);
     count_launches(1);
   }
   if (sel.n_prot > 0) {
