@@ -30,6 +30,11 @@ __global__ void init_min_kernel(uint32_t* minmax, int n_slabs);
 cudaError_t launch_quantize_keys(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0,
                                  int n_layers, int chunk, int64_t kgroup0, uint32_t* minmax, cudaStream_t stream);
 
+// Encode pass of Algorithm 3 for `n_slabs` slabs whose channel split (chunk table entry
+// `chunk`) is already written.
+cudaError_t launch_encode_keys(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0, int n_slabs,
+                               int slabs_per_layer, int chunk, int64_t kgroup0, cudaStream_t stream);
+
 // Algorithm 2 on the prefill tokens of one layer.  T_q (multiple of 32) tokens; the
 // unprotected ones go to ternary stream positions 0.., the protected ones to 2-bit groups.
 cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer,

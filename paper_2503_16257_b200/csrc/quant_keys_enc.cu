@@ -1,0 +1,337 @@
+// Key encode pass of Algorithm 3 (MixQuant) for one tile of 128 tokens x 128 channels:
+//   normal channels   (Eq. 5) orthonormal 64-point DFT over the channel axis as a matrix
+//                     product on the tensor cores (A = the tile's values, binary16, exact;
+//                     B = the DFT matrix split into a binary16 leading part and a binary16
+//                     remainder, so that products carry 22 bits; float32 accumulation), then
+//                     the sign bit and the per-group mean |.| of every spectrum column;
+//   anomalous channels (Eq. 4) min / max per (32-token group, channel), s = (max - min) / 3,
+//                     z = min rounded to binary16, code = clamp(rint((x - z) / s), 0, 3).
+//                     The division is not done per element: code >= k is a monotone predicate
+//                     of x, so per (group, channel) the three smallest element values X_k with
+//                     code(X_k) >= k are found once with the defining float32 arithmetic, and
+//                     the elements are compared against them two at a time.
+// grid = (tiles of 128 tokens, slabs); block = 256 threads = 8 warps; each warp owns 16 tokens
+// in the DFT phase.
+#include <math.h>
+
+#include "common.cuh"
+#include "kernels.cuh"
+
+namespace vidkv {
+
+namespace {
+
+constexpr int kEncTokens = 128;
+constexpr int kRowBytes = 272;                 // 256 bytes of data + 16 of padding per staged token
+constexpr int kDftWords = 4 * 8 * 32 * 4;      // [k step][column tile][lane][hi0, hi1, lo0, lo1]
+
+// B fragments of the DFT matrix in the order the MMA wants them (see dft_table_kernel).
+__device__ __align__(16) uint32_t g_dft_frag[kDftWords];
+
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ __half2 as_h2(uint32_t v) { return *reinterpret_cast<const __half2*>(&v); }
+__device__ __forceinline__ uint32_t as_u32(__half2 v) { return *reinterpret_cast<const uint32_t*>(&v); }
+
+// Element-type helpers: raw 16-bit patterns in, binary16 1.0 / 0.0 pairs out of the comparison.
+template <typename T> struct Ops;
+template <> struct Ops<__half> {
+  static __device__ __forceinline__ float to_float(uint16_t b) { return __half2float(__ushort_as_half(b)); }
+  static __device__ __forceinline__ uint16_t from_float_rn(float f) { return __half_as_ushort(__float2half_rn(f)); }
+  static __device__ __forceinline__ uint16_t vmin(uint16_t a, uint16_t b) { return __half_as_ushort(__hmin(__ushort_as_half(a), __ushort_as_half(b))); }
+  static __device__ __forceinline__ uint16_t vmax(uint16_t a, uint16_t b) { return __half_as_ushort(__hmax(__ushort_as_half(a), __ushort_as_half(b))); }
+  static __device__ __forceinline__ uint32_t ge(uint32_t a, uint32_t b) { return as_u32(__hge2(as_h2(a), as_h2(b))); }
+  static __device__ __forceinline__ uint32_t to_half_pair(uint32_t raw) { return raw; }
+  static constexpr uint16_t kInf = 0x7c00u;
+};
+template <> struct Ops<__nv_bfloat16> {
+  static __device__ __forceinline__ float to_float(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
+  static __device__ __forceinline__ uint16_t from_float_rn(float f) { return __bfloat16_as_ushort(__float2bfloat16_rn(f)); }
+  static __device__ __forceinline__ uint16_t vmin(uint16_t a, uint16_t b) { return to_float(a) <= to_float(b) ? a : b; }
+  static __device__ __forceinline__ uint16_t vmax(uint16_t a, uint16_t b) { return to_float(a) >= to_float(b) ? a : b; }
+  static __device__ __forceinline__ uint32_t ge(uint32_t a, uint32_t b) {
+    const __nv_bfloat162 r = __hge2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+    return *reinterpret_cast<const uint32_t*>(&r) & 0x3c003c00u;   // bfloat16 1.0 -> binary16 1.0
+  }
+  static __device__ __forceinline__ uint32_t to_half_pair(uint32_t raw) {
+    const __half2 h = __floats2half2_rn(__uint_as_float(raw << 16), __uint_as_float(raw & 0xffff0000u));
+    return as_u32(h);
+  }
+  static constexpr uint16_t kInf = 0x7f80u;
+};
+
+// Value order of 16-bit sign-magnitude patterns as integers (both zeros map to 0).
+__device__ __forceinline__ int ord_of(uint16_t b) { return (b & 0x8000u) ? -static_cast<int>(b & 0x7fffu) : static_cast<int>(b); }
+__device__ __forceinline__ uint16_t bits_of(int o) { return o >= 0 ? static_cast<uint16_t>(o) : static_cast<uint16_t>(0x8000u | static_cast<uint32_t>(-o)); }
+
+// Eq. 4 for one element, in the defining arithmetic (float32, IEEE division, round half to even).
+template <typename T>
+__device__ __forceinline__ int code_ref(int o, float z, float s) {
+  const float d = __fsub_rn(Ops<T>::to_float(bits_of(o)), z);
+  const float q = fminf(fmaxf(rintf(__fdiv_rn(d, s)), 0.0f), 3.0f);
+  return static_cast<int>(q);
+}
+
+}  // namespace
+
+// One block of 256 threads, 4 table words per thread.  Word layout for k step ks, column tile
+// nt and lane (n = lane / 4, r = lane % 4): rows k0 = 16 ks + 2 r (and k0 + 1; k0 + 8, k0 + 9)
+// of column f = 16 (n / 2) + 2 nt + (n % 2), so that after the product lane (., r) holds the
+// spectrum columns 16 r .. 16 r + 15 of its two tokens.  Column f of the matrix: f = 0: 1/8;
+// f = 1: (-1)^c / 8; f = 2k: cos(2 pi k c / 64) / 8; f = 2k + 1: -sin(2 pi k c / 64) / 8.
+__global__ void dft_table_kernel() {
+  for (int i = threadIdx.x; i < kDftWords / 4; i += blockDim.x) {
+    const int lane = i & 31, nt = (i >> 5) & 7, ks = i >> 8;
+    const int n = lane >> 2, r = lane & 3;
+    const int f = 16 * (n >> 1) + 2 * nt + (n & 1);
+    float w[4];
+    const int rows[4] = {16 * ks + 2 * r, 16 * ks + 2 * r + 1, 16 * ks + 2 * r + 8, 16 * ks + 2 * r + 9};
+    for (int j = 0; j < 4; ++j) {
+      const int c = rows[j];
+      double v;
+      if (f == 0) v = 1.0;
+      else if (f == 1) v = (c & 1) ? -1.0 : 1.0;
+      else {
+        double sn, cs;
+        sincospi(static_cast<double>(((f >> 1) * c) & 63) / 32.0, &sn, &cs);
+        v = (f & 1) ? -sn : cs;
+      }
+      w[j] = static_cast<float>(v * 0.125);
+    }
+    const __half h0 = __float2half_rn(w[0]), h1 = __float2half_rn(w[1]), h2 = __float2half_rn(w[2]), h3 = __float2half_rn(w[3]);
+    g_dft_frag[i * 4 + 0] = as_u32(__halves2half2(h0, h1));
+    g_dft_frag[i * 4 + 1] = as_u32(__halves2half2(h2, h3));
+    g_dft_frag[i * 4 + 2] = as_u32(__floats2half2_rn(w[0] - __half2float(h0), w[1] - __half2float(h1)));
+    g_dft_frag[i * 4 + 3] = as_u32(__floats2half2_rn(w[2] - __half2float(h2), w[3] - __half2float(h3)));
+  }
+}
+
+size_t k_encode_smem_bytes() {
+  return kEncTokens * kRowBytes + kDftWords * 4 + 4 * 3 * 32 * 4 + 8 * 64 * 4 + kD;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_tokens, CacheView cv, int layer0,
+                                                       int slabs_per_layer, int chunk, int64_t kgroup0) {
+  extern __shared__ __align__(16) uint8_t esm[];
+  uint8_t* tile = esm;                                                      // [128][272] raw elements
+  uint32_t* dft = reinterpret_cast<uint32_t*>(tile + kEncTokens * kRowBytes);   // DFT fragments
+  uint32_t* thr = dft + kDftWords;                                          // [4][3][32] threshold pairs
+  float* colsum = reinterpret_cast<float*>(thr + 4 * 3 * 32);               // [8][64]
+  uint8_t* perm = reinterpret_cast<uint8_t*>(colsum + 8 * 64);              // [128]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int slab = blockIdx.y;
+  const int layer = layer0 + slab / slabs_per_layer;
+  const int bh = slab % slabs_per_layer;
+  const T* base = reinterpret_cast<const T*>(src.ptr) + (slab / src.H) * src.stride_b + (slab % src.H) * src.stride_h;
+  uint8_t* slab_ptr = cv.slab(layer, bh / cv.H_kv, bh % cv.H_kv);
+  const int64_t t0 = static_cast<int64_t>(blockIdx.x) * kEncTokens;
+  const int n_tok = static_cast<int>(min(static_cast<int64_t>(kEncTokens), T_tokens - t0));   // multiple of 32
+  const int n_groups = n_tok / kG;
+  uint8_t* kg_base = slab_ptr + cv.kgroup_offset + (kgroup0 + t0 / kG) * kKGroupBytes;
+
+  // ---- stage the tile and the DFT fragments
+  for (int i = tid; i < n_tok * 16; i += 256) {
+    const int row = i >> 4, piece = i & 15;
+    cp_async16(tile + row * kRowBytes + piece * 16,
+               reinterpret_cast<const uint8_t*>(base + (t0 + row) * src.stride_t) + piece * 16);
+  }
+  for (int i = tid; i < kDftWords / 4; i += 256) cp_async16(dft + i * 4, g_dft_frag + i * 4);
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  if (tid < kD) perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  // ---- A: Eq. 4 metadata and thresholds, thread = (anomalous slot j, group g)
+  {
+    const int j = tid & 63, g = tid >> 6;
+    if (g < n_groups) {
+      const uint8_t* p = tile + (g * kG) * kRowBytes + perm[j] * 2;
+      uint16_t mn = *reinterpret_cast<const uint16_t*>(p), mx = mn;
+#pragma unroll 8
+      for (int t = 1; t < kG; ++t) {
+        const uint16_t v = *reinterpret_cast<const uint16_t*>(p + t * kRowBytes);
+        mn = Ops<T>::vmin(mn, v); mx = Ops<T>::vmax(mx, v);
+      }
+      const float fmn = Ops<T>::to_float(mn), fmx = Ops<T>::to_float(mx);
+      const uint16_t sh = f2h_bits(__fdiv_rn(__fsub_rn(fmx, fmn), 3.0f));
+      const uint16_t zh = f2h_bits(fmn);
+      uint8_t* kg = kg_base + g * kKGroupBytes;
+      reinterpret_cast<uint16_t*>(kg + kKG_S2)[j] = sh;
+      reinterpret_cast<uint16_t*>(kg + kKG_Z2)[j] = zh;
+      const float s = h2f(sh), z = h2f(zh);
+      uint16_t* th = reinterpret_cast<uint16_t*>(thr + g * 3 * 32);
+#pragma unroll 1
+      for (int k = 1; k <= 3; ++k) {
+        uint16_t X = Ops<T>::kInf;                     // s == 0: every code is 0
+        if (s != 0.0f) {
+          int o = ord_of(Ops<T>::from_float_rn(fmaf(static_cast<float>(k) - 0.5f, s, z)));
+#pragma unroll 1
+          for (int it = 0; it < 4 && code_ref<T>(o, z, s) < k; ++it) ++o;
+#pragma unroll 1
+          for (int it = 0; it < 4 && code_ref<T>(o - 1, z, s) >= k; ++it) --o;
+          X = bits_of(o);
+        }
+        th[(k - 1) * 64 + j] = X;
+      }
+    }
+  }
+
+  // ---- B: DFT of the normal channels, warp = 16 tokens
+  const int hd = lane >> 2, r = lane & 3;
+  if (warp * 16 < n_tok) {
+    const uint8_t* row0 = tile + (warp * 16 + hd) * kRowBytes;
+    const uint8_t* row1 = row0 + 8 * kRowBytes;
+    uint32_t a[4][4];
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      const uint32_t pc = *reinterpret_cast<const uint16_t*>(perm + kNA + 16 * ks + 2 * r);        // two channel ids
+      const uint32_t pd = *reinterpret_cast<const uint16_t*>(perm + kNA + 16 * ks + 2 * r + 8);
+      const int c0 = (pc & 0xffu) * 2, c1 = (pc >> 8) * 2, c2 = (pd & 0xffu) * 2, c3 = (pd >> 8) * 2;
+      a[ks][0] = Ops<T>::to_half_pair(*reinterpret_cast<const uint16_t*>(row0 + c0) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row0 + c1)) << 16));
+      a[ks][1] = Ops<T>::to_half_pair(*reinterpret_cast<const uint16_t*>(row1 + c0) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row1 + c1)) << 16));
+      a[ks][2] = Ops<T>::to_half_pair(*reinterpret_cast<const uint16_t*>(row0 + c2) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row0 + c3)) << 16));
+      a[ks][3] = Ops<T>::to_half_pair(*reinterpret_cast<const uint16_t*>(row1 + c2) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row1 + c3)) << 16));
+    }
+    float acc[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) { acc[nt][0] = 0.0f; acc[nt][1] = 0.0f; acc[nt][2] = 0.0f; acc[nt][3] = 0.0f; }
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const uint4 bw = *reinterpret_cast<const uint4*>(dft + ((ks * 8 + nt) * 32 + lane) * 4);
+        mma_f16(acc[nt], a[ks][0], a[ks][1], a[ks][2], a[ks][3], bw.x, bw.y);
+        mma_f16(acc[nt], a[ks][0], a[ks][1], a[ks][2], a[ks][3], bw.z, bw.w);
+      }
+    }
+    // sign bits: column e = 2 nt + c of half-word r goes to bit 15 - e; 1 = coefficient >= 0
+    uint32_t w0 = 0u, w1 = 0u;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        w0 = __funnelshift_l(__float_as_uint(acc[nt][c]), w0, 1);
+        w1 = __funnelshift_l(__float_as_uint(acc[nt][c + 2]), w1, 1);
+      }
+    }
+    const int g = warp >> 1, nt_tok = 2 * (warp & 1);
+    uint16_t* hw = reinterpret_cast<uint16_t*>(kg_base + g * kKGroupBytes + kKG_Bits1);
+    hw[(hd * 4 + r) * 4 + nt_tok] = static_cast<uint16_t>(~w0);
+    hw[(hd * 4 + r) * 4 + nt_tok + 1] = static_cast<uint16_t>(~w1);
+    // column sums of |X| over the warp's 16 tokens: reduce-scatter over the 8 lanes of equal r
+    float p[16];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      p[2 * nt] = fabsf(acc[nt][0]) + fabsf(acc[nt][2]);
+      p[2 * nt + 1] = fabsf(acc[nt][1]) + fabsf(acc[nt][3]);
+    }
+#pragma unroll
+    for (int width = 8, mask = 16; width >= 2; width >>= 1, mask >>= 1) {
+      const bool up = (lane & mask) != 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (i < width) {
+          const float send = up ? p[i] : p[i + width];
+          const float keep = up ? p[i + width] : p[i];
+          p[i] = keep + __shfl_xor_sync(0xffffffffu, send, mask);
+        }
+      }
+    }
+    const int e0 = ((lane & 16) ? 8 : 0) + ((lane & 8) ? 4 : 0) + ((lane & 4) ? 2 : 0);
+    colsum[warp * 64 + 16 * r + e0] = p[0];
+    colsum[warp * 64 + 16 * r + e0 + 1] = p[1];
+  }
+  __syncthreads();
+
+  // ---- C: s = Mean |X| per (group, column)
+  {
+    const int f = tid & 63, g = tid >> 6;
+    if (g < n_groups) {
+      const float sum = colsum[(2 * g) * 64 + f] + colsum[(2 * g + 1) * 64 + f];
+      reinterpret_cast<uint16_t*>(kg_base + g * kKGroupBytes + kKG_S1)[f] = f2h_bits(sum * (1.0f / 32.0f));
+    }
+  }
+
+  // ---- D: 2-bit codes, thread = one 32-bit word = (token, 16 slots), two words per thread
+  {
+    const int widx = tid & 127;
+    const int tl = widx >> 4, r4 = (widx >> 2) & 3, nt = widx & 3;
+    int cofs[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) cofs[i] = perm[16 * r4 + i] * 2;
+    const uint32_t k1024 = 0x64006400u;
+    const uint32_t wgt[4] = {0x3c003c00u, 0x44004400u, 0x4c004c00u, 0x54005400u};   // 1, 4, 16, 64
+#pragma unroll 1
+    for (int g = tid >> 7; g < n_groups; g += 2) {
+      const uint8_t* row = tile + (g * kG + 8 * nt + tl) * kRowBytes;
+      const uint32_t* th = thr + g * 3 * 32 + 8 * r4;
+      __half2 lo = as_h2(k1024), hi = as_h2(k1024);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint32_t v = *reinterpret_cast<const uint16_t*>(row + cofs[2 * i]) |
+                           (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row + cofs[2 * i + 1])) << 16);
+        const __half2 code = __hadd2(__hadd2(as_h2(Ops<T>::ge(v, th[i])), as_h2(Ops<T>::ge(v, th[32 + i]))),
+                                     as_h2(Ops<T>::ge(v, th[64 + i])));
+        if (i < 4) lo = __hfma2(code, as_h2(wgt[i & 3]), lo);
+        else hi = __hfma2(code, as_h2(wgt[i & 3]), hi);
+      }
+      // 1024 + n keeps n in the low byte of each lane: fields 0-3 and 4-7 of both half-words
+      uint32_t word;
+      asm("prmt.b32 %0, %1, %2, 0x6240;" : "=r"(word) : "r"(as_u32(lo)), "r"(as_u32(hi)));
+      reinterpret_cast<uint32_t*>(kg_base + g * kKGroupBytes + kKG_Codes2)[widx] = word;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// Host launcher of the encode pass
+// ---------------------------------------------------------------------------------
+template <typename T>
+static cudaError_t launch_encode_t(const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0, int n_slabs,
+                                   int slabs_per_layer, int chunk, int64_t kgroup0, cudaStream_t stream) {
+  cudaError_t e;
+  // the DFT fragments are written once per device, ordered before their first use on this stream
+  static bool table_done[64] = {};
+  int dev = 0;
+  if ((e = cudaGetDevice(&dev))) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!table_done[dev]) {
+    dft_table_kernel<<<1, 256, 0, stream>>>();
+    if ((e = cudaGetLastError())) return e;
+    // later calls may come on other streams: make the table visible to all of them
+    if ((e = cudaStreamSynchronize(stream))) return e;
+    table_done[dev] = true;
+    count_launches(1);
+  }
+  static bool attr_set = false;
+  const size_t smem = k_encode_smem_bytes();
+  if (!attr_set) {
+    if ((e = cudaFuncSetAttribute(k_encode_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    if ((e = cudaFuncSetAttribute(k_encode_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    attr_set = true;
+  }
+  const int64_t blocks = (T_tokens + kEncTokens - 1) / kEncTokens;
+  k_encode_kernel<T><<<dim3(static_cast<unsigned>(blocks), n_slabs), 256, smem, stream>>>(src, T_tokens, cv, layer0,
+                                                                                         slabs_per_layer, chunk, kgroup0);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_encode_keys(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0, int n_slabs,
+                               int slabs_per_layer, int chunk, int64_t kgroup0, cudaStream_t stream) {
+  if (dtype == VIDKV_F16) return launch_encode_t<__half>(src, T_tokens, cv, layer0, n_slabs, slabs_per_layer, chunk, kgroup0, stream);
+  return launch_encode_t<__nv_bfloat16>(src, T_tokens, cv, layer0, n_slabs, slabs_per_layer, chunk, kgroup0, stream);
+}
+
+}  // namespace vidkv
