@@ -116,7 +116,7 @@ __global__ void dft_table_kernel() {
 }
 
 size_t k_encode_smem_bytes() {
-  return kEncTokens * kRowBytes + kDftWords * 4 + 4 * 3 * 32 * 4 + 8 * 64 * 4 + kD;
+  return kEncTokens * kRowBytes + kDftWords * 4 + 4 * 3 * 32 * 4 + 8 * 64 * 4 + kD + 4 * 128 * 32;
 }
 
 template <typename T>
@@ -128,6 +128,8 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
   uint32_t* thr = dft + kDftWords;                                          // [4][3][32] threshold pairs
   float* colsum = reinterpret_cast<float*>(thr + 4 * 3 * 32);               // [8][64]
   uint8_t* perm = reinterpret_cast<uint8_t*>(colsum + 8 * 64);              // [128]
+  // anomalous values gathered per code word: [group][word of the group's 2-bit block][16 slots]
+  uint16_t* gath = reinterpret_cast<uint16_t*>(perm + kD);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int slab = blockIdx.y;
@@ -157,11 +159,15 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
     const int j = tid & 63, g = tid >> 6;
     if (g < n_groups) {
       const uint8_t* p = tile + (g * kG) * kRowBytes + perm[j] * 2;
+      // token t of the group goes to word ((t % 8) * 4 + j / 16) * 4 + t / 8, slot j % 16
+      uint16_t* gp = gath + (g * 128 + (j >> 4) * 4) * 16 + (j & 15);
       uint16_t mn = *reinterpret_cast<const uint16_t*>(p), mx = mn;
-#pragma unroll 8
+      gp[0] = mn;
+#pragma unroll
       for (int t = 1; t < kG; ++t) {
         const uint16_t v = *reinterpret_cast<const uint16_t*>(p + t * kRowBytes);
         mn = Ops<T>::vmin(mn, v); mx = Ops<T>::vmax(mx, v);
+        gp[((t & 7) * 16 + (t >> 3)) * 16] = v;
       }
       const float fmn = Ops<T>::to_float(mn), fmx = Ops<T>::to_float(mx);
       const uint16_t sh = f2h_bits(__fdiv_rn(__fsub_rn(fmx, fmn), 3.0f));
@@ -266,23 +272,24 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
   // ---- D: 2-bit codes, thread = one 32-bit word = (token, 16 slots), two words per thread
   {
     const int widx = tid & 127;
-    const int tl = widx >> 4, r4 = (widx >> 2) & 3, nt = widx & 3;
-    int cofs[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) cofs[i] = perm[16 * r4 + i] * 2;
+    const int r4 = (widx >> 2) & 3;
     const uint32_t k1024 = 0x64006400u;
     const uint32_t wgt[4] = {0x3c003c00u, 0x44004400u, 0x4c004c00u, 0x54005400u};   // 1, 4, 16, 64
 #pragma unroll 1
     for (int g = tid >> 7; g < n_groups; g += 2) {
-      const uint8_t* row = tile + (g * kG + 8 * nt + tl) * kRowBytes;
-      const uint32_t* th = thr + g * 3 * 32 + 8 * r4;
+      const uint4* gv = reinterpret_cast<const uint4*>(gath + (g * 128 + widx) * 16);
+      const uint4 v0 = gv[0], v1 = gv[1];
+      const uint32_t v[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+      const uint4* th = reinterpret_cast<const uint4*>(thr + g * 3 * 32 + 8 * r4);
+      uint32_t x1[8], x2[8], x3[8];
+      { const uint4 a0 = th[0], a1 = th[1]; x1[0] = a0.x; x1[1] = a0.y; x1[2] = a0.z; x1[3] = a0.w; x1[4] = a1.x; x1[5] = a1.y; x1[6] = a1.z; x1[7] = a1.w; }
+      { const uint4 a0 = th[8], a1 = th[9]; x2[0] = a0.x; x2[1] = a0.y; x2[2] = a0.z; x2[3] = a0.w; x2[4] = a1.x; x2[5] = a1.y; x2[6] = a1.z; x2[7] = a1.w; }
+      { const uint4 a0 = th[16], a1 = th[17]; x3[0] = a0.x; x3[1] = a0.y; x3[2] = a0.z; x3[3] = a0.w; x3[4] = a1.x; x3[5] = a1.y; x3[6] = a1.z; x3[7] = a1.w; }
       __half2 lo = as_h2(k1024), hi = as_h2(k1024);
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        const uint32_t v = *reinterpret_cast<const uint16_t*>(row + cofs[2 * i]) |
-                           (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row + cofs[2 * i + 1])) << 16);
-        const __half2 code = __hadd2(__hadd2(as_h2(Ops<T>::ge(v, th[i])), as_h2(Ops<T>::ge(v, th[32 + i]))),
-                                     as_h2(Ops<T>::ge(v, th[64 + i])));
+        const __half2 code = __hadd2(__hadd2(as_h2(Ops<T>::ge(v[i], x1[i])), as_h2(Ops<T>::ge(v[i], x2[i]))),
+                                     as_h2(Ops<T>::ge(v[i], x3[i])));
         if (i < 4) lo = __hfma2(code, as_h2(wgt[i & 3]), lo);
         else hi = __hfma2(code, as_h2(wgt[i & 3]), hi);
       }
