@@ -111,6 +111,9 @@ def _decode_steps(pair: Pair, n_steps, tol=TOL_ABS):
     ("tiny", 77, 2, 0.0, 5),
     ("tiny", 31, 1, 0.0, 3),
     ("qwen", 480, 2, 0.2, 4),
+    ("qwen", 480, 2, 0.0, 4),      # bf16 inputs without protection: the tensor-core kernel
+    ("tiny", 2000, 1, 0.0, 3),     # 1984 quantized tokens = 3.1 splits of 640, plus 16 residual tokens
+    ("tiny", 1300, 2, 0.0, 3),     # last split starts inside a supergroup (1280) and ends in the residual
 ])
 def test_decode_attention_parity(name, T, B, p, steps):
     pair = Pair(CONFIGS[name], T, B=B, L=1, p=p, max_new=steps).prefill()
@@ -124,6 +127,47 @@ def test_decode_parity_heavy_tailed():
     for _ in range(4):
         out, ref = pair.decode()
         assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
+
+
+def test_decode_parity_heavy_tailed_without_protection():
+    # Student-t keys and values through the tensor-core kernel, three splits
+    pair = Pair(CONFIGS["llava"], 1504, B=1, L=1, p=0.0, max_new=3).prefill()
+    for _ in range(3):
+        out, ref = pair.decode()
+        assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
+
+
+def test_full_size_slabs_in_the_benchmark_launch_shape():
+    """The benchmark's configuration (batched long video: T = 12544, batch 16, 640-token splits),
+    two layers in one call; the oracle recomputes four sampled (layer, batch, KV head) slabs."""
+    import paper_2503_16257_b200 as P
+    from workloads import make_layer_kv, make_step_inputs
+    wl = CONFIGS["batched"]
+    L, B, T, steps = 2, wl.batch, wl.T, 2
+    cfg = P.VidKVConfig(B=B, L=L, max_prefill_tokens=T, max_new_tokens=steps, p_ratio=0.0,
+                        in_dtype=P.VIDKV_F16, out_dtype=P.VIDKV_F32)
+    cache = P.VidKVCache(cfg, device="cuda")
+    samples = [(0, 0, 0), (0, 7, 2), (1, 15, 3), (1, 3, 1)]
+    slabs = {}
+    for layer in range(L):
+        K, V = make_layer_kv(wl, layer, "cuda")
+        cache.quantize_keys(layer, K)
+        cache.quantize_values(layer, V)
+        for (sl, b, h) in samples:
+            if sl == layer:
+                sc = O.SlabCache()
+                sc.prefill(to_np(K[b, h]), to_np(V[b, h]), None)
+                slabs[(sl, b, h)] = sc
+        del K, V
+    for step in range(steps):
+        q, k, v = (torch.stack(t) for t in zip(*[make_step_inputs(wl, layer, step, "cuda") for layer in range(L)]))
+        out = torch.empty((L, B, 28, 128), dtype=torch.float32, device="cuda")
+        cache.decode_attention(0, L, q, k, v, out)
+        out = out.cpu().numpy().astype(np.float64)
+        for (sl, b, h), sc in slabs.items():
+            ref = sc.decode_step(to_np(q[sl, b, 7 * h:7 * h + 7]), to_np(k[sl, b, h]), to_np(v[sl, b, h]))
+            assert np.abs(out[sl, b, 7 * h:7 * h + 7] - ref).max() <= TOL_ABS
+    assert cache.status() == 0
 
 
 def test_residual_flush_parity():
