@@ -62,8 +62,10 @@
  *                               ((((kt*2 + u)*4 + w)*4 + r)*8 + rho)*8 + 2 e + parity;
  *                    [4096,5376) s (binary16) [5][128].
  *     protected groups (STP) : per 32 protected tokens 1536 bytes:
- *                    [0,1024) 2-bit codes, token j at 32*j, channel c in word
- *                    c/16 at bits 2*(c%16); [1024,1280) s; [1280,1536) z.
+ *                    [0,1024) 2-bit codes as 256 32-bit words: with token
+ *                    j = 16 kt + 8 u + 2 r + hf of the group and channel c = 32 w + 4 rho + e
+ *                    the code is in word ((kt*4 + w)*4 + r)*8 + rho at bits
+ *                    2 (4 u + e) + 16 hf; [1024,1280) s; [1280,1536) z.
  *     residual     : K_r and V_r, 128 x 128 elements each, in in_dtype.
  *   per batch element: the protection mask E as bit words plus, per word, the
  *   number of protected tokens before it.
@@ -223,8 +225,8 @@ vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* handle, int32_t layer, flo
  * The split-KV scratch lives in a 16 MiB array inside the library, which every GPU that
  * loads the library keeps until the process exits.  It must hold 520 bytes per (query head,
  * split) record, n_layers * B * H_q * ceil(tokens / split) of them with split = 160, 320 or
- * 640 tokens, plus, when n_protected is 0, 3072 bytes per (layer, batch element, KV head,
- * chunk) -- larger problems return VIDKV_ERR_CAPACITY (use fewer layers per call).
+ * 640 tokens (320 at most when n_protected > 0), plus 3072 bytes per (layer, batch element,
+ * KV head, chunk) -- larger problems return VIDKV_ERR_CAPACITY (use fewer layers per call).
  * Nothing is allocated or freed.  The first call on each device looks up the array's device
  * address, so make that first call outside any stream capture.  All calls share the array:
  * two calls whose kernels may overlap on the GPU (different streams, no ordering) race on it;

@@ -105,6 +105,15 @@ __host__ __device__ __forceinline__ int k2_bit(int j) { return 2 * ((j & 15) >> 
 // the 16-bit half-word with the same index as the 2-bit word above, at bit 15 - e.
 __host__ __device__ __forceinline__ int k1_half_index(int t, int f) { return ((t & 7) * 4 + (f >> 4)) * 4 + (t >> 3); }
 __host__ __device__ __forceinline__ int k1_bit(int f) { return 15 - (f & 15); }
+// 2-bit codes of one protected (STP) value group (1024 bytes = 256 words): protected token
+// j = 16 kt + 8 u + 2 r + hf of the group, channel c = 32 w + 4 rho + e.  Word
+// ((kt * 4 + w) * 4 + r) * 8 + rho holds 4 channels x 4 tokens: the code sits at bit
+// 2 (4 u + e) + 16 hf, so the low half-word belongs to an even token, the high one to the
+// next token, and one word yields the eight operand registers of one 16-token MMA step.
+__host__ __device__ __forceinline__ int prot_word_index(int j, int c) {
+  return ((((j >> 4) * 4 + (c >> 5)) * 4 + ((j >> 1) & 3)) * 8) + ((c >> 2) & 7);
+}
+__host__ __device__ __forceinline__ int prot_bit(int j, int c) { return 2 * (4 * ((j >> 3) & 1) + (c & 3)) + 16 * (j & 1); }
 __host__ __device__ __forceinline__ int trit_digit(uint32_t b, int slot) {
   const uint32_t p3[5] = {81u, 27u, 9u, 3u, 1u};
   return static_cast<int>((b / p3[slot]) % 3u);

@@ -215,64 +215,49 @@ __global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int
 }
 
 // ---------------------------------------------------------------------------------
-// Shared memory of the attention kernel, for a split of ST tokens (a multiple of 160):
-//   kbuf  ST/32 key groups           (reused for the output staging after phase 1)
-//   vbuf  ST/160 ternary supergroups
-//   S     8 rows of ST + 4 floats: scores, then binary16 probabilities in place
-//   psum  [ST/32][8]  -5 * (sum of the rounded probabilities of the group)
-//   red   [16]        row maxima and sums
+// Per-thread view of one split: which tokens it covers and where its slab lives.
 // ---------------------------------------------------------------------------------
-size_t decode_mma_smem_bytes(int ST) {
-  return static_cast<size_t>(ST / 32) * kKGroupBytes + static_cast<size_t>(ST / 160) * kSGBytes +
-         sizeof(float) * (8 * (ST + 4) + 8 * (ST / 32) + 16);
+struct Split {
+  int tid, lane, warp, hd, r;             // hd = lane / 4 (MMA row group), r = lane % 4
+  uint32_t m_field, c_four, m_sign, c_neg1;
+  int split, slab, h, lb, rep;
+  const uint8_t* slab_ptr;
+  int64_t T_q0, T_qt, t0, t1, tq1, gk0;   // prefill-quantized / all quantized tokens; split range; first key group
+  int n_loc, nq, n_kg;                    // tokens, quantized tokens, key groups in the split
+};
+
+__device__ __forceinline__ Split make_split(const DecodeArgs& a) {
+  Split c;
+  c.tid = threadIdx.x; c.lane = c.tid & 31; c.warp = c.tid >> 5; c.hd = c.lane >> 2; c.r = c.lane & 3;
+  c.m_field = kExpand[0]; c.c_four = kExpand[1]; c.m_sign = kExpand[2]; c.c_neg1 = kExpand[3];
+  c.split = blockIdx.x; c.slab = blockIdx.y;
+  const CacheView& cv = a.cv;
+  c.h = c.slab % cv.H_kv; c.lb = c.slab / cv.H_kv; c.rep = cv.rep;
+  c.slab_ptr = cv.slab(a.layer0 + c.lb / cv.B, c.lb % cv.B, c.h);
+  c.T_q0 = a.st.T_q0;
+  c.T_qt = c.T_q0 + a.st.n_flush * kR;
+  const int64_t T_tot = c.T_qt + a.st.n_res;
+  c.t0 = static_cast<int64_t>(c.split) * a.split_tokens;
+  c.t1 = min(c.t0 + a.split_tokens, T_tot);
+  c.tq1 = max(min(c.t1, c.T_qt), c.t0);
+  c.n_loc = static_cast<int>(c.t1 - c.t0);
+  c.nq = static_cast<int>(c.tq1 - c.t0);
+  c.n_kg = c.nq / kG;
+  c.gk0 = c.t0 / kG;
+  return c;
 }
 
+// Phase 1: raw scores q . k (before the softmax scale) of every token of the split into
+// S[head][token - t0]: the packed key groups staged in kbuf, then the FP16 / BF16 residual rows.
 template <typename T>
-__global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, int n_chunks) {
-  extern __shared__ __align__(16) uint8_t smem_raw[];
-  const int ST = a.split_tokens;
-  const int SS = ST + 4;                                  // row stride of S in floats
-  uint8_t* kbuf = smem_raw;
-  uint8_t* vbuf = kbuf + (ST / 32) * kKGroupBytes;
-  float* S = reinterpret_cast<float*>(vbuf + (ST / 160) * kSGBytes);
-  float* psum = S + 8 * SS;
-  float* red = psum + 8 * (ST / 32);
-
+__device__ __forceinline__ void score_phase(const DecodeArgs& a, int n_chunks, const Split& c, const uint8_t* kbuf,
+                                            float* S, int SS) {
   const CacheView& cv = a.cv;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int hd = lane >> 2, r = lane & 3;
-  const uint32_t m_field = kExpand[0], c_four = kExpand[1], m_sign = kExpand[2], c_neg1 = kExpand[3];
-  const int split = blockIdx.x, slab = blockIdx.y;
-  const int h = slab % cv.H_kv, lb = slab / cv.H_kv;
-  const int b = lb % cv.B, layer_idx = lb / cv.B;
-  const int rep = cv.rep;
-  const uint8_t* slab_ptr = cv.slab(a.layer0 + layer_idx, b, h);
-
-  const int64_t T_q0 = a.st.T_q0;
-  const int64_t T_qt = T_q0 + a.st.n_flush * kR;          // quantized tokens (multiple of 32)
-  const int64_t T_tot = T_qt + a.st.n_res;
-  const int64_t t0 = static_cast<int64_t>(split) * ST;
-  const int64_t t1 = min(t0 + ST, T_tot);
-  const int64_t tq1 = max(min(t1, T_qt), t0);             // end of the quantized part of this split
-  const int n_loc = static_cast<int>(t1 - t0);
-  const int nq = static_cast<int>(tq1 - t0);              // quantized tokens here (multiple of 32)
-  const int n_kg = nq / kG;                               // key groups = ternary groups (p = 0)
-  const int n_sg = (n_kg + kSGGroups - 1) / kSGGroups;
-  const int64_t gk0 = t0 / kG;
-
-  // ---- stage the packed split
-  {
-    const uint8_t* ksrc = slab_ptr + cv.kgroup_offset + gk0 * kKGroupBytes;
-    for (int i = tid; i < n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
-    cp_async_commit();
-    const uint8_t* vsrc = slab_ptr + cv.tern_offset + (t0 / (kG * kSGGroups)) * kSGBytes;
-    for (int i = tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
-    cp_async_commit();
-  }
-
-  // ================= phase 1: scores =================
-  cp_async_wait<1>();
-  __syncthreads();
+  const int lane = c.lane, warp = c.warp, hd = c.hd, r = c.r, slab = c.slab, h = c.h, lb = c.lb, rep = c.rep;
+  const uint32_t m_field = c.m_field, c_four = c.c_four, m_sign = c.m_sign, c_neg1 = c.c_neg1;
+  const uint8_t* slab_ptr = c.slab_ptr;
+  const int64_t T_q0 = c.T_q0, T_qt = c.T_qt, t0 = c.t0, t1 = c.t1, gk0 = c.gk0;
+  const int n_kg = c.n_kg;
   {
     const int64_t g0n = T_q0 / kG;                        // key groups of the prefill chunk
     int cur_chunk = -1;
@@ -377,67 +362,20 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
       if (c0 + 1 < r_end) srow[c0 + 1] = acc[1];
     }
   }
-  __syncthreads();
+}
 
-  // ================= softmax numerators, in place as binary16 =================
+// Phase 2, ternary stream: tot[i][.] += sum over n_sg staged supergroups of s * (P V) for the
+// warp's 32 channels.  prow = this lane's probability row (binary16), its entry 0 matching
+// token 0 of the first staged supergroup; psum = -5 * group sums of those probabilities,
+// [group][8 heads]; groups from n_grp on do not exist (zero scale).
+__device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbuf, int n_sg, int n_grp,
+                                              const uint8_t* prow, const float* psum, float (&tot)[2][4]) {
+  const int warp = c.warp, hd = c.hd, r = c.r;
+  const uint32_t m_field = c.m_field, c_four = c.c_four;
   {
-    const float sl2 = a.scale * 1.4426950408889634f;
-    const int n_pad = max(n_sg * kSGGroups * kG, (n_loc + 1) & ~1);      // entries the P V loops may read
-    constexpr int kMaxPairs = 10;                                          // ST <= 640: 320 pairs per row
-#pragma unroll 1
-    for (int hh = 0; hh < 2; ++hh) {
-      const int row_h = warp * 2 + hh;
-      float* row = S + row_h * SS;
-      float2 v[kMaxPairs];
-      float m = -INFINITY;
-#pragma unroll
-      for (int k = 0; k < kMaxPairs; ++k) {
-        const int i = 2 * lane + 64 * k;
-        v[k] = i < n_loc ? *reinterpret_cast<const float2*>(row + i) : make_float2(-INFINITY, -INFINITY);
-        if (i + 1 >= n_loc) v[k].y = -INFINITY;
-        m = fmaxf(m, fmaxf(v[k].x, v[k].y));
-      }
-#pragma unroll
-      for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-      __syncwarp();
-      const float ms = m * sl2;
-      float l = 0.0f;
-      uint32_t* prow = reinterpret_cast<uint32_t*>(row);
-#pragma unroll
-      for (int k = 0; k < kMaxPairs; ++k) {
-        const int i = 2 * lane + 64 * k;
-        const float p0 = ex2_approx(fmaf(v[k].x, sl2, -ms)), p1 = ex2_approx(fmaf(v[k].y, sl2, -ms));
-        l += p0 + p1;
-        if (i < n_pad) prow[i >> 1] = pack_half2(p0, p1);
-      }
-#pragma unroll
-      for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-      if (lane == 0) { red[row_h] = m * a.scale; red[8 + row_h] = l; }
-    }
-  }
-  __syncthreads();
-  // -5 * sum of the rounded probabilities of every (group, head)
-  for (int i = tid; i < n_sg * kSGGroups * 8; i += kThreads) {
-    const int g = i >> 3, hh = i & 7;
-    const __half2* pr = reinterpret_cast<const __half2*>(reinterpret_cast<const __half*>(S + hh * SS) + g * kG);
-    float s = 0.0f;
-#pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      const float2 f = __half22float2(pr[k]);
-      s += f.x + f.y;
-    }
-    psum[g * 8 + hh] = -5.0f * s;
-  }
-
-  // ================= phase 2: P V =================
-  cp_async_wait<0>();
-  __syncthreads();
-  float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
-  {
-    const uint8_t* prow = reinterpret_cast<const uint8_t*>(S + hd * SS);
     for (int sg = 0; sg < n_sg; ++sg) {
       const uint8_t* sgp = vbuf + sg * kSGBytes;
-      const int n_valid = min(kSGGroups, n_kg - sg * kSGGroups);
+      const int n_valid = min(kSGGroups, n_grp - sg * kSGGroups);
       float acc[kSGGroups][2][4];
       float2 ps[kSGGroups];
 #pragma unroll
@@ -492,6 +430,17 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
       }
     }
   }
+}
+
+// Epilogue: stage tot as O[head][channel], add the residual rows' P V (probabilities of the
+// residual tokens sit in S in place, binary16, token order), write the split's partial record.
+template <typename T>
+__device__ __forceinline__ void epilogue(const DecodeArgs& a, const Split& c, uint8_t* kbuf, const float* S, int SS,
+                                         const float* red, const float (&tot)[2][4]) {
+  const CacheView& cv = a.cv;
+  const int tid = c.tid, warp = c.warp, hd = c.hd, r = c.r, h = c.h, lb = c.lb, rep = c.rep, split = c.split;
+  const uint8_t* slab_ptr = c.slab_ptr;
+  const int64_t T_qt = c.T_qt, t0 = c.t0, t1 = c.t1;
   // ---- output staging: O[head][channel] (reuses the key buffer, free since phase 1; the
   // smallest split, 160 tokens, has 5 x 1152 bytes there, more than the 4096 needed)
   float* O = reinterpret_cast<float*>(kbuf);
@@ -534,16 +483,294 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
   }
 }
 
+// Softmax numerators of the 8 score rows (warp w owns rows 2 w and 2 w + 1): p = exp(scale *
+// (score - row max)), rounded to binary16.  Without protected tokens the probabilities
+// replace the scores in place (entry i of the row, as binary16).  With them (STP) the
+// quantized tokens [0, nq) are scattered into the stream-ordered rows Ptern / Pprot through
+// `map` (bit 15 = protected stream) and only the residual tokens [nq, n_loc) stay in place.
+// red[row] = scaled row maximum, red[8 + row] = sum of the probabilities.
+template <bool STP>
+__device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& c, float* S, int SS, float* red,
+                                              int n_pad, const uint16_t* map, __half* Ptern, int PT, __half* Pprot,
+                                              int PP) {
+  const int lane = c.lane, n_loc = c.n_loc;
+  const float sl2 = a.scale * 1.4426950408889634f;
+  constexpr int kMaxPairs = 10;                                          // ST <= 640: 320 pairs per row
+#pragma unroll 1
+  for (int hh = 0; hh < 2; ++hh) {
+    const int row_h = c.warp * 2 + hh;
+    float* row = S + row_h * SS;
+    float2 v[kMaxPairs];
+    float m = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < kMaxPairs; ++k) {
+      const int i = 2 * lane + 64 * k;
+      v[k] = i < n_loc ? *reinterpret_cast<const float2*>(row + i) : make_float2(-INFINITY, -INFINITY);
+      if (i + 1 >= n_loc) v[k].y = -INFINITY;
+      m = fmaxf(m, fmaxf(v[k].x, v[k].y));
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    __syncwarp();
+    const float ms = m * sl2;
+    float l = 0.0f;
+    uint32_t* prow = reinterpret_cast<uint32_t*>(row);
+#pragma unroll
+    for (int k = 0; k < kMaxPairs; ++k) {
+      const int i = 2 * lane + 64 * k;
+      const float p0 = ex2_approx(fmaf(v[k].x, sl2, -ms)), p1 = ex2_approx(fmaf(v[k].y, sl2, -ms));
+      l += p0 + p1;
+      if (STP && i < c.nq) {
+        const uint32_t d = *reinterpret_cast<const uint32_t*>(map + i);
+        const uint32_t d0 = d & 0xffffu, d1 = d >> 16;
+        __half* q0 = (d0 & 0x8000u) ? Pprot + row_h * PP + (d0 & 0x7fffu) : Ptern + row_h * PT + d0;
+        __half* q1 = (d1 & 0x8000u) ? Pprot + row_h * PP + (d1 & 0x7fffu) : Ptern + row_h * PT + d1;
+        *q0 = __float2half_rn(p0);
+        *q1 = __float2half_rn(p1);
+      } else if (i < n_pad) {
+        prow[i >> 1] = pack_half2(p0, p1);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    if (lane == 0) { red[row_h] = m * a.scale; red[8 + row_h] = l; }
+  }
+}
+
+// out[g * 8 + head] = factor * sum of the 32 binary16 entries of group g of every row
+__device__ __forceinline__ void group_sums(const Split& c, const __half* P, int row_stride, int n_groups, float factor,
+                                           float* out) {
+  for (int i = c.tid; i < n_groups * 8; i += kThreads) {
+    const int g = i >> 3, hh = i & 7;
+    const __half2* pr = reinterpret_cast<const __half2*>(P + hh * row_stride + g * kG);
+    float s = 0.0f;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      const float2 f = __half22float2(pr[k]);
+      s += f.x + f.y;
+    }
+    out[i] = factor * s;
+  }
+}
+
+// ---------------------------------------------------------------------------------
+// Caches without protected tokens.  Shared memory for a split of ST tokens (a multiple of 160):
+//   kbuf  ST/32 key groups           (reused for the output staging after phase 1)
+//   vbuf  ST/160 ternary supergroups
+//   S     8 rows of ST + 4 floats: scores, then binary16 probabilities in place
+//   psum  [ST/32][8]  -5 * (sum of the rounded probabilities of the group)
+//   red   [16]        row maxima and sums
+// ---------------------------------------------------------------------------------
+size_t decode_mma_smem_bytes(int ST) {
+  return static_cast<size_t>(ST / 32) * kKGroupBytes + static_cast<size_t>(ST / 160) * kSGBytes +
+         sizeof(float) * (8 * (ST + 4) + 8 * (ST / 32) + 16);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, int n_chunks) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  const int ST = a.split_tokens;
+  const int SS = ST + 4;                                  // row stride of S in floats
+  uint8_t* kbuf = smem_raw;
+  uint8_t* vbuf = kbuf + (ST / 32) * kKGroupBytes;
+  float* S = reinterpret_cast<float*>(vbuf + (ST / 160) * kSGBytes);
+  float* psum = S + 8 * SS;
+  float* red = psum + 8 * (ST / 32);
+  const Split c = make_split(a);
+  const CacheView& cv = a.cv;
+  const int n_sg = (c.n_kg + kSGGroups - 1) / kSGGroups;   // ternary groups = key groups here
+
+  // ---- stage the packed split
+  {
+    const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
+    for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
+    cp_async_commit();
+    const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + (c.t0 / (kG * kSGGroups)) * kSGBytes;
+    for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
+    cp_async_commit();
+  }
+  cp_async_wait<1>();
+  __syncthreads();
+  score_phase<T>(a, n_chunks, c, kbuf, S, SS);
+  __syncthreads();
+  softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0);
+  __syncthreads();
+  group_sums(c, reinterpret_cast<const __half*>(S), 2 * SS, n_sg * kSGGroups, -5.0f, psum);
+  cp_async_wait<0>();
+  __syncthreads();
+  float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
+  ternary_phase(c, vbuf, n_sg, c.n_kg, reinterpret_cast<const uint8_t*>(S + c.hd * SS), psum, tot);
+  epilogue<T>(a, c, kbuf, S, SS, red, tot);
+}
+
+// ---------------------------------------------------------------------------------
+// Caches with protected tokens (STPQuant, Algorithm 2).  The values of the split's tokens sit
+// in two streams whose order differs from the key order: unprotected tokens in the ternary
+// stream (position = token - protected tokens before it; flushed tokens follow from the next
+// group boundary), protected ones in 2-bit groups.  The probabilities are therefore scattered
+// into stream-ordered rows, zero wherever a staged stream position belongs to another split.
+// Shared memory for a split of ST tokens (160 or 320):
+//   kbuf  ST/32 key groups; after phase 1: Pprot, 8 rows of (ST/32 + 1) * 32 + 8 binary16;
+//         at the end the output staging
+//   vbuf  ST/160 + 2 ternary supergroups     pbuf  ST/32 + 1 protected groups
+//   S     8 rows of ST + 4 floats            Ptern 8 rows of (ST/160 + 2) * 160 + 8 binary16
+//   map   ST destinations                    psum_t, psum_p, red
+// ---------------------------------------------------------------------------------
+__host__ __device__ inline int stp_sg_max(int ST) { return ST / 160 + 2; }
+__host__ __device__ inline int stp_pg_max(int ST) { return ST / 32 + 1; }
+
+size_t decode_stp_smem_bytes(int ST) {
+  const int PT = stp_sg_max(ST) * 160 + 8;
+  return static_cast<size_t>(ST / 32) * kKGroupBytes + static_cast<size_t>(stp_sg_max(ST)) * kSGBytes +
+         static_cast<size_t>(stp_pg_max(ST)) * kPGBytes + sizeof(float) * 8 * (ST + 4) + 16 * PT + 2 * ST +
+         sizeof(float) * (8 * stp_sg_max(ST) * kSGGroups + 8 * stp_pg_max(ST) + 16);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 3) decode_stp_kernel(DecodeArgs a, int n_chunks) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  const int ST = a.split_tokens;
+  const int SS = ST + 4;
+  const int PT = stp_sg_max(ST) * 160 + 8, PP = stp_pg_max(ST) * 32 + 8;
+  uint8_t* kbuf = smem_raw;
+  uint8_t* vbuf = kbuf + (ST / 32) * kKGroupBytes;
+  uint8_t* pbuf = vbuf + stp_sg_max(ST) * kSGBytes;
+  float* S = reinterpret_cast<float*>(pbuf + stp_pg_max(ST) * kPGBytes);
+  __half* Ptern = reinterpret_cast<__half*>(S + 8 * SS);
+  uint16_t* map = reinterpret_cast<uint16_t*>(Ptern + 8 * PT);
+  float* psum_t = reinterpret_cast<float*>(map + ST);
+  float* psum_p = psum_t + 8 * stp_sg_max(ST) * kSGGroups;
+  float* red = psum_p + 8 * stp_pg_max(ST);
+  __half* Pprot = reinterpret_cast<__half*>(kbuf);
+  const Split c = make_split(a);
+  const CacheView& cv = a.cv;
+  const int b = c.lb % cv.B;
+  const uint32_t* ew = cv.e_words(b);
+  const uint32_t* ep = cv.e_prefix(b);
+
+  // ---- where the split's tokens sit in the two value streams
+  const int64_t tp0 = min(c.t0, c.T_q0), tp1 = min(c.tq1, c.T_q0);              // prefill part
+  const int64_t pp0 = ep[tp0 / kG], pp1 = ep[tp1 / kG];                         // protected positions
+  const int64_t n_rest = c.T_q0 - a.n_prot;
+  const int64_t u_fl0 = (n_rest + kG - 1) / kG * kG;                            // flushed tokens start here
+  const int64_t ua0 = tp0 - pp0, ua1 = tp1 - pp1;
+  const int64_t tf0 = max(c.t0, c.T_q0), tf1 = max(c.tq1, tf0);                 // flushed part
+  const int64_t ub0 = u_fl0 + (tf0 - c.T_q0), ub1 = u_fl0 + (tf1 - c.T_q0);
+  const bool has_a = ua1 > ua0, has_b = tf1 > tf0;
+  const int64_t U0 = has_a ? ua0 : (has_b ? ub0 : 0), U1 = has_b ? ub1 : (has_a ? ua1 : 0);
+  const int64_t sgA = U0 / (kG * kSGGroups);
+  const int n_sg = U1 > U0 ? static_cast<int>((U1 - 1) / (kG * kSGGroups) - sgA + 1) : 0;
+  const int64_t Ubase = sgA * (kG * kSGGroups);
+  const int64_t pgA = pp0 / kG;
+  const int n_pg = pp1 > pp0 ? static_cast<int>((pp1 - 1) / kG - pgA + 1) : 0;
+  const int64_t Pbase = pgA * kG;
+  const int64_t tg_total = (n_rest + kG - 1) / kG + (kR / kG) * a.st.n_flush;   // ternary groups that exist
+
+  // ---- stage keys, ternary supergroups, protected groups
+  {
+    const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
+    for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
+    cp_async_commit();
+    const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + sgA * kSGBytes;
+    for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
+    const uint8_t* psrc = c.slab_ptr + cv.prot_offset + pgA * kPGBytes;
+    for (int i = c.tid; i < n_pg * (kPGBytes / 16); i += kThreads) cp_async16(pbuf + i * 16, psrc + i * 16);
+    cp_async_commit();
+  }
+  // ---- destinations of the quantized tokens, cleared ternary rows
+  for (int i = c.tid; i < c.nq; i += kThreads) {
+    const int64_t t = c.t0 + i;
+    uint32_t d;
+    if (t < c.T_q0) {
+      const uint32_t word = ew[t / kG];
+      const int64_t pb = ep[t / kG] + __popc(word & ((1u << (t & 31)) - 1u));
+      d = (word >> (t & 31)) & 1u ? 0x8000u | static_cast<uint32_t>(pb - Pbase) : static_cast<uint32_t>((t - pb) - Ubase);
+    } else {
+      d = static_cast<uint32_t>(u_fl0 + (t - c.T_q0) - Ubase);
+    }
+    map[i] = static_cast<uint16_t>(d);
+  }
+  for (int i = c.tid; i < PT; i += kThreads) reinterpret_cast<uint4*>(Ptern)[i] = make_uint4(0u, 0u, 0u, 0u);
+
+  cp_async_wait<1>();
+  __syncthreads();
+  score_phase<T>(a, n_chunks, c, kbuf, S, SS);
+  __syncthreads();
+  for (int i = c.tid; i < PP; i += kThreads) reinterpret_cast<uint4*>(Pprot)[i] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  softmax_phase<true>(a, c, S, SS, red, (c.n_loc + 1) & ~1, map, Ptern, PT, Pprot, PP);
+  __syncthreads();
+  group_sums(c, Ptern, PT, n_sg * kSGGroups, -5.0f, psum_t);
+  group_sums(c, Pprot, PP, n_pg, 1.0f, psum_p);
+  cp_async_wait<0>();
+  __syncthreads();
+
+  float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
+  ternary_phase(c, vbuf, n_sg, static_cast<int>(min(tg_total - sgA * kSGGroups, static_cast<int64_t>(n_sg * kSGGroups))),
+                reinterpret_cast<const uint8_t*>(Ptern + c.hd * PT), psum_t, tot);
+  // ---- protected stream: 2-bit codes (Eq. 4) as 4 + code, then s * (acc - 4 sum p) + z * sum p
+  {
+    const int warp = c.warp, hd = c.hd, r = c.r;
+    const uint8_t* prow = reinterpret_cast<const uint8_t*>(Pprot + hd * PP);
+    for (int pg = 0; pg < n_pg; ++pg) {
+      const uint8_t* gp = pbuf + pg * kPGBytes;
+      const float2 sp = *reinterpret_cast<const float2*>(psum_p + pg * 8 + 2 * r);
+      float acc[2][4];
+#pragma unroll
+      for (int kt = 0; kt < 2; ++kt) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(gp + ((((kt * 4 + warp) * 4 + r) * 8) + hd) * 4);
+        uint32_t x[8];
+        x[0] = and_or(w << 8, c.m_field, c.c_four);
+        x[1] = and_or(w << 6, c.m_field, c.c_four);
+        x[2] = and_or(w << 4, c.m_field, c.c_four);
+        x[3] = and_or(w << 2, c.m_field, c.c_four);
+        x[4] = and_or(w, c.m_field, c.c_four);
+        x[5] = and_or(w >> 2, c.m_field, c.c_four);
+        x[6] = and_or(w >> 4, c.m_field, c.c_four);
+        x[7] = and_or(w >> 6, c.m_field, c.c_four);
+        const uint8_t* pb = prow + (pg * kG + kt * 16 + 2 * r) * 2;
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(pb);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(pb + 16);
+        if (kt == 0) {
+          mma_f16_c(acc[0], x[0], x[1], x[4], x[5], b0, b1, -4.0f * sp.x, -4.0f * sp.y, -4.0f * sp.x, -4.0f * sp.y);
+          mma_f16_c(acc[1], x[2], x[3], x[6], x[7], b0, b1, -4.0f * sp.x, -4.0f * sp.y, -4.0f * sp.x, -4.0f * sp.y);
+        } else {
+          mma_f16(acc[0], x[0], x[1], x[4], x[5], b0, b1);
+          mma_f16(acc[1], x[2], x[3], x[6], x[7], b0, b1);
+        }
+      }
+      const uint2 sc = *reinterpret_cast<const uint2*>(gp + kPG_S + (32 * warp + 4 * hd) * 2);
+      const uint2 zc = *reinterpret_cast<const uint2*>(gp + kPG_Z + (32 * warp + 4 * hd) * 2);
+      const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));
+      const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));
+      const float2 za = __half22float2(*reinterpret_cast<const __half2*>(&zc.x));
+      const float2 zb = __half22float2(*reinterpret_cast<const __half2*>(&zc.y));
+      tot[0][0] += sa.x * acc[0][0] + za.x * sp.x; tot[0][1] += sa.x * acc[0][1] + za.x * sp.y;
+      tot[0][2] += sa.y * acc[0][2] + za.y * sp.x; tot[0][3] += sa.y * acc[0][3] + za.y * sp.y;
+      tot[1][0] += sb.x * acc[1][0] + zb.x * sp.x; tot[1][1] += sb.x * acc[1][1] + zb.x * sp.y;
+      tot[1][2] += sb.y * acc[1][2] + zb.y * sp.x; tot[1][3] += sb.y * acc[1][3] + zb.y * sp.y;
+    }
+  }
+  __syncthreads();                                       // Pprot shares kbuf with the output staging
+  epilogue<T>(a, c, kbuf, S, SS, red, tot);
+}
+
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t stream) {
   const int n_slabs = a.n_layers * a.cv.B * a.cv.H_kv;
   const int n_chunks = static_cast<int>((a.st.T_q0 > 0 ? 1 : 0) + a.st.n_flush);
-  const size_t smem = decode_mma_smem_bytes(a.split_tokens);
-  static size_t attr_smem = 0;
-  if (smem > attr_smem) {
+  const bool stp = a.n_prot > 0;
+  const size_t smem = stp ? decode_stp_smem_bytes(a.split_tokens) : decode_mma_smem_bytes(a.split_tokens);
+  static size_t attr_smem[2] = {0, 0};
+  if (smem > attr_smem[stp]) {
     cudaError_t e;
-    if ((e = cudaFuncSetAttribute(decode_mma_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    if ((e = cudaFuncSetAttribute(decode_mma_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    attr_smem = smem;
+    if (stp) {
+      if ((e = cudaFuncSetAttribute(decode_stp_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+      if ((e = cudaFuncSetAttribute(decode_stp_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    } else {
+      if ((e = cudaFuncSetAttribute(decode_mma_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+      if ((e = cudaFuncSetAttribute(decode_mma_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    }
+    attr_smem[stp] = smem;
   }
   const int chunk_stride = n_chunks > 0 ? n_chunks : 1;
   if (n_chunks > 0) {
@@ -554,8 +781,13 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t stream) {
   }
   const dim3 grid(a.n_splits, n_slabs);
   if (a.ev_begin) cudaEventRecord(a.ev_begin, stream);
-  if (a.in_dtype == VIDKV_F16) decode_mma_kernel<__half><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
-  else decode_mma_kernel<__nv_bfloat16><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
+  if (stp) {
+    if (a.in_dtype == VIDKV_F16) decode_stp_kernel<__half><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
+    else decode_stp_kernel<__nv_bfloat16><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
+  } else {
+    if (a.in_dtype == VIDKV_F16) decode_mma_kernel<__half><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
+    else decode_mma_kernel<__nv_bfloat16><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
+  }
   if (a.ev_end) cudaEventRecord(a.ev_end, stream);
   count_launches(1);
   return cudaGetLastError();

@@ -78,8 +78,8 @@ __global__ void __launch_bounds__(128) dequant_values_kernel(CacheView cv, int l
     if (prot) {
       const uint8_t* pg = sp + cv.prot_offset + (pb / kG) * kPGBytes;
       const int j = static_cast<int>(pb % kG);
-      const uint32_t word = reinterpret_cast<const uint32_t*>(pg)[j * 8 + (c >> 4)];
-      v = static_cast<float>((word >> (2 * (c & 15))) & 3u) * h2f(reinterpret_cast<const uint16_t*>(pg + kPG_S)[c]) +
+      const uint32_t word = reinterpret_cast<const uint32_t*>(pg)[prot_word_index(j, c)];
+      v = static_cast<float>((word >> prot_bit(j, c)) & 3u) * h2f(reinterpret_cast<const uint16_t*>(pg + kPG_S)[c]) +
           h2f(reinterpret_cast<const uint16_t*>(pg + kPG_Z)[c]);
     } else {
       const int64_t n_rest = T_q0 - n_prot;

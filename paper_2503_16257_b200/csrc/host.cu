@@ -66,11 +66,11 @@ void compute_layout(const vidkv_config_t& c, Layout* out) {
 }
 
 // Tokens per split: the largest of {640, 320, 160} that still gives >= 4 CTAs per SM on a
-// 148-SM part, else 160.
-int choose_split_tokens(int64_t T_tot, int64_t n_slabs) {
+// 148-SM part, else 160.  Caches with protected tokens stage two value streams and stop at 320.
+int choose_split_tokens(int64_t T_tot, int64_t n_slabs, bool stp) {
   const int cand[3] = {640, 320, 160};
   for (int s : cand)
-    if (n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
+    if ((!stp || s <= 320) && n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
   return 160;
 }
 
@@ -79,9 +79,11 @@ int64_t max_partial_entries(const vidkv_config_t& c, int64_t T_max) {
   if (T_max < 1) T_max = 1;
   for (int n = 1; n <= c.L; ++n) {
     const int64_t slabs = static_cast<int64_t>(n) * c.B * c.H_kv;
-    const int st = choose_split_tokens(T_max, slabs);
-    const int64_t e = static_cast<int64_t>(n) * c.B * c.H_q * ((T_max + st - 1) / st);
-    if (e > best) best = e;
+    for (int stp = 0; stp <= (c.p_ratio > 0.0f ? 1 : 0); ++stp) {
+      const int st = choose_split_tokens(T_max, slabs, stp != 0);
+      const int64_t e = static_cast<int64_t>(n) * c.B * c.H_q * ((T_max + st - 1) / st);
+      if (e > best) best = e;
+    }
   }
   return best;
 }
@@ -361,7 +363,7 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   a.st.T_q0 = first.T_q0; a.st.n_flush = first.n_flush; a.st.n_res = first.n_res + 1;
   const int64_t T_tot = first.T_q0 + first.n_flush * kR + a.st.n_res;
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv;
-  a.split_tokens = choose_split_tokens(T_tot, n_slabs);
+  a.split_tokens = choose_split_tokens(T_tot, n_slabs, h->n_prot > 0);
   a.n_splits = static_cast<int32_t>((T_tot + a.split_tokens - 1) / a.split_tokens);
   if (static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_q * a.n_splits > h->ws.partial_entries) return VIDKV_ERR_CAPACITY;
   if (launch_decode(a, s) != cudaSuccess) return VIDKV_ERR_CUDA;

@@ -191,17 +191,19 @@ __global__ void __launch_bounds__(128) v_protect_kernel(KSrc src, CacheView cv, 
   }
   __syncthreads();
   for (int item = threadIdx.x; item < kG * 8; item += 128) {
-    const int j = item >> 3, wi = item & 7;
+    // item = word index ((kt * 4 + w) * 4 + r) * 8 + rho: 4 channels x 4 tokens
+    const int rho = item & 7, r = (item >> 3) & 3, w = (item >> 5) & 3, kt = item >> 7;
     uint32_t word = 0;
-    if (j < n_rows) {
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int c = wi * 16 + i;
+    for (int f = 0; f < 16; ++f) {
+      const int e = f & 3, u = (f >> 2) & 1, hf = f >> 3;
+      const int j = 16 * kt + 8 * u + 2 * r + hf, c = 32 * w + 4 * rho + e;
+      if (j < n_rows) {
         const float s = h2f(s_s[c]), z = h2f(s_z[c]);
         const float v = Elem<T>::to_float(reinterpret_cast<const T*>(tile)[j * kD + c]);
         float q = rintf(__fdiv_rn(__fsub_rn(v, z), s));
         q = fminf(fmaxf(q, 0.0f), 3.0f);
-        word |= ((s == 0.0f) ? 0u : static_cast<uint32_t>(q)) << (2 * i);
+        word |= ((s == 0.0f) ? 0u : static_cast<uint32_t>(q)) << (2 * (4 * u + e) + 16 * hf);
       }
     }
     reinterpret_cast<uint32_t*>(pg)[item] = word;

@@ -80,11 +80,14 @@ def protected_groups(slab: np.ndarray, lay: dict, n_groups: int):
     codes = np.zeros((n_groups * G, D), np.int8)
     s = np.zeros((n_groups, D), np.float16)
     z = np.zeros((n_groups, D), np.float16)
-    sh = 2 * (np.arange(D) % 16)
+    j = np.arange(G)[:, None]
+    c = np.arange(D)[None, :]
+    widx = (((j // 16) * 4 + c // 32) * 4 + (j // 2) % 4) * 8 + (c // 4) % 8
+    bit = 2 * (4 * ((j // 8) % 2) + c % 4) + 16 * (j % 2)
     for g in range(n_groups):
         rec = slab[lay["prot_offset"] + g * PG_BYTES:][:PG_BYTES]
-        w = rec[:1024].view("<u4").reshape(G, 8)
-        codes[g * G:(g + 1) * G] = (w[:, np.arange(D) // 16] >> sh) & 3
+        w = rec[:1024].view("<u4")
+        codes[g * G:(g + 1) * G] = (w[widx] >> bit) & 3
         s[g] = rec[1024:1280].view("<f2")
         z[g] = rec[1280:1536].view("<f2")
     return codes, s, z
