@@ -562,37 +562,38 @@ __device__ __forceinline__ void group_sums(const Split& c, const __half* P, int 
 //   red   [16]        row maxima and sums
 // ---------------------------------------------------------------------------------
 size_t decode_mma_smem_bytes(int ST) {
-  return static_cast<size_t>(ST / 32) * kKGroupBytes + static_cast<size_t>(ST / 160) * kSGBytes +
-         sizeof(float) * (8 * (ST + 4) + 8 * (ST / 32) + 16);
+  return static_cast<size_t>(ST / 32) * kKGroupBytes + sizeof(float) * (8 * (ST + 4) + 8 * (ST / 32) + 16);
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, int n_chunks) {
+__global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, int n_chunks) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   const int ST = a.split_tokens;
   const int SS = ST + 4;                                  // row stride of S in floats
-  uint8_t* kbuf = smem_raw;
-  uint8_t* vbuf = kbuf + (ST / 32) * kKGroupBytes;
-  float* S = reinterpret_cast<float*>(vbuf + (ST / 160) * kSGBytes);
+  uint8_t* kbuf = smem_raw;                               // keys, then values (ST/160 * 5376 <= ST/32 * 1152)
+  uint8_t* vbuf = kbuf;
+  float* S = reinterpret_cast<float*>(kbuf + (ST / 32) * kKGroupBytes);
   float* psum = S + 8 * SS;
   float* red = psum + 8 * (ST / 32);
   const Split c = make_split(a);
   const CacheView& cv = a.cv;
   const int n_sg = (c.n_kg + kSGGroups - 1) / kSGGroups;   // ternary groups = key groups here
 
-  // ---- stage the packed split
   {
     const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
     for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
     cp_async_commit();
+  }
+  cp_async_wait<0>();
+  __syncthreads();
+  score_phase<T>(a, n_chunks, c, kbuf, S, SS);
+  __syncthreads();
+  {
+    // the key groups are spent: the ternary supergroups take their place while the softmax runs
     const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + (c.t0 / (kG * kSGGroups)) * kSGBytes;
     for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
     cp_async_commit();
   }
-  cp_async_wait<1>();
-  __syncthreads();
-  score_phase<T>(a, n_chunks, c, kbuf, S, SS);
-  __syncthreads();
   softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0);
   __syncthreads();
   group_sums(c, reinterpret_cast<const __half*>(S), 2 * SS, n_sg * kSGGroups, -5.0f, psum);
@@ -600,6 +601,7 @@ __global__ void __launch_bounds__(kThreads, 3) decode_mma_kernel(DecodeArgs a, i
   __syncthreads();
   float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
   ternary_phase(c, vbuf, n_sg, c.n_kg, reinterpret_cast<const uint8_t*>(S + c.hd * SS), psum, tot);
+  __syncthreads();                                        // the output staging reuses the same buffer
   epilogue<T>(a, c, kbuf, S, SS, red, tot);
 }
 
