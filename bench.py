@@ -347,7 +347,7 @@ def main():
         "quantize": {"tokens_per_s": world * q_tokens / (q_ms * 1e-3), "unit": "tokens/s (one position, 4 KV heads, "
                      "one layer, K and V)", "ms_per_bench_step": q_ms, "GBps": world * q_bytes / (q_ms * 1e-3) / 1e9,
                      "pct_of_8TBps": 100.0 * q_bytes / (q_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
-        "roofline": {"bound": "hbm", "kernel": "decode_split_kernel", "achieved": kern_gbs, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "decode_stp_kernel" if n_prot > 0 else "decode_mma_kernel", "achieved": kern_gbs, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": kern_gbs / peak, "traffic": traffic,
                      "avg_launch_ms": kern_avg_ms, "launches_timed": len(kern_ms)},
         "gpu_launches": int(launches),
