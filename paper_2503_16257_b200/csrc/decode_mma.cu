@@ -138,79 +138,73 @@ size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks) {
 }
 
 // ---------------------------------------------------------------------------------
-// Query preparation: one block per (chunk, slab).  Writes, per lane of a warp, the 24
-// register images the attention kernel needs for this chunk's channel split:
+// Query preparation: one warp per (chunk, slab).  Writes, per lane, the 24 register images the
+// attention kernel needs for this chunk's channel split:
 //   words  0.. 7  binary16 pairs of q at the anomalous slots (16 r + 2 i, 16 r + 2 i + 1)
 //   words  8..15  leading binary16 part of the transformed query Q at the spectrum
 //                 columns (16 r + 2 i, 16 r + 2 i + 1)
 //   words 16..23  binary16 remainder Q - leading part
 // for head lane / 4 (zero when that head does not exist) and r = lane % 4.
+// Q_f = sum_c q_c W[c, f] with W the weights with which spectrum column f enters channel c of
+// the inverse orthonormal 64-point transform of a Hermitian half spectrum: the forward DFT
+// matrix, doubled for the columns f >= 2 that stand for a conjugate pair.  The product runs
+// on the tensor cores against the same split-precision matrix fragments the encoder uses.
 // ---------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int n_chunks) {
-  __shared__ float q_raw[kMaxRep][kD];
-  __shared__ float q_hat[kMaxRep][kNF];
-  __shared__ float cs[64], sn[64];
-  __shared__ uint8_t perm[kD];
+__global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int n_chunks, int n_items) {
   const CacheView& cv = a.cv;
-  const int tid = threadIdx.x;
-  const int chunk = blockIdx.x, slab = blockIdx.y;
+  const int lane = threadIdx.x & 31;
+  const int item = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+  if (item >= n_items) return;
+  const int chunk = item % n_chunks, slab = item / n_chunks;
+  const int hd = lane >> 2, r = lane & 3;
   const int h = slab % cv.H_kv, lb = slab / cv.H_kv;
-  const int b = lb % cv.B, layer_idx = lb / cv.B;
   const int rep = cv.rep;
-  const uint8_t* slab_ptr = cv.slab(a.layer0 + layer_idx, b, h);
-  perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
-  const T* qp = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(lb) * cv.H_q + h * rep) * kD;
-  for (int i = tid; i < kMaxRep * kD; i += kThreads) {
-    const int r = i >> 7, c = i & 127;
-    q_raw[r][c] = r < rep ? Elem<T>::to_float(qp[r * kD + c]) : 0.0f;
-  }
-  if (tid < 64) {
-    float s, c;
-    sincospif(static_cast<float>(tid) / 32.0f, &s, &c);
-    cs[tid] = c; sn[tid] = s;
-  }
-  __syncthreads();
-  // Q_f = sum_c q_c W[c, f]: the weights with which spectrum column f enters channel c of
-  // the inverse orthonormal 64-point transform of a Hermitian half spectrum.
-  for (int i = tid; i < kMaxRep * kNF; i += kThreads) {
-    const int r = i >> 6, f = i & 63;
-    float acc = 0.0f;
-    if (f < 2) {
-      for (int c = 0; c < 64; ++c) {
-        const float qv = q_raw[r][perm[64 + c]];
-        acc += (f == 1 && (c & 1)) ? -qv : qv;
-      }
-      acc *= 0.125f;
-    } else {
-      const int k = f >> 1;
-      const bool im = f & 1;
-      for (int c = 0; c < 64; ++c) {
-        const float qv = q_raw[r][perm[64 + c]];
-        const int m = (k * c) & 63;
-        acc += qv * (im ? -sn[m] : cs[m]);
-      }
-      acc *= 0.25f;
+  const uint8_t* perm = cv.slab(a.layer0 + lb / cv.B, lb % cv.B, h) + cv.chunk_table_offset +
+                        static_cast<int64_t>(chunk) * kChunkBytes;
+  const T* qrow = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(lb) * cv.H_q + h * rep + hd) * kD;
+  const bool live = hd < rep;
+  auto q_at = [&](int c) -> float { return live ? Elem<T>::to_float(qrow[c]) : 0.0f; };
+  uint32_t* out = a.prep + (static_cast<int64_t>(slab) * n_chunks + chunk) * (kPrepWords * 32) + lane;
+  // anomalous slots
+  {
+    const uint4 p0 = __ldg(reinterpret_cast<const uint4*>(perm + 16 * r));
+    const uint32_t pw[4] = {p0.x, p0.y, p0.z, p0.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint32_t two = pw[i >> 1] >> (16 * (i & 1));
+      out[i * 32] = pack_half2(q_at(two & 0xffu), q_at((two >> 8) & 0xffu));
     }
-    q_hat[r][f] = acc;
   }
-  __syncthreads();
-  uint32_t* out = a.prep + (static_cast<int64_t>(slab) * n_chunks + chunk) * (kPrepWords * 32);
-  for (int i = tid; i < kPrepWords * 32; i += kThreads) {
-    const int word = i >> 5, lane = i & 31;
-    const int hd = lane >> 2, r = lane & 3;
-    const int kind = word >> 3, pi = word & 7;
-    const int e0 = 16 * r + 2 * pi;
-    uint32_t v;
-    if (kind == 0) {
-      v = pack_half2(q_raw[hd][perm[e0]], q_raw[hd][perm[e0 + 1]]);
-    } else {
-      const float x0 = q_hat[hd][e0], x1 = q_hat[hd][e0 + 1];
-      const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
-      if (kind == 1) v = pack_half2(__half2float(h0), __half2float(h1));
-      else v = pack_half2(x0 - __half2float(h0), x1 - __half2float(h1));
+  // transformed query: A = q at the normal channels (rows 8-15 unused), B = matrix fragments
+  uint32_t af[4][2];
+#pragma unroll
+  for (int ks = 0; ks < 4; ++ks) {
+    const uint32_t pa = __ldg(reinterpret_cast<const uint16_t*>(perm + kNA + 16 * ks + 2 * r));
+    const uint32_t pb = __ldg(reinterpret_cast<const uint16_t*>(perm + kNA + 16 * ks + 2 * r + 8));
+    af[ks][0] = pack_half2(q_at(pa & 0xffu), q_at(pa >> 8));
+    af[ks][1] = pack_half2(q_at(pb & 0xffu), q_at(pb >> 8));
+  }
+  float acc[8][4];
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) { acc[nt][0] = 0.0f; acc[nt][1] = 0.0f; acc[nt][2] = 0.0f; acc[nt][3] = 0.0f; }
+#pragma unroll
+  for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      const uint4 bw = __ldg(reinterpret_cast<const uint4*>(a.dft + ((ks * 8 + nt) * 32 + lane) * 4));
+      mma_f16(acc[nt], af[ks][0], 0u, af[ks][1], 0u, bw.x, bw.y);
+      mma_f16(acc[nt], af[ks][0], 0u, af[ks][1], 0u, bw.z, bw.w);
     }
-    out[i] = v;
+  }
+  // lane (hd, r) now holds Q of head hd at columns 16 r + 2 nt + {0, 1}
+#pragma unroll
+  for (int nt = 0; nt < 8; ++nt) {
+    const float w0 = (r == 0 && nt == 0) ? 1.0f : 2.0f;            // columns 0 and 1 are not doubled
+    const float x0 = acc[nt][0] * w0, x1 = acc[nt][1] * w0;
+    const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
+    out[(8 + nt) * 32] = pack_half2(__half2float(h0), __half2float(h1));
+    out[(16 + nt) * 32] = pack_half2(x0 - __half2float(h0), x1 - __half2float(h1));
   }
 }
 
@@ -757,7 +751,9 @@ __global__ void __launch_bounds__(kThreads, 3) decode_stp_kernel(DecodeArgs a, i
   epilogue<T>(a, c, kbuf, S, SS, red, tot);
 }
 
-cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t stream) {
+cudaError_t launch_decode_mma(const DecodeArgs& a_in, cudaStream_t stream) {
+  DecodeArgs a = a_in;
+  a.dft = nullptr;
   const int n_slabs = a.n_layers * a.cv.B * a.cv.H_kv;
   const int n_chunks = static_cast<int>((a.st.T_q0 > 0 ? 1 : 0) + a.st.n_flush);
   const bool stp = a.n_prot > 0;
@@ -776,9 +772,12 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t stream) {
   }
   const int chunk_stride = n_chunks > 0 ? n_chunks : 1;
   if (n_chunks > 0) {
-    const dim3 pgrid(n_chunks, n_slabs);
-    if (a.in_dtype == VIDKV_F16) decode_prep_kernel<__half><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride);
-    else decode_prep_kernel<__nv_bfloat16><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride);
+    cudaError_t e;
+    if ((e = dft_fragments(&a.dft, stream))) return e;
+    const int n_items = n_slabs * n_chunks;
+    const int pgrid = (n_items + kThreads / 32 - 1) / (kThreads / 32);
+    if (a.in_dtype == VIDKV_F16) decode_prep_kernel<__half><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride, n_items);
+    else decode_prep_kernel<__nv_bfloat16><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride, n_items);
     count_launches(1);
   }
   const dim3 grid(a.n_splits, n_slabs);

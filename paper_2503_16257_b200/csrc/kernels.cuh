@@ -35,6 +35,13 @@ cudaError_t launch_quantize_keys(int dtype, const KSrc& src, int64_t T_tokens, c
 cudaError_t launch_encode_keys(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0, int n_slabs,
                                int slabs_per_layer, int chunk, int64_t kgroup0, cudaStream_t stream);
 
+// Device address of the 64-point DFT matrix in MMA B-fragment order: word
+// ((ks * 8 + nt) * 32 + lane) * 4 + {0, 1} = leading binary16 pairs, + {2, 3} = remainders, for
+// rows 16 ks + 2 r (+1; +8, +9) and column 16 (n / 2) + 2 nt + (n % 2), lane = 4 n + r; column f
+// holds 1/8, (-1)^c / 8, cos(2 pi k c / 64) / 8 (f = 2k) or -sin(2 pi k c / 64) / 8 (f = 2k + 1).
+// Filled on first use on each device (one small kernel and a stream synchronisation).
+cudaError_t dft_fragments(const uint32_t** table, cudaStream_t stream);
+
 // Algorithm 2 on the prefill tokens of one layer.  T_q (multiple of 32) tokens; the
 // unprotected ones go to ternary stream positions 0.., the protected ones to 2-bit groups.
 cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer,
@@ -74,6 +81,7 @@ struct DecodeArgs {
   void* out;
   float* partials;     // [n_layers * B * H_q * n_splits][130]
   uint32_t* prep;      // per (slab, chunk) query images of the tensor-core path (decode_prep_bytes)
+  const uint32_t* dft; // DFT matrix fragments (dft_fragments), set by launch_decode_mma
   int32_t layer0, n_layers;
   int32_t in_dtype, out_dtype;
   int32_t split_tokens, n_splits;

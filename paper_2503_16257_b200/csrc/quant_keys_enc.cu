@@ -304,23 +304,35 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
 // ---------------------------------------------------------------------------------
 // Host launcher of the encode pass
 // ---------------------------------------------------------------------------------
+// The DFT fragments are written once per device, ordered before their first use on `stream`
+// (and, through the synchronisation, before any later use on another stream).
+cudaError_t dft_fragments(const uint32_t** table, cudaStream_t stream) {
+  static bool done[64] = {};
+  static const uint32_t* addr[64] = {};
+  cudaError_t e;
+  int dev = 0;
+  if ((e = cudaGetDevice(&dev))) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!done[dev]) {
+    void* p = nullptr;
+    if ((e = cudaGetSymbolAddress(&p, g_dft_frag))) return e;
+    dft_table_kernel<<<1, 256, 0, stream>>>();
+    if ((e = cudaGetLastError())) return e;
+    if ((e = cudaStreamSynchronize(stream))) return e;
+    addr[dev] = static_cast<const uint32_t*>(p);
+    done[dev] = true;
+    count_launches(1);
+  }
+  *table = addr[dev];
+  return cudaSuccess;
+}
+
 template <typename T>
 static cudaError_t launch_encode_t(const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0, int n_slabs,
                                    int slabs_per_layer, int chunk, int64_t kgroup0, cudaStream_t stream) {
   cudaError_t e;
-  // the DFT fragments are written once per device, ordered before their first use on this stream
-  static bool table_done[64] = {};
-  int dev = 0;
-  if ((e = cudaGetDevice(&dev))) return e;
-  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!table_done[dev]) {
-    dft_table_kernel<<<1, 256, 0, stream>>>();
-    if ((e = cudaGetLastError())) return e;
-    // later calls may come on other streams: make the table visible to all of them
-    if ((e = cudaStreamSynchronize(stream))) return e;
-    table_done[dev] = true;
-    count_launches(1);
-  }
+  const uint32_t* table = nullptr;
+  if ((e = dft_fragments(&table, stream))) return e;
   static bool attr_set = false;
   const size_t smem = k_encode_smem_bytes();
   if (!attr_set) {
