@@ -30,7 +30,7 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream) {
   const cudaError_t e = launch_decode_mma(a, stream);
   if (e != cudaSuccess) return e;
   count_launches(1);
-  decode_merge_kernel<<<a.n_layers * a.cv.B * a.cv.H_q, kD, 0, stream>>>(a.partials, a.n_splits, a.out, a.out_dtype);
+  decode_merge_kernel<<<a.n_layers * a.cv.B * a.cv.H_q, kD, 0, stream>>>(a.partials, a.n_parts, a.out, a.out_dtype);
   return cudaGetLastError();
 }
 

@@ -220,11 +220,11 @@ struct Split {
   int n_loc, nq, n_kg;                    // tokens, quantized tokens, key groups in the split
 };
 
-__device__ __forceinline__ Split make_split(const DecodeArgs& a) {
+__device__ __forceinline__ Split make_split(const DecodeArgs& a, int split) {
   Split c;
   c.tid = threadIdx.x; c.lane = c.tid & 31; c.warp = c.tid >> 5; c.hd = c.lane >> 2; c.r = c.lane & 3;
   c.m_field = kExpand[0]; c.c_four = kExpand[1]; c.m_sign = kExpand[2]; c.c_neg1 = kExpand[3];
-  c.split = blockIdx.x; c.slab = blockIdx.y;
+  c.split = split; c.slab = blockIdx.y;
   const CacheView& cv = a.cv;
   c.h = c.slab % cv.H_kv; c.lb = c.slab / cv.H_kv; c.rep = cv.rep;
   c.slab_ptr = cv.slab(a.layer0 + c.lb / cv.B, c.lb % cv.B, c.h);
@@ -426,53 +426,62 @@ __device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbu
   }
 }
 
-// Epilogue: stage tot as O[head][channel], add the residual rows' P V (probabilities of the
-// residual tokens sit in S in place, binary16, token order), write the split's partial record.
+// P V of the FP16 / BF16 residual rows of the split, added to tot.  The probabilities of the
+// residual tokens sit in S in place (binary16, token order).  Thread = channel computes the
+// eight heads' sums into O[head][channel] (the staging buffer, which must be free), then every
+// thread picks up the entries of its accumulator layout.  All threads call it or none.
 template <typename T>
-__device__ __forceinline__ void epilogue(const DecodeArgs& a, const Split& c, uint8_t* kbuf, const float* S, int SS,
-                                         const float* red, const float (&tot)[2][4]) {
+__device__ __forceinline__ void residual_pv(const DecodeArgs& a, const Split& c, float* O, const float* S, int SS,
+                                            float (&tot)[2][4]) {
   const CacheView& cv = a.cv;
-  const int tid = c.tid, warp = c.warp, hd = c.hd, r = c.r, h = c.h, lb = c.lb, rep = c.rep, split = c.split;
-  const uint8_t* slab_ptr = c.slab_ptr;
-  const int64_t T_qt = c.T_qt, t0 = c.t0, t1 = c.t1;
-  // ---- output staging: O[head][channel] (reuses the key buffer, free since phase 1; the
-  // smallest split, 160 tokens, has 5 x 1152 bytes there, more than the 4096 needed)
-  float* O = reinterpret_cast<float*>(kbuf);
-  {
-    const int c0 = 32 * warp + 4 * hd;
+  const int ch = c.tid;
+  const int r_begin = static_cast<int>(max(c.t0, c.T_qt) - c.T_qt), r_end = static_cast<int>(c.t1 - c.T_qt);
+  const T* vres = reinterpret_cast<const T*>(c.slab_ptr + cv.vres_offset);
+  const int off = static_cast<int>(c.T_qt - c.t0);
+  float o[kMaxRep];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      O[(2 * r) * kD + c0 + 2 * i] = tot[i][0];
-      O[(2 * r + 1) * kD + c0 + 2 * i] = tot[i][1];
-      O[(2 * r) * kD + c0 + 2 * i + 1] = tot[i][2];
-      O[(2 * r + 1) * kD + c0 + 2 * i + 1] = tot[i][3];
-    }
+  for (int k = 0; k < kMaxRep; ++k) o[k] = 0.0f;
+  for (int rr = r_begin; rr < r_end; ++rr) {
+    const float v = Elem<T>::to_float(vres[rr * kD + ch]);
+#pragma unroll
+    for (int k = 0; k < kMaxRep; ++k) o[k] += __half2float(reinterpret_cast<const __half*>(S + k * SS)[off + rr]) * v;
+  }
+#pragma unroll
+  for (int k = 0; k < kMaxRep; ++k) O[k * kD + ch] = o[k];
+  __syncthreads();
+  const int c0 = 32 * c.warp + 4 * c.hd, r = c.r;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    tot[i][0] += O[(2 * r) * kD + c0 + 2 * i];
+    tot[i][1] += O[(2 * r + 1) * kD + c0 + 2 * i];
+    tot[i][2] += O[(2 * r) * kD + c0 + 2 * i + 1];
+    tot[i][3] += O[(2 * r + 1) * kD + c0 + 2 * i + 1];
   }
   __syncthreads();
-  {
-    const int c = tid;
-    float o[kMaxRep];
+}
+
+// Write one partial record per query head: (max, sum, unnormalised out[128]).  ml[h] = scaled
+// maximum, ml[8 + h] = sum of the probabilities; O is the staging buffer (free, 4 KB).
+__device__ __forceinline__ void write_partial(const DecodeArgs& a, const Split& c, int part, float* O, const float* ml,
+                                              const float (&tot)[2][4]) {
+  const CacheView& cv = a.cv;
+  const int c0 = 32 * c.warp + 4 * c.hd, r = c.r;
 #pragma unroll
-    for (int k = 0; k < kMaxRep; ++k) o[k] = O[k * kD + c];
-    if (t1 > T_qt) {
-      const int r_begin = static_cast<int>(max(t0, T_qt) - T_qt), r_end = static_cast<int>(t1 - T_qt);
-      const T* vres = reinterpret_cast<const T*>(slab_ptr + cv.vres_offset);
-      const int off = static_cast<int>(T_qt - t0);
-      for (int rr = r_begin; rr < r_end; ++rr) {
-        const float v = Elem<T>::to_float(vres[rr * kD + c]);
+  for (int i = 0; i < 2; ++i) {
+    O[(2 * r) * kD + c0 + 2 * i] = tot[i][0];
+    O[(2 * r + 1) * kD + c0 + 2 * i] = tot[i][1];
+    O[(2 * r) * kD + c0 + 2 * i + 1] = tot[i][2];
+    O[(2 * r + 1) * kD + c0 + 2 * i + 1] = tot[i][3];
+  }
+  __syncthreads();
+  const int ch = c.tid;
 #pragma unroll
-        for (int k = 0; k < kMaxRep; ++k)
-          o[k] += __half2float(reinterpret_cast<const __half*>(S + k * SS)[off + rr]) * v;
-      }
-    }
-#pragma unroll
-    for (int k = 0; k < kMaxRep; ++k) {
-      if (k < rep) {
-        const int64_t qh = static_cast<int64_t>(lb) * cv.H_q + h * rep + k;
-        float* pr = a.partials + (qh * a.n_splits + split) * 130;
-        pr[2 + c] = o[k];
-        if (c == 0) { pr[0] = red[k]; pr[1] = red[8 + k]; }
-      }
+  for (int k = 0; k < kMaxRep; ++k) {
+    if (k < c.rep) {
+      const int64_t qh = static_cast<int64_t>(c.lb) * cv.H_q + c.h * c.rep + k;
+      float* pr = a.partials + (qh * a.n_parts + part) * 130;
+      pr[2 + ch] = O[k * kD + ch];
+      if (ch == 0) { pr[0] = ml[k]; pr[1] = ml[8 + k]; }
     }
   }
 }
@@ -569,34 +578,62 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
   float* S = reinterpret_cast<float*>(kbuf + (ST / 32) * kKGroupBytes);
   float* psum = S + 8 * SS;
   float* red = psum + 8 * (ST / 32);
-  const Split c = make_split(a);
   const CacheView& cv = a.cv;
-  const int n_sg = (c.n_kg + kSGGroups - 1) / kSGGroups;   // ternary groups = key groups here
-
-  {
-    const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
-    for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
-    cp_async_commit();
+  // One CTA walks a.splits_per_cta consecutive splits of its slab and keeps a running
+  // (max, sum, out) per head, rescaled as in a streaming softmax; one record leaves at the end.
+  float TOT[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
+  float Mr[2] = {-INFINITY, -INFINITY}, Lr[2] = {0.0f, 0.0f};
+  Split c = make_split(a, blockIdx.x * a.splits_per_cta);
+#pragma unroll 1
+  for (int it = 0; it < a.splits_per_cta; ++it) {
+    const int split = blockIdx.x * a.splits_per_cta + it;
+    if (split >= a.n_splits) break;
+    if (it > 0) c = make_split(a, split);
+    const int n_sg = (c.n_kg + kSGGroups - 1) / kSGGroups;   // ternary groups = key groups here
+    {
+      const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
+      for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
+      cp_async_commit();
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    score_phase<T>(a, n_chunks, c, kbuf, S, SS);
+    __syncthreads();
+    {
+      // the key groups are spent: the ternary supergroups take their place while the softmax runs
+      const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + (c.t0 / (kG * kSGGroups)) * kSGBytes;
+      for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
+      cp_async_commit();
+    }
+    softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0);
+    __syncthreads();
+    group_sums(c, reinterpret_cast<const __half*>(S), 2 * SS, n_sg * kSGGroups, -5.0f, psum);
+    cp_async_wait<0>();
+    __syncthreads();
+    float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
+    ternary_phase(c, vbuf, n_sg, c.n_kg, reinterpret_cast<const uint8_t*>(S + c.hd * SS), psum, tot);
+    __syncthreads();                                        // the staging buffer is the key / value buffer
+    if (c.t1 > c.T_qt) residual_pv<T>(a, c, reinterpret_cast<float*>(kbuf), S, SS, tot);
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const float m_i = red[2 * c.r + j], l_i = red[8 + 2 * c.r + j];
+      const float m_new = fmaxf(Mr[j], m_i);
+      const float so = __expf(Mr[j] - m_new), si = __expf(m_i - m_new);
+      Lr[j] = Lr[j] * so + l_i * si;
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        TOT[i][j] = TOT[i][j] * so + tot[i][j] * si;
+        TOT[i][2 + j] = TOT[i][2 + j] * so + tot[i][2 + j] * si;
+      }
+      Mr[j] = m_new;
+    }
+    __syncthreads();                                        // red, S and the buffers are rewritten next
   }
-  cp_async_wait<0>();
-  __syncthreads();
-  score_phase<T>(a, n_chunks, c, kbuf, S, SS);
-  __syncthreads();
-  {
-    // the key groups are spent: the ternary supergroups take their place while the softmax runs
-    const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + (c.t0 / (kG * kSGGroups)) * kSGBytes;
-    for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
-    cp_async_commit();
+  if (c.warp == 0 && c.hd == 0) {
+    red[2 * c.r] = Mr[0]; red[2 * c.r + 1] = Mr[1];
+    red[8 + 2 * c.r] = Lr[0]; red[8 + 2 * c.r + 1] = Lr[1];
   }
-  softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0);
-  __syncthreads();
-  group_sums(c, reinterpret_cast<const __half*>(S), 2 * SS, n_sg * kSGGroups, -5.0f, psum);
-  cp_async_wait<0>();
-  __syncthreads();
-  float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
-  ternary_phase(c, vbuf, n_sg, c.n_kg, reinterpret_cast<const uint8_t*>(S + c.hd * SS), psum, tot);
-  __syncthreads();                                        // the output staging reuses the same buffer
-  epilogue<T>(a, c, kbuf, S, SS, red, tot);
+  write_partial(a, c, blockIdx.x, reinterpret_cast<float*>(kbuf), red, TOT);
 }
 
 // ---------------------------------------------------------------------------------
@@ -638,7 +675,7 @@ __global__ void __launch_bounds__(kThreads, 3) decode_stp_kernel(DecodeArgs a, i
   float* psum_p = psum_t + 8 * stp_sg_max(ST) * kSGGroups;
   float* red = psum_p + 8 * stp_pg_max(ST);
   __half* Pprot = reinterpret_cast<__half*>(kbuf);
-  const Split c = make_split(a);
+  const Split c = make_split(a, blockIdx.x);
   const CacheView& cv = a.cv;
   const int b = c.lb % cv.B;
   const uint32_t* ew = cv.e_words(b);
@@ -748,7 +785,8 @@ __global__ void __launch_bounds__(kThreads, 3) decode_stp_kernel(DecodeArgs a, i
     }
   }
   __syncthreads();                                       // Pprot shares kbuf with the output staging
-  epilogue<T>(a, c, kbuf, S, SS, red, tot);
+  if (c.t1 > c.T_qt) residual_pv<T>(a, c, reinterpret_cast<float*>(kbuf), S, SS, tot);
+  write_partial(a, c, blockIdx.x, reinterpret_cast<float*>(kbuf), red, tot);
 }
 
 cudaError_t launch_decode_mma(const DecodeArgs& a_in, cudaStream_t stream) {
@@ -780,7 +818,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a_in, cudaStream_t stream) {
     else decode_prep_kernel<__nv_bfloat16><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride, n_items);
     count_launches(1);
   }
-  const dim3 grid(a.n_splits, n_slabs);
+  const dim3 grid(a.n_parts, n_slabs);
   if (a.ev_begin) cudaEventRecord(a.ev_begin, stream);
   if (stp) {
     if (a.in_dtype == VIDKV_F16) decode_stp_kernel<__half><<<grid, kThreads, smem, stream>>>(a, chunk_stride);

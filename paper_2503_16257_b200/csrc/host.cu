@@ -74,6 +74,14 @@ int choose_split_tokens(int64_t T_tot, int64_t n_slabs, bool stp) {
   return 160;
 }
 
+// Consecutive splits one CTA folds into a single partial record: as many as still leave about
+// eight waves of CTAs (4 per SM, 148 SMs), at most 8; 1 with protected tokens.
+int choose_splits_per_cta(int64_t n_splits, int64_t n_slabs, bool stp) {
+  if (stp) return 1;
+  const int64_t k = n_splits * n_slabs / 4736;
+  return static_cast<int>(k < 1 ? 1 : (k > 8 ? 8 : k));
+}
+
 int64_t max_partial_entries(const vidkv_config_t& c, int64_t T_max) {
   int64_t best = 0;
   if (T_max < 1) T_max = 1;
@@ -365,6 +373,8 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv;
   a.split_tokens = choose_split_tokens(T_tot, n_slabs, h->n_prot > 0);
   a.n_splits = static_cast<int32_t>((T_tot + a.split_tokens - 1) / a.split_tokens);
+  a.splits_per_cta = choose_splits_per_cta(a.n_splits, n_slabs, h->n_prot > 0);
+  a.n_parts = (a.n_splits + a.splits_per_cta - 1) / a.splits_per_cta;
   if (static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_q * a.n_splits > h->ws.partial_entries) return VIDKV_ERR_CAPACITY;
   if (launch_decode(a, s) != cudaSuccess) return VIDKV_ERR_CUDA;
   const bool flush = a.st.n_res == kR;

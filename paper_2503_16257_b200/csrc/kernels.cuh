@@ -85,6 +85,7 @@ struct DecodeArgs {
   int32_t layer0, n_layers;
   int32_t in_dtype, out_dtype;
   int32_t split_tokens, n_splits;
+  int32_t splits_per_cta, n_parts;   // consecutive splits one CTA folds into one partial record; records per head
   int64_t n_prot;      // protected tokens per batch element (0 = no STP)
   float scale;
   LayerState st;
