@@ -28,9 +28,11 @@ if ROOT not in sys.path:
 
 NOMINAL_HBM_GBS = 8000.0          # the 8 TB/s the targets are quoted against
 FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used if MEASURED_PEAKS.json is absent
-# DRAM bytes per launch of the split-KV decode kernel from the ncu capture summarised in
-# profiles/ (bytes per cached token per KV head, scaled to the launch); None until captured.
-NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = None
+# DRAM bytes per cached token per KV head moved by one launch of the split-KV decode kernel, from the
+# ncu captures summarised in profiles/decode_mma_kernel_batched_4layers.txt (p = 0) and
+# profiles/decode_stp_kernel_batched_4layers_p02.txt (p > 0): a 4-layer cut of the batched workload,
+# scaled to the launch by the token-heads it processes (traffic is proportional to them).
+NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = {"decode_mma_kernel": 75.17, "decode_stp_kernel": 82.01}
 
 
 def algorithmic_decode_bytes(B, L, H_kv, H_q, T_q0, n_flush, n_res, n_prot, elem=2):
@@ -331,9 +333,10 @@ def main():
     q_tokens = n_caches * B * T * L
     kern_bytes = dec_bytes / steps_dec
     kern_gbs = kern_bytes / (kern_avg_ms * 1e-3) / 1e9
-    traffic = None
-    if NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD is not None:
-        traffic = NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD * B * L * H * (T - T % 32)
+    kernel_name = "decode_stp_kernel" if n_prot > 0 else "decode_mma_kernel"
+    traffic = NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD.get(kernel_name)
+    if traffic is not None:
+        traffic = traffic * B * L * H * (T - T % 32)
 
     line = {
         "metric": "packed_kv_decode_attention_GBps", "value": decode_gbs, "unit": "GB/s",
@@ -347,7 +350,7 @@ def main():
         "quantize": {"tokens_per_s": world * q_tokens / (q_ms * 1e-3), "unit": "tokens/s (one position, 4 KV heads, "
                      "one layer, K and V)", "ms_per_bench_step": q_ms, "GBps": world * q_bytes / (q_ms * 1e-3) / 1e9,
                      "pct_of_8TBps": 100.0 * q_bytes / (q_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
-        "roofline": {"bound": "hbm", "kernel": "decode_stp_kernel" if n_prot > 0 else "decode_mma_kernel", "achieved": kern_gbs, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": kernel_name, "achieved": kern_gbs, "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": kern_gbs / peak, "traffic": traffic,
                      "avg_launch_ms": kern_avg_ms, "launches_timed": len(kern_ms)},
         "gpu_launches": int(launches),
