@@ -140,9 +140,11 @@ typedef struct {
 typedef struct vidkv_cache vidkv_cache_t;
 
 /* Sizes (host only).  cache_bytes / workspace_bytes are what vidkv_cache_init wants.
- * The workspace holds split-KV partial results, channel ranges and the gather
- * lists of the token selection; it carries no state between calls except the
- * gather lists, which vidkv_quantize_values reads. */
+ * The workspace holds split-KV partial results, prepared queries, channel ranges and
+ * the gather lists of the token selection.  Between calls it carries the gather lists,
+ * which vidkv_quantize_values reads, and the armed channel-range accumulators that
+ * vidkv_cache_init sets up: it belongs to one handle and must not be overwritten while
+ * that handle is in use. */
 vidkv_status_t vidkv_cache_bytes(const vidkv_config_t* cfg, size_t* cache_bytes, size_t* workspace_bytes);
 
 /* Offsets of every region of the packed cache for this configuration (host only). */

@@ -104,7 +104,7 @@ struct WsPlan {
 void plan_workspace(const vidkv_config_t& c, const Layout& L, WsPlan* w) {
   int64_t off = 0;
   w->minmax_off = off;
-  off = round_up(off + static_cast<int64_t>(c.L) * c.B * c.H_kv * 2 * kD * 4, kAlign);
+  off = round_up(off + 2 * static_cast<int64_t>(c.L) * c.B * c.H_kv * 2 * kD * 4, kAlign);   // two alternating buffers
   w->partial_entries = max_partial_entries(c, L.max_total_tokens);
   w->partials_off = off;
   off = round_up(off + w->partial_entries * 130 * 4, kAlign);
@@ -142,8 +142,25 @@ struct vidkv_cache {
   uint8_t* workspace;
   bool sel_set;
   int64_t sel_T, n_prot;
+  int mm_parity = 0;            // which min / max buffer the next key quantization accumulates into
+  int64_t mm_dirty[2] = {0, 0}; // words of each buffer written since it was last re-armed
   std::vector<LayerInfo> layers;
 };
+
+// The min / max buffers of the next key quantization over n_slabs slabs (see MinMaxBuffers).
+static MinMaxBuffers next_minmax(vidkv_cache* h, int64_t n_slabs) {
+  const int64_t words = static_cast<int64_t>(h->cfg.L) * h->cfg.B * h->cfg.H_kv * 2 * kD;
+  uint32_t* base = reinterpret_cast<uint32_t*>(h->workspace + h->ws.minmax_off);
+  const int p = h->mm_parity;
+  MinMaxBuffers mm;
+  mm.cur = base + p * words;
+  mm.next = base + (1 - p) * words;
+  mm.next_dirty_words = static_cast<int>(h->mm_dirty[1 - p]);
+  h->mm_dirty[1 - p] = 0;
+  h->mm_dirty[p] = n_slabs * 2 * kD;
+  h->mm_parity = 1 - p;
+  return mm;
+}
 
 extern "C" {
 
@@ -214,6 +231,11 @@ vidkv_status_t vidkv_cache_init(const vidkv_config_t* cfg, void* cache, size_t c
   h->layers.assign(cfg->L, LayerInfo());
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(h->cache, 0, static_cast<size_t>(l.total_bytes), s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }
+  if (launch_init_minmax(reinterpret_cast<uint32_t*>(h->workspace + h->ws.minmax_off),
+                         2 * static_cast<int64_t>(cfg->L) * cfg->B * cfg->H_kv * 2 * kD, s) != cudaSuccess) {
+    delete h;
+    return VIDKV_ERR_CUDA;
+  }
   const uint32_t hdr[3] = {kMagic, static_cast<uint32_t>(vidkv_version()), 0u};
   if (cudaMemcpyAsync(h->cache, hdr, sizeof(hdr), cudaMemcpyHostToDevice, s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }
   if (cudaStreamSynchronize(s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }   // hdr is a stack buffer
@@ -306,8 +328,10 @@ vidkv_status_t vidkv_quantize_keys(vidkv_cache_t* h, int32_t layer, const void* 
   const int r = static_cast<int>(T % kG);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   KSrc src{K, stride_b, stride_h, stride_t, h->cfg.H_kv};
-  uint32_t* minmax = reinterpret_cast<uint32_t*>(h->workspace + h->ws.minmax_off);
-  if (launch_quantize_keys(h->cfg.in_dtype, src, T_q, h->cv, layer, 1, 0, 0, minmax, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  if (T_q > 0) {
+    const MinMaxBuffers mm = next_minmax(h, static_cast<int64_t>(h->cfg.B) * h->cfg.H_kv);
+    if (launch_quantize_keys(h->cfg.in_dtype, src, T_q, h->cv, layer, 1, 0, 0, mm, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  }
   if (launch_copy_to_residual(h->cfg.in_dtype, src, T_q, r, h->cv, layer, false, 0, s) != cudaSuccess) return VIDKV_ERR_CUDA;
   li.k_done = true; li.T = T; li.T_q0 = T_q; li.n_res = r; li.n_flush = 0;
   return VIDKV_OK;
@@ -383,10 +407,10 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
     const uint8_t* slab0 = h->cache + h->cv.slab_offset + static_cast<int64_t>(layer_begin) * h->cfg.B * h->cfg.H_kv * h->cv.slab_stride;
     KSrc ksrc{slab0 + h->cv.kres_offset, es * h->cfg.H_kv, es, kD, h->cfg.H_kv};
     KSrc vsrc{slab0 + h->cv.vres_offset, es * h->cfg.H_kv, es, kD, h->cfg.H_kv};
-    uint32_t* minmax = reinterpret_cast<uint32_t*>(h->workspace + h->ws.minmax_off);
+    const MinMaxBuffers mm = next_minmax(h, static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv);
     const int chunk = 1 + static_cast<int>(first.n_flush);
     const int64_t kgroup0 = first.T_q0 / kG + (kR / kG) * first.n_flush;
-    if (launch_quantize_keys(dt, ksrc, kR, h->cv, layer_begin, n_layers, chunk, kgroup0, minmax, s) != cudaSuccess)
+    if (launch_quantize_keys(dt, ksrc, kR, h->cv, layer_begin, n_layers, chunk, kgroup0, mm, s) != cudaSuccess)
       return VIDKV_ERR_CUDA;
     const int64_t n_rest = first.T_q0 - h->n_prot;
     const int64_t tgroup0 = (n_rest + kG - 1) / kG + (kR / kG) * first.n_flush;

@@ -22,13 +22,22 @@ struct SelView {
   int64_t n_prot;
 };
 
-__global__ void init_min_kernel(uint32_t* minmax, int n_slabs);
+// Channel min / max accumulators of the range pass: 256 ordered-integer words per slab (128
+// minima that start at all ones, 128 maxima that start at zero).  Two buffers alternate: a call
+// accumulates into `cur`, which the call before it re-armed, and re-arms the first
+// `next_dirty_words` words of `next` for the call after it, so no call spends a launch on it.
+struct MinMaxBuffers {
+  uint32_t* cur;
+  uint32_t* next;
+  int next_dirty_words;
+};
+cudaError_t launch_init_minmax(uint32_t* minmax, int64_t n_words, cudaStream_t stream);
 
 // Algorithm 3 on `T_tokens` tokens (a multiple of 32) of every slab of layers
 // [layer0, layer0 + n_layers): writes chunk `chunk` of the chunk table and the key groups
-// starting at group index kgroup0.  minmax: scratch, 256 uint32 per slab.
+// starting at group index kgroup0.
 cudaError_t launch_quantize_keys(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0,
-                                 int n_layers, int chunk, int64_t kgroup0, uint32_t* minmax, cudaStream_t stream);
+                                 int n_layers, int chunk, int64_t kgroup0, const MinMaxBuffers& mm, cudaStream_t stream);
 
 // Encode pass of Algorithm 3 for `n_slabs` slabs whose channel split (chunk table entry
 // `chunk`) is already written.

@@ -57,7 +57,12 @@ __global__ void __launch_bounds__(256) k_range_kernel(KSrc src, int64_t T_tokens
 // 64 normal ids ascending.
 // ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kD) k_select_kernel(const uint32_t* __restrict__ minmax, CacheView cv,
-                                                      int layer0, int slabs_per_layer, int chunk) {
+                                                      int layer0, int slabs_per_layer, int chunk,
+                                                      uint32_t* __restrict__ rearm, int rearm_words) {
+  // Re-arm the buffer the next call accumulates into (min half all ones, max half zero).  Nobody
+  // reads it now: its last readers ran before this call's range pass in stream order.
+  for (int i = blockIdx.x * kD + threadIdx.x; i < rearm_words; i += gridDim.x * kD)
+    rearm[i] = (i & (2 * kD - 1)) < kD ? 0xffffffffu : 0u;
   const int slab = blockIdx.x;
   const int layer = layer0 + slab / slabs_per_layer;
   const int bh = slab % slabs_per_layer;
@@ -90,36 +95,40 @@ __global__ void __launch_bounds__(kD) k_select_kernel(const uint32_t* __restrict
 // ---------------------------------------------------------------------------------
 template <typename T>
 static cudaError_t launch_keys_t(const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0, int n_layers,
-                                 int chunk, int64_t kgroup0, uint32_t* minmax, cudaStream_t stream) {
+                                 int chunk, int64_t kgroup0, const MinMaxBuffers& mm, cudaStream_t stream) {
+  uint32_t* minmax = mm.cur;
   const int slabs_per_layer = cv.B * cv.H_kv;
   const int n_slabs = slabs_per_layer * n_layers;
   if (T_tokens <= 0 || n_slabs <= 0) return cudaSuccess;
   cudaError_t e;
-  // min array -> all ones (largest ordered key), max array -> zero, interleaved per slab
-  if ((e = cudaMemsetAsync(minmax, 0, static_cast<size_t>(n_slabs) * 2 * kD * sizeof(uint32_t), stream))) return e;
-  init_min_kernel<<<(n_slabs * kD + 255) / 256, 256, 0, stream>>>(minmax, n_slabs);
   int tokens_per_block = 512;
   const int64_t splits = (T_tokens + tokens_per_block - 1) / tokens_per_block;
   k_range_kernel<T><<<dim3(static_cast<unsigned>(splits), n_slabs), 256, 0, stream>>>(src, T_tokens, tokens_per_block,
                                                                                        minmax);
-  k_select_kernel<<<n_slabs, kD, 0, stream>>>(minmax, cv, layer0, slabs_per_layer, chunk);
+  k_select_kernel<<<n_slabs, kD, 0, stream>>>(minmax, cv, layer0, slabs_per_layer, chunk, mm.next, mm.next_dirty_words);
   if ((e = launch_encode_keys(std::is_same<T, __half>::value ? VIDKV_F16 : VIDKV_BF16, src, T_tokens, cv,
                               layer0, n_slabs, slabs_per_layer, chunk, kgroup0, stream)))
     return e;
-  count_launches(3);
+  count_launches(2);
   return cudaGetLastError();
 }
 
-__global__ void init_min_kernel(uint32_t* minmax, int n_slabs) {
+__global__ void init_min_kernel(uint32_t* minmax, int n_words) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n_slabs * kD) minmax[(i / kD) * 2 * kD + (i % kD)] = 0xffffffffu;
+  if (i < n_words) minmax[i] = (i & (2 * kD - 1)) < kD ? 0xffffffffu : 0u;
+}
+
+cudaError_t launch_init_minmax(uint32_t* minmax, int64_t n_words, cudaStream_t stream) {
+  init_min_kernel<<<static_cast<unsigned>((n_words + 255) / 256), 256, 0, stream>>>(minmax, static_cast<int>(n_words));
+  count_launches(1);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_keys(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0,
-                                 int n_layers, int chunk, int64_t kgroup0, uint32_t* minmax, cudaStream_t stream) {
+                                 int n_layers, int chunk, int64_t kgroup0, const MinMaxBuffers& mm, cudaStream_t stream) {
   if (dtype == VIDKV_F16)
-    return launch_keys_t<__half>(src, T_tokens, cv, layer0, n_layers, chunk, kgroup0, minmax, stream);
-  return launch_keys_t<__nv_bfloat16>(src, T_tokens, cv, layer0, n_layers, chunk, kgroup0, minmax, stream);
+    return launch_keys_t<__half>(src, T_tokens, cv, layer0, n_layers, chunk, kgroup0, mm, stream);
+  return launch_keys_t<__nv_bfloat16>(src, T_tokens, cv, layer0, n_layers, chunk, kgroup0, mm, stream);
 }
 
 }  // namespace vidkv
