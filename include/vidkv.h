@@ -227,7 +227,7 @@ vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* handle, int32_t layer, flo
  * The split-KV scratch lives in a 16 MiB array inside the library, which every GPU that
  * loads the library keeps until the process exits.  It must hold 520 bytes per (query head,
  * split) record, n_layers * B * H_q * ceil(tokens / split) of them with split = 160, 320 or
- * 640 tokens (320 at most when n_protected > 0), plus 3072 bytes per (layer, batch element,
+ * 640 tokens, plus 3072 bytes per (layer, batch element,
  * KV head, chunk) -- larger problems return VIDKV_ERR_CAPACITY (use fewer layers per call).
  * Nothing is allocated or freed.  The first call on each device looks up the array's device
  * address, so make that first call outside any stream capture.  All calls share the array:

@@ -362,7 +362,10 @@ __device__ __forceinline__ void score_phase(const DecodeArgs& a, int n_chunks, c
 // warp's 32 channels.  prow = this lane's probability row (binary16), its entry 0 matching
 // token 0 of the first staged supergroup; psum = -5 * group sums of those probabilities,
 // [group][8 heads]; groups from n_grp on do not exist (zero scale).
-__device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbuf, int n_sg, int n_grp,
+// With MASKED, groups before g_first hold no token of this split either: their MMAs, loads and
+// scale steps are skipped (the digit peel still has to pass over them).
+template <bool MASKED>
+__device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbuf, int n_sg, int g_first, int n_grp,
                                               const uint8_t* prow, const float* psum, float (&tot)[2][4]) {
   const int warp = c.warp, hd = c.hd, r = c.r;
   const uint32_t m_field = c.m_field, c_four = c.c_four;
@@ -370,6 +373,7 @@ __device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbu
     for (int sg = 0; sg < n_sg; ++sg) {
       const uint8_t* sgp = vbuf + sg * kSGBytes;
       const int n_valid = min(kSGGroups, n_grp - sg * kSGGroups);
+      const int g_lo = MASKED ? g_first - sg * kSGGroups : 0;
       float acc[kSGGroups][2][4];
       float2 ps[kSGGroups];
 #pragma unroll
@@ -388,6 +392,7 @@ __device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbu
         for (int k = 0; k < 8; ++k) W[k] = mad_u32(W[k], 3u, 0u);          // 3 * byte per 16-bit lane
 #pragma unroll
         for (int g = 0; g < kSGGroups; ++g) {
+          if (MASKED && g >= n_valid) continue;
           uint32_t A[8];
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
@@ -396,6 +401,7 @@ __device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbu
             A[k] = and_or(W[k], m_field, c_four);
             W[k] = mad_u32(A[k], 0xfffffffdu, mad_u32(W[k], 3u, 0xcc00cc00u));
           }
+          if (MASKED && g < g_lo) continue;
           // groups past the end of the cache meet zero probabilities (and a zero scale below)
           const uint8_t* pb = prow + (sg * (kSGGroups * kG) + g * kG + kt * 16 + 2 * r) * 2;
           const uint32_t b0 = *reinterpret_cast<const uint32_t*>(pb);
@@ -411,7 +417,7 @@ __device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbu
       }
 #pragma unroll
       for (int g = 0; g < kSGGroups; ++g) {
-        {
+        if (!MASKED || (g >= g_lo && g < n_valid)) {
           uint2 sc = *reinterpret_cast<const uint2*>(sgp + kSG_Scales + g * (kD * 2) + (32 * warp + 4 * hd) * 2);
           if (g >= n_valid) sc = make_uint2(0u, 0u);
           const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));
@@ -426,25 +432,25 @@ __device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbu
   }
 }
 
-// P V of the FP16 / BF16 residual rows of the split, added to tot.  The probabilities of the
-// residual tokens sit in S in place (binary16, token order).  Thread = channel computes the
-// eight heads' sums into O[head][channel] (the staging buffer, which must be free), then every
-// thread picks up the entries of its accumulator layout.  All threads call it or none.
+// P V of the FP16 / BF16 residual rows of the split, added to tot.  The probability of
+// residual row rr and head k is pres[k * pres_stride + pres_index0 + rr] (binary16).  Thread =
+// channel computes the eight heads' sums into O[head][channel] (the staging buffer, which must
+// be free), then every thread picks up the entries of its accumulator layout.  All threads
+// call it or none.
 template <typename T>
-__device__ __forceinline__ void residual_pv(const DecodeArgs& a, const Split& c, float* O, const float* S, int SS,
-                                            float (&tot)[2][4]) {
+__device__ __forceinline__ void residual_pv(const DecodeArgs& a, const Split& c, float* O, const __half* pres,
+                                            int pres_stride, int pres_index0, float (&tot)[2][4]) {
   const CacheView& cv = a.cv;
   const int ch = c.tid;
   const int r_begin = static_cast<int>(max(c.t0, c.T_qt) - c.T_qt), r_end = static_cast<int>(c.t1 - c.T_qt);
   const T* vres = reinterpret_cast<const T*>(c.slab_ptr + cv.vres_offset);
-  const int off = static_cast<int>(c.T_qt - c.t0);
   float o[kMaxRep];
 #pragma unroll
   for (int k = 0; k < kMaxRep; ++k) o[k] = 0.0f;
   for (int rr = r_begin; rr < r_end; ++rr) {
     const float v = Elem<T>::to_float(vres[rr * kD + ch]);
 #pragma unroll
-    for (int k = 0; k < kMaxRep; ++k) o[k] += __half2float(reinterpret_cast<const __half*>(S + k * SS)[off + rr]) * v;
+    for (int k = 0; k < kMaxRep; ++k) o[k] += __half2float(pres[k * pres_stride + pres_index0 + rr]) * v;
   }
 #pragma unroll
   for (int k = 0; k < kMaxRep; ++k) O[k * kD + ch] = o[k];
@@ -488,14 +494,15 @@ __device__ __forceinline__ void write_partial(const DecodeArgs& a, const Split& 
 
 // Softmax numerators of the 8 score rows (warp w owns rows 2 w and 2 w + 1): p = exp(scale *
 // (score - row max)), rounded to binary16.  Without protected tokens the probabilities
-// replace the scores in place (entry i of the row, as binary16).  With them (STP) the
-// quantized tokens [0, nq) are scattered into the stream-ordered rows Ptern / Pprot through
-// `map` (bit 15 = protected stream) and only the residual tokens [nq, n_loc) stay in place.
+// replace the scores in place (entry i of the row, as binary16).  With them (STP) the row is
+// cleared once its scores are in registers and becomes the ternary-stream row: quantized
+// tokens [0, nq) go to their stream position through `map` (bit 15 = protected stream, row of
+// Pprot), residual tokens [nq, n_loc) to Pres[row][i - nq].
 // red[row] = scaled row maximum, red[8 + row] = sum of the probabilities.
 template <bool STP>
 __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& c, float* S, int SS, float* red,
-                                              int n_pad, const uint16_t* map, __half* Ptern, int PT, __half* Pprot,
-                                              int PP) {
+                                              int n_pad, const uint16_t* map, __half* Pprot, int PP, __half* Pres,
+                                              int PRS) {
   const int lane = c.lane, n_loc = c.n_loc;
   const float sl2 = a.scale * 1.4426950408889634f;
   constexpr int kMaxPairs = 10;                                          // ST <= 640: 320 pairs per row
@@ -515,21 +522,30 @@ __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& 
 #pragma unroll
     for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     __syncwarp();
+    if (STP) {
+      for (int i = lane; i < SS / 4; i += 32) reinterpret_cast<uint4*>(row)[i] = make_uint4(0u, 0u, 0u, 0u);
+      __syncwarp();
+    }
     const float ms = m * sl2;
     float l = 0.0f;
     uint32_t* prow = reinterpret_cast<uint32_t*>(row);
+    __half* trow = reinterpret_cast<__half*>(row);
 #pragma unroll
     for (int k = 0; k < kMaxPairs; ++k) {
       const int i = 2 * lane + 64 * k;
       const float p0 = ex2_approx(fmaf(v[k].x, sl2, -ms)), p1 = ex2_approx(fmaf(v[k].y, sl2, -ms));
       l += p0 + p1;
-      if (STP && i < c.nq) {
-        const uint32_t d = *reinterpret_cast<const uint32_t*>(map + i);
-        const uint32_t d0 = d & 0xffffu, d1 = d >> 16;
-        __half* q0 = (d0 & 0x8000u) ? Pprot + row_h * PP + (d0 & 0x7fffu) : Ptern + row_h * PT + d0;
-        __half* q1 = (d1 & 0x8000u) ? Pprot + row_h * PP + (d1 & 0x7fffu) : Ptern + row_h * PT + d1;
-        *q0 = __float2half_rn(p0);
-        *q1 = __float2half_rn(p1);
+      if (STP) {
+        if (i < c.nq) {
+          const uint32_t d = *reinterpret_cast<const uint32_t*>(map + i);
+          const uint32_t d0 = d & 0xffffu, d1 = d >> 16;
+          __half* q0 = (d0 & 0x8000u) ? Pprot + row_h * PP + (d0 & 0x7fffu) : trow + d0;
+          __half* q1 = (d1 & 0x8000u) ? Pprot + row_h * PP + (d1 & 0x7fffu) : trow + d1;
+          *q0 = __float2half_rn(p0);
+          *q1 = __float2half_rn(p1);
+        } else if (i < n_loc) {
+          *reinterpret_cast<uint32_t*>(Pres + row_h * PRS + (i - c.nq)) = pack_half2(p0, p1);
+        }
       } else if (i < n_pad) {
         prow[i >> 1] = pack_half2(p0, p1);
       }
@@ -611,9 +627,11 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
     cp_async_wait<0>();
     __syncthreads();
     float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
-    ternary_phase(c, vbuf, n_sg, c.n_kg, reinterpret_cast<const uint8_t*>(S + c.hd * SS), psum, tot);
+    ternary_phase<false>(c, vbuf, n_sg, 0, c.n_kg, reinterpret_cast<const uint8_t*>(S + c.hd * SS), psum, tot);
     __syncthreads();                                        // the staging buffer is the key / value buffer
-    if (c.t1 > c.T_qt) residual_pv<T>(a, c, reinterpret_cast<float*>(kbuf), S, SS, tot);
+    if (c.t1 > c.T_qt)
+      residual_pv<T>(a, c, reinterpret_cast<float*>(kbuf), reinterpret_cast<const __half*>(S), 2 * SS,
+                     static_cast<int>(c.T_qt - c.t0), tot);
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
       const float m_i = red[2 * c.r + j], l_i = red[8 + 2 * c.r + j];
@@ -642,45 +660,53 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
 // stream (position = token - protected tokens before it; flushed tokens follow from the next
 // group boundary), protected ones in 2-bit groups.  The probabilities are therefore scattered
 // into stream-ordered rows, zero wherever a staged stream position belongs to another split.
-// Shared memory for a split of ST tokens (160 or 320):
-//   kbuf  ST/32 key groups; after phase 1: Pprot, 8 rows of (ST/32 + 1) * 32 + 8 binary16;
-//         at the end the output staging
-//   vbuf  ST/160 + 2 ternary supergroups     pbuf  ST/32 + 1 protected groups
-//   S     8 rows of ST + 4 floats            Ptern 8 rows of (ST/160 + 2) * 160 + 8 binary16
-//   map   ST destinations                    psum_t, psum_p, red
+// Shared memory for a split of ST tokens (160, 320 or 640):
+//   buf   ST/32 key groups, then ST/160 + 2 ternary supergroups, at the end the output staging
+//   S     8 rows of SSP floats: scores, then the ternary-stream probabilities (binary16)
+//   Pprot 8 rows of (ST/32 + 1) * 32 + 8 binary16    Pres 8 rows of 136 binary16 (residual)
+//   map   ST destinations                            psum_t, psum_p, red
+// The protected groups are read from global memory as they are consumed.
 // ---------------------------------------------------------------------------------
 __host__ __device__ inline int stp_sg_max(int ST) { return ST / 160 + 2; }
 __host__ __device__ inline int stp_pg_max(int ST) { return ST / 32 + 1; }
+__host__ __device__ inline int stp_row_floats(int ST) {       // a row must hold the scores and, later, the stream
+  const int need = stp_sg_max(ST) * 80 + 4;
+  return ST + 4 > need ? ST + 4 : need;
+}
+constexpr int kPresStride = kR + 8;
 
 size_t decode_stp_smem_bytes(int ST) {
-  const int PT = stp_sg_max(ST) * 160 + 8;
-  return static_cast<size_t>(ST / 32) * kKGroupBytes + static_cast<size_t>(stp_sg_max(ST)) * kSGBytes +
-         static_cast<size_t>(stp_pg_max(ST)) * kPGBytes + sizeof(float) * 8 * (ST + 4) + 16 * PT + 2 * ST +
+  const size_t buf = static_cast<size_t>(stp_sg_max(ST)) * kSGBytes;        // >= ST/32 key groups
+  return buf + sizeof(float) * 8 * stp_row_floats(ST) + 16 * (stp_pg_max(ST) * 32 + 8) + 16 * kPresStride + 2 * ST +
          sizeof(float) * (8 * stp_sg_max(ST) * kSGGroups + 8 * stp_pg_max(ST) + 16);
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads, 3) decode_stp_kernel(DecodeArgs a, int n_chunks) {
+__global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, int n_chunks) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   const int ST = a.split_tokens;
-  const int SS = ST + 4;
-  const int PT = stp_sg_max(ST) * 160 + 8, PP = stp_pg_max(ST) * 32 + 8;
-  uint8_t* kbuf = smem_raw;
-  uint8_t* vbuf = kbuf + (ST / 32) * kKGroupBytes;
-  uint8_t* pbuf = vbuf + stp_sg_max(ST) * kSGBytes;
-  float* S = reinterpret_cast<float*>(pbuf + stp_pg_max(ST) * kPGBytes);
-  __half* Ptern = reinterpret_cast<__half*>(S + 8 * SS);
-  uint16_t* map = reinterpret_cast<uint16_t*>(Ptern + 8 * PT);
+  const int SS = stp_row_floats(ST);
+  const int PT = 2 * SS, PP = stp_pg_max(ST) * 32 + 8;
+  uint8_t* buf = smem_raw;
+  float* S = reinterpret_cast<float*>(buf + stp_sg_max(ST) * kSGBytes);
+  __half* Pprot = reinterpret_cast<__half*>(S + 8 * SS);
+  __half* Pres = Pprot + 8 * PP;
+  uint16_t* map = reinterpret_cast<uint16_t*>(Pres + 8 * kPresStride);
   float* psum_t = reinterpret_cast<float*>(map + ST);
   float* psum_p = psum_t + 8 * stp_sg_max(ST) * kSGGroups;
   float* red = psum_p + 8 * stp_pg_max(ST);
-  __half* Pprot = reinterpret_cast<__half*>(kbuf);
   const Split c = make_split(a, blockIdx.x);
   const CacheView& cv = a.cv;
   const int b = c.lb % cv.B;
   const uint32_t* ew = cv.e_words(b);
   const uint32_t* ep = cv.e_prefix(b);
 
+  // ---- keys first
+  {
+    const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
+    for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(buf + i * 16, ksrc + i * 16);
+    cp_async_commit();
+  }
   // ---- where the split's tokens sit in the two value streams
   const int64_t tp0 = min(c.t0, c.T_q0), tp1 = min(c.tq1, c.T_q0);              // prefill part
   const int64_t pp0 = ep[tp0 / kG], pp1 = ep[tp1 / kG];                         // protected positions
@@ -699,18 +725,7 @@ __global__ void __launch_bounds__(kThreads, 3) decode_stp_kernel(DecodeArgs a, i
   const int64_t Pbase = pgA * kG;
   const int64_t tg_total = (n_rest + kG - 1) / kG + (kR / kG) * a.st.n_flush;   // ternary groups that exist
 
-  // ---- stage keys, ternary supergroups, protected groups
-  {
-    const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
-    for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
-    cp_async_commit();
-    const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + sgA * kSGBytes;
-    for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
-    const uint8_t* psrc = c.slab_ptr + cv.prot_offset + pgA * kPGBytes;
-    for (int i = c.tid; i < n_pg * (kPGBytes / 16); i += kThreads) cp_async16(pbuf + i * 16, psrc + i * 16);
-    cp_async_commit();
-  }
-  // ---- destinations of the quantized tokens, cleared ternary rows
+  // ---- destinations of the quantized tokens, cleared protected rows
   for (int i = c.tid; i < c.nq; i += kThreads) {
     const int64_t t = c.t0 + i;
     uint32_t d;
@@ -723,35 +738,56 @@ __global__ void __launch_bounds__(kThreads, 3) decode_stp_kernel(DecodeArgs a, i
     }
     map[i] = static_cast<uint16_t>(d);
   }
-  for (int i = c.tid; i < PT; i += kThreads) reinterpret_cast<uint4*>(Ptern)[i] = make_uint4(0u, 0u, 0u, 0u);
-
-  cp_async_wait<1>();
-  __syncthreads();
-  score_phase<T>(a, n_chunks, c, kbuf, S, SS);
-  __syncthreads();
   for (int i = c.tid; i < PP; i += kThreads) reinterpret_cast<uint4*>(Pprot)[i] = make_uint4(0u, 0u, 0u, 0u);
+
+  cp_async_wait<0>();
   __syncthreads();
-  softmax_phase<true>(a, c, S, SS, red, (c.n_loc + 1) & ~1, map, Ptern, PT, Pprot, PP);
+  score_phase<T>(a, n_chunks, c, buf, S, SS);
   __syncthreads();
-  group_sums(c, Ptern, PT, n_sg * kSGGroups, -5.0f, psum_t);
+  {
+    // the key groups are spent: the ternary supergroups take their place while the softmax runs
+    const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + sgA * kSGBytes;
+    for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(buf + i * 16, vsrc + i * 16);
+    cp_async_commit();
+  }
+  softmax_phase<true>(a, c, S, SS, red, 0, map, Pprot, PP, Pres, kPresStride);
+  __syncthreads();
+  group_sums(c, reinterpret_cast<const __half*>(S), PT, n_sg * kSGGroups, -5.0f, psum_t);
   group_sums(c, Pprot, PP, n_pg, 1.0f, psum_p);
   cp_async_wait<0>();
   __syncthreads();
 
   float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
-  ternary_phase(c, vbuf, n_sg, static_cast<int>(min(tg_total - sgA * kSGGroups, static_cast<int64_t>(n_sg * kSGGroups))),
-                reinterpret_cast<const uint8_t*>(Ptern + c.hd * PT), psum_t, tot);
+  // groups of the staged supergroups that hold tokens of this split: [U0 / 32, ceil(U1 / 32)), and no group past the stream's end
+  const int g_first = static_cast<int>(U0 / kG - sgA * kSGGroups);
+  const int g_end = static_cast<int>(min(tg_total, (U1 + kG - 1) / kG) - sgA * kSGGroups);
+  ternary_phase<true>(c, buf, n_sg, g_first, g_end, reinterpret_cast<const uint8_t*>(S + c.hd * SS), psum_t, tot);
   // ---- protected stream: 2-bit codes (Eq. 4) as 4 + code, then s * (acc - 4 sum p) + z * sum p
-  {
+  if (n_pg > 0) {
     const int warp = c.warp, hd = c.hd, r = c.r;
     const uint8_t* prow = reinterpret_cast<const uint8_t*>(Pprot + hd * PP);
+    const uint8_t* gbase = c.slab_ptr + cv.prot_offset + pgA * kPGBytes;
+    const int w_off = (((warp * 4) + r) * 8 + hd) * 4, m_off = (32 * warp + 4 * hd) * 2;
+    // operands of the group being consumed are loaded one group ahead
+    uint32_t w0 = __ldg(reinterpret_cast<const uint32_t*>(gbase + w_off));
+    uint32_t w1 = __ldg(reinterpret_cast<const uint32_t*>(gbase + 512 + w_off));
+    uint2 sc = __ldg(reinterpret_cast<const uint2*>(gbase + kPG_S + m_off));
+    uint2 zc = __ldg(reinterpret_cast<const uint2*>(gbase + kPG_Z + m_off));
     for (int pg = 0; pg < n_pg; ++pg) {
-      const uint8_t* gp = pbuf + pg * kPGBytes;
+      const uint32_t wk[2] = {w0, w1};
+      const uint2 scc = sc, zcc = zc;
+      if (pg + 1 < n_pg) {
+        const uint8_t* gp = gbase + (pg + 1) * kPGBytes;
+        w0 = __ldg(reinterpret_cast<const uint32_t*>(gp + w_off));
+        w1 = __ldg(reinterpret_cast<const uint32_t*>(gp + 512 + w_off));
+        sc = __ldg(reinterpret_cast<const uint2*>(gp + kPG_S + m_off));
+        zc = __ldg(reinterpret_cast<const uint2*>(gp + kPG_Z + m_off));
+      }
       const float2 sp = *reinterpret_cast<const float2*>(psum_p + pg * 8 + 2 * r);
       float acc[2][4];
 #pragma unroll
       for (int kt = 0; kt < 2; ++kt) {
-        const uint32_t w = *reinterpret_cast<const uint32_t*>(gp + ((((kt * 4 + warp) * 4 + r) * 8) + hd) * 4);
+        const uint32_t w = wk[kt];
         uint32_t x[8];
         x[0] = and_or(w << 8, c.m_field, c.c_four);
         x[1] = and_or(w << 6, c.m_field, c.c_four);
@@ -772,21 +808,21 @@ __global__ void __launch_bounds__(kThreads, 3) decode_stp_kernel(DecodeArgs a, i
           mma_f16(acc[1], x[2], x[3], x[6], x[7], b0, b1);
         }
       }
-      const uint2 sc = *reinterpret_cast<const uint2*>(gp + kPG_S + (32 * warp + 4 * hd) * 2);
-      const uint2 zc = *reinterpret_cast<const uint2*>(gp + kPG_Z + (32 * warp + 4 * hd) * 2);
-      const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));
-      const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));
-      const float2 za = __half22float2(*reinterpret_cast<const __half2*>(&zc.x));
-      const float2 zb = __half22float2(*reinterpret_cast<const __half2*>(&zc.y));
+      const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&scc.x));
+      const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&scc.y));
+      const float2 za = __half22float2(*reinterpret_cast<const __half2*>(&zcc.x));
+      const float2 zb = __half22float2(*reinterpret_cast<const __half2*>(&zcc.y));
       tot[0][0] += sa.x * acc[0][0] + za.x * sp.x; tot[0][1] += sa.x * acc[0][1] + za.x * sp.y;
       tot[0][2] += sa.y * acc[0][2] + za.y * sp.x; tot[0][3] += sa.y * acc[0][3] + za.y * sp.y;
       tot[1][0] += sb.x * acc[1][0] + zb.x * sp.x; tot[1][1] += sb.x * acc[1][1] + zb.x * sp.y;
       tot[1][2] += sb.y * acc[1][2] + zb.y * sp.x; tot[1][3] += sb.y * acc[1][3] + zb.y * sp.y;
     }
   }
-  __syncthreads();                                       // Pprot shares kbuf with the output staging
-  if (c.t1 > c.T_qt) residual_pv<T>(a, c, reinterpret_cast<float*>(kbuf), S, SS, tot);
-  write_partial(a, c, blockIdx.x, reinterpret_cast<float*>(kbuf), red, tot);
+  __syncthreads();                                       // the output staging reuses buf
+  if (c.t1 > c.T_qt)
+    residual_pv<T>(a, c, reinterpret_cast<float*>(buf), Pres, kPresStride,
+                   -static_cast<int>(max(c.t0, c.T_qt) - c.T_qt), tot);
+  write_partial(a, c, blockIdx.x, reinterpret_cast<float*>(buf), red, tot);
 }
 
 cudaError_t launch_decode_mma(const DecodeArgs& a_in, cudaStream_t stream) {

@@ -66,11 +66,11 @@ void compute_layout(const vidkv_config_t& c, Layout* out) {
 }
 
 // Tokens per split: the largest of {640, 320, 160} that still gives >= 4 CTAs per SM on a
-// 148-SM part, else 160.  Caches with protected tokens stage two value streams and stop at 320.
-int choose_split_tokens(int64_t T_tot, int64_t n_slabs, bool stp) {
+// 148-SM part, else 160.
+int choose_split_tokens(int64_t T_tot, int64_t n_slabs, bool /*stp*/) {
   const int cand[3] = {640, 320, 160};
   for (int s : cand)
-    if ((!stp || s <= 320) && n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
+    if (n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
   return 160;
 }
 

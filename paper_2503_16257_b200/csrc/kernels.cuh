@@ -108,7 +108,7 @@ inline void count_launches(int n) { g_launch_count += static_cast<unsigned long 
 // Split-KV attention over the packed cache + residual, then the merge of the partials.
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
 // The tensor-core split kernels and their query preparation; scratch for `n_slabs` slabs of
-// `n_chunks` chunks each.  With protected tokens the split may not exceed 320 tokens.
+// `n_chunks` chunks each.
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t stream);
 size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks);
 // Write k_new / v_new [n_layers, B, H_kv, D] into row `row` of the residual rings.

@@ -38,11 +38,11 @@ vidkv_status_t static_partials(float** out) {
 }
 
 // Tokens per split, by the same rule of thumb as the regular entry point: the largest of
-// {640, 320, 160} (320 at most with protected tokens) that still yields about four CTAs per SM.
-int split_tokens_for(int64_t T_tot, int64_t n_slabs, bool stp) {
+// {640, 320, 160} that still yields about four CTAs per SM.
+int split_tokens_for(int64_t T_tot, int64_t n_slabs, bool /*stp*/) {
   const int cand[3] = {640, 320, 160};
   for (int s : cand)
-    if ((!stp || s <= 320) && n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
+    if (n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
   return 160;
 }
 
