@@ -116,7 +116,7 @@ __global__ void dft_table_kernel() {
 }
 
 size_t k_encode_smem_bytes() {
-  return kEncTokens * kRowBytes + kDftWords * 4 + 4 * 3 * 32 * 4 + 8 * 64 * 4 + kD + 4 * 128 * 32;
+  return kEncTokens * kRowBytes + 4 * 3 * 32 * 4 + 8 * 64 * 4 + kD + 4 * 128 * 32;
 }
 
 template <typename T>
@@ -124,8 +124,8 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
                                                        int slabs_per_layer, int chunk, int64_t kgroup0) {
   extern __shared__ __align__(16) uint8_t esm[];
   uint8_t* tile = esm;                                                      // [128][272] raw elements
-  uint32_t* dft = reinterpret_cast<uint32_t*>(tile + kEncTokens * kRowBytes);   // DFT fragments
-  uint32_t* thr = dft + kDftWords;                                          // [4][3][32] threshold pairs
+  const uint32_t* dft = g_dft_frag;                                         // 16 KB, read through L1
+  uint32_t* thr = reinterpret_cast<uint32_t*>(tile + kEncTokens * kRowBytes);   // [4][3][32] threshold pairs
   float* colsum = reinterpret_cast<float*>(thr + 4 * 3 * 32);               // [8][64]
   uint8_t* perm = reinterpret_cast<uint8_t*>(colsum + 8 * 64);              // [128]
   // anomalous values gathered per code word: [group][word of the group's 2-bit block][16 slots]
@@ -142,13 +142,12 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
   const int n_groups = n_tok / kG;
   uint8_t* kg_base = slab_ptr + cv.kgroup_offset + (kgroup0 + t0 / kG) * kKGroupBytes;
 
-  // ---- stage the tile and the DFT fragments
+  // ---- stage the tile
   for (int i = tid; i < n_tok * 16; i += 256) {
     const int row = i >> 4, piece = i & 15;
     cp_async16(tile + row * kRowBytes + piece * 16,
                reinterpret_cast<const uint8_t*>(base + (t0 + row) * src.stride_t) + piece * 16);
   }
-  for (int i = tid; i < kDftWords / 4; i += 256) cp_async16(dft + i * 4, g_dft_frag + i * 4);
   asm volatile("cp.async.commit_group;" ::: "memory");
   if (tid < kD) perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
   asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -216,7 +215,7 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
     for (int ks = 0; ks < 4; ++ks) {
 #pragma unroll
       for (int nt = 0; nt < 8; ++nt) {
-        const uint4 bw = *reinterpret_cast<const uint4*>(dft + ((ks * 8 + nt) * 32 + lane) * 4);
+        const uint4 bw = __ldg(reinterpret_cast<const uint4*>(dft + ((ks * 8 + nt) * 32 + lane) * 4));
         mma_f16(acc[nt], a[ks][0], a[ks][1], a[ks][2], a[ks][3], bw.x, bw.y);
         mma_f16(acc[nt], a[ks][0], a[ks][1], a[ks][2], a[ks][3], bw.z, bw.w);
       }
