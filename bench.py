@@ -54,6 +54,24 @@ def algorithmic_quantize_bytes(B, L, H_kv, T, n_prot, elem=2):
     return L * B * H_kv * (read + write)
 
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum over the ranks of a list of floats (one all-reduce on `device`,
+    with whatever process group is initialised); the list itself at world == 1.  Every rank
+    processes the same amount of work, so job throughput = world * units / this maximum."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    tt = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return tt.tolist()
+
+
+def whole_job_throughput(units_per_rank, ms, world):
+    """Units per second of the whole job: every rank did `units_per_rank` in at most `ms`."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 def read_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -321,14 +339,11 @@ def main():
     d_ms = sum(t[1].elapsed_time(t[2]) for t in timers) / len(timers)
     kern_ms = [a.elapsed_time(b_) for t in timers for (a, b_) in t[3]]
     kern_avg_ms = sum(kern_ms) / len(kern_ms)
-    if world > 1:
-        tt = torch.tensor([total_ms, q_ms, d_ms, kern_avg_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, q_ms, d_ms, kern_avg_ms = tt.tolist()
+    total_ms, q_ms, d_ms, kern_avg_ms = max_over_ranks([total_ms, q_ms, d_ms, kern_avg_ms], dev, world)
     ms_per_step = total_ms / args.steps
 
     peak, peak_kind = read_peaks()
-    decode_gbs = world * dec_bytes / (d_ms * 1e-3) / 1e9
+    decode_gbs = whole_job_throughput(dec_bytes, d_ms, world) / 1e9
     q_bytes = n_caches * algorithmic_quantize_bytes(B, L, H, T, n_prot)
     q_tokens = n_caches * B * T * L
     kern_bytes = dec_bytes / steps_dec
