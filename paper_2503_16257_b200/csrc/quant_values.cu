@@ -30,8 +30,8 @@ template <> struct Simd2<__half> {
     const __half2 r = __hge2(*reinterpret_cast<const __half2*>(&a), *reinterpret_cast<const __half2*>(&b));
     return *reinterpret_cast<const uint32_t*>(&r);
   }
-  static __device__ __forceinline__ uint32_t le(uint32_t a, uint32_t b) {
-    const __half2 r = __hle2(*reinterpret_cast<const __half2*>(&a), *reinterpret_cast<const __half2*>(&b));
+  static __device__ __forceinline__ uint32_t gt(uint32_t a, uint32_t b) {
+    const __half2 r = __hgt2(*reinterpret_cast<const __half2*>(&a), *reinterpret_cast<const __half2*>(&b));
     return *reinterpret_cast<const uint32_t*>(&r);
   }
   // smallest element value strictly above x >= 0
@@ -45,8 +45,8 @@ template <> struct Simd2<__nv_bfloat16> {
     const __nv_bfloat162 r = __hge2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
     return *reinterpret_cast<const uint32_t*>(&r) & 0x3c003c00u;
   }
-  static __device__ __forceinline__ uint32_t le(uint32_t a, uint32_t b) {
-    const __nv_bfloat162 r = __hle2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+  static __device__ __forceinline__ uint32_t gt(uint32_t a, uint32_t b) {
+    const __nv_bfloat162 r = __hgt2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
     return *reinterpret_cast<const uint32_t*>(&r) & 0x3c003c00u;
   }
   static __device__ __forceinline__ uint16_t above(float x) {
@@ -121,21 +121,24 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
   }
   __syncthreads();
   // ---- pass 2: one word of the plane per thread and step
-#pragma unroll 1
-  for (int wd = tid; wd < kG * kD / 4; wd += 256) {
+#pragma unroll
+  for (int wi = 0; wi < kG * kD / 4 / 256; ++wi) {
+    const int wd = tid + 256 * wi;
     const int cp = 16 * ((wd >> 6) & 3) + 2 * ((wd >> 1) & 7) + (wd & 1);
     const int m = 8 * ((wd >> 9) & 1) + 4 * ((wd >> 8) & 1) + ((wd >> 4) & 3);
     uint32_t b0 = 0u, b1 = 0u;                        // binary16 pairs (even channel, odd channel) of tokens 2m, 2m+1
-    const uint32_t three = 0x42004200u, one = 0x3c003c00u;
+    const uint32_t three = 0x42004200u;
+    const uint8_t* rp0 = tile + (2 * m) * kVRowBytes + cp * 4;
+    const uint32_t* thp = thr + cp;
 #pragma unroll
     for (int g = 0; g < kSGGroups; ++g) {
-      const uint32_t A = thr[g * 64 + cp], nA = A ^ 0x80008000u;
-      const uint8_t* rp = tile + (g * kG + 2 * m) * kVRowBytes + cp * 4;
+      const uint32_t A = thp[g * 64], nA = A ^ 0x80008000u;
+      const uint8_t* rp = rp0 + g * (kG * kVRowBytes);
       const uint32_t v0 = *reinterpret_cast<const uint32_t*>(rp);
       const uint32_t v1 = *reinterpret_cast<const uint32_t*>(rp + kVRowBytes);
-      // digit = 1 + [v > alpha] - [v < -alpha]
-      __half2 d0 = __hsub2(__hadd2(*reinterpret_cast<const __half2*>(&one), as_half2(Simd2<T>::ge(v0, A))), as_half2(Simd2<T>::le(v0, nA)));
-      __half2 d1 = __hsub2(__hadd2(*reinterpret_cast<const __half2*>(&one), as_half2(Simd2<T>::ge(v1, A))), as_half2(Simd2<T>::le(v1, nA)));
+      // digit = [v > alpha] + [v >= -alpha] = [v >= A] + [v > -A]
+      const __half2 d0 = __hadd2(as_half2(Simd2<T>::ge(v0, A)), as_half2(Simd2<T>::gt(v0, nA)));
+      const __half2 d1 = __hadd2(as_half2(Simd2<T>::ge(v1, A)), as_half2(Simd2<T>::gt(v1, nA)));
       const __half2 t0 = __hfma2(as_half2(b0), *reinterpret_cast<const __half2*>(&three), d0);
       const __half2 t1 = __hfma2(as_half2(b1), *reinterpret_cast<const __half2*>(&three), d1);
       b0 = *reinterpret_cast<const uint32_t*>(&t0);
