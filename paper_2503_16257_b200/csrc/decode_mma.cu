@@ -165,6 +165,13 @@ __global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int
   const T* qrow = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(lb) * cv.H_q + h * rep + hd) * kD;
   const bool live = hd < rep;
   auto q_at = [&](int c) -> float { return live ? Elem<T>::to_float(qrow[c]) : 0.0f; };
+  if (chunk == 0 && a.append_row >= 0) {
+    // Algorithm 1, Decoding: the step's new key / value row joins the residual (lanes 0-15 copy
+    // the key row, 16-31 the value row); the attention kernel that follows reads it there.
+    uint8_t* sp = cv.slab(a.layer0 + lb / cv.B, lb % cv.B, h);
+    const uint4* srcp = reinterpret_cast<const uint4*>(lane < 16 ? a.k_new : a.v_new) + static_cast<int64_t>(slab) * 16 + (lane & 15);
+    reinterpret_cast<uint4*>(sp + (lane < 16 ? cv.kres_offset : cv.vres_offset))[a.append_row * 16 + (lane & 15)] = __ldg(srcp);
+  }
   uint32_t* out = a.prep + (static_cast<int64_t>(slab) * n_chunks + chunk) * (kPrepWords * 32) + lane;
   // anomalous slots
   {

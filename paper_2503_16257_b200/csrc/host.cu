@@ -381,12 +381,16 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int dt = h->cfg.in_dtype;
-  if (launch_append(dt, k_new, v_new, h->cv, layer_begin, n_layers, first.n_res, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  // the append rides on the query-preparation kernel when there is one (some chunk is quantized)
+  const bool has_chunks = first.T_q0 + first.n_flush > 0;
+  if (!has_chunks && launch_append(dt, k_new, v_new, h->cv, layer_begin, n_layers, first.n_res, s) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
   DecodeArgs a;
   a.cv = h->cv;
   a.q = q; a.k_new = k_new; a.v_new = v_new; a.out = out;
   a.partials = reinterpret_cast<float*>(h->workspace + h->ws.partials_off);
   a.prep = reinterpret_cast<uint32_t*>(h->workspace + h->ws.prep_off);
+  a.append_row = has_chunks ? first.n_res : -1;
   a.layer0 = layer_begin; a.n_layers = n_layers;
   a.in_dtype = dt; a.out_dtype = h->cfg.out_dtype;
   a.n_prot = h->n_prot;

@@ -91,6 +91,7 @@ struct DecodeArgs {
   float* partials;     // [n_layers * B * H_q * n_splits][130]
   uint32_t* prep;      // per (slab, chunk) query images of the tensor-core path (decode_prep_bytes)
   const uint32_t* dft; // DFT matrix fragments (dft_fragments), set by launch_decode_mma
+  int32_t append_row;  // >= 0: the preparation kernel also writes k_new / v_new into this residual row
   int32_t layer0, n_layers;
   int32_t in_dtype, out_dtype;
   int32_t split_tokens, n_splits;

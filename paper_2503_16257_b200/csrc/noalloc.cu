@@ -91,6 +91,7 @@ extern "C" vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const 
   a.split_tokens = split_tokens_for(T_tot, n_slabs, n_protected > 0);
   a.n_splits = static_cast<int32_t>((T_tot + a.split_tokens - 1) / a.split_tokens);
   a.splits_per_cta = 1;
+  a.append_row = -1;
   a.n_parts = a.n_splits;
   const int64_t records = static_cast<int64_t>(n_layers) * cfg->B * cfg->H_q * a.n_splits;
   // the array holds the partial records, then (256-byte aligned) the per-chunk query images
