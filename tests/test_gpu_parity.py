@@ -170,6 +170,31 @@ def test_full_size_slabs_in_the_benchmark_launch_shape():
     assert cache.status() == 0
 
 
+def test_longest_sequence_slab():
+    """The stress configuration's token count (1000 frames = 196 000 tokens, 307 splits per slab) on
+    one layer and one batch element; the oracle recomputes one KV head."""
+    import paper_2503_16257_b200 as P
+    from workloads import make_layer_kv, make_step_inputs
+    wl = CONFIGS["stress"]
+    T = wl.T
+    cfg = P.VidKVConfig(B=1, L=1, max_prefill_tokens=T, max_new_tokens=2, p_ratio=0.0,
+                        in_dtype=P.VIDKV_F16, out_dtype=P.VIDKV_F32)
+    cache = P.VidKVCache(cfg, device="cuda")
+    K, V = make_layer_kv(wl, 0, "cuda", T=T, B=1)
+    cache.quantize_keys(0, K)
+    cache.quantize_values(0, V)
+    h = 2
+    sc = O.SlabCache()
+    sc.prefill(to_np(K[0, h]), to_np(V[0, h]), None)
+    q, k, v = make_step_inputs(wl, 0, 0, "cuda", T=T, B=1)
+    out = torch.empty((1, 1, 28, 128), dtype=torch.float32, device="cuda")
+    cache.decode_attention(0, 1, q[None], k[None], v[None], out)
+    ref = sc.decode_step(to_np(q[0, 7 * h:7 * h + 7]), to_np(k[0, h]), to_np(v[0, h]))
+    assert np.abs(out[0, 0, 7 * h:7 * h + 7].cpu().numpy().astype(np.float64) - ref).max() <= TOL_ABS
+    assert cache.layer_state(0) == dict(n_quantized=196000 - 196000 % 32, n_residual=196000 % 32 + 1, n_chunks=1, n_protected=0)
+    assert cache.status() == 0
+
+
 def test_residual_flush_parity():
     # 64 quantized + 5 residual tokens; the residual fills at step 123 and is flushed
     wl = CONFIGS["tiny"]
