@@ -405,8 +405,11 @@ __device__ __forceinline__ void ternary_phase(const Split& c, const uint8_t* vbu
           for (int k = 0; k < 8; ++k) {
             // W holds 3 * (remaining byte) per 16-bit lane; the digit sits at bits 8-9.
             // Next W = 3 * (W - digit << 8) = 3 W - 3 A + 3 * 0x4400 (no lane ever borrows).
+            // Half of the lanes take that route (two multiply-adds), the other half mask the digit
+            // away and multiply (one logic, one multiply-add): the two pipes share the work evenly.
             A[k] = and_or(W[k], m_field, c_four);
-            W[k] = mad_u32(A[k], 0xfffffffdu, mad_u32(W[k], 3u, 0xcc00cc00u));
+            if (k & 1) W[k] = mad_u32(A[k], 0xfffffffdu, mad_u32(W[k], 3u, 0xcc00cc00u));
+            else W[k] = mad_u32(W[k] & 0x00ff00ffu, 3u, 0u);
           }
           if (MASKED && g < g_lo) continue;
           // groups past the end of the cache meet zero probabilities (and a zero scale below)
