@@ -78,6 +78,8 @@ def _compare_dequant(pair: Pair):
     ("tiny", 31, 1, 0.0),          # nothing quantized, everything in the residual
     ("llava", 352, 1, 0.2),        # heavy-tailed values, +-5 outlier offsets
     ("qwen", 480, 2, 0.2),         # bf16 inputs, rotary-structured keys
+    ("tiny", 1632, 1, 0.9),        # nearly every visual token protected
+    ("tiny", 800, 1, 0.002),       # a single protected token
 ])
 def test_prefill_codes_and_dequant(name, T, B, p):
     pair = Pair(CONFIGS[name], T, B=B, L=1, p=p).prefill()
@@ -114,6 +116,8 @@ def _decode_steps(pair: Pair, n_steps, tol=TOL_ABS):
     ("qwen", 480, 2, 0.0, 4),      # bf16 inputs without protection: the tensor-core kernel
     ("tiny", 2000, 1, 0.0, 3),     # 1984 quantized tokens = 3.1 splits of 640, plus 16 residual tokens
     ("tiny", 1300, 2, 0.0, 3),     # last split starts inside a supergroup (1280) and ends in the residual
+    ("tiny", 1632, 1, 0.9, 3),     # nearly every visual token protected: long protected stream, short ternary one
+    ("tiny", 800, 1, 0.002, 3),    # a single protected token
 ])
 def test_decode_attention_parity(name, T, B, p, steps):
     pair = Pair(CONFIGS[name], T, B=B, L=1, p=p, max_new=steps).prefill()
