@@ -72,6 +72,21 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
   const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
 }
+// Copy n16 16-byte pieces from global to shared memory, pieces interleaved over the CTA's threads;
+// unrolled by four so that the offsets are immediates.
+__device__ __forceinline__ void stage_async(uint8_t* dst, const uint8_t* src, int n16, int tid) {
+  constexpr int kStep = 128 * 16;
+  uint8_t* d = dst + tid * 16;
+  const uint8_t* s = src + tid * 16;
+  int i = tid;
+  for (; i + 3 * 128 < n16; i += 4 * 128, d += 4 * kStep, s += 4 * kStep) {
+    cp_async16(d, s);
+    cp_async16(d + kStep, s + kStep);
+    cp_async16(d + 2 * kStep, s + 2 * kStep);
+    cp_async16(d + 3 * kStep, s + 3 * kStep);
+  }
+  for (; i < n16; i += 128, d += kStep, s += kStep) cp_async16(d, s);
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -282,8 +297,9 @@ __device__ __forceinline__ void score_phase(const DecodeArgs& a, int n_chunks, c
         const uint4 x0 = *reinterpret_cast<const uint4*>(kg + kKG_S2 + 32 * r);
         const uint4 x1 = *reinterpret_cast<const uint4*>(kg + kKG_S2 + 32 * r + 16);
         s2[0] = x0.x; s2[1] = x0.y; s2[2] = x0.z; s2[3] = x0.w; s2[4] = x1.x; s2[5] = x1.y; s2[6] = x1.z; s2[7] = x1.w;
-        const uint4 y0 = *reinterpret_cast<const uint4*>(kg + kKG_Z2 + 32 * r);
-        const uint4 y1 = *reinterpret_cast<const uint4*>(kg + kKG_Z2 + 32 * r + 16);
+        const uint8_t* zs = kg + ((hd & 1) ? kKG_S2 : kKG_Z2) + 32 * r;   // B operand of the constants: z for even columns, s for odd
+        const uint4 y0 = *reinterpret_cast<const uint4*>(zs);
+        const uint4 y1 = *reinterpret_cast<const uint4*>(zs + 16);
         z2[0] = y0.x; z2[1] = y0.y; z2[2] = y0.z; z2[3] = y0.w; z2[4] = y1.x; z2[5] = y1.y; z2[6] = y1.z; z2[7] = y1.w;
         const uint4 w0 = *reinterpret_cast<const uint4*>(kg + kKG_S1 + 32 * r);
         const uint4 w1 = *reinterpret_cast<const uint4*>(kg + kKG_S1 + 32 * r + 16);
@@ -293,10 +309,8 @@ __device__ __forceinline__ void score_phase(const DecodeArgs& a, int n_chunks, c
       float cst;
       {
         float cz[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        const bool odd = hd & 1;
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          mma_f16(cz, qa[2 * ks], 0u, qa[2 * ks + 1], 0u, odd ? s2[2 * ks] : z2[2 * ks], odd ? s2[2 * ks + 1] : z2[2 * ks + 1]);
+        for (int ks = 0; ks < 4; ++ks) mma_f16(cz, qa[2 * ks], 0u, qa[2 * ks + 1], 0u, z2[2 * ks], z2[2 * ks + 1]);
         cst = cz[0] - 4.0f * cz[1];
       }
       // q s as exact binary16 pairs hi + lo
@@ -618,7 +632,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
     const int n_sg = (c.n_kg + kSGGroups - 1) / kSGGroups;   // ternary groups = key groups here
     {
       const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
-      for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(kbuf + i * 16, ksrc + i * 16);
+      stage_async(kbuf, ksrc, c.n_kg * (kKGroupBytes / 16), c.tid);
       cp_async_commit();
     }
     cp_async_wait<0>();
@@ -628,7 +642,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
     {
       // the key groups are spent: the ternary supergroups take their place while the softmax runs
       const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + (c.t0 / (kG * kSGGroups)) * kSGBytes;
-      for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(vbuf + i * 16, vsrc + i * 16);
+      stage_async(vbuf, vsrc, n_sg * (kSGBytes / 16), c.tid);
       cp_async_commit();
     }
     softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0);
@@ -714,7 +728,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
   // ---- keys first
   {
     const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
-    for (int i = c.tid; i < c.n_kg * (kKGroupBytes / 16); i += kThreads) cp_async16(buf + i * 16, ksrc + i * 16);
+    stage_async(buf, ksrc, c.n_kg * (kKGroupBytes / 16), c.tid);
     cp_async_commit();
   }
   // ---- where the split's tokens sit in the two value streams
@@ -757,7 +771,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
   {
     // the key groups are spent: the ternary supergroups take their place while the softmax runs
     const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + sgA * kSGBytes;
-    for (int i = c.tid; i < n_sg * (kSGBytes / 16); i += kThreads) cp_async16(buf + i * 16, vsrc + i * 16);
+    stage_async(buf, vsrc, n_sg * (kSGBytes / 16), c.tid);
     cp_async_commit();
   }
   softmax_phase<true>(a, c, S, SS, red, 0, map, Pprot, PP, Pres, kPresStride);
