@@ -523,7 +523,7 @@ __device__ __forceinline__ void write_partial(const DecodeArgs& a, const Split& 
 // tokens [0, nq) go to their stream position through `map` (bit 15 = protected stream, row of
 // Pprot), residual tokens [nq, n_loc) to Pres[row][i - nq].
 // red[row] = scaled row maximum, red[8 + row] = sum of the probabilities.
-template <bool STP>
+template <bool STP, bool FULL = false>     // FULL: the split holds exactly 640 tokens, no bound checks
 __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& c, float* S, int SS, float* red,
                                               int n_pad, const uint16_t* map, __half* Pprot, int PP, __half* Pres,
                                               int PRS) {
@@ -539,8 +539,12 @@ __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& 
 #pragma unroll
     for (int k = 0; k < kMaxPairs; ++k) {
       const int i = 2 * lane + 64 * k;
-      v[k] = i < n_loc ? *reinterpret_cast<const float2*>(row + i) : make_float2(-INFINITY, -INFINITY);
-      if (i + 1 >= n_loc) v[k].y = -INFINITY;
+      if (FULL) {
+        v[k] = *reinterpret_cast<const float2*>(row + i);
+      } else {
+        v[k] = i < n_loc ? *reinterpret_cast<const float2*>(row + i) : make_float2(-INFINITY, -INFINITY);
+        if (i + 1 >= n_loc) v[k].y = -INFINITY;
+      }
       m = fmaxf(m, fmaxf(v[k].x, v[k].y));
     }
 #pragma unroll
@@ -570,7 +574,7 @@ __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& 
         } else if (i < n_loc) {
           *reinterpret_cast<uint32_t*>(Pres + row_h * PRS + (i - c.nq)) = pack_half2(p0, p1);
         }
-      } else if (i < n_pad) {
+      } else if (FULL || i < n_pad) {
         prow[i >> 1] = pack_half2(p0, p1);
       }
     }
@@ -645,7 +649,10 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
       stage_async(vbuf, vsrc, n_sg * (kSGBytes / 16), c.tid);
       cp_async_commit();
     }
-    softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0);
+    if (c.n_loc == 640)
+      softmax_phase<false, true>(a, c, S, SS, red, 640, nullptr, nullptr, 0, nullptr, 0);
+    else
+      softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0);
     __syncthreads();
     group_sums(c, reinterpret_cast<const __half*>(S), 2 * SS, n_sg * kSGGroups, -5.0f, psum);
     cp_async_wait<0>();
