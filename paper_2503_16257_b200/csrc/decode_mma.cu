@@ -589,14 +589,19 @@ __device__ __forceinline__ void group_sums(const Split& c, const __half* P, int 
                                            float* out) {
   for (int i = c.tid; i < n_groups * 8; i += kThreads) {
     const int g = i >> 3, hh = i & 7;
-    const __half2* pr = reinterpret_cast<const __half2*>(P + hh * row_stride + g * kG);
-    float s = 0.0f;
+    const uint4* pr = reinterpret_cast<const uint4*>(P + hh * row_stride + g * kG);   // 64 bytes, 16-byte aligned
+    float s0 = 0.0f, s1 = 0.0f;
 #pragma unroll
-    for (int k = 0; k < 16; ++k) {
-      const float2 f = __half22float2(pr[k]);
-      s += f.x + f.y;
+    for (int k = 0; k < 4; ++k) {
+      const uint4 v = pr[k];
+      const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+      const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+      const float2 f2 = __half22float2(*reinterpret_cast<const __half2*>(&v.z));
+      const float2 f3 = __half22float2(*reinterpret_cast<const __half2*>(&v.w));
+      s0 += (f0.x + f0.y) + (f1.x + f1.y);
+      s1 += (f2.x + f2.y) + (f3.x + f3.y);
     }
-    out[i] = factor * s;
+    out[i] = factor * (s0 + s1);
   }
 }
 
