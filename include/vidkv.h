@@ -23,7 +23,9 @@
  *     and passes the buffers in.  The handle is a small host object.
  *   - All device work is enqueued on the caller's stream (a cudaStream_t passed
  *     as void*) and is asynchronous.  Argument errors are detected on the host
- *     before anything is launched.
+ *     before anything is launched.  One exception: the first key quantization or
+ *     decode call on each device fills a 16 KB table of DFT coefficients inside the
+ *     library and synchronises the stream once.
  *   - Fixed by this build: D = 128, G = 32, R = 128, k = 0.5 (64 two-bit and 64
  *     one-bit channels), H_q a multiple of H_kv with H_q / H_kv <= 8.  Other
  *     shapes return VIDKV_ERR_UNSUPPORTED.

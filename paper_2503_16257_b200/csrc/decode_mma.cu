@@ -1,5 +1,6 @@
 // Decode attention over the packed cache on the tensor cores (Algorithm 1 "Decoding",
-// Eq. 3), split-KV, for caches without protected tokens (p = 0).
+// Eq. 3), split-KV: decode_mma_kernel for caches without protected tokens, decode_stp_kernel
+// for caches with them (STPQuant), decode_prep_kernel for the per-chunk query images.
 //
 // The packed codes never become FP16 K or V in memory.  They are expanded in registers to
 // small exact binary16 numbers and fed to mma.sync.m16n8k16 as one operand; everything that
@@ -22,10 +23,12 @@
 //     5 + trit in binary16; the 5 is removed through the accumulator's initial value
 //     -5 sum_t p_t, and the per-(group, channel) scale multiplies the group's accumulator.
 //
-// One CTA (4 warps) = one split of the token axis of one (layer, batch element, KV head).
-// The split's key groups and ternary supergroups are copied to shared memory with cp.async;
-// phase 1 (warps split the 32-token groups) writes scores, a softmax pass turns them into
-// binary16 probabilities in place, phase 2 (warps split the channels) accumulates P V.
+// One CTA (4 warps) walks one or more consecutive splits of the token axis of one (layer, batch
+// element, KV head).  A split's key groups, then its ternary supergroups, are copied into the same
+// shared-memory buffer with cp.async; phase 1 (warps split the 32-token groups) writes scores, a
+// softmax pass turns them into binary16 probabilities in place, phase 2 (warps split the channels)
+// accumulates P V.  With protected tokens the probabilities are scattered into stream order and
+// the protected 2-bit groups are read from global memory as they are consumed.
 #include "common.cuh"
 #include "kernels.cuh"
 
