@@ -14,30 +14,67 @@ namespace vidkv {
 // Range pass.  grid = (token splits, slabs); block = 256 threads = 16 rows x 16 lanes,
 // each lane owns 8 consecutive channels (one 16-byte load per row).
 // ---------------------------------------------------------------------------------
+template <typename T> struct Pair2;
+template <> struct Pair2<__half> {
+  using V = __half2;
+  static __device__ __forceinline__ V mn(V a, V b) { return __hmin2(a, b); }
+  static __device__ __forceinline__ V mx(V a, V b) { return __hmax2(a, b); }
+  static __device__ __forceinline__ float2 f2(V a) { return __half22float2(a); }
+};
+template <> struct Pair2<__nv_bfloat16> {
+  using V = __nv_bfloat162;
+  static __device__ __forceinline__ V mn(V a, V b) { return __hmin2(a, b); }
+  static __device__ __forceinline__ V mx(V a, V b) { return __hmax2(a, b); }
+  static __device__ __forceinline__ float2 f2(V a) { return __bfloat1622float2(a); }
+};
+
 template <typename T>
 __global__ void __launch_bounds__(256) k_range_kernel(KSrc src, int64_t T_tokens, int tokens_per_block,
                                                       uint32_t* __restrict__ minmax) {
+  using P = Pair2<T>;
+  using V = typename P::V;
   const int slab = blockIdx.y;
   const T* base = reinterpret_cast<const T*>(src.ptr) + (slab / src.H) * src.stride_b + (slab % src.H) * src.stride_h;
   const int lane16 = threadIdx.x & 15, row = threadIdx.x >> 4;
   const int64_t t0 = static_cast<int64_t>(blockIdx.x) * tokens_per_block;
   const int64_t t1 = min(t0 + tokens_per_block, T_tokens);
-  float mn[8], mx[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) { mn[i] = INFINITY; mx[i] = -INFINITY; }
-  for (int64_t t = t0 + row; t < t1; t += 16) {
+  // element pairs stay in their 16-bit type: min / max need no conversion
+  V mn[4], mx[4];
+  bool any = false;
+  int64_t t = t0 + row;
+  if (t < t1) {
     const uint4 v = __ldg(reinterpret_cast<const uint4*>(base + t * src.stride_t) + lane16);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    const V* pv = reinterpret_cast<const V*>(&v);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 f = Elem<T>::to_float2(w[i]);
-      mn[2 * i] = fminf(mn[2 * i], f.x);      mx[2 * i] = fmaxf(mx[2 * i], f.x);
-      mn[2 * i + 1] = fminf(mn[2 * i + 1], f.y); mx[2 * i + 1] = fmaxf(mx[2 * i + 1], f.y);
+    for (int i = 0; i < 4; ++i) { mn[i] = pv[i]; mx[i] = pv[i]; }
+    any = true;
+    t += 16;
+  }
+  for (; t + 48 < t1; t += 64) {                       // four rows in flight per thread
+    uint4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) v[k] = __ldg(reinterpret_cast<const uint4*>(base + (t + 16 * k) * src.stride_t) + lane16);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const V* pv = reinterpret_cast<const V*>(&v[k]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { mn[i] = P::mn(mn[i], pv[i]); mx[i] = P::mx(mx[i], pv[i]); }
     }
+  }
+  for (; t < t1; t += 16) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(base + t * src.stride_t) + lane16);
+    const V* pv = reinterpret_cast<const V*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { mn[i] = P::mn(mn[i], pv[i]); mx[i] = P::mx(mx[i], pv[i]); }
   }
   __shared__ float s_mn[16][kD + 1], s_mx[16][kD + 1];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) { s_mn[row][lane16 * 8 + i] = mn[i]; s_mx[row][lane16 * 8 + i] = mx[i]; }
+  for (int i = 0; i < 4; ++i) {
+    float2 a = make_float2(INFINITY, INFINITY), c = make_float2(-INFINITY, -INFINITY);
+    if (any) { a = P::f2(mn[i]); c = P::f2(mx[i]); }
+    s_mn[row][lane16 * 8 + 2 * i] = a.x; s_mn[row][lane16 * 8 + 2 * i + 1] = a.y;
+    s_mx[row][lane16 * 8 + 2 * i] = c.x; s_mx[row][lane16 * 8 + 2 * i + 1] = c.y;
+  }
   __syncthreads();
   if (threadIdx.x < kD) {
     float a = INFINITY, c = -INFINITY;
