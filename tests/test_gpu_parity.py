@@ -199,6 +199,47 @@ def test_longest_sequence_slab():
     assert cache.status() == 0
 
 
+@pytest.mark.parametrize("H_kv,H_q,p", [(2, 16, 0.0), (2, 16, 0.25), (8, 8, 0.0), (1, 4, 0.25)])
+def test_other_head_counts(H_kv, H_q, p):
+    """GQA ratios 8, 1 and 4 (the named workloads all use 7): seeded Gaussian K, V, q with a few
+    wide key channels, two decode steps, every slab against the oracle."""
+    import paper_2503_16257_b200 as P
+    T, B, rep = 704, 2, H_q // H_kv
+    g = torch.Generator().manual_seed(1234 + 17 * H_kv + H_q)
+    wide = torch.ones(128); wide[torch.randperm(128, generator=g)[:6]] = 8.0
+    K = (torch.randn((B, H_kv, T, 128), generator=g) * wide).to(torch.float16)
+    V = torch.randn((B, H_kv, T, 128), generator=g).to(torch.float16)
+    cfg = P.VidKVConfig(B=B, L=1, H_kv=H_kv, H_q=H_q, max_prefill_tokens=T, max_new_tokens=2, p_ratio=p,
+                        in_dtype=P.VIDKV_F16, out_dtype=P.VIDKV_F32)
+    cache = P.VidKVCache(cfg, device="cuda")
+    E = [None] * B
+    if p > 0:
+        sal = torch.randn((B, 640), generator=g)
+        cache.select_tokens(sal.cuda(), 0, 640, T)
+        for b in range(B):
+            E[b] = np.zeros(T, dtype=bool)
+            E[b][:T - T % 32] = O.select_tokens(sal[b].numpy(), p, 0, T - T % 32)
+    cache.quantize_keys(0, K.cuda())
+    cache.quantize_values(0, V.cuda())
+    slabs = {}
+    for b in range(B):
+        for h in range(H_kv):
+            sc = O.SlabCache()
+            sc.prefill(to_np(K[b, h]), to_np(V[b, h]), E[b])
+            slabs[(b, h)] = sc
+    for step in range(2):
+        q = (torch.randn((1, B, H_q, 128), generator=g)).to(torch.float16)
+        k = (torch.randn((1, B, H_kv, 128), generator=g) * wide).to(torch.float16)
+        v = torch.randn((1, B, H_kv, 128), generator=g).to(torch.float16)
+        out = torch.empty((1, B, H_q, 128), dtype=torch.float32, device="cuda")
+        cache.decode_attention(0, 1, q.cuda(), k.cuda(), v.cuda(), out)
+        out = out.cpu().numpy().astype(np.float64)
+        for (b, h), sc in slabs.items():
+            ref = sc.decode_step(to_np(q[0, b, h * rep:(h + 1) * rep]), to_np(k[0, b, h]), to_np(v[0, b, h]))
+            assert np.abs(out[0, b, h * rep:(h + 1) * rep] - ref).max() <= TOL_ABS
+    assert cache.status() == 0
+
+
 def test_residual_flush_parity():
     # 64 quantized + 5 residual tokens; the residual fills at step 123 and is flushed
     wl = CONFIGS["tiny"]
