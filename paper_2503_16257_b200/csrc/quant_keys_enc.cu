@@ -181,10 +181,20 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
         uint16_t X = Ops<T>::kInf;                     // s == 0: every code is 0
         if (s != 0.0f) {
           int o = ord_of(Ops<T>::from_float_rn(fmaf(static_cast<float>(k) - 0.5f, s, z)));
+          // the threshold is almost always the candidate or a neighbour: three independent evaluations
+          const int cm = code_ref<T>(o - 1, z, s), c0 = code_ref<T>(o, z, s), cp = code_ref<T>(o + 1, z, s);
+          if (cm < k && c0 >= k) {
+          } else if (c0 < k && cp >= k) {
+            o += 1;
+          } else if (cm >= k) {
+            o -= 1;
 #pragma unroll 1
-          for (int it = 0; it < 4 && code_ref<T>(o, z, s) < k; ++it) ++o;
+            for (int it = 0; it < 4 && code_ref<T>(o - 1, z, s) >= k; ++it) --o;
+          } else {
+            o += 2;
 #pragma unroll 1
-          for (int it = 0; it < 4 && code_ref<T>(o - 1, z, s) >= k; ++it) --o;
+            for (int it = 0; it < 4 && code_ref<T>(o, z, s) < k; ++it) ++o;
+          }
           X = bits_of(o);
         }
         th[(k - 1) * 64 + j] = X;
