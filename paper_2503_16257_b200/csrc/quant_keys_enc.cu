@@ -1,17 +1,18 @@
 // Key encode pass of Algorithm 3 (MixQuant) for one tile of 128 tokens x 128 channels:
-//   normal channels   (Eq. 5) orthonormal 64-point DFT over the channel axis as a matrix
-//                     product on the tensor cores (A = the tile's values, binary16, exact;
-//                     B = the DFT matrix split into a binary16 leading part and a binary16
-//                     remainder, so that products carry 22 bits; float32 accumulation), then
-//                     the sign bit and the per-group mean |.| of every spectrum column;
+//   normal channels   (Eq. 5) orthonormal 64-point DFT over the channel axis as one 128 x 64 x 64
+//                     matrix product on the fifth-generation tensor cores (tcgen05.mma, operands
+//                     in shared memory in the 128-byte-swizzled K-major layout, accumulator in
+//                     tensor memory).  A = the tile's values, binary16, exact; B = the DFT matrix
+//                     split into a binary16 leading part and a binary16 remainder, so that
+//                     products carry 22 bits; float32 accumulation.  Then the sign bit and the
+//                     per-group mean |.| of every spectrum column, one thread per token;
 //   anomalous channels (Eq. 4) min / max per (32-token group, channel), s = (max - min) / 3,
 //                     z = min rounded to binary16, code = clamp(rint((x - z) / s), 0, 3).
 //                     The division is not done per element: code >= k is a monotone predicate
 //                     of x, so per (group, channel) the three smallest element values X_k with
 //                     code(X_k) >= k are found once with the defining float32 arithmetic, and
 //                     the elements are compared against them two at a time.
-// grid = (tiles of 128 tokens, slabs); block = 256 threads = 8 warps; each warp owns 16 tokens
-// in the DFT phase.
+// grid = (tiles of 128 tokens, slabs); block = 256 threads = 8 warps.
 #include <math.h>
 
 #include "common.cuh"
@@ -28,13 +29,17 @@ constexpr int kDftWords = 4 * 8 * 32 * 4;      // [k step][column tile][lane][hi
 // B fragments of the DFT matrix in the order the MMA wants them (see dft_table_kernel).
 __device__ __align__(16) uint32_t g_dft_frag[kDftWords];
 
-__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                        uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+// The same matrix as the B operand of tcgen05.mma: two blocks (leading part, remainder) of
+// [64 spectrum columns][64 channel positions] binary16, K-major with the 128-byte swizzle.
+constexpr int kUmmaBlockBytes = 64 * 128;
+__device__ __align__(1024) uint8_t g_dft_umma[2 * kUmmaBlockBytes];
+
+// Byte offset of element (row, k) of a K-major operand with 64 binary16 per row under the
+// 128-byte swizzle: 8-row atoms of 1024 bytes, 16-byte pieces XORed with the row within the atom.
+__host__ __device__ constexpr int sw128_offset(int row, int k) {
+  return (row >> 3) * 1024 + (row & 7) * 128 + ((((k >> 3) ^ row) & 7) << 4) + (k & 7) * 2;
 }
+
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
   const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
@@ -83,11 +88,20 @@ __device__ __forceinline__ int code_ref(int o, float z, float s) {
 
 }  // namespace
 
-// One block of 256 threads, 4 table words per thread.  Word layout for k step ks, column tile
-// nt and lane (n = lane / 4, r = lane % 4): rows k0 = 16 ks + 2 r (and k0 + 1; k0 + 8, k0 + 9)
-// of column f = 16 (n / 2) + 2 nt + (n % 2), so that after the product lane (., r) holds the
-// spectrum columns 16 r .. 16 r + 15 of its two tokens.  Column f of the matrix: f = 0: 1/8;
-// f = 1: (-1)^c / 8; f = 2k: cos(2 pi k c / 64) / 8; f = 2k + 1: -sin(2 pi k c / 64) / 8.
+// Column f of the DFT matrix at channel position c: f = 0: 1/8; f = 1: (-1)^c / 8;
+// f = 2k: cos(2 pi k c / 64) / 8; f = 2k + 1: -sin(2 pi k c / 64) / 8.
+__device__ double dft_weight(int f, int c) {
+  if (f == 0) return 0.125;
+  if (f == 1) return (c & 1) ? -0.125 : 0.125;
+  double sn, cs;
+  sincospi(static_cast<double>(((f >> 1) * c) & 63) / 32.0, &sn, &cs);
+  return ((f & 1) ? -sn : cs) * 0.125;
+}
+
+// One block of 256 threads.  mma.sync fragments (used by the decode path for the query): word
+// layout for k step ks, column tile nt and lane (n = lane / 4, r = lane % 4): rows
+// k0 = 16 ks + 2 r (and k0 + 1; k0 + 8, k0 + 9) of column f = 16 (n / 2) + 2 nt + (n % 2), so
+// that after the product lane (., r) holds the spectrum columns 16 r .. 16 r + 15 of its two rows.
 __global__ void dft_table_kernel() {
   for (int i = threadIdx.x; i < kDftWords / 4; i += blockDim.x) {
     const int lane = i & 31, nt = (i >> 5) & 7, ks = i >> 8;
@@ -95,41 +109,82 @@ __global__ void dft_table_kernel() {
     const int f = 16 * (n >> 1) + 2 * nt + (n & 1);
     float w[4];
     const int rows[4] = {16 * ks + 2 * r, 16 * ks + 2 * r + 1, 16 * ks + 2 * r + 8, 16 * ks + 2 * r + 9};
-    for (int j = 0; j < 4; ++j) {
-      const int c = rows[j];
-      double v;
-      if (f == 0) v = 1.0;
-      else if (f == 1) v = (c & 1) ? -1.0 : 1.0;
-      else {
-        double sn, cs;
-        sincospi(static_cast<double>(((f >> 1) * c) & 63) / 32.0, &sn, &cs);
-        v = (f & 1) ? -sn : cs;
-      }
-      w[j] = static_cast<float>(v * 0.125);
-    }
+    for (int j = 0; j < 4; ++j) w[j] = static_cast<float>(dft_weight(f, rows[j]));
     const __half h0 = __float2half_rn(w[0]), h1 = __float2half_rn(w[1]), h2 = __float2half_rn(w[2]), h3 = __float2half_rn(w[3]);
     g_dft_frag[i * 4 + 0] = as_u32(__halves2half2(h0, h1));
     g_dft_frag[i * 4 + 1] = as_u32(__halves2half2(h2, h3));
     g_dft_frag[i * 4 + 2] = as_u32(__floats2half2_rn(w[0] - __half2float(h0), w[1] - __half2float(h1)));
     g_dft_frag[i * 4 + 3] = as_u32(__floats2half2_rn(w[2] - __half2float(h2), w[3] - __half2float(h3)));
   }
+  // tcgen05 operand: row = spectrum column f, k = position c among the normal channels
+  for (int i = threadIdx.x; i < 64 * 64; i += blockDim.x) {
+    const int f = i >> 6, c = i & 63;
+    const float w = static_cast<float>(dft_weight(f, c));
+    const __half hi = __float2half_rn(w);
+    const __half lo = __float2half_rn(w - __half2float(hi));
+    *reinterpret_cast<__half*>(g_dft_umma + sw128_offset(f, c)) = hi;
+    *reinterpret_cast<__half*>(g_dft_umma + kUmmaBlockBytes + sw128_offset(f, c)) = lo;
+  }
 }
 
-size_t k_encode_smem_bytes() {
-  return kEncTokens * kRowBytes + 4 * 3 * 32 * 4 + 8 * 64 * 4 + kD + 4 * 128 * 32;
+// ---- tcgen05 helpers -------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+// Shared-memory matrix descriptor of a K-major operand with one 128-byte swizzle atom along K:
+// start address / 16, 8-row groups 1024 bytes apart, descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+  return static_cast<uint64_t>((smem_addr >> 4) & 0x3fffu) | (static_cast<uint64_t>(1u) << 16) |
+         (static_cast<uint64_t>(1024u >> 4) << 32) | (static_cast<uint64_t>(1u) << 46) | (static_cast<uint64_t>(2u) << 61);
 }
+// Instruction descriptor: float32 accumulator, binary16 A and B, both K-major, N = 64, M = 128.
+constexpr uint32_t kUmmaIdesc = (1u << 4) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr int kTmemCols = 64;
+constexpr int kWaitLimit = 1 << 14;
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(kUmmaIdesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// 32 consecutive accumulator columns of the calling warp's 32 lanes of tensor memory.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared memory of one block, from a 1024-byte boundary:
+//   [0, 16384)       A operand: the normal channels of the tile, [128 tokens][64 positions]
+//   [16384, 51200)   the staged tile, [128][272] raw elements; once the tile has been sorted into
+//                    the A operand and the gathered anomalous values, its first 16 KB take the B operand
+//   [51200, 67584)   anomalous values gathered per code word
+//   then thresholds [4][3][32] pairs, the channel order [128], the mbarrier, the tensor-memory address
+constexpr int kSmAop = 0, kSmTile = 16384, kSmGath = kSmTile + kEncTokens * kRowBytes, kSmThr = kSmGath + 4 * 128 * 32,
+              kSmPerm = kSmThr + 4 * 3 * 32 * 4, kSmBar = kSmPerm + kD, kSmEnd = kSmBar + 16;
+
+size_t k_encode_smem_bytes() { return kSmEnd + 1024; }
 
 template <typename T>
-__global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_tokens, CacheView cv, int layer0,
-                                                       int slabs_per_layer, int chunk, int64_t kgroup0) {
-  extern __shared__ __align__(16) uint8_t esm[];
-  uint8_t* tile = esm;                                                      // [128][272] raw elements
-  const uint32_t* dft = g_dft_frag;                                         // 16 KB, read through L1
-  uint32_t* thr = reinterpret_cast<uint32_t*>(tile + kEncTokens * kRowBytes);   // [4][3][32] threshold pairs
-  float* colsum = reinterpret_cast<float*>(thr + 4 * 3 * 32);               // [8][64]
-  uint8_t* perm = reinterpret_cast<uint8_t*>(colsum + 8 * 64);              // [128]
-  // anomalous values gathered per code word: [group][word of the group's 2-bit block][16 slots]
-  uint16_t* gath = reinterpret_cast<uint16_t*>(perm + kD);
+__global__ void __launch_bounds__(256, 3) k_encode_kernel(KSrc src, int64_t T_tokens, CacheView cv, int layer0,
+                                                          int slabs_per_layer, int chunk, int64_t kgroup0) {
+  extern __shared__ uint8_t esm_raw[];
+  uint8_t* esm = esm_raw + ((1024u - (smem_u32(esm_raw) & 1023u)) & 1023u);
+  uint8_t* aop = esm + kSmAop;
+  uint8_t* tile = esm + kSmTile;
+  uint16_t* gath = reinterpret_cast<uint16_t*>(esm + kSmGath);   // [group][word of the group's 2-bit block][16 slots]
+  uint32_t* thr = reinterpret_cast<uint32_t*>(esm + kSmThr);
+  uint8_t* perm = esm + kSmPerm;
+  uint64_t* mbar = reinterpret_cast<uint64_t*>(esm + kSmBar);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(esm + kSmBar + 8);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int slab = blockIdx.y;
@@ -142,7 +197,7 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
   const int n_groups = n_tok / kG;
   uint8_t* kg_base = slab_ptr + cv.kgroup_offset + (kgroup0 + t0 / kG) * kKGroupBytes;
 
-  // ---- stage the tile
+  // ---- stage the tile; meanwhile set up the barrier and 64 columns of tensor memory
   for (int i = tid; i < n_tok * 16; i += 256) {
     const int row = i >> 4, piece = i & 15;
     cp_async16(tile + row * kRowBytes + piece * 16,
@@ -150,8 +205,19 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
   if (tid < kD) perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(mbar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = *tmem_slot;
 
   // ---- A: Eq. 4 metadata and thresholds, thread = (anomalous slot j, group g)
   {
@@ -202,80 +268,27 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
     }
   }
 
-  // ---- B: DFT of the normal channels, warp = 16 tokens
-  const int hd = lane >> 2, r = lane & 3;
+  // ---- B: the normal channels as the A operand; warp = 16 tokens, lane = two channel positions
   if (warp * 16 < n_tok) {
-    const uint8_t* row0 = tile + (warp * 16 + hd) * kRowBytes;
-    const uint8_t* row1 = row0 + 8 * kRowBytes;
-    uint32_t a[4][4];
+    const uint32_t pc = *reinterpret_cast<const uint16_t*>(perm + kNA + 2 * lane);
+    const int c0 = (pc & 0xffu) * 2, c1 = (pc >> 8) * 2;
 #pragma unroll
-    for (int ks = 0; ks < 4; ++ks) {
-      const uint32_t pc = *reinterpret_cast<const uint16_t*>(perm + kNA + 16 * ks + 2 * r);        // two channel ids
-      const uint32_t pd = *reinterpret_cast<const uint16_t*>(perm + kNA + 16 * ks + 2 * r + 8);
-      const int c0 = (pc & 0xffu) * 2, c1 = (pc >> 8) * 2, c2 = (pd & 0xffu) * 2, c3 = (pd >> 8) * 2;
-      a[ks][0] = Ops<T>::to_half_pair(*reinterpret_cast<const uint16_t*>(row0 + c0) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row0 + c1)) << 16));
-      a[ks][1] = Ops<T>::to_half_pair(*reinterpret_cast<const uint16_t*>(row1 + c0) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row1 + c1)) << 16));
-      a[ks][2] = Ops<T>::to_half_pair(*reinterpret_cast<const uint16_t*>(row0 + c2) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row0 + c3)) << 16));
-      a[ks][3] = Ops<T>::to_half_pair(*reinterpret_cast<const uint16_t*>(row1 + c2) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(row1 + c3)) << 16));
+    for (int i = 0; i < 16; ++i) {
+      const int row = warp * 16 + i;
+      const uint8_t* rp = tile + row * kRowBytes;
+      const uint32_t raw = *reinterpret_cast<const uint16_t*>(rp + c0) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(rp + c1)) << 16);
+      *reinterpret_cast<uint32_t*>(aop + sw128_offset(row, 2 * lane)) = Ops<T>::to_half_pair(raw);
     }
-    float acc[8][4];
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) { acc[nt][0] = 0.0f; acc[nt][1] = 0.0f; acc[nt][2] = 0.0f; acc[nt][3] = 0.0f; }
-#pragma unroll
-    for (int ks = 0; ks < 4; ++ks) {
-#pragma unroll
-      for (int nt = 0; nt < 8; ++nt) {
-        const uint4 bw = __ldg(reinterpret_cast<const uint4*>(dft + ((ks * 8 + nt) * 32 + lane) * 4));
-        mma_f16(acc[nt], a[ks][0], a[ks][1], a[ks][2], a[ks][3], bw.x, bw.y);
-        mma_f16(acc[nt], a[ks][0], a[ks][1], a[ks][2], a[ks][3], bw.z, bw.w);
-      }
-    }
-    // sign bits: column e = 2 nt + c of half-word r goes to bit 15 - e; 1 = coefficient >= 0
-    uint32_t w0 = 0u, w1 = 0u;
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        w0 = __funnelshift_l(__float_as_uint(acc[nt][c]), w0, 1);
-        w1 = __funnelshift_l(__float_as_uint(acc[nt][c + 2]), w1, 1);
-      }
-    }
-    const int g = warp >> 1, nt_tok = 2 * (warp & 1);
-    uint16_t* hw = reinterpret_cast<uint16_t*>(kg_base + g * kKGroupBytes + kKG_Bits1);
-    hw[(hd * 4 + r) * 4 + nt_tok] = static_cast<uint16_t>(~w0);
-    hw[(hd * 4 + r) * 4 + nt_tok + 1] = static_cast<uint16_t>(~w1);
-    // column sums of |X| over the warp's 16 tokens: reduce-scatter over the 8 lanes of equal r
-    float p[16];
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      p[2 * nt] = fabsf(acc[nt][0]) + fabsf(acc[nt][2]);
-      p[2 * nt + 1] = fabsf(acc[nt][1]) + fabsf(acc[nt][3]);
-    }
-#pragma unroll
-    for (int width = 8, mask = 16; width >= 2; width >>= 1, mask >>= 1) {
-      const bool up = (lane & mask) != 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (i < width) {
-          const float send = up ? p[i] : p[i + width];
-          const float keep = up ? p[i + width] : p[i];
-          p[i] = keep + __shfl_xor_sync(0xffffffffu, send, mask);
-        }
-      }
-    }
-    const int e0 = ((lane & 16) ? 8 : 0) + ((lane & 8) ? 4 : 0) + ((lane & 4) ? 2 : 0);
-    colsum[warp * 64 + 16 * r + e0] = p[0];
-    colsum[warp * 64 + 16 * r + e0 + 1] = p[1];
   }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
 
-  // ---- C: s = Mean |X| per (group, column)
+  // ---- the tile is no longer needed: fetch the B operand (both parts of the matrix) over it
   {
-    const int f = tid & 63, g = tid >> 6;
-    if (g < n_groups) {
-      const float sum = colsum[(2 * g) * 64 + f] + colsum[(2 * g + 1) * 64 + f];
-      reinterpret_cast<uint16_t*>(kg_base + g * kKGroupBytes + kKG_S1)[f] = f2h_bits(sum * (1.0f / 32.0f));
-    }
+    uint8_t* wdst = tile;
+#pragma unroll
+    for (int i = 0; i < 2 * kUmmaBlockBytes / (256 * 16); ++i) cp_async16(wdst + (i * 256 + tid) * 16, g_dft_umma + (i * 256 + tid) * 16);
+    asm volatile("cp.async.commit_group;" ::: "memory");
   }
 
   // ---- D: 2-bit codes, thread = one 32-bit word = (token, 16 slots), two words per thread
@@ -307,6 +320,74 @@ __global__ void __launch_bounds__(256) k_encode_kernel(KSrc src, int64_t T_token
       asm("prmt.b32 %0, %1, %2, 0x6240;" : "=r"(word) : "r"(as_u32(lo)), "r"(as_u32(hi)));
       reinterpret_cast<uint32_t*>(kg_base + g * kKGroupBytes + kKG_Codes2)[widx] = word;
     }
+  }
+
+  // ---- the product: X[128 x 64] = A (leading part of the matrix) + A (remainder), K = 64 in four steps each
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (tid == 0) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint64_t da = umma_desc_sw128(smem_u32(aop));
+    const uint64_t db = umma_desc_sw128(smem_u32(tile));
+#pragma unroll
+    for (int part = 0; part < 2; ++part) {
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks)   // 16 binary16 = 32 bytes along K per step: the start address field counts 16 bytes
+        umma_f16(tmem, da + static_cast<uint64_t>(2 * ks), db + static_cast<uint64_t>(part * (kUmmaBlockBytes >> 4) + 2 * ks),
+                 (part | ks) != 0 ? 1u : 0u);
+    }
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(mbar)) : "memory");
+  }
+  // every thread waits for the accumulator; the wait is bounded, a timeout is reported in the status word
+  uint32_t done = 0;
+  for (int it = 0; it < kWaitLimit && !done; ++it) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_u32(mbar)), "r"(0u) : "memory");
+  }
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  done = __all_sync(0xffffffffu, done != 0);
+
+  // ---- sign bits and s = Mean |X| (Eq. 5): warp = (group g, 32 spectrum columns), lane = token
+  const int g = warp & 3, half = warp >> 2;
+  if (!done) {
+    if (tid == 0) atomicCAS(reinterpret_cast<int*>(cv.base + kHdrStatus), 0, static_cast<int>(VIDKV_ERR_TIMEOUT));
+  } else if (g < n_groups) {
+    uint32_t x[32];
+    tmem_ld32(tmem + (static_cast<uint32_t>(g * 32) << 16) + static_cast<uint32_t>(half * 32), x);
+    // column e of a 16-column block goes to bit 15 - e of the block's half-word; 1 = coefficient >= 0
+    uint32_t w = 0u;
+#pragma unroll
+    for (int c = 0; c < 32; ++c) w = __funnelshift_l(x[c], w, 1);
+    w = ~w;
+    uint16_t* hw = reinterpret_cast<uint16_t*>(kg_base + g * kKGroupBytes + kKG_Bits1);
+    const int hidx = ((lane & 7) * 4 + 2 * half) * 4 + (lane >> 3);
+    hw[hidx] = static_cast<uint16_t>(w >> 16);
+    hw[hidx + 4] = static_cast<uint16_t>(w);
+    // column sums of |X| over the group's 32 tokens: reduce-scatter over the lanes, lane l ends with column l
+    float p[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) p[c] = fabsf(__uint_as_float(x[c]));
+#pragma unroll
+    for (int width = 16; width >= 1; width >>= 1) {
+      const bool up = (lane & width) != 0;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        if (i < width) {
+          const float send = up ? p[i] : p[i + width];
+          const float keep = up ? p[i + width] : p[i];
+          p[i] = keep + __shfl_xor_sync(0xffffffffu, send, width);
+        }
+      }
+    }
+    reinterpret_cast<uint16_t*>(kg_base + g * kKGroupBytes + kKG_S1)[half * 32 + lane] = f2h_bits(p[0] * (1.0f / 32.0f));
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
 }
 
