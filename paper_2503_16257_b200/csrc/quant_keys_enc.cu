@@ -78,12 +78,13 @@ template <> struct Ops<__nv_bfloat16> {
 __device__ __forceinline__ int ord_of(uint16_t b) { return (b & 0x8000u) ? -static_cast<int>(b & 0x7fffu) : static_cast<int>(b); }
 __device__ __forceinline__ uint16_t bits_of(int o) { return o >= 0 ? static_cast<uint16_t>(o) : static_cast<uint16_t>(0x8000u | static_cast<uint32_t>(-o)); }
 
-// Eq. 4 for one element, in the defining arithmetic (float32, IEEE division, round half to even).
+// Eq. 4 for one element, in the defining arithmetic (float32, IEEE division, round half to even):
+// is the code of the element with value order o at least k?  (k = 1..3, so the clamp to [0, 3]
+// does not change the answer.)
 template <typename T>
-__device__ __forceinline__ int code_ref(int o, float z, float s) {
+__device__ __forceinline__ bool code_at_least(int o, float z, float s, float k) {
   const float d = __fsub_rn(Ops<T>::to_float(bits_of(o)), z);
-  const float q = fminf(fmaxf(rintf(__fdiv_rn(d, s)), 0.0f), 3.0f);
-  return static_cast<int>(q);
+  return rintf(__fdiv_rn(d, s)) >= k;
 }
 
 }  // namespace
@@ -198,10 +199,14 @@ __global__ void __launch_bounds__(256, 3) k_encode_kernel(KSrc src, int64_t T_to
   uint8_t* kg_base = slab_ptr + cv.kgroup_offset + (kgroup0 + t0 / kG) * kKGroupBytes;
 
   // ---- stage the tile; meanwhile set up the barrier and 64 columns of tensor memory
-  for (int i = tid; i < n_tok * 16; i += 256) {
-    const int row = i >> 4, piece = i & 15;
-    cp_async16(tile + row * kRowBytes + piece * 16,
-               reinterpret_cast<const uint8_t*>(base + (t0 + row) * src.stride_t) + piece * 16);
+  {
+    const int row0 = tid >> 4, piece = tid & 15;   // 16 threads per token row, 16 rows per sweep
+    const uint8_t* srow = reinterpret_cast<const uint8_t*>(base + (t0 + row0) * src.stride_t) + piece * 16;
+    uint8_t* drow = tile + row0 * kRowBytes + piece * 16;
+    const int64_t sstep = 16 * src.stride_t * static_cast<int64_t>(sizeof(T));
+#pragma unroll
+    for (int it = 0; it < kEncTokens / 16; ++it)
+      if (row0 + 16 * it < n_tok) cp_async16(drow + it * 16 * kRowBytes, srow + it * sstep);
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
   if (tid < kD) perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
@@ -247,19 +252,20 @@ __global__ void __launch_bounds__(256, 3) k_encode_kernel(KSrc src, int64_t T_to
         uint16_t X = Ops<T>::kInf;                     // s == 0: every code is 0
         if (s != 0.0f) {
           int o = ord_of(Ops<T>::from_float_rn(fmaf(static_cast<float>(k) - 0.5f, s, z)));
-          // the threshold is almost always the candidate or a neighbour: three independent evaluations
-          const int cm = code_ref<T>(o - 1, z, s), c0 = code_ref<T>(o, z, s), cp = code_ref<T>(o + 1, z, s);
-          if (cm < k && c0 >= k) {
-          } else if (c0 < k && cp >= k) {
-            o += 1;
-          } else if (cm >= k) {
+          // the threshold is almost always the candidate or its upper neighbour: two evaluations
+          const float kf = static_cast<float>(k);
+          const bool p0 = code_at_least<T>(o, z, s, kf);
+          const bool p1 = code_at_least<T>(p0 ? o - 1 : o + 1, z, s, kf);
+          if (p0 != p1) {
+            o += p0 ? 0 : 1;
+          } else if (p0) {
             o -= 1;
 #pragma unroll 1
-            for (int it = 0; it < 4 && code_ref<T>(o - 1, z, s) >= k; ++it) --o;
+            for (int it = 0; it < 4 && code_at_least<T>(o - 1, z, s, kf); ++it) --o;
           } else {
             o += 2;
 #pragma unroll 1
-            for (int it = 0; it < 4 && code_ref<T>(o, z, s) < k; ++it) ++o;
+            for (int it = 0; it < 4 && !code_at_least<T>(o, z, s, kf); ++it) ++o;
           }
           X = bits_of(o);
         }
