@@ -15,6 +15,9 @@
 // grid = (tiles of 128 tokens, slabs); block = 256 threads = 8 warps.
 #include <math.h>
 
+#include <algorithm>
+#include <cstdint>
+
 #include "common.cuh"
 #include "kernels.cuh"
 
@@ -23,16 +26,16 @@ namespace vidkv {
 namespace {
 
 constexpr int kEncTokens = 128;
-constexpr int kRowBytes = 272;                 // 256 bytes of data + 16 of padding per staged token
 constexpr int kDftWords = 4 * 8 * 32 * 4;      // [k step][column tile][lane][hi0, hi1, lo0, lo1]
 
 // B fragments of the DFT matrix in the order the MMA wants them (see dft_table_kernel).
 __device__ __align__(16) uint32_t g_dft_frag[kDftWords];
 
-// The same matrix as the B operand of tcgen05.mma: two blocks (leading part, remainder) of
-// [64 spectrum columns][64 channel positions] binary16, K-major with the 128-byte swizzle.
-constexpr int kUmmaBlockBytes = 64 * 128;
-__device__ __align__(1024) uint8_t g_dft_umma[2 * kUmmaBlockBytes];
+// The same matrix as plain 16-bit patterns [part][spectrum column f][channel position c]:
+// parts 0, 1: binary16 leading part and remainder; parts 2, 3, 4: bfloat16 leading, middle and
+// last part (w = sum of the parts to 22 resp. 24 bits).
+constexpr int kWParts = 5;
+__device__ __align__(16) uint16_t g_dft_w[kWParts * 64 * 64];
 
 // Byte offset of element (row, k) of a K-major operand with 64 binary16 per row under the
 // 128-byte swizzle: 8-row atoms of 1024 bytes, 16-byte pieces XORed with the row within the atom.
@@ -117,14 +120,19 @@ __global__ void dft_table_kernel() {
     g_dft_frag[i * 4 + 2] = as_u32(__floats2half2_rn(w[0] - __half2float(h0), w[1] - __half2float(h1)));
     g_dft_frag[i * 4 + 3] = as_u32(__floats2half2_rn(w[2] - __half2float(h2), w[3] - __half2float(h3)));
   }
-  // tcgen05 operand: row = spectrum column f, k = position c among the normal channels
   for (int i = threadIdx.x; i < 64 * 64; i += blockDim.x) {
     const int f = i >> 6, c = i & 63;
     const float w = static_cast<float>(dft_weight(f, c));
     const __half hi = __float2half_rn(w);
-    const __half lo = __float2half_rn(w - __half2float(hi));
-    *reinterpret_cast<__half*>(g_dft_umma + sw128_offset(f, c)) = hi;
-    *reinterpret_cast<__half*>(g_dft_umma + kUmmaBlockBytes + sw128_offset(f, c)) = lo;
+    g_dft_w[i] = __half_as_ushort(hi);
+    g_dft_w[4096 + i] = __half_as_ushort(__float2half_rn(w - __half2float(hi)));
+    const __nv_bfloat16 b0 = __float2bfloat16_rn(w);
+    const float r1 = w - __bfloat162float(b0);
+    const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(b1);
+    g_dft_w[2 * 4096 + i] = __bfloat16_as_ushort(b0);
+    g_dft_w[3 * 4096 + i] = __bfloat16_as_ushort(b1);
+    g_dft_w[4 * 4096 + i] = __bfloat16_as_ushort(__float2bfloat16_rn(r2));
   }
 }
 
@@ -137,16 +145,14 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
   return static_cast<uint64_t>((smem_addr >> 4) & 0x3fffu) | (static_cast<uint64_t>(1u) << 16) |
          (static_cast<uint64_t>(1024u >> 4) << 32) | (static_cast<uint64_t>(1u) << 46) | (static_cast<uint64_t>(2u) << 61);
 }
-// Instruction descriptor: float32 accumulator, binary16 A and B, both K-major, N = 64, M = 128.
-constexpr uint32_t kUmmaIdesc = (1u << 4) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr int kTmemCols = 64;
+constexpr int kTmemCols = 256;        // two float32 accumulators of 128 x 128
 constexpr int kWaitLimit = 1 << 14;
 
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
-      ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(kUmmaIdesc), "r"(accumulate), "r"(0u)
+      ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
       : "memory");
 }
 // 32 consecutive accumulator columns of the calling warp's 32 lanes of tensor memory.
@@ -162,234 +168,337 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
+}
 
-// Shared memory of one block, from a 1024-byte boundary:
-//   [0, 16384)       A operand: the normal channels of the tile, [128 tokens][64 positions]
-//   [16384, 51200)   the staged tile, [128][272] raw elements; once the tile has been sorted into
-//                    the A operand and the gathered anomalous values, its first 16 KB take the B operand
-//   [51200, 67584)   anomalous values gathered per code word
-//   then thresholds [4][3][32] pairs, the channel order [128], the mbarrier, the tensor-memory address
-constexpr int kSmAop = 0, kSmTile = 16384, kSmGath = kSmTile + kEncTokens * kRowBytes, kSmThr = kSmGath + 4 * 128 * 32,
-              kSmPerm = kSmThr + 4 * 3 * 32 * 4, kSmBar = kSmPerm + kD, kSmEnd = kSmBar + 16;
+// Per element type: how the DFT matrix is split (binary16: 2 parts, bfloat16: 3 parts), the
+// operand format code of the instruction descriptor, and 1.0.
+template <typename T> struct Enc;
+template <> struct Enc<__half> {
+  static constexpr int kParts = 2, kFmt = 0, kTab = 0;
+  static constexpr uint16_t kOne = 0x3c00u;
+  static __device__ __forceinline__ uint32_t pack(float a, float b) { return as_u32(__floats2half2_rn(a, b)); }
+};
+template <> struct Enc<__nv_bfloat16> {
+  static constexpr int kParts = 3, kFmt = 1, kTab = 2;
+  static constexpr uint16_t kOne = 0x3f80u;
+  static __device__ __forceinline__ uint32_t pack(float a, float b) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&v);
+  }
+};
 
-size_t k_encode_smem_bytes() { return kSmEnd + 1024; }
+// Shared memory of one block, from a 1024-byte boundary.  All operands are K-major with the
+// 128-byte swizzle, one 64-channel block of K after the other.
+//   [0, 32768)        the tile as the B operand: [2 K blocks][128 tokens][64 channels]
+//   [32768, 65536)    A, leading part: [2 K blocks][128 rows][64 channels]; row m < 64 selects the
+//                     anomalous channel of slot m, row 64 + f holds column f of the DFT matrix
+//                     spread over the normal channels (zero elsewhere)
+//   [65536, ...)      A, remaining parts of the DFT rows only: per part [2 K blocks][64 rows][64 channels].
+//                     Their products use M = 128 with a descriptor that starts 64 rows early; those
+//                     rows read whatever precedes (finite numbers) and land in accumulator rows
+//                     that nobody reads.
+//   then the channel order [128], the mbarrier, the tensor-memory address, the fault flag
+constexpr int kSmTile = 0, kSmAhi = 32768, kSmAex = 65536;
+template <typename T> __host__ __device__ constexpr int enc_sm_perm() { return kSmAex + 16384 * (Enc<T>::kParts - 1); }
+template <typename T> __host__ __device__ constexpr int enc_sm_bytes() { return enc_sm_perm<T>() + kD + 32 + 1024; }
 
+size_t k_encode_smem_bytes(int dtype) { return dtype == VIDKV_F16 ? enc_sm_bytes<__half>() : enc_sm_bytes<__nv_bfloat16>(); }
+
+// Persistent blocks, two per SM: block b encodes the tiles [n b / G, n (b + 1) / G) of the
+// launch's n = slabs x tiles-per-slab tiles.  Warp w works on tensor-memory lanes 32 (w % 4):
+// warps with w % 4 < 2 own 32 anomalous slots each, the others 32 spectrum columns each (and
+// issue the tile loads); w / 4 picks two of the tile's four 32-token groups.
 template <typename T>
-__global__ void __launch_bounds__(256, 3) k_encode_kernel(KSrc src, int64_t T_tokens, CacheView cv, int layer0,
-                                                          int slabs_per_layer, int chunk, int64_t kgroup0) {
+__global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_tokens, CacheView cv, int layer0,
+                                                          int slabs_per_layer, int chunk, int64_t kgroup0,
+                                                          int tiles_per_slab, int total_tiles) {
   extern __shared__ uint8_t esm_raw[];
   uint8_t* esm = esm_raw + ((1024u - (smem_u32(esm_raw) & 1023u)) & 1023u);
-  uint8_t* aop = esm + kSmAop;
   uint8_t* tile = esm + kSmTile;
-  uint16_t* gath = reinterpret_cast<uint16_t*>(esm + kSmGath);   // [group][word of the group's 2-bit block][16 slots]
-  uint32_t* thr = reinterpret_cast<uint32_t*>(esm + kSmThr);
-  uint8_t* perm = esm + kSmPerm;
-  uint64_t* mbar = reinterpret_cast<uint64_t*>(esm + kSmBar);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(esm + kSmBar + 8);
+  uint8_t* a_hi = esm + kSmAhi;
+  uint8_t* a_ex = esm + kSmAex;
+  uint8_t* perm = esm + enc_sm_perm<T>();
+  uint64_t* mbar = reinterpret_cast<uint64_t*>(perm + kD);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(perm + kD + 8);
+  volatile uint32_t* fault = reinterpret_cast<volatile uint32_t*>(perm + kD + 12);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int slab = blockIdx.y;
-  const int layer = layer0 + slab / slabs_per_layer;
-  const int bh = slab % slabs_per_layer;
-  const T* base = reinterpret_cast<const T*>(src.ptr) + (slab / src.H) * src.stride_b + (slab % src.H) * src.stride_h;
-  uint8_t* slab_ptr = cv.slab(layer, bh / cv.H_kv, bh % cv.H_kv);
-  const int64_t t0 = static_cast<int64_t>(blockIdx.x) * kEncTokens;
-  const int n_tok = static_cast<int>(min(static_cast<int64_t>(kEncTokens), T_tokens - t0));   // multiple of 32
-  const int n_groups = n_tok / kG;
-  uint8_t* kg_base = slab_ptr + cv.kgroup_offset + (kgroup0 + t0 / kG) * kKGroupBytes;
+  const int quad = warp & 3, half = warp >> 2;
+  const bool loader = quad >= 2;
+  const int lt = half * 64 + (quad - 2) * 32 + lane;   // 0 .. 127 among the loading threads
 
-  // ---- stage the tile; meanwhile set up the barrier and 64 columns of tensor memory
-  {
-    const int row0 = tid >> 4, piece = tid & 15;   // 16 threads per token row, 16 rows per sweep
-    const uint8_t* srow = reinterpret_cast<const uint8_t*>(base + (t0 + row0) * src.stride_t) + piece * 16;
-    uint8_t* drow = tile + row0 * kRowBytes + piece * 16;
-    const int64_t sstep = 16 * src.stride_t * static_cast<int64_t>(sizeof(T));
-#pragma unroll
-    for (int it = 0; it < kEncTokens / 16; ++it)
-      if (row0 + 16 * it < n_tok) cp_async16(drow + it * 16 * kRowBytes, srow + it * sstep);
-  }
-  asm volatile("cp.async.commit_group;" ::: "memory");
-  if (tid < kD) perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
   if (tid == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(mbar)) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    *fault = 0u;
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
 
-  // ---- A: Eq. 4 metadata and thresholds, thread = (anomalous slot j, group g)
-  {
-    const int j = tid & 63, g = tid >> 6;
-    if (g < n_groups) {
-      const uint8_t* p = tile + (g * kG) * kRowBytes + perm[j] * 2;
-      // token t of the group goes to word ((t % 8) * 4 + j / 16) * 4 + t / 8, slot j % 16
-      uint16_t* gp = gath + (g * 128 + (j >> 4) * 4) * 16 + (j & 15);
-      uint16_t mn = *reinterpret_cast<const uint16_t*>(p), mx = mn;
-      gp[0] = mn;
-#pragma unroll
-      for (int t = 1; t < kG; ++t) {
-        const uint16_t v = *reinterpret_cast<const uint16_t*>(p + t * kRowBytes);
-        mn = Ops<T>::vmin(mn, v); mx = Ops<T>::vmax(mx, v);
-        gp[((t & 7) * 16 + (t >> 3)) * 16] = v;
-      }
-      const float fmn = Ops<T>::to_float(mn), fmx = Ops<T>::to_float(mx);
-      const uint16_t sh = f2h_bits(__fdiv_rn(__fsub_rn(fmx, fmn), 3.0f));
-      const uint16_t zh = f2h_bits(fmn);
-      uint8_t* kg = kg_base + g * kKGroupBytes;
-      reinterpret_cast<uint16_t*>(kg + kKG_S2)[j] = sh;
-      reinterpret_cast<uint16_t*>(kg + kKG_Z2)[j] = zh;
-      const float s = h2f(sh), z = h2f(zh);
-      uint16_t* th = reinterpret_cast<uint16_t*>(thr + g * 3 * 32);
-#pragma unroll 1
-      for (int k = 1; k <= 3; ++k) {
-        uint16_t X = Ops<T>::kInf;                     // s == 0: every code is 0
-        if (s != 0.0f) {
-          int o = ord_of(Ops<T>::from_float_rn(fmaf(static_cast<float>(k) - 0.5f, s, z)));
-          // the threshold is almost always the candidate or its upper neighbour: two evaluations
-          const float kf = static_cast<float>(k);
-          const bool p0 = code_at_least<T>(o, z, s, kf);
-          const bool p1 = code_at_least<T>(p0 ? o - 1 : o + 1, z, s, kf);
-          if (p0 != p1) {
-            o += p0 ? 0 : 1;
-          } else if (p0) {
-            o -= 1;
-#pragma unroll 1
-            for (int it = 0; it < 4 && code_at_least<T>(o - 1, z, s, kf); ++it) --o;
-          } else {
-            o += 2;
-#pragma unroll 1
-            for (int it = 0; it < 4 && !code_at_least<T>(o, z, s, kf); ++it) ++o;
-          }
-          X = bits_of(o);
-        }
-        th[(k - 1) * 64 + j] = X;
-      }
-    }
-  }
+  const int tile_begin = static_cast<int>(static_cast<int64_t>(total_tiles) * blockIdx.x / gridDim.x);
+  const int tile_end = static_cast<int>(static_cast<int64_t>(total_tiles) * (blockIdx.x + 1) / gridDim.x);
 
-  // ---- B: the normal channels as the A operand; warp = 16 tokens, lane = two channel positions
-  if (warp * 16 < n_tok) {
-    const uint32_t pc = *reinterpret_cast<const uint16_t*>(perm + kNA + 2 * lane);
-    const int c0 = (pc & 0xffu) * 2, c1 = (pc >> 8) * 2;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int row = warp * 16 + i;
-      const uint8_t* rp = tile + row * kRowBytes;
-      const uint32_t raw = *reinterpret_cast<const uint16_t*>(rp + c0) | (static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(rp + c1)) << 16);
-      *reinterpret_cast<uint32_t*>(aop + sw128_offset(row, 2 * lane)) = Ops<T>::to_half_pair(raw);
-    }
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  __syncthreads();
+  // Tiles are walked as (slab, tile of the slab) pairs so that divisions happen once per block,
+  // once for the tile being encoded and once for the tile being fetched.
+  int slab = tile_begin / tiles_per_slab, ti = tile_begin - slab * tiles_per_slab;
+  int lslab = slab, lti = ti, lbase_slab = -1;
+  const T* lbase = nullptr;
 
-  // ---- the tile is no longer needed: fetch the B operand (both parts of the matrix) over it
-  {
-    uint8_t* wdst = tile;
+  // 16-byte pieces of a tile: thread lt moves piece lt % 16 of the rows lt / 16 + 8 i
+  auto load_next_tile = [&]() {
+    if (lslab != lbase_slab) {
+      lbase_slab = lslab;
+      lbase = reinterpret_cast<const T*>(src.ptr) + (lslab / src.H) * src.stride_b + (lslab % src.H) * src.stride_h;
+    }
+    const int64_t t0 = static_cast<int64_t>(lti) * kEncTokens;
+    const int n_tok = static_cast<int>(min(static_cast<int64_t>(kEncTokens), T_tokens - t0));
+    const int row0 = lt >> 4, piece = lt & 15;
+    const uint8_t* srow = reinterpret_cast<const uint8_t*>(lbase + (t0 + row0) * src.stride_t) + piece * 16;
+    uint8_t* drow = tile + (piece >> 3) * 16384 + row0 * 128 + (((piece & 7) ^ row0) << 4);
+    const int64_t sstep = 8 * src.stride_t * static_cast<int64_t>(sizeof(T));
 #pragma unroll
-    for (int i = 0; i < 2 * kUmmaBlockBytes / (256 * 16); ++i) cp_async16(wdst + (i * 256 + tid) * 16, g_dft_umma + (i * 256 + tid) * 16);
+    for (int i = 0; i < kEncTokens / 8; ++i)
+      if (row0 + 8 * i < n_tok) cp_async16(drow + i * 1024, srow + i * sstep);
     asm volatile("cp.async.commit_group;" ::: "memory");
-  }
+    if (++lti == tiles_per_slab) { lti = 0; ++lslab; }
+  };
 
-  // ---- D: 2-bit codes, thread = one 32-bit word = (token, 16 slots), two words per thread
-  {
-    const int widx = tid & 127;
-    const int r4 = (widx >> 2) & 3;
-    const uint32_t k1024 = 0x64006400u;
-    const uint32_t wgt[4] = {0x3c003c00u, 0x44004400u, 0x4c004c00u, 0x54005400u};   // 1, 4, 16, 64
-#pragma unroll 1
-    for (int g = tid >> 7; g < n_groups; g += 2) {
-      const uint4* gv = reinterpret_cast<const uint4*>(gath + (g * 128 + widx) * 16);
-      const uint4 v0 = gv[0], v1 = gv[1];
-      const uint32_t v[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-      const uint4* th = reinterpret_cast<const uint4*>(thr + g * 3 * 32 + 8 * r4);
-      uint32_t x1[8], x2[8], x3[8];
-      { const uint4 a0 = th[0], a1 = th[1]; x1[0] = a0.x; x1[1] = a0.y; x1[2] = a0.z; x1[3] = a0.w; x1[4] = a1.x; x1[5] = a1.y; x1[6] = a1.z; x1[7] = a1.w; }
-      { const uint4 a0 = th[8], a1 = th[9]; x2[0] = a0.x; x2[1] = a0.y; x2[2] = a0.z; x2[3] = a0.w; x2[4] = a1.x; x2[5] = a1.y; x2[6] = a1.z; x2[7] = a1.w; }
-      { const uint4 a0 = th[16], a1 = th[17]; x3[0] = a0.x; x3[1] = a0.y; x3[2] = a0.z; x3[3] = a0.w; x3[4] = a1.x; x3[5] = a1.y; x3[6] = a1.z; x3[7] = a1.w; }
-      __half2 lo = as_h2(k1024), hi = as_h2(k1024);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const __half2 code = __hadd2(__hadd2(as_h2(Ops<T>::ge(v[i], x1[i])), as_h2(Ops<T>::ge(v[i], x2[i]))),
-                                     as_h2(Ops<T>::ge(v[i], x3[i])));
-        if (i < 4) lo = __hfma2(code, as_h2(wgt[i & 3]), lo);
-        else hi = __hfma2(code, as_h2(wgt[i & 3]), hi);
+  int cur_slab = -1;
+  uint32_t phase = 0;
+  uint8_t* slab_ptr = nullptr;
+  if (loader && tile_begin < tile_end) load_next_tile();
+  for (int t = tile_begin; t < tile_end; ++t, ti = (ti + 1 == tiles_per_slab) ? 0 : ti + 1, slab += (ti == 0) ? 1 : 0) {
+    if (slab != cur_slab) {
+      const int layer = layer0 + slab / slabs_per_layer;
+      const int bh = slab % slabs_per_layer;
+      slab_ptr = cv.slab(layer, bh / cv.H_kv, bh % cv.H_kv);
+    }
+    const int64_t t0 = static_cast<int64_t>(ti) * kEncTokens;
+    const int n_tok = static_cast<int>(min(static_cast<int64_t>(kEncTokens), T_tokens - t0));   // multiple of 32
+    const int n_groups = n_tok / kG;
+    uint8_t* kg_base = slab_ptr + cv.kgroup_offset + (kgroup0 + t0 / kG) * kKGroupBytes;
+
+    // ---- a new slab: its channel order and the A operand built from it
+    if (slab != cur_slab) {
+      cur_slab = slab;
+      if (tid < kD) perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
+      constexpr int kAVec = (32768 + 16384 * (Enc<T>::kParts - 1)) / 16;
+      for (int i = tid; i < kAVec; i += 256) reinterpret_cast<uint4*>(a_hi)[i] = make_uint4(0u, 0u, 0u, 0u);
+      __syncthreads();
+      if (tid < kNA) {
+        const int c = perm[tid];
+        *reinterpret_cast<uint16_t*>(a_hi + (c >> 6) * 16384 + sw128_offset(tid, c & 63)) = Enc<T>::kOne;
       }
-      // 1024 + n keeps n in the low byte of each lane: fields 0-3 and 4-7 of both half-words
-      uint32_t word;
-      asm("prmt.b32 %0, %1, %2, 0x6240;" : "=r"(word) : "r"(as_u32(lo)), "r"(as_u32(hi)));
-      reinterpret_cast<uint32_t*>(kg_base + g * kKGroupBytes + kKG_Codes2)[widx] = word;
+      for (int i = tid; i < 64 * 64; i += 256) {
+        const int f = i >> 6, c = perm[kNA + (i & 63)];
+        *reinterpret_cast<uint16_t*>(a_hi + (c >> 6) * 16384 + sw128_offset(64 + f, c & 63)) = g_dft_w[Enc<T>::kTab * 4096 + i];
+#pragma unroll
+        for (int part = 1; part < Enc<T>::kParts; ++part)
+          *reinterpret_cast<uint16_t*>(a_ex + (part - 1) * 16384 + (c >> 6) * 8192 + sw128_offset(f, c & 63)) =
+              g_dft_w[(Enc<T>::kTab + part) * 4096 + i];
+      }
     }
-  }
 
-  // ---- the product: X[128 x 64] = A (leading part of the matrix) + A (remainder), K = 64 in four steps each
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  if (tid == 0) {
+    // ---- the tile has landed; the accumulators of the previous tile have been read
+    if (loader) asm volatile("cp.async.wait_group 0;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint64_t da = umma_desc_sw128(smem_u32(aop));
-    const uint64_t db = umma_desc_sw128(smem_u32(tile));
-#pragma unroll
-    for (int part = 0; part < 2; ++part) {
-#pragma unroll
-      for (int ks = 0; ks < 4; ++ks)   // 16 binary16 = 32 bytes along K per step: the start address field counts 16 bytes
-        umma_f16(tmem, da + static_cast<uint64_t>(2 * ks), db + static_cast<uint64_t>(part * (kUmmaBlockBytes >> 4) + 2 * ks),
-                 (part | ks) != 0 ? 1u : 0u);
-    }
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(mbar)) : "memory");
-  }
-  // every thread waits for the accumulator; the wait is bounded, a timeout is reported in the status word
-  uint32_t done = 0;
-  for (int it = 0; it < kWaitLimit && !done; ++it) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(smem_u32(mbar)), "r"(0u) : "memory");
-  }
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  done = __all_sync(0xffffffffu, done != 0);
+    if (*fault) break;
 
-  // ---- sign bits and s = Mean |X| (Eq. 5): warp = (group g, 32 spectrum columns), lane = token
-  const int g = warp & 3, half = warp >> 2;
-  if (!done) {
-    if (tid == 0) atomicCAS(reinterpret_cast<int*>(cv.base + kHdrStatus), 0, static_cast<int>(VIDKV_ERR_TIMEOUT));
-  } else if (g < n_groups) {
-    uint32_t x[32];
-    tmem_ld32(tmem + (static_cast<uint32_t>(g * 32) << 16) + static_cast<uint32_t>(half * 32), x);
-    // column e of a 16-column block goes to bit 15 - e of the block's half-word; 1 = coefficient >= 0
-    uint32_t w = 0u;
+    // ---- D[128 rows x 128 tokens] = A (leading) x tile^T; D'[.. x ..] = A (remaining parts) x tile^T
+    if (tid == 0) {
+      constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(Enc<T>::kFmt) << 7) | (static_cast<uint32_t>(Enc<T>::kFmt) << 10) |
+                                 ((128u >> 3) << 17) | ((128u >> 4) << 24);
 #pragma unroll
-    for (int c = 0; c < 32; ++c) w = __funnelshift_l(x[c], w, 1);
-    w = ~w;
-    uint16_t* hw = reinterpret_cast<uint16_t*>(kg_base + g * kKGroupBytes + kKG_Bits1);
-    const int hidx = ((lane & 7) * 4 + 2 * half) * 4 + (lane >> 3);
-    hw[hidx] = static_cast<uint16_t>(w >> 16);
-    hw[hidx + 4] = static_cast<uint16_t>(w);
-    // column sums of |X| over the group's 32 tokens: reduce-scatter over the lanes, lane l ends with column l
-    float p[32];
+      for (int kb = 0; kb < 2; ++kb) {
+        const uint64_t da = umma_desc_sw128(smem_u32(a_hi + kb * 16384)), db = umma_desc_sw128(smem_u32(tile + kb * 16384));
 #pragma unroll
-    for (int c = 0; c < 32; ++c) p[c] = fabsf(__uint_as_float(x[c]));
+        for (int ks = 0; ks < 4; ++ks)   // 16 elements = 32 bytes along K per step; the address field counts 16 bytes
+          umma_f16(tmem, da + static_cast<uint64_t>(2 * ks), db + static_cast<uint64_t>(2 * ks), idesc, (kb | ks) != 0 ? 1u : 0u);
+      }
 #pragma unroll
-    for (int width = 16; width >= 1; width >>= 1) {
-      const bool up = (lane & width) != 0;
+      for (int part = 1; part < Enc<T>::kParts; ++part) {
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        if (i < width) {
-          const float send = up ? p[i] : p[i + width];
-          const float keep = up ? p[i + width] : p[i];
-          p[i] = keep + __shfl_xor_sync(0xffffffffu, send, width);
+        for (int kb = 0; kb < 2; ++kb) {
+          // rows 64 .. 127 of the operand are the part's data: start 64 rows (8192 bytes) early
+          const uint64_t da = umma_desc_sw128(smem_u32(a_ex + (part - 1) * 16384 + kb * 8192 - 8192));
+          const uint64_t db = umma_desc_sw128(smem_u32(tile + kb * 16384));
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            umma_f16(tmem + 128u, da + static_cast<uint64_t>(2 * ks), db + static_cast<uint64_t>(2 * ks), idesc,
+                     (part - 1) | kb | ks ? 1u : 0u);
         }
       }
+      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(mbar)) : "memory");
     }
-    reinterpret_cast<uint16_t*>(kg_base + g * kKGroupBytes + kKG_S1)[half * 32 + lane] = f2h_bits(p[0] * (1.0f / 32.0f));
+    // every thread waits for the accumulators; the wait is bounded, a timeout is reported in the status word
+    uint32_t done = 0;
+    for (int it = 0; it < kWaitLimit && !done; ++it) {
+      asm volatile(
+          "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(done) : "r"(smem_u32(mbar)), "r"(phase) : "memory");
+    }
+    phase ^= 1u;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    done = __all_sync(0xffffffffu, done != 0);
+    if (!done) {
+      if (lane == 0) {
+        *fault = 1u;
+        atomicCAS(reinterpret_cast<int*>(cv.base + kHdrStatus), 0, static_cast<int>(VIDKV_ERR_TIMEOUT));
+      }
+      continue;
+    }
+    // the products are done with shared memory: fetch the next tile behind the epilogue
+    if (loader && t + 1 < tile_end) load_next_tile();
+
+    if (!loader) {
+      // ---- Eq. 4: lane = anomalous slot j, the accumulator row holds its 128 tokens (exact values)
+      const int j = quad * 32 + lane, wg = j >> 4;
+      const int pos = (lane >> 1) & 3;                            // field of the slot inside its code byte
+      const bool pb0 = (lane & 2) != 0, pb1 = (lane & 4) != 0;    // bits of pos
+      const bool bb0 = (lane & 8) != 0, bb1 = (lane & 1) != 0;    // bits of the slot's byte index 2 (e % 2) + e / 8
+      const uint32_t wgt = pos == 0 ? 0x3c003c00u : pos == 1 ? 0x44004400u : pos == 2 ? 0x4c004c00u : 0x54005400u;   // 4^pos
+#pragma unroll 1
+      for (int g = 2 * half; g < 2 * half + 2 && g < n_groups; ++g) {
+        uint32_t x[32];
+        tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(g * 32), x);
+        float fmn = __uint_as_float(x[0]), fmx = fmn;
+#pragma unroll
+        for (int i = 1; i < 32; ++i) { fmn = fminf(fmn, __uint_as_float(x[i])); fmx = fmaxf(fmx, __uint_as_float(x[i])); }
+        const uint16_t sh = f2h_bits(__fdiv_rn(__fsub_rn(fmx, fmn), 3.0f));
+        const uint16_t zh = f2h_bits(fmn);
+        uint8_t* kg = kg_base + g * kKGroupBytes;
+        reinterpret_cast<uint16_t*>(kg + kKG_S2)[j] = sh;
+        reinterpret_cast<uint16_t*>(kg + kKG_Z2)[j] = zh;
+        const float sc = h2f(sh), z = h2f(zh);
+        uint32_t thr[3];
+#pragma unroll
+        for (int k = 1; k <= 3; ++k) {
+          uint16_t X = Ops<T>::kInf;                     // s == 0: every code is 0
+          if (sc != 0.0f) {
+            int o = ord_of(Ops<T>::from_float_rn(fmaf(static_cast<float>(k) - 0.5f, sc, z)));
+            // the threshold is almost always the candidate or its upper neighbour: two evaluations
+            const float kf = static_cast<float>(k);
+            const bool p0 = code_at_least<T>(o, z, sc, kf);
+            const bool p1 = code_at_least<T>(p0 ? o - 1 : o + 1, z, sc, kf);
+            if (p0 != p1) {
+              o += p0 ? 0 : 1;
+            } else if (p0) {
+              o -= 1;
+#pragma unroll 1
+              for (int it = 0; it < 4 && code_at_least<T>(o - 1, z, sc, kf); ++it) --o;
+            } else {
+              o += 2;
+#pragma unroll 1
+              for (int it = 0; it < 4 && !code_at_least<T>(o, z, sc, kf); ++it) ++o;
+            }
+            X = bits_of(o);
+          }
+          thr[k - 1] = static_cast<uint32_t>(X) * 0x10001u;
+        }
+        // codes of token pairs as 1024 + code * 4^pos per 16-bit lane: the low byte of a lane is the
+        // slot's contribution to the code byte of that token
+        uint32_t w[8];   // w[tl]: bytes nt = 0..3 for the tokens tl + 8 nt
+#pragma unroll
+        for (int sp = 0; sp < 4; ++sp) {
+          uint32_t h[4];
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) {
+            const int tp = sp + 4 * nt;   // tokens 2 sp + 8 nt and the next one
+            const uint32_t v = Enc<T>::pack(__uint_as_float(x[2 * tp]), __uint_as_float(x[2 * tp + 1]));
+            __half2 acc = __hfma2(as_h2(Ops<T>::ge(v, thr[0])), as_h2(wgt), as_h2(0x64006400u));
+            acc = __hfma2(as_h2(Ops<T>::ge(v, thr[1])), as_h2(wgt), acc);
+            acc = __hfma2(as_h2(Ops<T>::ge(v, thr[2])), as_h2(wgt), acc);
+            h[nt] = as_u32(acc);
+          }
+          const uint32_t p01 = prmt(h[0], h[1], 0x6240u), p23 = prmt(h[2], h[3], 0x6240u);
+          w[2 * sp] = prmt(p01, p23, 0x5410u);
+          w[2 * sp + 1] = prmt(p01, p23, 0x7632u);
+        }
+        // OR over the four slots of a byte (lanes ^ 4, ^ 2), each lane keeping the token sets tl = 2 pos, 2 pos + 1
+        uint32_t w1[4], w2[2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t keep = pb1 ? w[4 + i] : w[i], send = pb1 ? w[i] : w[4 + i];
+          w1[i] = keep | __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const uint32_t keep = pb0 ? w1[2 + i] : w1[i], send = pb0 ? w1[i] : w1[2 + i];
+          w2[i] = keep | __shfl_xor_sync(0xffffffffu, send, 2);
+        }
+        // gather the four bytes of a word from the four lanes that hold them (lanes ^ 8, ^ 1); the
+        // lane ends with the words of token nt = 2 bb0 + bb1 of both of its token sets
+        uint32_t u0, u1;
+        {
+          const uint32_t lo = prmt(w2[0], w2[1], 0x5410u), hi = prmt(w2[0], w2[1], 0x7632u);
+          const uint32_t keep = bb0 ? hi : lo, recv = __shfl_xor_sync(0xffffffffu, bb0 ? lo : hi, 8);
+          const uint32_t a = bb0 ? recv : keep, b = bb0 ? keep : recv;   // a: even byte of the pair, b: odd byte
+          u0 = prmt(a, b, 0x5140u);
+          u1 = prmt(a, b, 0x7362u);
+        }
+        {
+          const uint32_t first = prmt(u0, u1, 0x5410u), second = prmt(u0, u1, 0x7632u);
+          const uint32_t keep = bb1 ? second : first, recv = __shfl_xor_sync(0xffffffffu, bb1 ? first : second, 1);
+          const uint32_t lowpair = bb1 ? recv : keep, highpair = bb1 ? keep : recv;
+          const int nt = (bb0 ? 2 : 0) + (bb1 ? 1 : 0);
+          uint32_t* codes = reinterpret_cast<uint32_t*>(kg + kKG_Codes2);
+          codes[((2 * pos) * 4 + wg) * 4 + nt] = prmt(lowpair, highpair, 0x5410u);
+          codes[((2 * pos + 1) * 4 + wg) * 4 + nt] = prmt(lowpair, highpair, 0x7632u);
+        }
+      }
+    } else {
+      // ---- Eq. 5: lane = spectrum column f, the two accumulators' rows 64 + f hold its 128 tokens
+      const int hq = quad - 2, f = hq * 32 + lane;
+#pragma unroll 1
+      for (int g = 2 * half; g < 2 * half + 2 && g < n_groups; ++g) {
+        uint32_t xa[32], xb[32];
+        tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(g * 32), xa);
+        tmem_ld32(tmem + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(128 + g * 32), xb);
+        float sum = 0.0f;
+        uint32_t bits = 0u;   // bit i = sign bit of the column's coefficient of token i
+#pragma unroll
+        for (int i = 31; i >= 0; --i) {
+          const float X = __uint_as_float(xa[i]) + __uint_as_float(xb[i]);
+          sum += fabsf(X);
+          bits = __funnelshift_l(__float_as_uint(X), bits, 1);
+        }
+        uint8_t* kg = kg_base + g * kKGroupBytes;
+        reinterpret_cast<uint16_t*>(kg + kKG_S1)[f] = f2h_bits(sum * (1.0f / 32.0f));
+        // 32 x 32 bit transpose over the warp: afterwards lane = token, bit l = column 32 hq + l
+#pragma unroll
+        for (int jb = 4; jb >= 0; --jb) {
+          const int js = 1 << jb;
+          const uint32_t m = jb == 4 ? 0x0000ffffu : jb == 3 ? 0x00ff00ffu : jb == 2 ? 0x0f0f0f0fu : jb == 1 ? 0x33333333u : 0x55555555u;
+          const uint32_t y = __shfl_xor_sync(0xffffffffu, bits, js);
+          const bool up = (lane & js) != 0;
+          const uint32_t keep = up ? ~m : m;
+          const uint32_t ysh = up ? (y >> js) : (y << js);
+          bits = (bits & keep) | (ysh & ~keep);
+        }
+        // column e of a 16-column block goes to bit 15 - e of the block's half-word, 1 = coefficient >= 0
+        const uint32_t mine = ~__brev(bits);
+        uint16_t* hw = reinterpret_cast<uint16_t*>(kg + kKG_Bits1);
+        const int hidx = ((lane & 7) * 4 + 2 * hq) * 4 + (lane >> 3);
+        hw[hidx] = static_cast<uint16_t>(mine >> 16);
+        hw[hidx + 4] = static_cast<uint16_t>(mine);
+      }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
+  if (loader) asm volatile("cp.async.wait_group 0;" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 0) {
@@ -430,15 +539,23 @@ static cudaError_t launch_encode_t(const KSrc& src, int64_t T_tokens, const Cach
   const uint32_t* table = nullptr;
   if ((e = dft_fragments(&table, stream))) return e;
   static bool attr_set = false;
-  const size_t smem = k_encode_smem_bytes();
+  static int n_sms[64] = {};
+  constexpr int smem = enc_sm_bytes<T>();
   if (!attr_set) {
-    if ((e = cudaFuncSetAttribute(k_encode_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    if ((e = cudaFuncSetAttribute(k_encode_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    if ((e = cudaFuncSetAttribute(k_encode_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem))) return e;
     attr_set = true;
   }
-  const int64_t blocks = (T_tokens + kEncTokens - 1) / kEncTokens;
-  k_encode_kernel<T><<<dim3(static_cast<unsigned>(blocks), n_slabs), 256, smem, stream>>>(src, T_tokens, cv, layer0,
-                                                                                         slabs_per_layer, chunk, kgroup0);
+  int dev = 0;
+  if ((e = cudaGetDevice(&dev))) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (n_sms[dev] == 0 && (e = cudaDeviceGetAttribute(&n_sms[dev], cudaDevAttrMultiProcessorCount, dev))) return e;
+  const int64_t tiles_per_slab = (T_tokens + kEncTokens - 1) / kEncTokens;
+  const int64_t total = tiles_per_slab * n_slabs;
+  if (total <= 0) return cudaSuccess;
+  if (total > INT32_MAX) return cudaErrorInvalidValue;
+  const int blocks = static_cast<int>(std::min<int64_t>(total, 2 * n_sms[dev]));
+  k_encode_kernel<T><<<blocks, 256, smem, stream>>>(src, T_tokens, cv, layer0, slabs_per_layer, chunk, kgroup0,
+                                                    static_cast<int>(tiles_per_slab), static_cast<int>(total));
   count_launches(1);
   return cudaGetLastError();
 }
