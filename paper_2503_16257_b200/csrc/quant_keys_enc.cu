@@ -81,13 +81,20 @@ template <> struct Ops<__nv_bfloat16> {
 __device__ __forceinline__ int ord_of(uint16_t b) { return (b & 0x8000u) ? -static_cast<int>(b & 0x7fffu) : static_cast<int>(b); }
 __device__ __forceinline__ uint16_t bits_of(int o) { return o >= 0 ? static_cast<uint16_t>(o) : static_cast<uint16_t>(0x8000u | static_cast<uint32_t>(-o)); }
 
-// Eq. 4 for one element, in the defining arithmetic (float32, IEEE division, round half to even):
-// is the code of the element with value order o at least k?  (k = 1..3, so the clamp to [0, 3]
-// does not change the answer.)
+// Eq. 4 for one element: is clamp(rint(RN(RN(x - z) / s)), 0, 3) >= k for the element with value
+// order o (k = 1..3, s > 0)?  Decided without the division.  rint(q) >= k holds from q = 0.5 + 2^-24,
+// 1.5 and 2.5 + 2^-22 on (round half to even), and the rounded quotient reaches that float exactly
+// when the real quotient passes the midpoint below it: d / s > 0.5 + 2^-25, >= 1.5 - 2^-24,
+// > 2.5 + 2^-23 (ties go to the even neighbour 0.5, 1.5, 2.5).  With c = k - 0.5 the sign of
+// d - (c + delta) s is that of u - delta s, u = fma(-c, s, d): c s is exact, u is exact whenever
+// d is within a factor two of c s (the only case where delta matters), delta s is a power of two times s.
 template <typename T>
-__device__ __forceinline__ bool code_at_least(int o, float z, float s, float k) {
+__device__ __forceinline__ bool code_at_least(int o, float z, float s, int k) {
   const float d = __fsub_rn(Ops<T>::to_float(bits_of(o)), z);
-  return rintf(__fdiv_rn(d, s)) >= k;
+  const float u = fmaf(0.5f - static_cast<float>(k), s, d);
+  if (k == 1) return u > 0x1p-25f * s;
+  if (k == 2) return u >= -0x1p-24f * s;
+  return u > 0x1p-23f * s;
 }
 
 }  // namespace
@@ -193,17 +200,19 @@ template <> struct Enc<__nv_bfloat16> {
 
 // Shared memory of one block, from a 1024-byte boundary.  All operands are K-major with the
 // 128-byte swizzle, one 64-channel block of K after the other.
-//   [0, 32768)        the tile as the B operand: [2 K blocks][128 tokens][64 channels]
-//   [32768, 65536)    A, leading part: [2 K blocks][128 rows][64 channels]; row m < 64 selects the
-//                     anomalous channel of slot m, row 64 + f holds column f of the DFT matrix
-//                     spread over the normal channels (zero elsewhere)
-//   [65536, ...)      A, remaining parts of the DFT rows only: per part [2 K blocks][64 rows][64 channels].
-//                     Their products use M = 128 with a descriptor that starts 64 rows early; those
-//                     rows read whatever precedes (finite numbers) and land in accumulator rows
-//                     that nobody reads.
+//   [0, 32768)     the tile as the B operand: [2 K blocks][128 tokens][64 channels]
+//   then           X: the remaining parts of the DFT rows, per part [2 K blocks][64 rows][64 channels]
+//                  A: the leading part, [2 K blocks][128 rows][64 channels].  Arrangement 0: row
+//                  m < 64 selects the anomalous channel of slot m, row 64 + f holds column f of the
+//                  DFT matrix spread over the normal channels (zero elsewhere); arrangement 1 swaps
+//                  the two halves.
+//                  The products of X use M = 128 too: in arrangement 0 the descriptor starts 64
+//                  rows early, in arrangement 1 it runs 64 rows long; the extra rows read
+//                  neighbouring shared memory and land in accumulator rows that nobody reads.
 //   then the channel order [128], the mbarrier, the tensor-memory address, the fault flag
-constexpr int kSmTile = 0, kSmAhi = 32768, kSmAex = 65536;
-template <typename T> __host__ __device__ constexpr int enc_sm_perm() { return kSmAex + 16384 * (Enc<T>::kParts - 1); }
+constexpr int kSmTile = 0, kSmAex = 32768;
+template <typename T> __host__ __device__ constexpr int enc_sm_ahi() { return kSmAex + 16384 * (Enc<T>::kParts - 1); }
+template <typename T> __host__ __device__ constexpr int enc_sm_perm() { return enc_sm_ahi<T>() + 32768; }
 template <typename T> __host__ __device__ constexpr int enc_sm_bytes() { return enc_sm_perm<T>() + kD + 32 + 1024; }
 
 size_t k_encode_smem_bytes(int dtype) { return dtype == VIDKV_F16 ? enc_sm_bytes<__half>() : enc_sm_bytes<__nv_bfloat16>(); }
@@ -219,7 +228,7 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
   extern __shared__ uint8_t esm_raw[];
   uint8_t* esm = esm_raw + ((1024u - (smem_u32(esm_raw) & 1023u)) & 1023u);
   uint8_t* tile = esm + kSmTile;
-  uint8_t* a_hi = esm + kSmAhi;
+  uint8_t* a_hi = esm + enc_sm_ahi<T>();
   uint8_t* a_ex = esm + kSmAex;
   uint8_t* perm = esm + enc_sm_perm<T>();
   uint64_t* mbar = reinterpret_cast<uint64_t*>(perm + kD);
@@ -228,8 +237,13 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int quad = warp & 3, half = warp >> 2;
-  const bool loader = quad >= 2;
-  const int lt = half * 64 + (quad - 2) * 32 + lane;   // 0 .. 127 among the loading threads
+  // Row arrangement of the A operand: 0 puts the anomalous slots in rows 0 .. 63 and the DFT
+  // columns in rows 64 .. 127, 1 the other way round.  The two blocks that share an SM (b and
+  // b + G / 2 when blocks are handed out breadth first) take different arrangements so that the
+  // heavier anomalous warps of one block sit on the schedulers of the lighter warps of the other.
+  const int arr = (2 * blockIdx.x >= gridDim.x) ? 1 : 0;
+  const bool loader = (quad >= 2) != (arr == 1);        // the spectrum warps also move the tiles
+  const int lt = half * 64 + (quad & 1) * 32 + lane;    // 0 .. 127 among the loading threads
 
   if (tid == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(mbar)) : "memory");
@@ -293,15 +307,15 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
       cur_slab = slab;
       if (tid < kD) perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
       constexpr int kAVec = (32768 + 16384 * (Enc<T>::kParts - 1)) / 16;
-      for (int i = tid; i < kAVec; i += 256) reinterpret_cast<uint4*>(a_hi)[i] = make_uint4(0u, 0u, 0u, 0u);
+      for (int i = tid; i < kAVec; i += 256) reinterpret_cast<uint4*>(a_ex)[i] = make_uint4(0u, 0u, 0u, 0u);
       __syncthreads();
       if (tid < kNA) {
         const int c = perm[tid];
-        *reinterpret_cast<uint16_t*>(a_hi + (c >> 6) * 16384 + sw128_offset(tid, c & 63)) = Enc<T>::kOne;
+        *reinterpret_cast<uint16_t*>(a_hi + (c >> 6) * 16384 + sw128_offset(64 * arr + tid, c & 63)) = Enc<T>::kOne;
       }
       for (int i = tid; i < 64 * 64; i += 256) {
         const int f = i >> 6, c = perm[kNA + (i & 63)];
-        *reinterpret_cast<uint16_t*>(a_hi + (c >> 6) * 16384 + sw128_offset(64 + f, c & 63)) = g_dft_w[Enc<T>::kTab * 4096 + i];
+        *reinterpret_cast<uint16_t*>(a_hi + (c >> 6) * 16384 + sw128_offset(64 - 64 * arr + f, c & 63)) = g_dft_w[Enc<T>::kTab * 4096 + i];
 #pragma unroll
         for (int part = 1; part < Enc<T>::kParts; ++part)
           *reinterpret_cast<uint16_t*>(a_ex + (part - 1) * 16384 + (c >> 6) * 8192 + sw128_offset(f, c & 63)) =
@@ -332,8 +346,8 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
       for (int part = 1; part < Enc<T>::kParts; ++part) {
 #pragma unroll
         for (int kb = 0; kb < 2; ++kb) {
-          // rows 64 .. 127 of the operand are the part's data: start 64 rows (8192 bytes) early
-          const uint64_t da = umma_desc_sw128(smem_u32(a_ex + (part - 1) * 16384 + kb * 8192 - 8192));
+          // the part's 64 rows are rows 64 .. 127 of arrangement 0 (start 8192 bytes early), rows 0 .. 63 of arrangement 1
+          const uint64_t da = umma_desc_sw128(smem_u32(a_ex + (part - 1) * 16384 + kb * 8192 - (arr ? 0 : 8192)));
           const uint64_t db = umma_desc_sw128(smem_u32(tile + kb * 16384));
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
@@ -365,7 +379,7 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
 
     if (!loader) {
       // ---- Eq. 4: lane = anomalous slot j, the accumulator row holds its 128 tokens (exact values)
-      const int j = quad * 32 + lane, wg = j >> 4;
+      const int j = (quad & 1) * 32 + lane, wg = j >> 4;
       const int pos = (lane >> 1) & 3;                            // field of the slot inside its code byte
       const bool pb0 = (lane & 2) != 0, pb1 = (lane & 4) != 0;    // bits of pos
       const bool bb0 = (lane & 8) != 0, bb1 = (lane & 1) != 0;    // bits of the slot's byte index 2 (e % 2) + e / 8
@@ -390,19 +404,18 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
           if (sc != 0.0f) {
             int o = ord_of(Ops<T>::from_float_rn(fmaf(static_cast<float>(k) - 0.5f, sc, z)));
             // the threshold is almost always the candidate or its upper neighbour: two evaluations
-            const float kf = static_cast<float>(k);
-            const bool p0 = code_at_least<T>(o, z, sc, kf);
-            const bool p1 = code_at_least<T>(p0 ? o - 1 : o + 1, z, sc, kf);
+            const bool p0 = code_at_least<T>(o, z, sc, k);
+            const bool p1 = code_at_least<T>(p0 ? o - 1 : o + 1, z, sc, k);
             if (p0 != p1) {
               o += p0 ? 0 : 1;
             } else if (p0) {
               o -= 1;
 #pragma unroll 1
-              for (int it = 0; it < 4 && code_at_least<T>(o - 1, z, sc, kf); ++it) --o;
+              for (int it = 0; it < 4 && code_at_least<T>(o - 1, z, sc, k); ++it) --o;
             } else {
               o += 2;
 #pragma unroll 1
-              for (int it = 0; it < 4 && !code_at_least<T>(o, z, sc, kf); ++it) ++o;
+              for (int it = 0; it < 4 && !code_at_least<T>(o, z, sc, k); ++it) ++o;
             }
             X = bits_of(o);
           }
@@ -461,7 +474,7 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
       }
     } else {
       // ---- Eq. 5: lane = spectrum column f, the two accumulators' rows 64 + f hold its 128 tokens
-      const int hq = quad - 2, f = hq * 32 + lane;
+      const int hq = quad & 1, f = hq * 32 + lane;
 #pragma unroll 1
       for (int g = 2 * half; g < 2 * half + 2 && g < n_groups; ++g) {
         uint32_t xa[32], xb[32];
