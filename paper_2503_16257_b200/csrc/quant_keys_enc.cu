@@ -1,18 +1,22 @@
-// Key encode pass of Algorithm 3 (MixQuant) for one tile of 128 tokens x 128 channels:
-//   normal channels   (Eq. 5) orthonormal 64-point DFT over the channel axis as one 128 x 64 x 64
-//                     matrix product on the fifth-generation tensor cores (tcgen05.mma, operands
-//                     in shared memory in the 128-byte-swizzled K-major layout, accumulator in
-//                     tensor memory).  A = the tile's values, binary16, exact; B = the DFT matrix
-//                     split into a binary16 leading part and a binary16 remainder, so that
-//                     products carry 22 bits; float32 accumulation.  Then the sign bit and the
-//                     per-group mean |.| of every spectrum column, one thread per token;
-//   anomalous channels (Eq. 4) min / max per (32-token group, channel), s = (max - min) / 3,
-//                     z = min rounded to binary16, code = clamp(rint((x - z) / s), 0, 3).
-//                     The division is not done per element: code >= k is a monotone predicate
-//                     of x, so per (group, channel) the three smallest element values X_k with
-//                     code(X_k) >= k are found once with the defining float32 arithmetic, and
-//                     the elements are compared against them two at a time.
-// grid = (tiles of 128 tokens, slabs); block = 256 threads = 8 warps.
+// Key encode pass of Algorithm 3 (MixQuant), one tile of 128 tokens x 128 channels at a time.
+// The tile is the B operand of one product on the fifth-generation tensor cores (tcgen05.mma,
+// operands in shared memory in the 128-byte-swizzled K-major layout, accumulators in tensor
+// memory); the A operand has one row per output of the channel sort:
+//   anomalous channels (Eq. 4) 64 selector rows (a single 1.0) copy the 64 anomalous channels
+//                     exactly, so that accumulator row = slot, columns = tokens.  Per (slot,
+//                     32-token group): min / max, s = (max - min) / 3, z = min rounded to
+//                     binary16, code = clamp(rint((x - z) / s), 0, 3).  No division: code >= k
+//                     is a monotone predicate of x, so the three smallest element values X_k
+//                     with code(X_k) >= k are found once, with an exact test (code_at_least),
+//                     and the elements are compared against them two at a time; the 2-bit
+//                     fields are assembled into the cache's code words across lanes.
+//   normal channels   (Eq. 5) 64 rows hold the columns of the orthonormal 64-point DFT over the
+//                     channel axis, spread over the slab's normal channels and split into
+//                     parts (binary16: 2, bfloat16: 3) so that products carry 22 - 24 bits;
+//                     float32 accumulation.  Accumulator row = spectrum column: the sign bits
+//                     and the per-group mean |.| are per-thread work, a warp-wide bit
+//                     transpose gives the cache's (token, 16 columns) half-words.
+// Persistent grid of two blocks per SM; block = 256 threads = 8 warps.
 #include <math.h>
 
 #include <algorithm>
