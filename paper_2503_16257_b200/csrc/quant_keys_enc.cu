@@ -555,17 +555,15 @@ static cudaError_t launch_encode_t(const KSrc& src, int64_t T_tokens, const Cach
   cudaError_t e;
   const uint32_t* table = nullptr;
   if ((e = dft_fragments(&table, stream))) return e;
-  static bool attr_set = false;
-  static int n_sms[64] = {};
+  static int n_sms[64] = {};   // per device; 0 = the kernel's attributes are not set there yet
   constexpr int smem = enc_sm_bytes<T>();
-  if (!attr_set) {
-    if ((e = cudaFuncSetAttribute(k_encode_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem))) return e;
-    attr_set = true;
-  }
   int dev = 0;
   if ((e = cudaGetDevice(&dev))) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (n_sms[dev] == 0 && (e = cudaDeviceGetAttribute(&n_sms[dev], cudaDevAttrMultiProcessorCount, dev))) return e;
+  if (n_sms[dev] == 0) {
+    if ((e = cudaFuncSetAttribute(k_encode_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem))) return e;
+    if ((e = cudaDeviceGetAttribute(&n_sms[dev], cudaDevAttrMultiProcessorCount, dev))) return e;
+  }
   const int64_t tiles_per_slab = (T_tokens + kEncTokens - 1) / kEncTokens;
   const int64_t total = tiles_per_slab * n_slabs;
   if (total <= 0) return cudaSuccess;
