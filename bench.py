@@ -123,8 +123,9 @@ class ClockSampler:
 
 
 def oracle_sample(wl, p, device_tensors=None):
-    """Time the CPU oracle, as it stands, on a bounded sample of the workload: one
-    (layer 0, batch 0) slab set = 4 KV heads, full T, K+V quantize and 2 decode steps."""
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload (about ten seconds of
+    host time on the batched shape): layer 0, up to 8 batch elements, all KV heads, full T, K+V
+    quantize once and 8 decode steps."""
     import numpy as np
     from oracle import vidkv_oracle as O
     from workloads import make_layer_kv, make_saliency, make_step_inputs
@@ -134,40 +135,45 @@ def oracle_sample(wl, p, device_tensors=None):
     except Exception:
         threads = os.cpu_count() or 1
     T = min(wl.T, 12544)
+    nb = min(wl.batch, 8)
     if device_tensors is not None:
         K, V = device_tensors
-        K, V = K[:1, :, :T].float().cpu(), V[:1, :, :T].float().cpu()
+        K, V = K[:nb, :, :T].float().cpu(), V[:nb, :, :T].float().cpu()
     else:
-        K, V = make_layer_kv(wl, 0, "cpu", T=T, B=1)
+        K, V = make_layer_kv(wl, 0, "cpu", T=T, B=nb)
     l_v = min(wl.l_v, T - T % 32)
     E = None
     n_prot = 0
     if p > 0:
-        sal = make_saliency(wl, "cpu", l_v=l_v, B=1)
-        E = O.select_tokens(sal[0].numpy(), p, 0, T)
-        n_prot = int(E.sum())
+        sal = make_saliency(wl, "cpu", l_v=l_v, B=nb)
+        E = [O.select_tokens(sal[b].numpy(), p, 0, T) for b in range(nb)]
+        n_prot = int(E[0].sum())
     H = K.shape[1]
     t0 = time.perf_counter()
     slabs = []
-    for h in range(H):
-        sc = O.SlabCache()
-        sc.prefill(K[0, h].float().numpy(), V[0, h].float().numpy(), E)
-        slabs.append(sc)
+    for b in range(nb):
+        for h in range(H):
+            sc = O.SlabCache()
+            sc.prefill(K[b, h].float().numpy(), V[b, h].float().numpy(), E[b] if E is not None else None)
+            slabs.append(sc)
     t_quant = time.perf_counter() - t0
-    n_steps = 2
+    n_steps = 8
+    rep = 7   # query heads per KV head in every workload
     t0 = time.perf_counter()
     for s in range(n_steps):
-        q, k, v = make_step_inputs(wl, 0, s, "cpu", T=T, B=1)
-        for h in range(H):
-            slabs[h].decode_step(q[0, 7 * h:7 * h + 7].float().numpy(), k[0, h].float().numpy(), v[0, h].float().numpy())
+        q, k, v = make_step_inputs(wl, 0, s, "cpu", T=T, B=nb)
+        for b in range(nb):
+            for h in range(H):
+                slabs[b * H + h].decode_step(q[b, rep * h:rep * h + rep].float().numpy(), k[b, h].float().numpy(),
+                                             v[b, h].float().numpy())
     t_dec = (time.perf_counter() - t0) / n_steps
-    dec_bytes = algorithmic_decode_bytes(1, 1, H, 7 * H, T - T % 32, 0, T % 32 + 1, n_prot)
+    dec_bytes = algorithmic_decode_bytes(nb, 1, H, rep * H, T - T % 32, 0, T % 32 + 1, n_prot)
     return {
         "decode_gbs": dec_bytes / t_dec / 1e9,
-        "quantize_tokens_per_s": T / t_quant,
+        "quantize_tokens_per_s": nb * T / t_quant,
         "seconds": t_quant + t_dec * n_steps,
         "cores": threads,
-        "sample": f"layer 0, batch element 0, {H} KV heads, T={T}: K+V quantize once, {n_steps} decode steps "
+        "sample": f"layer 0, batch elements 0..{nb - 1}, {H} KV heads, T={T}: K+V quantize once, {n_steps} decode steps "
                   f"(first step includes the oracle's one-time dequantization)",
     }
 
