@@ -12,6 +12,7 @@ What follows the paper, step by step, in its notation:
 * ``fft_1bit``          Eq. 5   sign code + mean-|.| scale in the frequency domain
 * ``mixquant``          Algorithm 3 MixQuant (k = 0.5 : 64 two-bit + 64 one-bit)
 * ``quant_1p58``        Eq. 6 / Algorithm 2 "1.58Quant" (ternary, gamma = 0.7)
+* ``stp_saliency``      Eq. 7   cross-modal scores I = X_v X_t^T, summed over the text tokens
 * ``select_tokens``     Eq. 7 / Sec. 3.3(2): top n = floor(p * l_v) visual tokens
 * ``stpquant``          Algorithm 2 STPQuant
 * ``SlabCache``         Algorithm 1 Prefill / Decoding for one (layer, batch,
@@ -276,6 +277,16 @@ def dequant_1p58_groups(trits, s):
 def n_protected(p, l_v: int) -> int:
     """n = floor(p * l_v) with p held in float32 (the config stores a float)."""
     return int(math.floor(float(np.float32(p)) * l_v))
+
+
+def stp_saliency(x_v: np.ndarray, x_t: np.ndarray) -> np.ndarray:
+    """Eq. 7: the cross-modal score matrix I[i, j] = X_v(i) . X_t(j) between the hidden
+    states of the l_v visual tokens (x_v [l_v, d]) and of the l_t text tokens (x_t [l_t, d]).
+    The paper ranks visual tokens by these scores without saying how the text axis is
+    reduced; the reading taken here is the sum over the text tokens (the mean up to a
+    constant, which does not change a ranking).  Returns the l_v row sums, float64."""
+    I = x_v.astype(np.float64) @ x_t.astype(np.float64).T
+    return I.sum(axis=1)
 
 
 def select_tokens(saliency: np.ndarray, p, vis_begin: int, T: int) -> np.ndarray:

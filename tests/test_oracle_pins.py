@@ -325,6 +325,43 @@ def test_select_tokens_matches_argsort_and_counts():
     assert np.nonzero(E)[0].tolist() == [4, 5]
 
 
+def test_stp_saliency_brute_force_and_closed_forms():
+    r = rng(41)
+    x_v = fp16_values((7, 12), 42)
+    x_t = fp16_values((5, 12), 43)
+    got = O.stp_saliency(x_v, x_t)
+    # Eq. 7 element by element, then the row sums
+    want = np.zeros(7)
+    for i in range(7):
+        for j in range(5):
+            want[i] += sum(float(x_v[i, c]) * float(x_t[j, c]) for c in range(12))
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    # text tokens that are unit vectors pick coordinates of the visual tokens
+    e = np.zeros((3, 12), np.float32)
+    e[0, 2] = e[1, 5] = e[2, 5] = 1.0
+    np.testing.assert_allclose(O.stp_saliency(x_v, e), x_v[:, 2].astype(np.float64) + 2.0 * x_v[:, 5], rtol=0, atol=1e-12)
+    # the order of the text tokens does not matter; the score is linear in the visual token
+    np.testing.assert_allclose(O.stp_saliency(x_v, x_t[r.permutation(5)]), got, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(O.stp_saliency(2.0 * x_v, x_t), 2.0 * got, rtol=1e-12, atol=1e-12)
+    # a single text token: one matrix-vector product (library routine)
+    np.testing.assert_allclose(O.stp_saliency(x_v, x_t[:1]), np.dot(x_v.astype(np.float64), x_t[0].astype(np.float64)),
+                               rtol=1e-12, atol=1e-12)
+
+
+def test_stp_saliency_ranks_planted_tokens_first():
+    # visual tokens aligned with the text direction must come out on top of the ranking
+    r = rng(44)
+    d, l_v, l_t = 64, 200, 9
+    direction = r.standard_normal(d)
+    direction /= np.linalg.norm(direction)
+    x_t = (direction[None, :] * r.uniform(1.0, 2.0, (l_t, 1)) + 0.01 * r.standard_normal((l_t, d))).astype(np.float32)
+    x_v = (0.1 * r.standard_normal((l_v, d))).astype(np.float32)
+    planted = np.sort(r.choice(l_v, 40, replace=False))
+    x_v[planted] += 3.0 * direction[None, :].astype(np.float32)
+    E = O.select_tokens(O.stp_saliency(x_v, x_t), 0.2, 0, l_v)
+    assert np.array_equal(np.nonzero(E)[0], planted)
+
+
 def test_stpquant_streams():
     v = fp16_values((96, 16), 20)
     E = np.zeros(96, dtype=bool)
