@@ -163,6 +163,18 @@ vidkv_status_t vidkv_cache_destroy(vidkv_cache_t* handle);
 /* Forget all tokens (host state only; the next quantize calls overwrite the buffers). */
 vidkv_status_t vidkv_cache_reset(vidkv_cache_t* handle, void* stream);
 
+/* Sec. 3.3(2) / Eq. 7: the cross-modal scores I = X_v X_t^T from hidden states, summed over
+ * the text tokens (the paper does not say how the text axis is reduced; a sum and a mean
+ * rank alike):  saliency[b, i] = sum_j x_v[b, i, :] . x_t[b, j, :]  in float32.
+ *   x_v      [B, l_v, d]  device, dtype VIDKV_F16 or VIDKV_BF16, contiguous
+ *   x_t      [B, l_t, d]  device, same dtype, contiguous (l_t == 0: all scores are 0)
+ *   text_sum [B, d]       device float32 scratch owned by the caller, overwritten
+ *   saliency [B, l_v]     device float32, written; feed it to vidkv_select_tokens
+ * d must be a multiple of 8 and at most 16384, B at most 65535 (else UNSUPPORTED); all
+ * pointers 16-byte aligned.  Needs no cache handle.  Two launches on `stream`. */
+vidkv_status_t vidkv_saliency_scores(int32_t dtype, const void* x_v, const void* x_t, int64_t B, int64_t l_v,
+                                     int64_t l_t, int64_t d, float* text_sum, float* saliency, void* stream);
+
 /* Sec. 3.3(2) / Eq. 7: choose the protected tokens.  saliency [B, l_v] float32 scores
  * the visual tokens vis_begin .. vis_begin + l_v - 1 of a prompt of T tokens; the top
  * n = floor(p_ratio * l_v) (ties: lower token index) are protected in every layer and

@@ -71,6 +71,8 @@ _SIGNATURES = {
                                      C.c_void_p, C.POINTER(C.c_void_p)]),
     "vidkv_cache_destroy": (C.c_int32, [C.c_void_p]),
     "vidkv_cache_reset": (C.c_int32, [C.c_void_p, C.c_void_p]),
+    "vidkv_saliency_scores": (C.c_int32, [C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
+                                          C.c_void_p, C.c_void_p, C.c_void_p]),
     "vidkv_select_tokens": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p]),
     "vidkv_set_token_mask": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
     "vidkv_quantize_keys": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
@@ -135,6 +137,24 @@ def vidkv_attend_noalloc(cfg: VidKVConfig, cache, n_prefill_quantized: int, n_fl
     _check("vidkv_attend_noalloc", load_library().vidkv_attend_noalloc(
         C.byref(c), C.c_void_p(cache.data_ptr()), n_prefill_quantized, n_flushed_chunks, n_residual, n_protected,
         layer_begin, n_layers, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()), softmax_scale, _stream_ptr()))
+
+
+def vidkv_saliency_scores(x_v, x_t, text_sum=None, saliency=None):
+    """Eq. 7 scores of the visual tokens: x_v [B, l_v, d], x_t [B, l_t, d] (float16 or bfloat16 device
+    tensors) -> saliency [B, l_v] float32.  `text_sum` [B, d] float32 is scratch; both are
+    allocated here when not given."""
+    import torch
+    B, l_v, d = x_v.shape
+    l_t = x_t.shape[1]
+    dtype = VIDKV_F16 if x_v.dtype == torch.float16 else VIDKV_BF16
+    if text_sum is None:
+        text_sum = torch.empty((B, d), dtype=torch.float32, device=x_v.device)
+    if saliency is None:
+        saliency = torch.empty((B, l_v), dtype=torch.float32, device=x_v.device)
+    _check("vidkv_saliency_scores", load_library().vidkv_saliency_scores(
+        dtype, C.c_void_p(x_v.data_ptr()), C.c_void_p(x_t.data_ptr()), B, l_v, l_t, d,
+        C.c_void_p(text_sum.data_ptr()), C.c_void_p(saliency.data_ptr()), _stream_ptr()))
+    return saliency
 
 
 def vidkv_cache_bytes(cfg: VidKVConfig):

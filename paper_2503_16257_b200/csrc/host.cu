@@ -257,6 +257,19 @@ vidkv_status_t vidkv_cache_reset(vidkv_cache_t* h, void* stream) {
   return VIDKV_OK;
 }
 
+vidkv_status_t vidkv_saliency_scores(int32_t dtype, const void* x_v, const void* x_t, int64_t B, int64_t l_v, int64_t l_t,
+                                     int64_t d, float* text_sum, float* saliency, void* stream) {
+  if (dtype != VIDKV_F16 && dtype != VIDKV_BF16) return VIDKV_ERR_INVALID_ARG;
+  if (B < 0 || l_v < 0 || l_t < 0 || d < 1) return VIDKV_ERR_INVALID_ARG;
+  if (B == 0 || l_v == 0) return VIDKV_OK;
+  if (!x_v || !text_sum || !saliency || (l_t > 0 && !x_t)) return VIDKV_ERR_INVALID_ARG;
+  if (d % 8 != 0 || d > 16384 || B > 65535) return VIDKV_ERR_UNSUPPORTED;
+  if (!aligned16(x_v) || !aligned16(text_sum) || !aligned16(saliency) || (l_t > 0 && !aligned16(x_t))) return VIDKV_ERR_ALIGNMENT;
+  if (launch_saliency(dtype, x_v, x_t, B, l_v, l_t, d, text_sum, saliency, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  return VIDKV_OK;
+}
+
 vidkv_status_t vidkv_select_tokens(vidkv_cache_t* h, const float* saliency, int64_t vis_begin, int64_t l_v, int64_t T,
                                    void* stream) {
   if (!h || T < 0) return VIDKV_ERR_INVALID_ARG;

@@ -102,6 +102,10 @@ struct DecodeArgs {
   cudaEvent_t ev_begin, ev_end;   // optional: recorded around the split-KV kernel (profiling)
 };
 
+// Eq. 7 scores from hidden states: text_sum [B, d] (scratch) and saliency [B, l_v], both float32.
+cudaError_t launch_saliency(int dtype, const void* x_v, const void* x_t, int64_t B, int64_t l_v, int64_t l_t, int64_t d,
+                            float* text_sum, float* saliency, cudaStream_t stream);
+
 // Number of kernels launched by this library since it was loaded (host counter).
 extern unsigned long long g_launch_count;
 inline void count_launches(int n) { g_launch_count += static_cast<unsigned long long>(n); }

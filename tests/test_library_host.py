@@ -109,6 +109,18 @@ def test_null_arguments_are_rejected_without_a_device(lib):
     assert lib.vidkv_decode_attention(None, 0, 1, None, None, None, None, 0.0, None) == -1
 
 
+def test_saliency_scores_argument_checks_without_a_device(lib):
+    f = lib.vidkv_saliency_scores
+    a = ctypes.c_void_p(0x1000)
+    assert f(7, a, a, 1, 4, 2, 64, a, a, None) == -1                      # unknown dtype
+    assert f(P.VIDKV_F16, a, a, -1, 4, 2, 64, a, a, None) == -1           # negative size
+    assert f(P.VIDKV_F16, None, a, 1, 4, 2, 64, a, a, None) == -1         # null input
+    assert f(P.VIDKV_F16, a, a, 0, 4, 2, 64, a, a, None) == 0             # nothing to do
+    assert f(P.VIDKV_F16, a, a, 1, 4, 2, 12, a, a, None) == -2            # d not a multiple of 8
+    assert f(P.VIDKV_F16, a, a, 1, 4, 2, 32768, a, a, None) == -2         # d beyond the supported width
+    assert f(P.VIDKV_F16, ctypes.c_void_p(0x1004), a, 1, 4, 2, 64, a, a, None) == -3   # misaligned
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     import paper_2503_16257_b200.api as api
     monkeypatch.setattr(api, "_LIB", None)

@@ -23,7 +23,8 @@ H_Q = 28
 D = 128
 TOKENS_PER_FRAME = 196
 
-_T_K, _T_V, _T_CH, _T_MU, _T_SIG, _T_SAL, _T_STEP = 0, 1, 2, 3, 4, 5, 6
+_T_K, _T_V, _T_CH, _T_MU, _T_SIG, _T_SAL, _T_STEP, _T_HV, _T_HT = 0, 1, 2, 3, 4, 5, 6, 7, 8
+D_MODEL = 3584   # hidden size of the 7B video LLMs the workloads are shaped after
 
 
 @dataclass(frozen=True)
@@ -184,3 +185,19 @@ def make_saliency(cfg: WorkloadConfig, device="cpu", l_v: int | None = None,
     B = cfg.batch if B is None else B
     return torch.randn((B, l_v), generator=_gen(cfg, 0, _T_SAL, device), device=device,
                        dtype=torch.float32)
+
+
+def make_hidden_states(cfg: WorkloadConfig, device="cpu", l_v: int | None = None, l_t: int | None = None,
+                       B: int | None = None, d_model: int = D_MODEL):
+    """Hidden states of the visual tokens ``[B, l_v, d_model]`` and of the text tokens
+    ``[B, l_t, d_model]`` in the config's storage dtype, ~ N(0, 1); the text tokens share a
+    common direction (scale 0.5) so that their sum does not average out."""
+    l_v = cfg.l_v if l_v is None else l_v
+    l_t = cfg.text_tokens if l_t is None else l_t
+    B = cfg.batch if B is None else B
+    x_v = torch.randn((B, l_v, d_model), generator=_gen(cfg, 0, _T_HV, device), device=device, dtype=torch.float32)
+    g = _gen(cfg, 0, _T_HT, device)
+    common = torch.randn((B, 1, d_model), generator=g, device=device, dtype=torch.float32)
+    x_t = torch.randn((B, l_t, d_model), generator=g, device=device, dtype=torch.float32) + 0.5 * common
+    dt = cfg.torch_dtype
+    return x_v.to(dt).contiguous(), x_t.to(dt).contiguous()
