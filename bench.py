@@ -223,6 +223,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=None, help="override the decode steps per bench step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-token-scores", action="store_true", help="skip the stand-alone timing of vidkv_saliency_scores")
     args = ap.parse_args()
 
     from dataclasses import replace
@@ -385,10 +386,42 @@ def main():
         line["cpu_baseline"] = {"value": res["decode_gbs"], "unit": "GB/s", "cores": res["cores"], "kind": "oracle",
                                 "sample": res["sample"], "quantize_tokens_per_s": res["quantize_tokens_per_s"],
                                 "seconds": res["seconds"]}
+    if rank == 0 and not args.no_token_scores:
+        line["token_scores"] = run_token_scores(P, torch, wl, dev, peak)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_token_scores(P, torch, wl, dev, peak):
+    """Upstream of the hot path (not part of a step): the Eq. 7 scores of the visual tokens from hidden
+    states of the workload's shape, timed alone with CUDA events; two input copies alternate so that
+    no call finds its input in L2.  Algorithmic bytes = the two inputs read once + the scores written."""
+    from workloads import make_hidden_states
+    l_t = wl.text_tokens if wl.text_tokens > 0 else 64    # a 64-token text query where the workload has none
+    x_v, x_t = make_hidden_states(wl, dev, l_t=l_t)
+    xs = [x_v, x_v.clone()] if x_v.numel() * 2 < 400e6 else [x_v]
+    B, l_v, d = x_v.shape
+    text_sum = torch.empty((B, d), dtype=torch.float32, device=dev)
+    sal = torch.empty((B, l_v), dtype=torch.float32, device=dev)
+    for i in range(8):
+        P.vidkv_saliency_scores(xs[i % len(xs)], x_t, text_sum, sal)
+    times = []
+    for i in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        P.vidkv_saliency_scores(xs[i % len(xs)], x_t, text_sum, sal)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = sum(times) / len(times)
+    nbytes = x_v.numel() * 2 + x_t.numel() * 2 + sal.numel() * 4
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"GBps": gbs, "frac_of_measured_hbm": gbs / peak, "pct_of_8TBps": 100.0 * gbs / NOMINAL_HBM_GBS, "ms_per_call": ms,
+            "bytes_per_call": nbytes, "shape": {"B": B, "l_v": l_v, "l_t": int(x_t.shape[1]), "d_model": d},
+            "launches_per_call": 2, "ms_each": [round(t, 4) for t in times]}
 
 
 def run_e2e(P, torch, wl, cfg, cache, Ks, Vs, qs, ks, vs, sal, out, n_prot, dev, world):

@@ -30,7 +30,8 @@ __global__ void __launch_bounds__(kSalThreads) text_sum_kernel(const T* __restri
 }
 
 // saliency[b, i] = x_v[b, i, :] . text_sum[b, :].  grid = (blocks of 64 rows, B); a warp owns 8
-// consecutive rows and walks each in 16-byte pieces per lane, the vector sits in shared memory.
+// consecutive rows and walks four of them at a time in 16-byte pieces per lane (four independent
+// loads in flight per lane), the vector sits in shared memory.
 template <typename T>
 __global__ void __launch_bounds__(kSalThreads) saliency_kernel(const T* __restrict__ x_v, int64_t l_v, int64_t d,
                                                                const float* __restrict__ text_sum,
@@ -44,35 +45,34 @@ __global__ void __launch_bounds__(kSalThreads) saliency_kernel(const T* __restri
   const int64_t row0 = static_cast<int64_t>(blockIdx.x) * kSalRowsPerBlock + warp * kSalRowsPerWarp;
   const int64_t pieces = d / 8;                 // 16-byte pieces per row
 #pragma unroll 1
-  for (int r = 0; r < kSalRowsPerWarp; r += 2) {
-    // two rows at a time: their loads are independent
-    const int64_t i0 = row0 + r, i1 = i0 + 1;
+  for (int r = 0; r < kSalRowsPerWarp; r += 4) {
+    const int64_t i0 = row0 + r;
     if (i0 >= l_v) break;
-    const bool two = i1 < l_v;
-    const uint4* p0 = reinterpret_cast<const uint4*>(x_v + (b * l_v + i0) * d);
-    const uint4* p1 = reinterpret_cast<const uint4*>(x_v + (b * l_v + (two ? i1 : i0)) * d);
-    float acc0 = 0.0f, acc1 = 0.0f;
-#pragma unroll 2
+    const uint4* p[4];
+    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) p[q] = reinterpret_cast<const uint4*>(x_v + (b * l_v + min(i0 + q, l_v - 1)) * d);
+#pragma unroll 1
     for (int64_t k = lane; k < pieces; k += 32) {
-      const uint4 u0 = __ldcs(p0 + k);
-      const uint4 u1 = __ldcs(p1 + k);
+      uint4 u[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) u[q] = __ldcs(p[q] + k);
       const float4 ta = *reinterpret_cast<const float4*>(tsum + 8 * k);
       const float4 tb = *reinterpret_cast<const float4*>(tsum + 8 * k + 4);
-      const float2 a0 = Elem<T>::to_float2(u0.x), a1 = Elem<T>::to_float2(u0.y), a2 = Elem<T>::to_float2(u0.z), a3 = Elem<T>::to_float2(u0.w);
-      const float2 b0 = Elem<T>::to_float2(u1.x), b1 = Elem<T>::to_float2(u1.y), b2 = Elem<T>::to_float2(u1.z), b3 = Elem<T>::to_float2(u1.w);
-      acc0 = fmaf(a0.x, ta.x, acc0); acc0 = fmaf(a0.y, ta.y, acc0); acc0 = fmaf(a1.x, ta.z, acc0); acc0 = fmaf(a1.y, ta.w, acc0);
-      acc0 = fmaf(a2.x, tb.x, acc0); acc0 = fmaf(a2.y, tb.y, acc0); acc0 = fmaf(a3.x, tb.z, acc0); acc0 = fmaf(a3.y, tb.w, acc0);
-      acc1 = fmaf(b0.x, ta.x, acc1); acc1 = fmaf(b0.y, ta.y, acc1); acc1 = fmaf(b1.x, ta.z, acc1); acc1 = fmaf(b1.y, ta.w, acc1);
-      acc1 = fmaf(b2.x, tb.x, acc1); acc1 = fmaf(b2.y, tb.y, acc1); acc1 = fmaf(b3.x, tb.z, acc1); acc1 = fmaf(b3.y, tb.w, acc1);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 a0 = Elem<T>::to_float2(u[q].x), a1 = Elem<T>::to_float2(u[q].y), a2 = Elem<T>::to_float2(u[q].z), a3 = Elem<T>::to_float2(u[q].w);
+        float a = acc[q];
+        a = fmaf(a0.x, ta.x, a); a = fmaf(a0.y, ta.y, a); a = fmaf(a1.x, ta.z, a); a = fmaf(a1.y, ta.w, a);
+        a = fmaf(a2.x, tb.x, a); a = fmaf(a2.y, tb.y, a); a = fmaf(a3.x, tb.z, a); a = fmaf(a3.y, tb.w, a);
+        acc[q] = a;
+      }
     }
 #pragma unroll
-    for (int m = 16; m >= 1; m >>= 1) {
-      acc0 += __shfl_xor_sync(0xffffffffu, acc0, m);
-      acc1 += __shfl_xor_sync(0xffffffffu, acc1, m);
-    }
-    if (lane == 0) {
-      saliency[b * l_v + i0] = acc0;
-      if (two) saliency[b * l_v + i1] = acc1;
+    for (int q = 0; q < 4; ++q) {
+#pragma unroll
+      for (int m = 16; m >= 1; m >>= 1) acc[q] += __shfl_xor_sync(0xffffffffu, acc[q], m);
+      if (lane == 0 && i0 + q < l_v) saliency[b * l_v + i0 + q] = acc[q];
     }
   }
 }

@@ -79,8 +79,8 @@ def test_full_size_scores_on_sampled_rows():
     """The batched workload's shape as bench.py launches it (16 sequences, every visual token, hidden
     size 3584): sampled rows against the oracle, which handles a row at a time."""
     wl = CONFIGS["batched"]
-    x_v, x_t = make_hidden_states(wl, "cuda")
-    assert x_v.shape == (wl.batch, wl.l_v, D_MODEL)
+    x_v, x_t = make_hidden_states(wl, "cuda", l_t=wl.text_tokens if wl.text_tokens > 0 else 64)
+    assert x_v.shape == (wl.batch, wl.l_v, D_MODEL) and x_t.shape[1] > 0
     got = P.vidkv_saliency_scores(x_v, x_t).cpu().numpy()
     r = np.random.default_rng(5)
     for b in (0, wl.batch // 2, wl.batch - 1):
