@@ -26,7 +26,7 @@
  *     before anything is launched.  One exception: the first key quantization or
  *     decode call on each device fills a 16 KB table of DFT coefficients inside the
  *     library and synchronises the stream once.
- *   - Fixed by this build: D = 128, G = 32, R = 128, k = 0.5 (64 two-bit and 64
+ *   - Fixed in this library: D = 128, G = 32, R = 128, k = 0.5 (64 two-bit and 64
  *     one-bit channels), H_q a multiple of H_kv with H_q / H_kv <= 8.  Other
  *     shapes return VIDKV_ERR_UNSUPPORTED.
  *   - Element types: VIDKV_F16 / VIDKV_BF16 for K, V, q, k_new, v_new (in_dtype);
@@ -87,7 +87,7 @@ typedef int32_t vidkv_status_t;
 enum {
   VIDKV_OK = 0,
   VIDKV_ERR_INVALID_ARG = -1,   /* null pointer, negative size, bad enum value, p outside [0,1] ... */
-  VIDKV_ERR_UNSUPPORTED = -2,   /* a shape or mode this build does not implement */
+  VIDKV_ERR_UNSUPPORTED = -2,   /* a shape or mode this library does not implement */
   VIDKV_ERR_ALIGNMENT = -3,     /* a pointer or stride that is not 16-byte aligned */
   VIDKV_ERR_CAPACITY = -4,      /* more tokens than the cache was sized for, buffer too small */
   VIDKV_ERR_STATE = -5,         /* call order: decode before quantize, quantize twice, ... */

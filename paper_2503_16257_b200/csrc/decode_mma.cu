@@ -871,7 +871,10 @@ cudaError_t launch_decode_mma(const DecodeArgs& a_in, cudaStream_t stream) {
   const int n_chunks = static_cast<int>((a.st.T_q0 > 0 ? 1 : 0) + a.st.n_flush);
   const bool stp = a.n_prot > 0;
   const size_t smem = stp ? decode_stp_smem_bytes(a.split_tokens) : decode_mma_smem_bytes(a.split_tokens);
-  static size_t attr_smem[2] = {0, 0};
+  static size_t attr_smem_dev[64][2] = {};   // function attributes are per device
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  size_t* attr_smem = attr_smem_dev[dev];
   if (smem > attr_smem[stp]) {
     cudaError_t e;
     if (stp) {

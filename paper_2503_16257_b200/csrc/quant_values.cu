@@ -407,7 +407,10 @@ static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheVi
   if (n_rest > 0) {
     const int64_t sgs = (n_rest + kSGTokens - 1) / kSGTokens;
     const size_t smem = kSGTokens * kVRowBytes + sizeof(float) * kSGGroups * 4 * kD + sizeof(uint32_t) * kSGGroups * 64 + 256;
-    static bool attr_set = false;
+    static bool attr_set_dev[64] = {};   // function attributes are per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    bool& attr_set = attr_set_dev[dev];
     if (!attr_set) {
       cudaError_t e;
       if ((e = cudaFuncSetAttribute(v_ternary_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
