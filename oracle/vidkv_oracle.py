@@ -240,26 +240,39 @@ def mixquant_dequant(mq) -> np.ndarray:
 # --------------------------------------------------------------------------
 # Eq. 6 / Algorithm 2 : 1.58-bit (ternary) quantizer
 # --------------------------------------------------------------------------
-def quant_1p58(v: np.ndarray, gamma=GAMMA):
+def quant_1p58(v: np.ndarray, gamma=GAMMA, scale: str = "mean_abs"):
     """Eq. 6 on one group v [n_tokens, C]: s = Mean|v| per channel (binary16),
-    alpha = gamma * s, trit = +1 if v > alpha, -1 if v < -alpha, else 0."""
+    alpha = gamma * s, trit = +1 if v > alpha, -1 if v < -alpha, else 0.
+
+    The paper gives the codes only; the scale that multiplies them back is a reading.
+    ``scale="mean_abs"`` (the default) stores the same s.  ``scale="nonzero_mean"`` stores
+    the mean of |v| over the elements whose trit is not 0 (0 where there is none), the
+    least-squares scale for the given codes as in ternary weight networks, from which
+    Eq. 6 takes its threshold; the codes are the same in both modes."""
     v = np.asarray(v, dtype=np.float32)
     s_h = np.abs(v.astype(np.float64)).mean(axis=0).astype(np.float16)
     alpha = np.float32(gamma) * s_h.astype(np.float32)
     trit = np.zeros(v.shape, dtype=np.int8)
     trit[v > alpha] = 1
     trit[v < -alpha] = -1
-    return trit, s_h
+    if scale == "mean_abs":
+        return trit, s_h
+    assert scale == "nonzero_mean"
+    nz = trit != 0
+    total = (np.abs(v.astype(np.float64)) * nz).sum(axis=0)
+    count = nz.sum(axis=0)
+    s_nz = np.where(count > 0, total / np.maximum(count, 1), 0.0).astype(np.float16)
+    return trit, s_nz
 
 
-def quant_1p58_groups(v: np.ndarray, gamma=GAMMA):
+def quant_1p58_groups(v: np.ndarray, gamma=GAMMA, scale: str = "mean_abs"):
     T = v.shape[0]
     ng = (T + G - 1) // G
     trits = np.zeros(v.shape, dtype=np.int8)
     s = np.zeros((ng, v.shape[1]), dtype=np.float16)
     for g in range(ng):
         sl = slice(g * G, min((g + 1) * G, T))
-        trits[sl], s[g] = quant_1p58(v[sl], gamma)
+        trits[sl], s[g] = quant_1p58(v[sl], gamma, scale)
     return trits, s
 
 
@@ -300,7 +313,7 @@ def select_tokens(saliency: np.ndarray, p, vis_begin: int, T: int) -> np.ndarray
     return E
 
 
-def stpquant(v: np.ndarray, E: np.ndarray, gamma=GAMMA):
+def stpquant(v: np.ndarray, E: np.ndarray, gamma=GAMMA, scale: str = "mean_abs"):
     """Algorithm 2 STPQuant: X[E] -> 2-bit GQuant per channel, X[~E] -> 1.58Quant;
     both streams keep ascending token order and are grouped by 32 in that order."""
     v = np.asarray(v, dtype=np.float32)
@@ -309,7 +322,7 @@ def stpquant(v: np.ndarray, E: np.ndarray, gamma=GAMMA):
     codes2, s2, z2 = gquant_groups(v[prot_idx], 2) if len(prot_idx) else (
         np.zeros((0, v.shape[1]), np.int8), np.zeros((0, v.shape[1]), np.float16),
         np.zeros((0, v.shape[1]), np.float16))
-    trits, st = quant_1p58_groups(v[rest_idx], gamma)
+    trits, st = quant_1p58_groups(v[rest_idx], gamma, scale)
     return dict(prot_idx=prot_idx, rest_idx=rest_idx, codes2=codes2, s2=s2, z2=z2,
                 trits=trits, st=st, T=v.shape[0])
 
@@ -343,9 +356,10 @@ class SlabCache:
     Algorithm 1, Q(X_Kq), X_Kr, Q(X_Vq), X_Vr, with the key part kept as a list
     of independently MixQuant-ed chunks (prefill chunk, then one per flush)."""
 
-    def __init__(self, ratio: float = 0.5, gamma=GAMMA):
+    def __init__(self, ratio: float = 0.5, gamma=GAMMA, ternary_scale: str = "mean_abs"):
         self.ratio = ratio
         self.gamma = gamma
+        self.ternary_scale = ternary_scale
         self.k_chunks = []        # list of mixquant dicts
         self.v_prefill = None     # stpquant dict of the prefill tokens
         self.v_flush = []         # list of (trits, s) per flushed residual
@@ -362,7 +376,7 @@ class SlabCache:
         vq, self.v_res = v[:l - r], v[l - r:].copy()
         if E is None:
             E = np.zeros(l, dtype=bool)
-        self.v_prefill = stpquant(vq, np.asarray(E[:l - r], dtype=bool), self.gamma)
+        self.v_prefill = stpquant(vq, np.asarray(E[:l - r], dtype=bool), self.gamma, self.ternary_scale)
         self.k_chunks = [mixquant(kq, self.ratio)] if l - r > 0 else []
 
     def dequant_k(self) -> np.ndarray:
@@ -399,7 +413,7 @@ class SlabCache:
         V = np.concatenate([self.dequant_v(), self.v_res.astype(np.float64)])
         out = attention(q, K, V, scale)
         if self.v_res.shape[0] == R:                      # residual flush
-            self.v_flush.append(quant_1p58_groups(self.v_res, self.gamma))
+            self.v_flush.append(quant_1p58_groups(self.v_res, self.gamma, self.ternary_scale))
             self.k_chunks.append(mixquant(self.k_res, self.ratio))
             self.k_res = np.zeros((0, d), dtype=np.float32)
             self.v_res = np.zeros((0, d), dtype=np.float32)

@@ -300,6 +300,35 @@ def test_ternary_nonzero_fraction_gaussian():
     assert (t != 0).mean() == pytest.approx(expect, abs=5e-3)
 
 
+def test_ternary_nonzero_mean_scale():
+    v = fp16_values((32, 16), 61, scale=2.0)
+    t, s = O.quant_1p58(v)
+    t2, s2 = O.quant_1p58(v, scale="nonzero_mean")
+    assert (t == t2).all()                                   # the codes do not depend on the stored scale
+    # brute force per channel
+    for c in range(16):
+        vals = [abs(float(v[i, c])) for i in range(32) if t[i, c] != 0]
+        want = np.float16(sum(vals) / len(vals)) if vals else np.float16(0)
+        assert s2[c] == want
+    # least squares: for fixed codes the unrounded non-zero mean minimises |v - s t|^2, so it cannot lose to Mean|v|
+    vv, tt = v.astype(np.float64), t.astype(np.float64)
+    nz = tt != 0
+    s_opt = (np.abs(vv) * nz).sum(0) / np.maximum(nz.sum(0), 1)
+    err_opt = ((vv - s_opt * tt) ** 2).sum(0)
+    err_mean = ((vv - s.astype(np.float64) * tt) ** 2).sum(0)
+    assert (err_opt <= err_mean + 1e-12).all()
+    # closed form: equal magnitudes m with some zeros -> the non-zero mean is m itself
+    w = np.zeros((32, 1), np.float32)
+    w[:8, 0] = 3.0
+    w[8:12, 0] = -3.0
+    t3, s3 = O.quant_1p58(w, scale="nonzero_mean")
+    assert t3[:8, 0].tolist() == [1] * 8 and t3[8:12, 0].tolist() == [-1] * 4 and not t3[12:].any()
+    assert float(s3[0]) == 3.0
+    # a channel of zeros has no non-zero code: scale 0
+    z = np.zeros((32, 2), np.float32)
+    assert (O.quant_1p58(z, scale="nonzero_mean")[1] == 0).all()
+
+
 def test_ternary_short_group_uses_present_elements():
     v = fp16_values((40, 4), 19)
     t, s = O.quant_1p58_groups(v)
