@@ -97,6 +97,11 @@ enum {
 
 enum { VIDKV_F16 = 0, VIDKV_BF16 = 1, VIDKV_F32 = 2 };
 enum { VIDKV_KEY1BIT_FFT_SIGN = 0 };
+/* Scale stored with the ternary codes of Eq. 6 (the paper gives the codes only): the Mean |v|
+ * that also sets the threshold, or the mean of |v| over the elements whose code is not 0
+ * (the least-squares scale for those codes, as in ternary weight networks; 0 where every
+ * code is 0).  The codes are the same in both modes. */
+enum { VIDKV_TERNARY_SCALE_MEAN_ABS = 0, VIDKV_TERNARY_SCALE_NONZERO_MEAN = 1 };
 
 /* Problem description (Algorithm 1 parameters G, R, p, k; Algorithm 2 gamma). */
 typedef struct {
@@ -113,7 +118,7 @@ typedef struct {
   int32_t in_dtype;           /* VIDKV_F16 | VIDKV_BF16 */
   int32_t out_dtype;          /* VIDKV_F16 | VIDKV_BF16 | VIDKV_F32 */
   int32_t key_1bit_mode;      /* VIDKV_KEY1BIT_FFT_SIGN */
-  int32_t reserved;           /* must be 0 */
+  int32_t ternary_scale;      /* VIDKV_TERNARY_SCALE_MEAN_ABS (default) | VIDKV_TERNARY_SCALE_NONZERO_MEAN */
   int64_t max_prefill_tokens; /* largest T passed to vidkv_quantize_* */
   int64_t max_new_tokens;     /* decode steps the cache must be able to absorb */
 } vidkv_config_t;

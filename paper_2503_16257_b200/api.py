@@ -6,6 +6,7 @@ import os
 from dataclasses import dataclass
 
 VIDKV_F16, VIDKV_BF16, VIDKV_F32 = 0, 1, 2
+VIDKV_TERNARY_SCALE_MEAN_ABS, VIDKV_TERNARY_SCALE_NONZERO_MEAN = 0, 1
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "ALIGNMENT", -4: "CAPACITY",
                 -5: "STATE", -6: "CUDA", -7: "TIMEOUT"}
 
@@ -24,7 +25,7 @@ class _Config(C.Structure):
                 ("D", C.c_int32), ("G", C.c_int32), ("R", C.c_int32),
                 ("k_ratio", C.c_float), ("p_ratio", C.c_float), ("gamma", C.c_float),
                 ("in_dtype", C.c_int32), ("out_dtype", C.c_int32), ("key_1bit_mode", C.c_int32),
-                ("reserved", C.c_int32),
+                ("ternary_scale", C.c_int32),
                 ("max_prefill_tokens", C.c_int64), ("max_new_tokens", C.c_int64)]
 
 
@@ -52,10 +53,11 @@ class VidKVConfig:
     in_dtype: int = VIDKV_F16
     out_dtype: int = VIDKV_F32
     key_1bit_mode: int = 0
+    ternary_scale: int = 0          # VIDKV_TERNARY_SCALE_MEAN_ABS | VIDKV_TERNARY_SCALE_NONZERO_MEAN
 
     def to_c(self) -> _Config:
         return _Config(self.B, self.L, self.H_kv, self.H_q, self.D, self.G, self.R, self.k_ratio,
-                       self.p_ratio, self.gamma, self.in_dtype, self.out_dtype, self.key_1bit_mode, 0,
+                       self.p_ratio, self.gamma, self.in_dtype, self.out_dtype, self.key_1bit_mode, self.ternary_scale,
                        self.max_prefill_tokens, self.max_new_tokens)
 
 

@@ -29,7 +29,8 @@ vidkv_status_t check_config(const vidkv_config_t* c) {
   if (!(c->gamma >= 0.0f) || !std::isfinite(c->gamma)) return VIDKV_ERR_INVALID_ARG;
   if (c->in_dtype != VIDKV_F16 && c->in_dtype != VIDKV_BF16) return VIDKV_ERR_INVALID_ARG;
   if (c->out_dtype != VIDKV_F16 && c->out_dtype != VIDKV_BF16 && c->out_dtype != VIDKV_F32) return VIDKV_ERR_INVALID_ARG;
-  if (c->reserved != 0) return VIDKV_ERR_INVALID_ARG;
+  if (c->ternary_scale != VIDKV_TERNARY_SCALE_MEAN_ABS && c->ternary_scale != VIDKV_TERNARY_SCALE_NONZERO_MEAN)
+    return VIDKV_ERR_INVALID_ARG;
   if (c->D != kD || c->G != kG || c->R != kR) return VIDKV_ERR_UNSUPPORTED;
   if (c->k_ratio != 0.5f) return VIDKV_ERR_UNSUPPORTED;
   if (c->key_1bit_mode != VIDKV_KEY1BIT_FFT_SIGN) return VIDKV_ERR_UNSUPPORTED;
@@ -371,7 +372,8 @@ vidkv_status_t vidkv_quantize_values(vidkv_cache_t* h, int32_t layer, const void
     sel.stride_rest = h->cfg.max_prefill_tokens;
     sel.n_prot = h->n_prot;
   }
-  if (T_q > 0 && launch_quantize_values(h->cfg.in_dtype, src, T_q, h->cv, layer, sel, h->cfg.gamma, s) != cudaSuccess)
+  if (T_q > 0 && launch_quantize_values(h->cfg.in_dtype, src, T_q, h->cv, layer, sel, h->cfg.gamma,
+                                        h->cfg.ternary_scale == VIDKV_TERNARY_SCALE_NONZERO_MEAN, s) != cudaSuccess)
     return VIDKV_ERR_CUDA;
   if (launch_copy_to_residual(h->cfg.in_dtype, src, T_q, r, h->cv, layer, true, 0, s) != cudaSuccess) return VIDKV_ERR_CUDA;
   li.v_done = true; li.T = T; li.T_q0 = T_q; li.n_res = r; li.n_flush = 0;
@@ -431,7 +433,8 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
       return VIDKV_ERR_CUDA;
     const int64_t n_rest = first.T_q0 - h->n_prot;
     const int64_t tgroup0 = (n_rest + kG - 1) / kG + (kR / kG) * first.n_flush;
-    if (launch_flush_values(dt, vsrc, h->cv, layer_begin, n_layers, tgroup0, h->cfg.gamma, s) != cudaSuccess)
+    if (launch_flush_values(dt, vsrc, h->cv, layer_begin, n_layers, tgroup0, h->cfg.gamma,
+                            h->cfg.ternary_scale == VIDKV_TERNARY_SCALE_NONZERO_MEAN, s) != cudaSuccess)
       return VIDKV_ERR_CUDA;
   }
   for (int l = layer_begin; l < layer_begin + n_layers; ++l) {

@@ -54,12 +54,12 @@ cudaError_t dft_fragments(const uint32_t** table, cudaStream_t stream);
 // Algorithm 2 on the prefill tokens of one layer.  T_q (multiple of 32) tokens; the
 // unprotected ones go to ternary stream positions 0.., the protected ones to 2-bit groups.
 cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer,
-                                   const SelView& sel, float gamma, cudaStream_t stream);
+                                   const SelView& sel, float gamma, bool nonzero_mean_scale, cudaStream_t stream);
 
 // 1.58Quant of a full 128-token residual of every slab of the given layers, appended at
 // ternary stream group index tgroup0 (read-modify-write of shared supergroup bytes).
 cudaError_t launch_flush_values(int dtype, const KSrc& src, const CacheView& cv, int layer0, int n_layers,
-                                int64_t tgroup0, float gamma, cudaStream_t stream);
+                                int64_t tgroup0, float gamma, bool nonzero_mean_scale, cudaStream_t stream);
 
 // Copy `n_tok` tokens starting at token t_begin of every slab of one layer into the
 // residual rings (rows r0 .. r0 + n_tok - 1).

@@ -59,7 +59,9 @@ __device__ __forceinline__ void cp_async16_v(void* smem_dst, const void* gmem_sr
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
 }
 
-template <typename T>
+// NZ: the stored scale is the mean of |v| over the non-zero codes instead of Mean |v| (one more
+// sweep over the staged tile; needs kSGGroups * 4 * kD more floats of shared memory).
+template <typename T, bool NZ>
 __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest, CacheView cv, int layer,
                                                         SelView sel, float gamma) {
   extern __shared__ __align__(16) uint8_t vsm[];
@@ -67,6 +69,7 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
   float* part = reinterpret_cast<float*>(tile + kSGTokens * kVRowBytes);       // [5][4][128]
   uint32_t* thr = reinterpret_cast<uint32_t*>(part + kSGGroups * 4 * kD);      // [5][64] threshold pairs
   uint8_t* lut = reinterpret_cast<uint8_t*>(thr + kSGGroups * 64);             // [256]
+  float* cnt = reinterpret_cast<float*>(lut + 256);                            // [5][4][128], NZ only
   const int tid = threadIdx.x;
   const int slab = blockIdx.y;
   const int b = slab / cv.H_kv, h = slab % cv.H_kv;
@@ -114,12 +117,43 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
       const float* pp = part + g * 4 * kD + c;
       const float sum = ((pp[0] + pp[kD]) + pp[2 * kD]) + pp[3 * kD];
       const uint16_t sh = f2h_bits(__fdiv_rn(sum, static_cast<float>(n)));
-      reinterpret_cast<uint16_t*>(sg + kSG_Scales)[g * kD + c] = sh;
+      if (!NZ) reinterpret_cast<uint16_t*>(sg + kSG_Scales)[g * kD + c] = sh;
       a = Simd2<T>::above(__fmul_rn(gamma, h2f(sh)));
     }
     reinterpret_cast<uint16_t*>(thr)[item] = a;
   }
   __syncthreads();
+  if (NZ) {
+    // ---- sums and counts of |v| over the elements whose code is not 0 (v >= A or v <= -A)
+    const int cp = tid & 63, q = tid >> 6;
+    const uint32_t one = 0x3c003c00u;
+#pragma unroll
+    for (int g = 0; g < kSGGroups; ++g) {
+      const uint32_t A = thr[g * 64 + cp], nA = A ^ 0x80008000u;
+      float a0 = 0.0f, a1 = 0.0f, c0 = 0.0f, c1 = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(tile + (g * kG + q * 8 + j) * kVRowBytes + cp * 4);
+        const __half2 nz = __hsub2(__hadd2(as_half2(Simd2<T>::ge(w, A)), as_half2(one)), as_half2(Simd2<T>::gt(w, nA)));
+        const float2 m = __half22float2(nz), f = Elem<T>::to_float2(w);
+        a0 = fmaf(m.x, fabsf(f.x), a0); a1 = fmaf(m.y, fabsf(f.y), a1);
+        c0 += m.x; c1 += m.y;
+      }
+      *reinterpret_cast<float2*>(part + (g * 4 + q) * kD + 2 * cp) = make_float2(a0, a1);
+      *reinterpret_cast<float2*>(cnt + (g * 4 + q) * kD + 2 * cp) = make_float2(c0, c1);
+    }
+    __syncthreads();
+    for (int item = tid; item < kSGGroups * kD; item += 256) {
+      const int c = item & (kD - 1), g = item >> 7;
+      if (n_rows - g * kG > 0) {
+        const float* pp = part + g * 4 * kD + c;
+        const float* pc = cnt + g * 4 * kD + c;
+        const float sum = ((pp[0] + pp[kD]) + pp[2 * kD]) + pp[3 * kD];
+        const float n_nz = ((pc[0] + pc[kD]) + pc[2 * kD]) + pc[3 * kD];
+        reinterpret_cast<uint16_t*>(sg + kSG_Scales)[g * kD + c] = n_nz > 0.0f ? f2h_bits(__fdiv_rn(sum, n_nz)) : static_cast<uint16_t>(0);
+      }
+    }
+  }
   // ---- pass 2: one word of the plane per thread and step
 #pragma unroll
   for (int wi = 0; wi < kG * kD / 4 / 256; ++wi) {
@@ -219,7 +253,7 @@ __global__ void __launch_bounds__(128) v_protect_kernel(KSrc src, CacheView cv, 
 // may land in a supergroup that already holds earlier groups, so bytes are updated digit
 // by digit.  grid = slabs (over layers); block = 128 threads (thread = channel).
 // ---------------------------------------------------------------------------------
-template <typename T>
+template <typename T, bool NZ>
 __global__ void __launch_bounds__(kD) v_flush_kernel(KSrc src, CacheView cv, int layer0, int slabs_per_layer,
                                                      int64_t tgroup0, float gamma) {
   const int slab = blockIdx.x;
@@ -236,15 +270,19 @@ __global__ void __launch_bounds__(kD) v_flush_kernel(KSrc src, CacheView cv, int
     float sum = 0.0f;
     for (int j = 0; j < kG; ++j) sum += fabsf(Elem<T>::to_float(base[(g4 * kG + j) * src.stride_t + c]));
     const uint16_t sh = f2h_bits(__fdiv_rn(sum, static_cast<float>(kG)));
-    reinterpret_cast<uint16_t*>(sg + kSG_Scales)[slot * kD + c] = sh;
     const float a = __fmul_rn(gamma, h2f(sh));
+    float nz_sum = 0.0f, nz_cnt = 0.0f;
     for (int j = 0; j < kG; ++j) {
       const float v = Elem<T>::to_float(base[(g4 * kG + j) * src.stride_t + c]);
       const uint32_t d = v > a ? 2u : (v < -a ? 0u : 1u);
+      if (NZ && d != 1u) { nz_sum += fabsf(v); nz_cnt += 1.0f; }
       const uint32_t bold = trit_byte_decode(sg[tern_byte_offset(j, c)]);
       const uint32_t dold = (bold / p3[slot]) % 3u;
       sg[tern_byte_offset(j, c)] = static_cast<uint8_t>(trit_byte_encode(bold - dold * p3[slot] + d * p3[slot]));
     }
+    // the stored scale: Mean |v|, or the mean of |v| over the non-zero codes (0 where there is none)
+    reinterpret_cast<uint16_t*>(sg + kSG_Scales)[slot * kD + c] =
+        !NZ ? sh : (nz_cnt > 0.0f ? f2h_bits(__fdiv_rn(nz_sum, nz_cnt)) : static_cast<uint16_t>(0));
   }
 }
 
@@ -399,25 +437,25 @@ __global__ void __launch_bounds__(1024) select_tokens_kernel(const float* __rest
 // ---------------------------------------------------------------------------------
 // Host launchers
 // ---------------------------------------------------------------------------------
-template <typename T>
+template <typename T, bool NZ>
 static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheView& cv, int layer, const SelView& sel,
                                      float gamma, cudaStream_t stream) {
   const int n_slabs = cv.B * cv.H_kv;
   const int64_t n_rest = T_q - sel.n_prot;
   if (n_rest > 0) {
     const int64_t sgs = (n_rest + kSGTokens - 1) / kSGTokens;
-    const size_t smem = kSGTokens * kVRowBytes + sizeof(float) * kSGGroups * 4 * kD + sizeof(uint32_t) * kSGGroups * 64 + 256;
-    static bool attr_set_dev[64] = {};   // function attributes are per device
+    const size_t smem = kSGTokens * kVRowBytes + sizeof(float) * kSGGroups * 4 * kD + sizeof(uint32_t) * kSGGroups * 64 + 256 +
+                        (NZ ? sizeof(float) * kSGGroups * 4 * kD : 0);
+    static bool attr_set_dev[64] = {};   // function attributes are per device (and per instantiation)
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     bool& attr_set = attr_set_dev[dev];
     if (!attr_set) {
       cudaError_t e;
-      if ((e = cudaFuncSetAttribute(v_ternary_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-      if ((e = cudaFuncSetAttribute(v_ternary_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+      if ((e = cudaFuncSetAttribute(v_ternary_kernel<T, NZ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
       attr_set = true;
     }
-    v_ternary_kernel<T><<<dim3(static_cast<unsigned>(sgs), n_slabs), 256, smem, stream>>>(src, n_rest, cv, layer, sel, gamma);
+    v_ternary_kernel<T, NZ><<<dim3(static_cast<unsigned>(sgs), n_slabs), 256, smem, stream>>>(src, n_rest, cv, layer, sel, gamma);
     count_launches(1);
   }
   if (sel.n_prot > 0) {
@@ -429,18 +467,30 @@ static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheVi
 }
 
 cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer,
-                                   const SelView& sel, float gamma, cudaStream_t stream) {
-  if (dtype == VIDKV_F16) return quantize_values_t<__half>(src, T_q, cv, layer, sel, gamma, stream);
-  return quantize_values_t<__nv_bfloat16>(src, T_q, cv, layer, sel, gamma, stream);
+                                   const SelView& sel, float gamma, bool nonzero_mean_scale, cudaStream_t stream) {
+  if (dtype == VIDKV_F16)
+    return nonzero_mean_scale ? quantize_values_t<__half, true>(src, T_q, cv, layer, sel, gamma, stream)
+                              : quantize_values_t<__half, false>(src, T_q, cv, layer, sel, gamma, stream);
+  return nonzero_mean_scale ? quantize_values_t<__nv_bfloat16, true>(src, T_q, cv, layer, sel, gamma, stream)
+                            : quantize_values_t<__nv_bfloat16, false>(src, T_q, cv, layer, sel, gamma, stream);
+}
+
+template <typename T, bool NZ>
+static void flush_values_t(const KSrc& src, const CacheView& cv, int layer0, int n_layers, int64_t tgroup0, float gamma,
+                           cudaStream_t stream) {
+  const int spl = cv.B * cv.H_kv;
+  v_flush_kernel<T, NZ><<<spl * n_layers, kD, 0, stream>>>(src, cv, layer0, spl, tgroup0, gamma);
 }
 
 cudaError_t launch_flush_values(int dtype, const KSrc& src, const CacheView& cv, int layer0, int n_layers,
-                                int64_t tgroup0, float gamma, cudaStream_t stream) {
-  const int spl = cv.B * cv.H_kv;
-  if (dtype == VIDKV_F16)
-    v_flush_kernel<__half><<<spl * n_layers, kD, 0, stream>>>(src, cv, layer0, spl, tgroup0, gamma);
-  else
-    v_flush_kernel<__nv_bfloat16><<<spl * n_layers, kD, 0, stream>>>(src, cv, layer0, spl, tgroup0, gamma);
+                                int64_t tgroup0, float gamma, bool nonzero_mean_scale, cudaStream_t stream) {
+  if (dtype == VIDKV_F16) {
+    if (nonzero_mean_scale) flush_values_t<__half, true>(src, cv, layer0, n_layers, tgroup0, gamma, stream);
+    else flush_values_t<__half, false>(src, cv, layer0, n_layers, tgroup0, gamma, stream);
+  } else {
+    if (nonzero_mean_scale) flush_values_t<__nv_bfloat16, true>(src, cv, layer0, n_layers, tgroup0, gamma, stream);
+    else flush_values_t<__nv_bfloat16, false>(src, cv, layer0, n_layers, tgroup0, gamma, stream);
+  }
   count_launches(1);
   return cudaGetLastError();
 }

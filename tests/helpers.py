@@ -28,7 +28,7 @@ def to_np(x: torch.Tensor) -> np.ndarray:
 class Pair:
     """One configuration run through both implementations (all layers, all slabs)."""
 
-    def __init__(self, wl, T, B=None, L=None, p=0.0, max_new=16, device="cuda"):
+    def __init__(self, wl, T, B=None, L=None, p=0.0, max_new=16, device="cuda", ternary_scale="mean_abs"):
         import paper_2503_16257_b200 as P
         self.P = P
         self.wl, self.T, self.p = wl, T, p
@@ -37,7 +37,10 @@ class Pair:
         self.device = device
         in_dt = P.VIDKV_F16 if wl.dtype == "fp16" else P.VIDKV_BF16
         self.cfg = P.VidKVConfig(B=self.B, L=self.L, max_prefill_tokens=T, max_new_tokens=max_new, p_ratio=p,
-                                 in_dtype=in_dt, out_dtype=P.VIDKV_F32)
+                                 in_dtype=in_dt, out_dtype=P.VIDKV_F32,
+                                 ternary_scale=P.VIDKV_TERNARY_SCALE_NONZERO_MEAN if ternary_scale == "nonzero_mean"
+                                 else P.VIDKV_TERNARY_SCALE_MEAN_ABS)
+        self.ternary_scale = ternary_scale
         self.cache = P.VidKVCache(self.cfg, device=device)
         self.lay = self.cache.layout
         self.l_v = min(wl.l_v, T - T % 32)
@@ -63,7 +66,7 @@ class Pair:
             self.cache.quantize_values(layer, Vd)
             for b in range(self.B):
                 for h in range(self.cfg.H_kv):
-                    sc = O.SlabCache()
+                    sc = O.SlabCache(ternary_scale=self.ternary_scale)
                     E = None
                     if self.E is not None:
                         E = np.zeros(self.T, dtype=bool)
@@ -131,17 +134,27 @@ def compare_key_chunk(slab, lay, chunk_idx, g_begin, mq, k_chunk, stats):
         assert (np.abs(cols[bad]) <= TIE_REL * scale[bad] + 1e-12).all(), "a sign bit differs away from zero"
 
 
-def compare_ternary(trits, s, o_trits, o_s, v_stream, stats, gamma=0.7):
-    ulp = f16_ulp_distance(s, o_s)
-    assert ulp.max() <= 1, f"ternary scales differ by {ulp.max()} ulp"
-    stats["st_n"] += ulp.size; stats["st_off"] += int((ulp > 0).sum())
+def compare_ternary(trits, s, o_trits, o_s, v_stream, stats, gamma=0.7, o_s_thr=None):
+    """o_s_thr: the oracle's Mean |v| scales where the stored scale is a different statistic (the
+    threshold always comes from Mean |v|)."""
     n = o_trits.shape[0]
     bad = trits[:n] != o_trits
+    ulp = f16_ulp_distance(s, o_s)
+    if o_s_thr is not None and bad.any():
+        # a stored scale that averages over the non-zero codes moves when a code at a tie differs
+        ng = o_s.shape[0]
+        pad = np.zeros((ng * 32, bad.shape[1]), dtype=bool)
+        pad[:n] = bad
+        ulp = np.where(pad.reshape(ng, 32, -1).any(axis=1), 0, ulp)
+    assert ulp.max() <= 1, f"ternary scales differ by {ulp.max()} ulp"
+    stats["st_n"] += ulp.size; stats["st_off"] += int((ulp > 0).sum())
     stats["trit_n"] += bad.size; stats["trit_off"] += int(bad.sum())
     if bad.any():
+        thr_s = o_s if o_s_thr is None else o_s_thr
+        ulp_thr = ulp if o_s_thr is None else np.ones_like(ulp)
         ng = o_s.shape[0]
-        srow = np.repeat(o_s.astype(np.float64), 32, axis=0)[:n]
-        urow = np.repeat(ulp, 32, axis=0)[:n]
+        srow = np.repeat(thr_s.astype(np.float64), 32, axis=0)[:n]
+        urow = np.repeat(ulp_thr, 32, axis=0)[:n]
         dist = np.abs(np.abs(v_stream.astype(np.float64)) - gamma * srow)
         tol = TIE_REL * srow + urow * srow * 2.0 ** -10
         assert (dist[bad] <= tol[bad] + 1e-12).all(), "a trit differs away from the threshold"

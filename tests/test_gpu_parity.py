@@ -29,7 +29,8 @@ def _compare_prefill(pair: Pair):
         if n_rest:
             ng = (n_rest + 31) // 32
             trits, s = U.ternary_groups(slab, pair.lay, 0, ng)
-            compare_ternary(trits, s, sq["trits"], sq["st"], v[sq["rest_idx"]], stats)
+            thr = None if pair.ternary_scale == "mean_abs" else O.quant_1p58_groups(v[sq["rest_idx"]])[1]
+            compare_ternary(trits, s, sq["trits"], sq["st"], v[sq["rest_idx"]], stats, o_s_thr=thr)
         n_prot = len(sq["prot_idx"])
         if n_prot:
             E, prefix = U.selection_mask(cache, pair.lay, b, Tq)
@@ -240,10 +241,27 @@ def test_other_head_counts(H_kv, H_q, p):
     assert cache.status() == 0
 
 
-def test_residual_flush_parity():
+@pytest.mark.parametrize("name,T,B,p", [
+    ("tiny", 1632, 1, 0.0), ("tiny", 77, 2, 0.0), ("llava", 352, 1, 0.2), ("qwen", 480, 2, 0.2),
+])
+def test_nonzero_mean_ternary_scale_prefill(name, T, B, p):
+    """The optional stored scale (mean of |v| over the non-zero codes): same codes, other scales."""
+    pair = Pair(CONFIGS[name], T, B=B, L=1, p=p, ternary_scale="nonzero_mean").prefill()
+    _compare_prefill(pair)
+    _compare_dequant(pair)
+    ref = Pair(CONFIGS[name], T, B=B, L=1, p=p).prefill()
+    a, b = pair.cache_bytes(), ref.cache_bytes()
+    assert (a != b).any()                       # the scales differ from the default mode's ...
+    for key, sc in pair.slabs.items():          # ... the codes do not
+        assert (sc.v_prefill["trits"] == ref.slabs[key].v_prefill["trits"]).all()
+    assert pair.cache.status() == 0
+
+
+@pytest.mark.parametrize("ternary_scale", ["mean_abs", "nonzero_mean"])
+def test_residual_flush_parity(ternary_scale):
     # 64 quantized + 5 residual tokens; the residual fills at step 123 and is flushed
     wl = CONFIGS["tiny"]
-    pair = Pair(wl, 69, B=1, L=2, p=0.0, max_new=140).prefill()
+    pair = Pair(wl, 69, B=1, L=2, p=0.0, max_new=140, ternary_scale=ternary_scale).prefill()
     _decode_steps(pair, 123)
     st = pair.cache.layer_state(0)
     assert st == dict(n_quantized=192, n_residual=0, n_chunks=2, n_protected=0)
@@ -256,7 +274,8 @@ def test_residual_flush_parity():
         compare_key_chunk(slab, pair.lay, 1, 2, sc.k_chunks[1], kin, stats)
         trits, s = U.ternary_groups(slab, pair.lay, 2, 4)
         o_t, o_s = sc.v_flush[0]
-        compare_ternary(trits, s, o_t, o_s, vin, stats)
+        compare_ternary(trits, s, o_t, o_s, vin, stats,
+                        o_s_thr=None if ternary_scale == "mean_abs" else O.quant_1p58_groups(vin)[1])
     check_stats(stats)
     _compare_dequant(pair)
     _decode_steps(pair, 10)          # attention over two chunks + a fresh residual

@@ -86,6 +86,7 @@ def test_layout_regions_do_not_overlap(lib):
     (dict(H_q=30), -2), (dict(H_q=64), -2), (dict(key_1bit_mode=1), -2),
     (dict(B=0), -1), (dict(p_ratio=1.5), -1), (dict(p_ratio=-0.1), -1), (dict(in_dtype=2), -1),
     (dict(out_dtype=7), -1), (dict(max_new_tokens=-1), -1), (dict(gamma=float("nan")), -1),
+    (dict(ternary_scale=2), -1),
 ])
 def test_config_validation(lib, kw, status):
     base = dict(B=1, L=1, max_prefill_tokens=64, max_new_tokens=4)
