@@ -7,6 +7,7 @@ What follows the paper, step by step, in its notation:
 
 * ``gquant``            Eq. 4   n-bit asymmetric min/max quantizer ("GQuant")
 * ``select_channels``   Algorithm 3 (range / TopK / D-mask / N-mask), Sec. 3.2(1)
+* ``channel_variance`` / ``channel_outliers``   the two other channel metrics of Sec. 4.1(1)
 * ``dft64`` / ``idft64``        the discrete Fourier transform written out as
                                  its defining matrix (no FFT routine)
 * ``fft_1bit``          Eq. 5   sign code + mean-|.| scale in the frequency domain
@@ -128,6 +129,22 @@ def channel_range(k: np.ndarray) -> np.ndarray:
     """Sec. 3.2(1): R = max(K) - min(K) per channel over all tokens (float32)."""
     k = np.asarray(k, dtype=np.float32)
     return k.max(axis=0) - k.min(axis=0)
+
+
+def channel_variance(k: np.ndarray) -> np.ndarray:
+    """Sec. 4.1(1), the Variance metric: population variance of each channel over the tokens (float64)."""
+    k = np.asarray(k, dtype=np.float64)
+    mean = k.sum(axis=0) / k.shape[0]
+    return ((k - mean) ** 2).sum(axis=0) / k.shape[0]
+
+
+def channel_outliers(k: np.ndarray, M: float = 3.0) -> np.ndarray:
+    """Sec. 4.1(1), the Outliers metric: N = sum_i 1[K_i > M * mean(K)] per channel with M = 3.  The paper
+    writes the comparison without magnitudes; for channels that are centred near zero that would count
+    about half of the tokens whatever their spread, so the reading taken here compares magnitudes:
+    |K_i| > M * mean_i |K_i|."""
+    a = np.abs(np.asarray(k, dtype=np.float64))
+    return (a > M * (a.sum(axis=0) / a.shape[0])).sum(axis=0).astype(np.int64)
 
 
 def select_channels(k: np.ndarray, ratio: float = 0.5):

@@ -128,6 +128,32 @@ def test_select_channels_matches_sort_and_is_permutation_invariant():
     assert (abn2 == abn).all()
 
 
+def test_channel_variance_and_outliers():
+    k = fp16_values((200, 6), 71, scale=3.0)
+    var = O.channel_variance(k)
+    np.testing.assert_allclose(var, np.var(k.astype(np.float64), axis=0), rtol=1e-12)     # library routine
+    for c in range(6):                                                                        # brute force
+        col = [float(x) for x in k[:, c]]
+        m = sum(col) / len(col)
+        assert var[c] == pytest.approx(sum((x - m) ** 2 for x in col) / len(col), rel=1e-12)
+    # closed forms: a constant channel has variance 0, +-a alternating has a^2; a shift changes nothing
+    z = np.zeros((64, 2), np.float32)
+    z[:, 0] = 1.5
+    z[0::2, 1], z[1::2, 1] = 2.0, -2.0
+    assert O.channel_variance(z).tolist() == [0.0, 4.0]
+    np.testing.assert_allclose(O.channel_variance(k + 7.0), var, rtol=1e-9)
+    # outliers: element by element, M = 3 (the paper's setting)
+    out = O.channel_outliers(k)
+    for c in range(6):
+        a = [abs(float(x)) for x in k[:, c]]
+        assert out[c] == sum(1 for x in a if x > 3.0 * (sum(a) / len(a)))
+    # planted: 5 values of 100 among 995 ones -> mean |K| = 1.495, threshold 4.485, exactly the 5 planted ones count
+    p = np.ones((1000, 1), np.float32)
+    p[::200, 0] = -100.0
+    assert O.channel_outliers(p)[0] == 5
+    assert O.channel_outliers(np.ones((50, 3), np.float32)).tolist() == [0, 0, 0]
+
+
 def test_select_channels_tie_break():
     k = np.zeros((4, 8), dtype=np.float32)
     k[0, :] = 1.0           # all ranges equal -> lowest indices win
