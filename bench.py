@@ -388,10 +388,34 @@ def main():
                                 "seconds": res["seconds"]}
     if rank == 0 and not args.no_token_scores:
         line["token_scores"] = run_token_scores(P, torch, wl, dev, peak)
+        line["channel_metrics"] = run_channel_metrics(P, torch, Ks, peak)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_channel_metrics(P, torch, Ks, peak):
+    """Upstream of the hot path: the Variance and Outliers channel metrics of one layer's keys, timed alone
+    with CUDA events, alternating between two layers' tensors when there are two.  Bytes = K read once
+    (variance) or twice (outliers: a mean pass and a counting pass).  The arithmetic is float64."""
+    res = {}
+    for metric, name, passes in ((P.VIDKV_METRIC_VARIANCE, "variance", 1), (P.VIDKV_METRIC_OUTLIERS, "outliers", 2)):
+        for i in range(4):
+            P.vidkv_channel_metrics(Ks[i % min(2, len(Ks))], metric)
+        times = []
+        for i in range(6):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            P.vidkv_channel_metrics(Ks[i % min(2, len(Ks))], metric)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = sum(times) / len(times)
+        gbs = passes * Ks[0].numel() * 2 / (ms * 1e-3) / 1e9
+        res[name] = {"GBps": gbs, "frac_of_measured_hbm": gbs / peak, "ms_per_call": ms}
+    return res
 
 
 def run_token_scores(P, torch, wl, dev, peak):

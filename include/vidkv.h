@@ -97,6 +97,8 @@ enum {
 
 enum { VIDKV_F16 = 0, VIDKV_BF16 = 1, VIDKV_F32 = 2 };
 enum { VIDKV_KEY1BIT_FFT_SIGN = 0 };
+/* Channel metrics of Sec. 4.1(1) other than the range (which the method uses and computes itself). */
+enum { VIDKV_METRIC_VARIANCE = 1, VIDKV_METRIC_OUTLIERS = 2 };
 /* Scale stored with the ternary codes of Eq. 6 (the paper gives the codes only): the Mean |v|
  * that also sets the threshold, or the mean of |v| over the elements whose code is not 0
  * (the least-squares scale for those codes, as in ternary weight networks; 0 where every
@@ -179,6 +181,20 @@ vidkv_status_t vidkv_cache_reset(vidkv_cache_t* handle, void* stream);
  * pointers 16-byte aligned.  Needs no cache handle.  Two launches on `stream`. */
 vidkv_status_t vidkv_saliency_scores(int32_t dtype, const void* x_v, const void* x_t, int64_t B, int64_t l_v,
                                      int64_t l_t, int64_t d, float* text_sum, float* saliency, void* stream);
+
+/* Sec. 4.1(1): the channel metrics the paper compares the range against, per (batch element,
+ * head, channel) of a key tensor K [B, H, T, 128] (dtype VIDKV_F16 / VIDKV_BF16, element
+ * strides as for vidkv_quantize_keys, T >= 1):
+ *   VIDKV_METRIC_VARIANCE  population variance of the channel over the T tokens
+ *   VIDKV_METRIC_OUTLIERS  number of tokens with |K_i| > M * mean_i |K_i|  (the paper sets M = 3
+ *                          and writes the comparison without magnitudes; magnitudes are taken
+ *                          here, or zero-centred channels would always count about T / 2)
+ * out [B, H, 128] float32 device; scratch [B, H, 2, 128] float64 device, caller-owned,
+ * overwritten.  Accumulation is in float64.  The cache is not involved: MixQuant's own channel
+ * split stays range-based.  Three or four launches and one memset on `stream`. */
+vidkv_status_t vidkv_channel_metrics(int32_t dtype, const void* K, int64_t B, int64_t H, int64_t T, int64_t stride_b,
+                                     int64_t stride_h, int64_t stride_t, int32_t metric, float M, double* scratch,
+                                     float* out, void* stream);
 
 /* Sec. 3.3(2) / Eq. 7: choose the protected tokens.  saliency [B, l_v] float32 scores
  * the visual tokens vis_begin .. vis_begin + l_v - 1 of a prompt of T tokens; the top

@@ -7,6 +7,7 @@ from dataclasses import dataclass
 
 VIDKV_F16, VIDKV_BF16, VIDKV_F32 = 0, 1, 2
 VIDKV_TERNARY_SCALE_MEAN_ABS, VIDKV_TERNARY_SCALE_NONZERO_MEAN = 0, 1
+VIDKV_METRIC_VARIANCE, VIDKV_METRIC_OUTLIERS = 1, 2
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "ALIGNMENT", -4: "CAPACITY",
                 -5: "STATE", -6: "CUDA", -7: "TIMEOUT"}
 
@@ -73,6 +74,8 @@ _SIGNATURES = {
                                      C.c_void_p, C.POINTER(C.c_void_p)]),
     "vidkv_cache_destroy": (C.c_int32, [C.c_void_p]),
     "vidkv_cache_reset": (C.c_int32, [C.c_void_p, C.c_void_p]),
+    "vidkv_channel_metrics": (C.c_int32, [C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
+                                          C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]),
     "vidkv_saliency_scores": (C.c_int32, [C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
                                           C.c_void_p, C.c_void_p, C.c_void_p]),
     "vidkv_select_tokens": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p]),
@@ -139,6 +142,21 @@ def vidkv_attend_noalloc(cfg: VidKVConfig, cache, n_prefill_quantized: int, n_fl
     _check("vidkv_attend_noalloc", load_library().vidkv_attend_noalloc(
         C.byref(c), C.c_void_p(cache.data_ptr()), n_prefill_quantized, n_flushed_chunks, n_residual, n_protected,
         layer_begin, n_layers, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()), softmax_scale, _stream_ptr()))
+
+
+def vidkv_channel_metrics(K, metric: int, M: float = 3.0):
+    """Variance or outlier count of every key channel: K [B, H, T, 128] (float16 / bfloat16 device
+    tensor, channel stride 1) -> float32 [B, H, 128]."""
+    import torch
+    B, H, T, D = K.shape
+    assert D == 128 and K.stride(3) == 1
+    dtype = VIDKV_F16 if K.dtype == torch.float16 else VIDKV_BF16
+    scratch = torch.empty((B, H, 2, D), dtype=torch.float64, device=K.device)
+    out = torch.empty((B, H, D), dtype=torch.float32, device=K.device)
+    _check("vidkv_channel_metrics", load_library().vidkv_channel_metrics(
+        dtype, C.c_void_p(K.data_ptr()), B, H, T, K.stride(0), K.stride(1), K.stride(2), metric, M,
+        C.c_void_p(scratch.data_ptr()), C.c_void_p(out.data_ptr()), _stream_ptr()))
+    return out
 
 
 def vidkv_saliency_scores(x_v, x_t, text_sum=None, saliency=None):

@@ -258,6 +258,24 @@ vidkv_status_t vidkv_cache_reset(vidkv_cache_t* h, void* stream) {
   return VIDKV_OK;
 }
 
+vidkv_status_t vidkv_channel_metrics(int32_t dtype, const void* K, int64_t B, int64_t H, int64_t T, int64_t stride_b,
+                                     int64_t stride_h, int64_t stride_t, int32_t metric, float M, double* scratch,
+                                     float* out, void* stream) {
+  if (dtype != VIDKV_F16 && dtype != VIDKV_BF16) return VIDKV_ERR_INVALID_ARG;
+  if (metric != VIDKV_METRIC_VARIANCE && metric != VIDKV_METRIC_OUTLIERS) return VIDKV_ERR_INVALID_ARG;
+  if (B < 0 || H < 0 || T < 1 || !(M > 0.0f) || !std::isfinite(M)) return VIDKV_ERR_INVALID_ARG;
+  if (B == 0 || H == 0) return VIDKV_OK;
+  if (!K || !scratch || !out) return VIDKV_ERR_INVALID_ARG;
+  if (B * H > 65535 || H > INT32_MAX) return VIDKV_ERR_UNSUPPORTED;
+  if (stride_b % 8 || stride_h % 8 || stride_t % 8 || stride_t < kD) return VIDKV_ERR_ALIGNMENT;
+  if (!aligned16(K) || !aligned16(scratch) || !aligned16(out)) return VIDKV_ERR_ALIGNMENT;
+  const KSrc src{K, stride_b, stride_h, stride_t, static_cast<int32_t>(H)};
+  if (launch_channel_metrics(dtype, src, B * H, T, metric, static_cast<double>(M), scratch, out,
+                             static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  return VIDKV_OK;
+}
+
 vidkv_status_t vidkv_saliency_scores(int32_t dtype, const void* x_v, const void* x_t, int64_t B, int64_t l_v, int64_t l_t,
                                      int64_t d, float* text_sum, float* saliency, void* stream) {
   if (dtype != VIDKV_F16 && dtype != VIDKV_BF16) return VIDKV_ERR_INVALID_ARG;

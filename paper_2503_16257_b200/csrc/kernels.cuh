@@ -106,6 +106,10 @@ struct DecodeArgs {
 cudaError_t launch_saliency(int dtype, const void* x_v, const void* x_t, int64_t B, int64_t l_v, int64_t l_t, int64_t d,
                             float* text_sum, float* saliency, cudaStream_t stream);
 
+// Variance / outlier count per (slab, channel) of a key tensor; stats [n_slabs][2][128] float64 scratch.
+cudaError_t launch_channel_metrics(int dtype, const KSrc& src, int64_t n_slabs, int64_t T_tokens, int metric, double M,
+                                   double* stats, float* out, cudaStream_t stream);
+
 // Number of kernels launched by this library since it was loaded (host counter).
 extern unsigned long long g_launch_count;
 inline void count_launches(int n) { g_launch_count += static_cast<unsigned long long>(n); }

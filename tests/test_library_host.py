@@ -122,6 +122,24 @@ def test_saliency_scores_argument_checks_without_a_device(lib):
     assert f(P.VIDKV_F16, ctypes.c_void_p(0x1004), a, 1, 4, 2, 64, a, a, None) == -3   # misaligned
 
 
+def test_channel_metrics_argument_checks_without_a_device(lib):
+    f = lib.vidkv_channel_metrics
+    a = ctypes.c_void_p(0x1000)
+    ok = (P.VIDKV_F16, a, 1, 4, 64, 4 * 64 * 128, 64 * 128, 128, P.VIDKV_METRIC_VARIANCE, 3.0, a, a, None)
+    def call(**kw):
+        names = ["dtype", "K", "B", "H", "T", "sb", "sh", "st", "metric", "M", "scratch", "out", "stream"]
+        args = list(ok)
+        for k, v in kw.items():
+            args[names.index(k)] = v
+        return f(*args)
+    assert call(dtype=5) == -1 and call(metric=0) == -1 and call(metric=3) == -1     # unknown dtype / metric
+    assert call(T=0) == -1 and call(M=0.0) == -1 and call(M=float("nan")) == -1
+    assert call(K=None) == -1 and call(out=None) == -1
+    assert call(B=0) == 0                                                              # nothing to do
+    assert call(st=100) == -3 and call(sh=4) == -3                                     # strides
+    assert call(K=ctypes.c_void_p(0x1002)) == -3                                       # misaligned
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     import paper_2503_16257_b200.api as api
     monkeypatch.setattr(api, "_LIB", None)
