@@ -44,15 +44,26 @@ __global__ void __launch_bounds__(kCmThreads) chan_moments_kernel(KSrc src, int6
   const int lane16 = threadIdx.x & 15, row = threadIdx.x >> 4;
   const int64_t t0 = static_cast<int64_t>(blockIdx.x) * kCmTokens, t1 = min(t0 + kCmTokens, T_tokens);
   double a0[8] = {0, 0, 0, 0, 0, 0, 0, 0}, a1[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  for (int64_t t = t0 + row; t < t1; t += 16) {
-    float f[8];
-    load8<T>(base + t * src.stride_t, lane16, f);
+  auto add = [&](const float (&f)[8]) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const double x = static_cast<double>(f[i]);
       if (VARIANCE) { a0[i] += x; a1[i] = fma(x, x, a1[i]); }
       else a0[i] += fabs(x);
     }
+  };
+  int64_t t = t0 + row;
+  for (; t + 48 < t1; t += 64) {                       // four rows in flight per thread
+    float f[4][8];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) load8<T>(base + (t + 16 * k) * src.stride_t, lane16, f[k]);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) add(f[k]);
+  }
+  for (; t < t1; t += 16) {
+    float f[8];
+    load8<T>(base + t * src.stride_t, lane16, f);
+    add(f);
   }
   block_add(red, a0, stats + static_cast<int64_t>(slab) * 2 * kD);
   if (VARIANCE) block_add(red, a1, stats + static_cast<int64_t>(slab) * 2 * kD + kD);
@@ -69,7 +80,17 @@ __global__ void __launch_bounds__(kCmThreads) chan_outlier_kernel(KSrc src, int6
   double thr[8], cnt[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #pragma unroll
   for (int i = 0; i < 8; ++i) thr[i] = M * (stats[static_cast<int64_t>(slab) * 2 * kD + lane16 * 8 + i] / static_cast<double>(T_tokens));
-  for (int64_t t = t0 + row; t < t1; t += 16) {
+  int64_t t = t0 + row;
+  for (; t + 48 < t1; t += 64) {                       // four rows in flight per thread
+    float f[4][8];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) load8<T>(base + (t + 16 * k) * src.stride_t, lane16, f[k]);
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) cnt[i] += fabs(static_cast<double>(f[k][i])) > thr[i] ? 1.0 : 0.0;
+  }
+  for (; t < t1; t += 16) {
     float f[8];
     load8<T>(base + t * src.stride_t, lane16, f);
 #pragma unroll
