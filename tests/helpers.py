@@ -48,6 +48,7 @@ class Pair:
         self.slabs = {}
         self.E = None
         self.step = 0
+        self.sign_tie_tokens = {}  # per slab: prefill tokens whose sign bits differ from the oracle's at a tie
         self.res_in = {}          # inputs currently in the residual, per slab
         self.flushed_in = {}      # inputs of the most recent flush, per slab
 
@@ -132,6 +133,7 @@ def compare_key_chunk(slab, lay, chunk_idx, g_begin, mq, k_chunk, stats):
         cols = np.concatenate([xf.real, xf.imag], -1)[:, pk]
         scale = np.repeat(o_s1.astype(np.float64), 32, axis=0)
         assert (np.abs(cols[bad]) <= TIE_REL * scale[bad] + 1e-12).all(), "a sign bit differs away from zero"
+    return np.nonzero(bad.any(axis=1))[0]          # tokens of the chunk with a sign bit at a tie
 
 
 def compare_ternary(trits, s, o_trits, o_s, v_stream, stats, gamma=0.7, o_s_thr=None):

@@ -23,7 +23,20 @@ def _compare_prefill(pair: Pair):
         k = to_np(pair.K[layer][b, h])
         v = to_np(pair.V[layer][b, h])
         if Tq:
-            compare_key_chunk(slab, pair.lay, 0, 0, sc.k_chunks[0], k[:Tq], stats)
+            ties = compare_key_chunk(slab, pair.lay, 0, 0, sc.k_chunks[0], k[:Tq], stats)
+            # Tokens with a spectrum coefficient that is zero (to rounding).  The oracle codes all 64 bins, the
+            # cache the Hermitian half: for a zero coefficient the oracle's two mirror bins both get the bit of
+            # +0, which the half spectrum cannot express, so the dequantized rows of such tokens may differ
+            # although every stored bit agrees.  (A sign bit at zero is a tie either way.)
+            mq = sc.k_chunks[0]
+            xf = O.dft64(k[:Tq][:, mq["nom_idx"]])
+            cols = np.concatenate([xf.real, xf.imag], -1)
+            scale = np.repeat(mq["s1"].astype(np.float64), 32, axis=0)
+            at_tie = (np.abs(cols) <= 1e-9 * scale) & (scale > 0)
+            ties = np.union1d(ties, np.nonzero(at_tie.any(axis=1))[0]).astype(np.int64)
+            if len(ties):
+                assert len(ties) <= max(2, 2e-3 * Tq), "too many tokens with a coefficient at a tie"
+                pair.sign_tie_tokens[(layer, b, h)] = ties
         sq = sc.v_prefill
         n_rest = len(sq["rest_idx"])
         if n_rest:
@@ -65,7 +78,14 @@ def _compare_dequant(pair: Pair):
                 if ok.size == 0:
                     continue
                 s1max = max([float(c["s1"].astype(np.float64).max()) for c in sc.k_chunks] + [0.0])
-                assert np.abs(Kd[b, h] - ok).max() <= _scale_tol([s1max])
+                kerr = np.abs(Kd[b, h] - ok)
+                # a sign bit that differs at a tie (coefficient within 1e-3 of its scale of zero, checked in
+                # _compare_prefill) moves the token's normal channels by up to half that column's scale
+                ties = pair.sign_tie_tokens.get((layer, b, h), [])
+                if len(ties):
+                    assert kerr[ties].max() <= 0.5 * s1max * 64
+                    kerr[ties] = 0.0
+                assert kerr.max() <= _scale_tol([s1max])
                 stmax = float(sc.v_prefill["st"].astype(np.float64).max()) if sc.v_prefill["st"].size else 0.0
                 for (_, s) in sc.v_flush:
                     stmax = max(stmax, float(s.astype(np.float64).max()))
@@ -123,6 +143,34 @@ def _decode_steps(pair: Pair, n_steps, tol=TOL_ABS):
 def test_decode_attention_parity(name, T, B, p, steps):
     pair = Pair(CONFIGS[name], T, B=B, L=1, p=p, max_new=steps).prefill()
     _decode_steps(pair, steps)
+    assert pair.cache.status() == 0
+
+
+def _random_cases(n, seed):
+    r = np.random.default_rng(seed)
+    cases = []
+    for _ in range(n):
+        name = ["tiny", "llava", "qwen"][int(r.integers(0, 3))]
+        cases.append((name, int(r.integers(1, 1500)), int(r.integers(1, 3)), int(r.integers(1, 3)),
+                      [0.0, 0.0, 0.1, 0.5][int(r.integers(0, 4))], int(r.integers(1, 4)),
+                      ["mean_abs", "nonzero_mean"][int(r.integers(0, 2))]))
+    return cases
+
+
+@pytest.mark.parametrize("name,T,B,L,p,steps,ternary_scale", _random_cases(10, 20250316))
+def test_seeded_random_shapes(name, T, B, L, p, steps, ternary_scale):
+    """Shapes nobody picked by hand: token counts anywhere in [1, 1500) (any remainder modulo 32, 128, 160 and
+    640), one or two sequences and layers, with and without protected tokens, both scale modes."""
+    wl = CONFIGS[name]
+    if min(wl.l_v, T - T % 32) < 1:
+        p = 0.0                                      # no quantized visual token to protect
+    pair = Pair(wl, T, B=B, L=L, p=p, max_new=steps, ternary_scale=ternary_scale).prefill()
+    _compare_prefill(pair)
+    _compare_dequant(pair)
+    for _ in range(steps):
+        out, ref = pair.decode()
+        # as in the heavy-tail tests: where the outputs are large the bound scales with their magnitude
+        assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
     assert pair.cache.status() == 0
 
 
