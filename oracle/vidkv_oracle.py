@@ -195,6 +195,17 @@ def fft_1bit(x: np.ndarray):
     cols = np.concatenate([xf.real, xf.imag], axis=-1)           # [n, 2N]
     bits = (cols >= 0).astype(np.uint8)
     s_h = np.abs(cols).mean(axis=0).astype(np.float16)
+    # The input is real, so bins N/2+1 .. N-1 are the conjugates of bins N/2-1 .. 1, and one bit per
+    # normal channel (the paper's bit count) pays for the N columns of the Hermitian half only
+    # (``hermitian_pack_columns``).  The mirror bins are therefore not coded on their own: their bits
+    # and scales follow from the half (real part equal, imaginary part negated).  This differs from
+    # coding every column by its own sign only where a coefficient is exactly zero.
+    n = x.shape[-1]
+    for k in range(1, n // 2):
+        bits[..., n - k] = bits[..., k]
+        bits[..., n + n - k] = 1 - bits[..., n + k]
+        s_h[n - k] = s_h[k]
+        s_h[n + n - k] = s_h[n + k]
     return bits, s_h
 
 

@@ -24,18 +24,8 @@ def _compare_prefill(pair: Pair):
         v = to_np(pair.V[layer][b, h])
         if Tq:
             ties = compare_key_chunk(slab, pair.lay, 0, 0, sc.k_chunks[0], k[:Tq], stats)
-            # Tokens with a spectrum coefficient that is zero (to rounding).  The oracle codes all 64 bins, the
-            # cache the Hermitian half: for a zero coefficient the oracle's two mirror bins both get the bit of
-            # +0, which the half spectrum cannot express, so the dequantized rows of such tokens may differ
-            # although every stored bit agrees.  (A sign bit at zero is a tie either way.)
-            mq = sc.k_chunks[0]
-            xf = O.dft64(k[:Tq][:, mq["nom_idx"]])
-            cols = np.concatenate([xf.real, xf.imag], -1)
-            scale = np.repeat(mq["s1"].astype(np.float64), 32, axis=0)
-            at_tie = (np.abs(cols) <= 1e-9 * scale) & (scale > 0)
-            ties = np.union1d(ties, np.nonzero(at_tie.any(axis=1))[0]).astype(np.int64)
             if len(ties):
-                assert len(ties) <= max(2, 2e-3 * Tq), "too many tokens with a coefficient at a tie"
+                assert len(ties) <= max(2, 2e-3 * Tq), "too many tokens with a sign bit at a tie"
                 pair.sign_tie_tokens[(layer, b, h)] = ties
         sq = sc.v_prefill
         n_rest = len(sq["rest_idx"])

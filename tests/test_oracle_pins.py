@@ -504,6 +504,27 @@ def test_residual_flush_after_R_tokens():
     assert np.allclose(out, ref)
 
 
+def test_fft_1bit_codes_the_hermitian_half():
+    # mirror bins follow from the half for any input ...
+    x = fp16_values((32, 64), 81)
+    bits, s = O.fft_1bit(x)
+    for k in range(1, 32):
+        assert (bits[:, 64 - k] == bits[:, k]).all() and (bits[:, 128 - k] == 1 - bits[:, 64 + k]).all()
+        assert s[64 - k] == s[k] and s[128 - k] == s[64 + k]
+    # ... so the dequantized spectrum is Hermitian and its inverse transform real, also when imaginary
+    # coefficients are exactly zero (an input that is even in the channel index has a real spectrum):
+    # coding each mirror bin by its own sign would give both the bit of +0 and leave an imaginary part
+    e = np.zeros((32, 64), np.float32)
+    e[:, 0] = fp16_values((32,), 82)
+    e[:, 32] = fp16_values((32,), 83)
+    for c in range(1, 32):
+        e[:, c] = e[:, 64 - c] = fp16_values((32,), 84 + c)
+    e[1] += x[1]                                   # one generic row so that the imaginary columns have a scale
+    xr, imag_max = O.fft_1bit_dequant(*O.fft_1bit(e))
+    assert imag_max <= 1e-12
+    assert xr.shape == e.shape
+
+
 def test_fft_smooths_one_bit_error_direction():
     # Direction of the paper's Fig. 5 only (its numbers come from a real model's
     # key channel): for tokens with a sharp outlier at a varying channel, sign coding in the
