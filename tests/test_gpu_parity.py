@@ -320,6 +320,21 @@ def test_residual_flush_parity(ternary_scale):
     assert pair.cache.layer_state(1)["n_residual"] == 10
 
 
+@pytest.mark.parametrize("name,T,B,p,ternary_scale", [
+    ("qwen", 577, 2, 0.2, "nonzero_mean"),      # bf16, protected tokens, the flush lands at stream group 18.4
+    ("llava", 475, 2, 0.0, "nonzero_mean"),     # heavy-tailed, 27 residual tokens at prefill
+    ("tiny", 118, 2, 0.0, "mean_abs"),
+])
+def test_decode_across_a_flush_on_other_shapes(name, T, B, p, ternary_scale):
+    steps = 128 - T % 32 + 3
+    pair = Pair(CONFIGS[name], T, B=B, L=1, p=p, max_new=steps + 1, ternary_scale=ternary_scale).prefill()
+    for _ in range(steps):
+        out, ref = pair.decode()
+        assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
+    st = pair.cache.layer_state(0)
+    assert st["n_chunks"] == 2 and st["n_residual"] == 3 and pair.cache.status() == 0
+
+
 def test_flush_with_protected_tokens_keeps_streams_apart():
     wl = CONFIGS["tiny"]
     pair = Pair(wl, 256, B=1, L=1, p=0.2, max_new=135).prefill()     # 51 protected, 205 ternary (6.4 groups)
