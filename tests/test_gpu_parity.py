@@ -238,7 +238,7 @@ def test_longest_sequence_slab():
     assert cache.status() == 0
 
 
-@pytest.mark.parametrize("H_kv,H_q,p", [(2, 16, 0.0), (2, 16, 0.25), (8, 8, 0.0), (1, 4, 0.25)])
+@pytest.mark.parametrize("H_kv,H_q,p", [(2, 16, 0.0), (2, 16, 0.25), (8, 8, 0.0), (1, 4, 0.25), (4, 8, 0.0), (4, 12, 0.25), (2, 10, 0.0), (1, 6, 0.25), (3, 9, 0.0), (16, 16, 0.25)])
 def test_other_head_counts(H_kv, H_q, p):
     """GQA ratios 8, 1 and 4 (the named workloads all use 7): seeded Gaussian K, V, q with a few
     wide key channels, two decode steps, every slab against the oracle."""
