@@ -335,6 +335,19 @@ def test_decode_across_a_flush_on_other_shapes(name, T, B, p, ternary_scale):
     assert st["n_chunks"] == 2 and st["n_residual"] == 3 and pair.cache.status() == 0
 
 
+@pytest.mark.parametrize("name,T,p,ternary_scale,steps", [
+    ("tiny", 69, 0.0, "mean_abs", 262), ("qwen", 200, 0.2, "nonzero_mean", 270),
+])
+def test_decode_across_two_flushes(name, T, p, ternary_scale, steps):
+    """Three key chunks with their own channel splits, two appended value runs, a residual on top."""
+    pair = Pair(CONFIGS[name], T, B=1, L=1, p=p, max_new=steps + 1, ternary_scale=ternary_scale).prefill()
+    for _ in range(steps):
+        out, ref = pair.decode()
+        assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
+    st = pair.cache.layer_state(0)
+    assert st["n_chunks"] == 3 and st["n_quantized"] == T - T % 32 + 256 and pair.cache.status() == 0
+
+
 def test_flush_with_protected_tokens_keeps_streams_apart():
     wl = CONFIGS["tiny"]
     pair = Pair(wl, 256, B=1, L=1, p=0.2, max_new=135).prefill()     # 51 protected, 205 ternary (6.4 groups)
