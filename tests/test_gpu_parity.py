@@ -8,7 +8,7 @@ from oracle import vidkv_oracle as O
 from tests import unpack as U
 from tests.helpers import (Pair, TOL_ABS, check_stats, compare_key_chunk, compare_ternary, f16_ulp_distance,
                            new_stats, to_np)
-from workloads import CONFIGS
+from workloads import CONFIGS, make_layer_kv, make_saliency
 
 pytestmark = pytest.mark.gpu
 
@@ -354,6 +354,34 @@ def test_flush_with_protected_tokens_keeps_streams_apart():
     _decode_steps(pair, 130)
     assert pair.cache.layer_state(0) == dict(n_quantized=384, n_residual=2, n_chunks=2, n_protected=51)
     _compare_dequant(pair)
+
+
+@pytest.mark.parametrize("name,p", [("tiny", 0.2), ("qwen", 0.0)])
+def test_strided_inputs_give_the_same_cache(name, p):
+    """K and V kept token-major ([B, T, H, D], as a projection writes them) and handed over as a
+    [B, H, T, D] view must pack to the same bytes as contiguous copies."""
+    import paper_2503_16257_b200 as P
+    wl = CONFIGS[name]
+    T, B = 1000, 2
+    K, V = make_layer_kv(wl, 0, "cuda", T=T, B=B)
+    in_dt = P.VIDKV_F16 if wl.dtype == "fp16" else P.VIDKV_BF16
+    cfg = P.VidKVConfig(B=B, L=1, max_prefill_tokens=T, max_new_tokens=1, p_ratio=p, in_dtype=in_dt, out_dtype=P.VIDKV_F32)
+    caches = []
+    for strided in (False, True):
+        c = P.VidKVCache(cfg, device="cuda")
+        if p > 0:
+            c.select_tokens(make_saliency(wl, "cuda", l_v=960, B=B), 0, 960, T)
+        if strided:
+            Kt = K.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)     # [B, H, T, D] view of [B, T, H, D]
+            Vt = V.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+            assert not Kt.is_contiguous() and Kt.stride(2) == K.shape[1] * 128
+            c.quantize_keys(0, Kt); c.quantize_values(0, Vt)
+        else:
+            c.quantize_keys(0, K); c.quantize_values(0, V)
+        torch.cuda.synchronize()
+        assert c.status() == 0
+        caches.append(c.cache.cpu().numpy())
+    assert np.array_equal(caches[0], caches[1])
 
 
 def test_multi_layer_call_equals_per_layer_calls():
