@@ -24,8 +24,8 @@
  *   - All device work is enqueued on the caller's stream (a cudaStream_t passed
  *     as void*) and is asynchronous.  Argument errors are detected on the host
  *     before anything is launched.  One exception: the first key quantization or
- *     decode call on each device fills a 16 KB table of DFT coefficients inside the
- *     library and synchronises the stream once.
+ *     decode call on each device fills the tables of DFT coefficients inside the
+ *     library (56 KB) and synchronises the stream once.
  *   - Fixed in this library: D = 128, G = 32, R = 128, k = 0.5 (64 two-bit and 64
  *     one-bit channels), H_q a multiple of H_kv with H_q / H_kv <= 8.  Other
  *     shapes return VIDKV_ERR_UNSUPPORTED.
@@ -34,6 +34,9 @@
  *     Input values must be finite and representable in binary16.
  *   - One handle must not be used from two host threads at once, and calls on
  *     one handle must be issued on one stream (or on streams the caller orders).
+ *     Different handles may be worked on from different streams at the same time.
+ *     The one-time set-up per device (tables, kernel attributes) is not guarded
+ *     against concurrent host threads: make the first call on a device from one thread.
  *
  * Packed cache layout (little endian; all offsets are given by vidkv_layout_t)
  *   per slab = (layer, batch element, KV head):

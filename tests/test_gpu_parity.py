@@ -384,6 +384,56 @@ def test_strided_inputs_give_the_same_cache(name, p):
     assert np.array_equal(caches[0], caches[1])
 
 
+def test_two_caches_on_two_streams():
+    """Two caches worked on from two streams at once (prefill and decode interleaved) end up exactly
+    as when each runs alone: the library keeps no per-call state outside the handle."""
+    import paper_2503_16257_b200 as P
+    wl = CONFIGS["tiny"]
+    T, B, L = 1632, 2, 2
+    cfg = P.VidKVConfig(B=B, L=L, max_prefill_tokens=T, max_new_tokens=4, p_ratio=0.0, in_dtype=P.VIDKV_F16, out_dtype=P.VIDKV_F32)
+    KV = [make_layer_kv(wl, layer, "cuda", T=T, B=B) for layer in range(L)]
+    from workloads import make_step_inputs
+    steps = [[make_step_inputs(wl, layer, s, "cuda", T=T, B=B) for layer in range(L)] for s in range(3)]
+
+    def calls(cache, outs):
+        """The work on one cache as a list of calls."""
+        todo = []
+        for layer in range(L):
+            todo.append(lambda layer=layer: cache.quantize_keys(layer, KV[layer][0]))
+            todo.append(lambda layer=layer: cache.quantize_values(layer, KV[layer][1]))
+        for s in range(3):
+            def step(s=s):
+                q = torch.stack([steps[s][layer][0] for layer in range(L)])
+                k = torch.stack([steps[s][layer][1] for layer in range(L)])
+                v = torch.stack([steps[s][layer][2] for layer in range(L)])
+                out = torch.empty((L, B, 28, 128), dtype=torch.float32, device="cuda")
+                cache.decode_attention(0, L, q, k, v, out)
+                outs.append(out)
+            todo.append(step)
+        return todo
+
+    alone = P.VidKVCache(cfg, device="cuda")
+    ref = []
+    for f in calls(alone, ref):
+        f()
+    torch.cuda.synchronize()
+    a, b = P.VidKVCache(cfg, device="cuda"), P.VidKVCache(cfg, device="cuda")
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    s1.wait_stream(torch.cuda.current_stream()); s2.wait_stream(torch.cuda.current_stream())
+    oa, ob = [], []
+    # call by call, alternating streams, so that kernels of both caches are in flight together
+    for fa, fb in zip(calls(a, oa), calls(b, ob)):
+        with torch.cuda.stream(s1):
+            fa()
+        with torch.cuda.stream(s2):
+            fb()
+    torch.cuda.synchronize()
+    for x, y, z in zip(ref, oa, ob):
+        assert torch.equal(x, y) and torch.equal(x, z)
+    assert torch.equal(alone.cache, a.cache) and torch.equal(alone.cache, b.cache)
+    assert a.status() == 0 and b.status() == 0
+
+
 def test_multi_layer_call_equals_per_layer_calls():
     wl = CONFIGS["tiny"]
     a = Pair(wl, 320, B=2, L=3, p=0.0, max_new=2).prefill()
