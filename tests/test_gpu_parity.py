@@ -129,6 +129,7 @@ def _decode_steps(pair: Pair, n_steps, tol=TOL_ABS):
     ("tiny", 1300, 2, 0.0, 3),     # last split starts inside a supergroup (1280) and ends in the residual
     ("tiny", 1632, 1, 0.9, 3),     # nearly every visual token protected: long protected stream, short ternary one
     ("tiny", 800, 1, 0.002, 3),    # a single protected token
+    ("tiny", 1568, 1, 1.0, 3),     # every token is visual and protected: the ternary stream is empty
 ])
 def test_decode_attention_parity(name, T, B, p, steps):
     pair = Pair(CONFIGS[name], T, B=B, L=1, p=p, max_new=steps).prefill()
@@ -324,6 +325,7 @@ def test_residual_flush_parity(ternary_scale):
     ("qwen", 577, 2, 0.2, "nonzero_mean"),      # bf16, protected tokens, the flush lands at stream group 18.4
     ("llava", 475, 2, 0.0, "nonzero_mean"),     # heavy-tailed, 27 residual tokens at prefill
     ("tiny", 118, 2, 0.0, "mean_abs"),
+    ("tiny", 320, 1, 1.0, "mean_abs"),          # the flush appends to a ternary stream that was empty
 ])
 def test_decode_across_a_flush_on_other_shapes(name, T, B, p, ternary_scale):
     steps = 128 - T % 32 + 3
