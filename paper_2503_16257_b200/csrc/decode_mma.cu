@@ -149,6 +149,38 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
   return d;
 }
 
+// 2^k as a float, |k| <= 126
+__device__ __forceinline__ float pow2i(int k) { return __uint_as_float(static_cast<uint32_t>(127 + k) << 23); }
+
+// Query normalisation.  The score operands q_j s_j and Q_f s_f are binary16 numbers, so a large
+// query entry times a large key scale would overflow although the score itself is an ordinary
+// float.  Every query head is therefore multiplied by the power of two 2^(-e - kQShift), e =
+// floor(log2(max_c |q_c|)), which puts its largest entry into [1/8, 1/4): no product of a scaled
+// entry (or of a spectrum coefficient, at most 16 times the largest entry) with a binary16 scale
+// below 16376 leaves the binary16 range.  Scores are linear in q, so the softmax multiplies by the
+// inverse power of two; both factors are exact.  head_exponent returns e (0 for a head that is all
+// zero or holds no finite maximum); the NSUB lanes sub = 0..NSUB-1 share the 128 entries of the row,
+// and all 32 lanes of the warp must call it.
+constexpr int kQShift = 3;
+template <typename T, int NSUB>
+__device__ __forceinline__ int head_exponent(const T* qrow, int sub, bool live) {
+  float m = 0.0f;
+  if (live) {
+    const uint2* p = reinterpret_cast<const uint2*>(qrow + sub * (kD / NSUB));
+#pragma unroll
+    for (int i = 0; i < kD / NSUB / 4; ++i) {
+      const uint2 v = __ldg(p + i);
+      const float2 a = Elem<T>::to_float2(v.x), b = Elem<T>::to_float2(v.y);
+      m = fmaxf(m, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(b.x), fabsf(b.y))));
+    }
+  }
+#pragma unroll
+  for (int o = NSUB / 2; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (!(m > 0.0f) || m > 3.0e38f) return 0;
+  const int e = static_cast<int>(__float_as_uint(m) >> 23) - 127;
+  return max(-100, min(100, e));
+}
+
 }  // namespace
 
 size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks) {
@@ -162,7 +194,8 @@ size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks) {
 //   words  8..15  leading binary16 part of the transformed query Q at the spectrum
 //                 columns (16 r + 2 i, 16 r + 2 i + 1)
 //   words 16..23  binary16 remainder Q - leading part
-// for head lane / 4 (zero when that head does not exist) and r = lane % 4.
+// for head lane / 4 (zero when that head does not exist) and r = lane % 4, all of the query
+// normalised by its head's power of two (head_exponent).
 // Q_f = sum_c q_c W[c, f] with W the weights with which spectrum column f enters channel c of
 // the inverse orthonormal 64-point transform of a Hermitian half spectrum: the forward DFT
 // matrix, doubled for the columns f >= 2 that stand for a conjugate pair.  The product runs
@@ -182,7 +215,8 @@ __global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int
                         static_cast<int64_t>(chunk) * kChunkBytes;
   const T* qrow = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(lb) * cv.H_q + h * rep + hd) * kD;
   const bool live = hd < rep;
-  auto q_at = [&](int c) -> float { return live ? Elem<T>::to_float(qrow[c]) : 0.0f; };
+  const float qf = pow2i(-head_exponent<T, 4>(qrow, r, live) - kQShift);   // normalised query, see head_exponent
+  auto q_at = [&](int c) -> float { return live ? Elem<T>::to_float(qrow[c]) * qf : 0.0f; };
   if (chunk == 0 && a.append_row >= 0) {
     // Algorithm 1, Decoding: the step's new key / value row joins the residual (lanes 0-15 copy
     // the key row, 16-31 the value row); the attention kernel that follows reads it there.
@@ -266,11 +300,25 @@ __device__ __forceinline__ Split make_split(const DecodeArgs& a, int split) {
   return c;
 }
 
-// Phase 1: raw scores q . k (before the softmax scale) of every token of the split into
-// S[head][token - t0]: the packed key groups staged in kbuf, then the FP16 / BF16 residual rows.
+// qexp[k] = head_exponent of query head k of the CTA's slab (0 for a head that does not exist);
+// warp w fills entries 2 w and 2 w + 1.
+template <typename T>
+__device__ __forceinline__ void query_exponents(const DecodeArgs& a, const Split& c, int* qexp) {
+  const T* qp = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(c.lb) * a.cv.H_q + c.h * c.rep) * kD;
+#pragma unroll
+  for (int hh = 0; hh < 2; ++hh) {
+    const int k = 2 * c.warp + hh;
+    const int e = head_exponent<T, 32>(qp + k * kD, c.lane, k < c.rep);
+    if (c.lane == 0) qexp[k] = e;
+  }
+}
+
+// Phase 1: raw scores q . k (before the softmax scale, in units of the head's query normalisation
+// 2^(-qexp[head] - kQShift)) of every token of the split into S[head][token - t0]: the packed key
+// groups staged in kbuf, then the FP16 / BF16 residual rows.
 template <typename T>
 __device__ __forceinline__ void score_phase(const DecodeArgs& a, int n_chunks, const Split& c, const uint8_t* kbuf,
-                                            float* S, int SS) {
+                                            float* S, int SS, const int* qexp) {
   const CacheView& cv = a.cv;
   const int lane = c.lane, warp = c.warp, hd = c.hd, r = c.r, slab = c.slab, h = c.h, lb = c.lb, rep = c.rep;
   const uint32_t m_field = c.m_field, c_four = c.c_four, m_sign = c.m_sign, c_neg1 = c.c_neg1;
@@ -367,6 +415,7 @@ __device__ __forceinline__ void score_phase(const DecodeArgs& a, int n_chunks, c
 #pragma unroll
     for (int i = 0; i < 16; ++i)
       qn[i] = hd < rep ? __ldg(reinterpret_cast<const uint32_t*>(qp + hd * kD + 8 * i + 2 * r)) : 0u;
+    const float qf = pow2i(-qexp[hd] - kQShift);                         // the raw query is used here: same units as above
     const int n_tiles = (r_end - r_begin + 7) / 8;
     for (int tile = warp; tile < n_tiles; tile += 4) {
       const int row = min(r_begin + tile * 8 + hd, r_end - 1);          // clamped: extra columns are dropped
@@ -376,8 +425,8 @@ __device__ __forceinline__ void score_phase(const DecodeArgs& a, int n_chunks, c
       for (int ks = 0; ks < 8; ++ks) mma_in<T>(acc, qn[2 * ks], qn[2 * ks + 1], kr[ks * 8], kr[ks * 8 + 4]);
       const int c0 = r_begin + tile * 8 + 2 * r;
       float* srow = S + hd * SS + static_cast<int>(T_qt - t0);
-      if (c0 < r_end) srow[c0] = acc[0];
-      if (c0 + 1 < r_end) srow[c0 + 1] = acc[1];
+      if (c0 < r_end) srow[c0] = acc[0] * qf;
+      if (c0 + 1 < r_end) srow[c0 + 1] = acc[1] * qf;
     }
   }
 }
@@ -525,17 +574,19 @@ __device__ __forceinline__ void write_partial(const DecodeArgs& a, const Split& 
 // cleared once its scores are in registers and becomes the ternary-stream row: quantized
 // tokens [0, nq) go to their stream position through `map` (bit 15 = protected stream, row of
 // Pprot), residual tokens [nq, n_loc) to Pres[row][i - nq].
-// red[row] = scaled row maximum, red[8 + row] = sum of the probabilities.
+// red[row] = scaled row maximum, red[8 + row] = sum of the probabilities.  The scores arrive in
+// units of the head's query normalisation; the inverse power of two joins the softmax scale.
 template <bool STP, bool FULL = false>     // FULL: the split holds exactly 640 tokens, no bound checks
 __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& c, float* S, int SS, float* red,
                                               int n_pad, const uint16_t* map, __half* Pprot, int PP, __half* Pres,
-                                              int PRS) {
+                                              int PRS, const int* qexp) {
   const int lane = c.lane, n_loc = c.n_loc;
-  const float sl2 = a.scale * 1.4426950408889634f;
   constexpr int kMaxPairs = 10;                                          // ST <= 640: 320 pairs per row
 #pragma unroll 1
   for (int hh = 0; hh < 2; ++hh) {
     const int row_h = c.warp * 2 + hh;
+    const float scale_h = a.scale * pow2i(qexp[row_h] + kQShift);
+    const float sl2 = scale_h * 1.4426950408889634f;
     float* row = S + row_h * SS;
     float2 v[kMaxPairs];
     float m = -INFINITY;
@@ -583,7 +634,7 @@ __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& 
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-    if (lane == 0) { red[row_h] = m * a.scale; red[8 + row_h] = l; }
+    if (lane == 0) { red[row_h] = m * scale_h; red[8 + row_h] = l; }
   }
 }
 
@@ -615,9 +666,10 @@ __device__ __forceinline__ void group_sums(const Split& c, const __half* P, int 
 //   S     8 rows of ST + 4 floats: scores, then binary16 probabilities in place
 //   psum  [ST/32][8]  -5 * (sum of the rounded probabilities of the group)
 //   red   [16]        row maxima and sums
+//   qexp  [8]         exponents of the query normalisation (head_exponent)
 // ---------------------------------------------------------------------------------
 size_t decode_mma_smem_bytes(int ST) {
-  return static_cast<size_t>(ST / 32) * kKGroupBytes + sizeof(float) * (8 * (ST + 4) + 8 * (ST / 32) + 16);
+  return static_cast<size_t>(ST / 32) * kKGroupBytes + sizeof(float) * (8 * (ST + 4) + 8 * (ST / 32) + 16 + 8);
 }
 
 template <typename T>
@@ -630,12 +682,14 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
   float* S = reinterpret_cast<float*>(kbuf + (ST / 32) * kKGroupBytes);
   float* psum = S + 8 * SS;
   float* red = psum + 8 * (ST / 32);
+  int* qexp = reinterpret_cast<int*>(red + 16);
   const CacheView& cv = a.cv;
   // One CTA walks a.splits_per_cta consecutive splits of its slab and keeps a running
   // (max, sum, out) per head, rescaled as in a streaming softmax; one record leaves at the end.
   float TOT[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
   float Mr[2] = {-INFINITY, -INFINITY}, Lr[2] = {0.0f, 0.0f};
   Split c = make_split(a, blockIdx.x * a.splits_per_cta);
+  query_exponents<T>(a, c, qexp);                           // visible after the first barrier below
 #pragma unroll 1
   for (int it = 0; it < a.splits_per_cta; ++it) {
     const int split = blockIdx.x * a.splits_per_cta + it;
@@ -649,7 +703,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
     }
     cp_async_wait<0>();
     __syncthreads();
-    score_phase<T>(a, n_chunks, c, kbuf, S, SS);
+    score_phase<T>(a, n_chunks, c, kbuf, S, SS, qexp);
     __syncthreads();
     {
       // the key groups are spent: the ternary supergroups take their place while the softmax runs
@@ -658,9 +712,9 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
       cp_async_commit();
     }
     if (c.n_loc == 640)
-      softmax_phase<false, true>(a, c, S, SS, red, 640, nullptr, nullptr, 0, nullptr, 0);
+      softmax_phase<false, true>(a, c, S, SS, red, 640, nullptr, nullptr, 0, nullptr, 0, qexp);
     else
-      softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0);
+      softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0, qexp);
     __syncthreads();
     group_sums(c, reinterpret_cast<const __half*>(S), 2 * SS, n_sg * kSGGroups, -5.0f, psum);
     cp_async_wait<0>();
@@ -703,7 +757,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
 //   buf   ST/32 key groups, then ST/160 + 2 ternary supergroups, at the end the output staging
 //   S     8 rows of SSP floats: scores, then the ternary-stream probabilities (binary16)
 //   Pprot 8 rows of (ST/32 + 1) * 32 + 8 binary16    Pres 8 rows of 136 binary16 (residual)
-//   map   ST destinations                            psum_t, psum_p, red
+//   map   ST destinations                            psum_t, psum_p, red, qexp
 // The protected groups are read from global memory as they are consumed.
 // ---------------------------------------------------------------------------------
 __host__ __device__ inline int stp_sg_max(int ST) { return ST / 160 + 2; }
@@ -717,7 +771,7 @@ constexpr int kPresStride = kR + 8;
 size_t decode_stp_smem_bytes(int ST) {
   const size_t buf = static_cast<size_t>(stp_sg_max(ST)) * kSGBytes;        // >= ST/32 key groups
   return buf + sizeof(float) * 8 * stp_row_floats(ST) + 16 * (stp_pg_max(ST) * 32 + 8) + 16 * kPresStride + 2 * ST +
-         sizeof(float) * (8 * stp_sg_max(ST) * kSGGroups + 8 * stp_pg_max(ST) + 16);
+         sizeof(float) * (8 * stp_sg_max(ST) * kSGGroups + 8 * stp_pg_max(ST) + 16 + 8);
 }
 
 template <typename T>
@@ -734,7 +788,9 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
   float* psum_t = reinterpret_cast<float*>(map + ST);
   float* psum_p = psum_t + 8 * stp_sg_max(ST) * kSGGroups;
   float* red = psum_p + 8 * stp_pg_max(ST);
+  int* qexp = reinterpret_cast<int*>(red + 16);
   const Split c = make_split(a, blockIdx.x);
+  query_exponents<T>(a, c, qexp);                          // visible after the barrier before the scores
   const CacheView& cv = a.cv;
   const int b = c.lb % cv.B;
   const uint32_t* ew = cv.e_words(b);
@@ -781,7 +837,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
 
   cp_async_wait<0>();
   __syncthreads();
-  score_phase<T>(a, n_chunks, c, buf, S, SS);
+  score_phase<T>(a, n_chunks, c, buf, S, SS, qexp);
   __syncthreads();
   {
     // the key groups are spent: the ternary supergroups take their place while the softmax runs
@@ -789,7 +845,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
     stage_async(buf, vsrc, n_sg * (kSGBytes / 16), c.tid);
     cp_async_commit();
   }
-  softmax_phase<true>(a, c, S, SS, red, 0, map, Pprot, PP, Pres, kPresStride);
+  softmax_phase<true>(a, c, S, SS, red, 0, map, Pprot, PP, Pres, kPresStride, qexp);
   __syncthreads();
   group_sums(c, reinterpret_cast<const __half*>(S), PT, n_sg * kSGGroups, -5.0f, psum_t);
   group_sums(c, Pprot, PP, n_pg, 1.0f, psum_p);

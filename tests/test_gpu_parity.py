@@ -181,6 +181,37 @@ def test_decode_parity_heavy_tailed_without_protection():
         assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
 
 
+@pytest.mark.parametrize("name,T,p,k_mul,q_mul", [
+    ("tiny", 300, 0.0, 100.0, 1.0),     # outlier channels reach +-6000: key scales near 2000 meet query entries near 40
+    ("tiny", 704, 0.25, 100.0, 1.0),
+    ("qwen", 480, 0.0, 10.0, 64.0),     # bfloat16; query entries of several hundred
+    ("tiny", 300, 0.0, 1.0, 2.0 ** -12),  # a tiny query: its binary16 image must not lose its bits
+])
+def test_large_keys_and_queries_stay_finite(monkeypatch, name, T, p, k_mul, q_mul):
+    """q_j * s_j would leave the binary16 range if the query went into the score operands as it
+    is; the kernels normalise each query head by a power of two, so the result stays an ordinary
+    number and still matches the oracle."""
+    from tests import helpers as Hm
+    make_kv, make_step = Hm.make_layer_kv, Hm.make_step_inputs
+
+    def big_kv(wl, layer, device="cpu", T=None, B=None):
+        K, V = make_kv(wl, layer, device, T=T, B=B)
+        return (K.float() * k_mul).clamp(-60000, 60000).to(K.dtype), V
+
+    def big_step(wl, layer, step, device="cpu", T=None, B=None):
+        q, k, v = make_step(wl, layer, step, device, T=T, B=B)
+        return (q.float() * q_mul).to(q.dtype), k, v
+
+    monkeypatch.setattr(Hm, "make_layer_kv", big_kv)
+    monkeypatch.setattr(Hm, "make_step_inputs", big_step)
+    pair = Pair(CONFIGS[name], T, B=1, L=1, p=p, max_new=3).prefill()
+    for _ in range(3):
+        out, ref = pair.decode()
+        assert np.isfinite(out).all()
+        assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
+    assert pair.cache.status() == 0
+
+
 def test_full_size_slabs_in_the_benchmark_launch_shape():
     """The benchmark's configuration (batched long video: T = 12544, batch 16, 640-token splits),
     two layers in one call; the oracle recomputes four sampled (layer, batch, KV head) slabs."""
