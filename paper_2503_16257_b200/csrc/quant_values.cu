@@ -78,14 +78,22 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
   const int n_rows = static_cast<int>(min(static_cast<int64_t>(kSGTokens), n_rest - u0));
   const int32_t* idx = sel.idx_rest ? sel.idx_rest + b * sel.stride_rest : nullptr;
   // ---- stage (rows past the end of the stream are zero: their trits come out 0)
-  for (int i = tid; i < kSGTokens * 16; i += 256) {
-    const int row = i >> 4, piece = i & 15;
-    uint8_t* dst = tile + row * kVRowBytes + piece * 16;
-    if (row < n_rows) {
-      const int64_t t = idx ? idx[u0 + row] : (u0 + row);
-      cp_async16_v(dst, reinterpret_cast<const uint8_t*>(base + t * src.stride_t) + piece * 16);
-    } else {
-      *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+  {
+    // thread = 16-byte piece (tid % 16) of rows tid / 16 + 16 k.  The stream positions of all its
+    // rows are fetched first, so that the gather list costs one memory latency, not one per row.
+    constexpr int kRowsPerThread = kSGTokens * 16 / 256;
+    const int row0 = tid >> 4, piece = tid & 15;
+    int64_t tok[kRowsPerThread];
+#pragma unroll
+    for (int k = 0; k < kRowsPerThread; ++k) {
+      const int row = row0 + 16 * k;
+      tok[k] = row < n_rows ? (idx ? static_cast<int64_t>(__ldg(idx + u0 + row)) : (u0 + row)) : -1;
+    }
+#pragma unroll
+    for (int k = 0; k < kRowsPerThread; ++k) {
+      uint8_t* dst = tile + (row0 + 16 * k) * kVRowBytes + piece * 16;
+      if (tok[k] >= 0) cp_async16_v(dst, reinterpret_cast<const uint8_t*>(base + tok[k] * src.stride_t) + piece * 16);
+      else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
     }
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
