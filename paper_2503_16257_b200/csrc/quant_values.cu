@@ -201,11 +201,66 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
 
 // ---------------------------------------------------------------------------------
 // 2-bit GQuant (Eq. 4) of one group of up to 32 protected tokens.  grid = (groups, slabs).
+//
+// code(v) = clamp(rint((v - z) / s), 0, 3) does not decrease with v, so it equals the number of
+// k in {1, 2, 3} with v >= t_k, t_k the smallest value of the input type whose code reaches k.
+// One thread per channel finds the three t_k with the literal formula (IEEE division included)
+// evaluated on a handful of candidates around z + (k - 1/2) s; the elements are then coded with
+// three comparisons each instead of a division each.
 // ---------------------------------------------------------------------------------
+template <typename T> struct Ordered16;     // 16-bit patterns of T <-> integers in value order
+template <> struct Ordered16<__half> {
+  static constexpr int kMin = 0x0400, kMax = 0xfbff;          // keys of -65504 and +65504
+  static __device__ __forceinline__ float value(int key) {
+    const uint16_t b = static_cast<uint16_t>(key ^ ((key & 0x8000) ? 0x8000 : 0xffff));
+    return __half2float(__ushort_as_half(b));
+  }
+  static __device__ __forceinline__ int key(float x) {
+    const uint16_t b = __half_as_ushort(__float2half_rn(x));
+    return b ^ ((b & 0x8000u) ? 0xffffu : 0x8000u);
+  }
+};
+template <> struct Ordered16<__nv_bfloat16> {
+  static constexpr int kMin = 0x0080, kMax = 0xff7f;          // keys of the largest finite magnitudes
+  static __device__ __forceinline__ float value(int key) {
+    const uint32_t b = static_cast<uint32_t>(key ^ ((key & 0x8000) ? 0x8000 : 0xffff));
+    return __uint_as_float(b << 16);
+  }
+  static __device__ __forceinline__ int key(float x) {
+    const uint16_t b = __bfloat16_as_ushort(__float2bfloat16_rn(x));
+    return b ^ ((b & 0x8000u) ? 0xffffu : 0x8000u);
+  }
+};
+
+// Smallest value of type T (as a float) whose Eq. 4 code with (s, z) is >= k; +infinity if none.
+template <typename T>
+__device__ __forceinline__ float code_threshold(float s, float z, int k) {
+  using O = Ordered16<T>;
+  if (!(s > 0.0f)) return INFINITY;                            // zero range: every code is 0
+  const float kf = static_cast<float>(k);
+  auto reaches = [&](int key) -> bool {
+    float q = rintf(__fdiv_rn(__fsub_rn(O::value(key), z), s));
+    q = fminf(fmaxf(q, 0.0f), 3.0f);
+    return q >= kf;
+  };
+  const int ck = min(max(O::key(fmaf(kf - 0.5f, s, z)), O::kMin), O::kMax);
+  int lo = max(ck - 4, O::kMin - 1), hi = min(ck + 4, O::kMax);   // invariant: code(lo) < k <= code(hi)
+  if (!reaches(hi)) {
+    lo = hi; hi = O::kMax;
+    if (!reaches(hi)) return INFINITY;
+  }
+  if (lo >= O::kMin && reaches(lo)) { hi = lo; lo = O::kMin - 1; }
+  while (hi - lo > 1) {                                        // at most 16 rounds
+    const int mid = (lo + hi) >> 1;
+    if (reaches(mid)) hi = mid; else lo = mid;
+  }
+  return O::value(hi);
+}
+
 template <typename T>
 __global__ void __launch_bounds__(128) v_protect_kernel(KSrc src, CacheView cv, int layer, SelView sel) {
   __shared__ __align__(16) uint16_t tile[kG * kD];
-  __shared__ uint16_t s_s[kD], s_z[kD];
+  __shared__ float s_thr[3][kD];
   const int slab = blockIdx.y;
   const int b = slab / cv.H_kv, h = slab % cv.H_kv;
   const T* base = reinterpret_cast<const T*>(src.ptr) + b * src.stride_b + h * src.stride_h;
@@ -230,25 +285,29 @@ __global__ void __launch_bounds__(128) v_protect_kernel(KSrc src, CacheView cv, 
       mn = fminf(mn, v); mx = fmaxf(mx, v);
     }
     const uint16_t sh = f2h_bits(__fdiv_rn(__fsub_rn(mx, mn), 3.0f)), zh = f2h_bits(mn);
-    s_s[c] = sh; s_z[c] = zh;
     reinterpret_cast<uint16_t*>(pg + kPG_S)[c] = sh;
     reinterpret_cast<uint16_t*>(pg + kPG_Z)[c] = zh;
+    const float s = h2f(sh), z = h2f(zh);
+#pragma unroll
+    for (int k = 1; k <= 3; ++k) s_thr[k - 1][c] = code_threshold<T>(s, z, k);
   }
   __syncthreads();
   for (int item = threadIdx.x; item < kG * 8; item += 128) {
     // item = word index ((kt * 4 + w) * 4 + r) * 8 + rho: 4 channels x 4 tokens
     const int rho = item & 7, r = (item >> 3) & 3, w = (item >> 5) & 3, kt = item >> 7;
+    const int c0 = 32 * w + 4 * rho;
+    float t1[4], t2[4], t3[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { t1[e] = s_thr[0][c0 + e]; t2[e] = s_thr[1][c0 + e]; t3[e] = s_thr[2][c0 + e]; }
     uint32_t word = 0;
 #pragma unroll
     for (int f = 0; f < 16; ++f) {
       const int e = f & 3, u = (f >> 2) & 1, hf = f >> 3;
-      const int j = 16 * kt + 8 * u + 2 * r + hf, c = 32 * w + 4 * rho + e;
+      const int j = 16 * kt + 8 * u + 2 * r + hf;
       if (j < n_rows) {
-        const float s = h2f(s_s[c]), z = h2f(s_z[c]);
-        const float v = Elem<T>::to_float(reinterpret_cast<const T*>(tile)[j * kD + c]);
-        float q = rintf(__fdiv_rn(__fsub_rn(v, z), s));
-        q = fminf(fmaxf(q, 0.0f), 3.0f);
-        word |= ((s == 0.0f) ? 0u : static_cast<uint32_t>(q)) << (2 * (4 * u + e) + 16 * hf);
+        const float v = Elem<T>::to_float(reinterpret_cast<const T*>(tile)[j * kD + c0 + e]);
+        const uint32_t code = static_cast<uint32_t>(v >= t1[e]) + static_cast<uint32_t>(v >= t2[e]) + static_cast<uint32_t>(v >= t3[e]);
+        word |= code << (2 * (4 * u + e) + 16 * hf);
       }
     }
     reinterpret_cast<uint32_t*>(pg)[item] = word;
