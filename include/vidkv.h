@@ -233,7 +233,12 @@ vidkv_status_t vidkv_quantize_values(vidkv_cache_t* handle, int32_t layer, const
  *   out    [n_layers, B, H_q,  D]  (out_dtype)   Softmax(q K^T * softmax_scale) V
  * softmax_scale <= 0 selects 1 / sqrt(D).  When a layer's residual reaches R tokens it
  * is quantized into a new 128-token chunk (own channel split; values by 1.58Quant) and
- * emptied.  All contiguous.  Returns CAPACITY when max_new_tokens would be exceeded. */
+ * emptied.  All contiguous.  Returns CAPACITY when max_new_tokens would be exceeded.
+ * Range: every query head is normalised by a power of two before it meets the stored
+ * binary16 scales, so finite inputs give finite outputs as long as the Eq. 5 scales of the
+ * spectrum stay below 16376 (normal-channel keys of magnitude up to a few thousand); the
+ * Eq. 4 scales may take any binary16 value, and a bfloat16 query may exceed the binary16
+ * range. */
 vidkv_status_t vidkv_decode_attention(vidkv_cache_t* handle, int32_t layer_begin, int32_t n_layers,
                                       const void* q, const void* k_new, const void* v_new, void* out,
                                       float softmax_scale, void* stream);
