@@ -21,7 +21,7 @@ __device__ __forceinline__ __half2 as_half2(uint32_t v) { return *reinterpret_ca
 //           chained in binary16 (exact, <= 242), and the byte code comes from a 243-entry table.
 // ---------------------------------------------------------------------------------
 constexpr int kSGTokens = kSGGroups * kG;   // 160
-constexpr int kVRowBytes = 288;             // 256 bytes of data + padding: rows two apart land 16 banks apart
+constexpr int kVRowBytes = 272;             // 256 bytes of data + padding: rows four apart land 16 banks apart
 
 template <typename T> struct Simd2;
 template <> struct Simd2<__half> {
@@ -165,7 +165,11 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
   // ---- pass 2: one word of the plane per thread and step
 #pragma unroll
   for (int wi = 0; wi < kG * kD / 4 / 256; ++wi) {
-    const int wd = tid + 256 * wi;
+    // bits 4 and 5 of the word index trade places: a warp then reads 16 words of each of two rows
+    // that lie four rows apart (conflict-free with the 272-byte row stride) and still writes
+    // whole 64-byte pieces of the plane
+    const int w0 = tid + 256 * wi;
+    const int wd = (w0 & ~0x30) | ((w0 & 0x10) << 1) | ((w0 & 0x20) >> 1);
     const int cp = 16 * ((wd >> 6) & 3) + 2 * ((wd >> 1) & 7) + (wd & 1);
     const int m = 8 * ((wd >> 9) & 1) + 4 * ((wd >> 8) & 1) + ((wd >> 4) & 3);
     uint32_t b0 = 0u, b1 = 0u;                        // binary16 pairs (even channel, odd channel) of tokens 2m, 2m+1
