@@ -212,6 +212,41 @@ def test_large_keys_and_queries_stay_finite(monkeypatch, name, T, p, k_mul, q_mu
     assert pair.cache.status() == 0
 
 
+def _degenerate(kind, K, V):
+    K, V = K.clone(), V.clone()
+    if kind == "zeros":                       # zero range everywhere: s = 0, every code 0
+        K.zero_(); V.zero_()
+    elif kind == "constant_channels":         # zero-range groups next to ordinary ones
+        K[..., 5] = 1.5; K[..., 77] = -2.0; V[..., 9] = 0.0; V[..., 100] = 3.0
+    elif kind == "huge":                      # near the end of the binary16 range
+        K = (K.float() * 6000).clamp(-60000, 60000).to(K.dtype); V = (V.float() * 6000).clamp(-60000, 60000).to(V.dtype)
+    elif kind == "tiny_values":               # subnormal binary16 (flushed to zero in bfloat16)
+        K = (K.float() * 1e-6).to(K.dtype); V = (V.float() * 1e-6).to(V.dtype)
+    elif kind == "equal_rows":                # every token the same: all ranges zero, nothing to rank
+        K[:, :, 1:] = K[:, :, :1]; V[:, :, 1:] = V[:, :, :1]
+    return K, V
+
+
+@pytest.mark.parametrize("kind", ["zeros", "constant_channels", "huge", "tiny_values", "equal_rows"])
+@pytest.mark.parametrize("name,T,p", [("tiny", 300, 0.0), ("tiny", 300, 0.2), ("qwen", 200, 0.2)])
+def test_degenerate_inputs(monkeypatch, kind, name, T, p):
+    """The degenerate cases of the method: zero-range groups (s = 0), constant channels, values at
+    both ends of the binary16 range, identical tokens.  Codes, metadata, dequantized tensors and
+    two decode steps against the oracle."""
+    from tests import helpers as Hm
+    make_kv = Hm.make_layer_kv
+    monkeypatch.setattr(Hm, "make_layer_kv",
+                        lambda wl, layer, device="cpu", T=None, B=None: _degenerate(kind, *make_kv(wl, layer, device, T=T, B=B)))
+    pair = Pair(CONFIGS[name], T, B=1, L=1, p=p, max_new=3).prefill()
+    _compare_prefill(pair)
+    _compare_dequant(pair)
+    for _ in range(2):
+        out, ref = pair.decode()
+        assert np.isfinite(out).all()
+        assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
+    assert pair.cache.status() == 0
+
+
 def test_full_size_slabs_in_the_benchmark_launch_shape():
     """The benchmark's configuration (batched long video: T = 12544, batch 16, 640-token splits),
     two layers in one call; the oracle recomputes four sampled (layer, batch, KV head) slabs."""
