@@ -755,22 +755,24 @@ __global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, i
 // into stream-ordered rows, zero wherever a staged stream position belongs to another split.
 // Shared memory for a split of ST tokens (160, 320 or 640):
 //   buf   ST/32 key groups, then ST/160 + 2 ternary supergroups, at the end the output staging
-//   S     8 rows of SSP floats: scores, then the ternary-stream probabilities (binary16)
-//   Pprot 8 rows of (ST/32 + 1) * 32 + 8 binary16    Pres 8 rows of 136 binary16 (residual)
+//   S     8 rows of SSP floats: scores, then the row's probabilities as binary16 in three pieces:
+//         [0, 160 n_sg) the staged ternary stream, then 32 n_pg entries of the protected stream,
+//         then the residual tokens.  The pieces hold the split's tokens plus the slack of their
+//         group alignment: at most ST + 349 + 62 + 2 entries.
 //   map   ST destinations                            psum_t, psum_p, red, qexp
 // The protected groups are read from global memory as they are consumed.
 // ---------------------------------------------------------------------------------
 __host__ __device__ inline int stp_sg_max(int ST) { return ST / 160 + 2; }
 __host__ __device__ inline int stp_pg_max(int ST) { return ST / 32 + 1; }
-__host__ __device__ inline int stp_row_floats(int ST) {       // a row must hold the scores and, later, the stream
-  const int need = stp_sg_max(ST) * 80 + 4;
-  return ST + 4 > need ? ST + 4 : need;
+__host__ __device__ inline int stp_row_floats(int ST) {       // a row must hold the scores and, later, the streams
+  const int scores = ST + 4;
+  const int streams = ((ST + 349 + 62 + 2 + 1) / 2 + 7) / 8 * 8 + 4;   // = 4 mod 8 floats: the 8 rows start in different banks
+  return scores > streams ? scores : streams;
 }
-constexpr int kPresStride = kR + 8;
 
 size_t decode_stp_smem_bytes(int ST) {
   const size_t buf = static_cast<size_t>(stp_sg_max(ST)) * kSGBytes;        // >= ST/32 key groups
-  return buf + sizeof(float) * 8 * stp_row_floats(ST) + 16 * (stp_pg_max(ST) * 32 + 8) + 16 * kPresStride + 2 * ST +
+  return buf + sizeof(float) * 8 * stp_row_floats(ST) + 2 * ST +
          sizeof(float) * (8 * stp_sg_max(ST) * kSGGroups + 8 * stp_pg_max(ST) + 16 + 8);
 }
 
@@ -779,12 +781,10 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
   extern __shared__ __align__(16) uint8_t smem_raw[];
   const int ST = a.split_tokens;
   const int SS = stp_row_floats(ST);
-  const int PT = 2 * SS, PP = stp_pg_max(ST) * 32 + 8;
+  const int PT = 2 * SS;                                   // row stride in binary16 entries
   uint8_t* buf = smem_raw;
   float* S = reinterpret_cast<float*>(buf + stp_sg_max(ST) * kSGBytes);
-  __half* Pprot = reinterpret_cast<__half*>(S + 8 * SS);
-  __half* Pres = Pprot + 8 * PP;
-  uint16_t* map = reinterpret_cast<uint16_t*>(Pres + 8 * kPresStride);
+  uint16_t* map = reinterpret_cast<uint16_t*>(S + 8 * SS);
   float* psum_t = reinterpret_cast<float*>(map + ST);
   float* psum_p = psum_t + 8 * stp_sg_max(ST) * kSGGroups;
   float* red = psum_p + 8 * stp_pg_max(ST);
@@ -819,8 +819,11 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
   const int n_pg = pp1 > pp0 ? static_cast<int>((pp1 - 1) / kG - pgA + 1) : 0;
   const int64_t Pbase = pgA * kG;
   const int64_t tg_total = (n_rest + kG - 1) / kG + (kR / kG) * a.st.n_flush;   // ternary groups that exist
+  // the protected and the residual probabilities follow the staged ternary stream in each row of S
+  __half* Pprot = reinterpret_cast<__half*>(S) + n_sg * (kSGGroups * kG);
+  __half* Pres = Pprot + n_pg * kG;
 
-  // ---- destinations of the quantized tokens, cleared protected rows
+  // ---- destinations of the quantized tokens
   for (int i = c.tid; i < c.nq; i += kThreads) {
     const int64_t t = c.t0 + i;
     uint32_t d;
@@ -833,7 +836,6 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
     }
     map[i] = static_cast<uint16_t>(d);
   }
-  for (int i = c.tid; i < PP; i += kThreads) reinterpret_cast<uint4*>(Pprot)[i] = make_uint4(0u, 0u, 0u, 0u);
 
   cp_async_wait<0>();
   __syncthreads();
@@ -845,10 +847,10 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
     stage_async(buf, vsrc, n_sg * (kSGBytes / 16), c.tid);
     cp_async_commit();
   }
-  softmax_phase<true>(a, c, S, SS, red, 0, map, Pprot, PP, Pres, kPresStride, qexp);
+  softmax_phase<true>(a, c, S, SS, red, 0, map, Pprot, PT, Pres, PT, qexp);
   __syncthreads();
   group_sums(c, reinterpret_cast<const __half*>(S), PT, n_sg * kSGGroups, -5.0f, psum_t);
-  group_sums(c, Pprot, PP, n_pg, 1.0f, psum_p);
+  group_sums(c, Pprot, PT, n_pg, 1.0f, psum_p);
   cp_async_wait<0>();
   __syncthreads();
 
@@ -860,7 +862,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
   // ---- protected stream: 2-bit codes (Eq. 4) as 4 + code, then s * (acc - 4 sum p) + z * sum p
   if (n_pg > 0) {
     const int warp = c.warp, hd = c.hd, r = c.r;
-    const uint8_t* prow = reinterpret_cast<const uint8_t*>(Pprot + hd * PP);
+    const uint8_t* prow = reinterpret_cast<const uint8_t*>(Pprot + hd * PT);
     const uint8_t* gbase = c.slab_ptr + cv.prot_offset + pgA * kPGBytes;
     const int w_off = (((warp * 4) + r) * 8 + hd) * 4, m_off = (32 * warp + 4 * hd) * 2;
     // operands of the group being consumed are loaded one group ahead
@@ -915,7 +917,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
   }
   __syncthreads();                                       // the output staging reuses buf
   if (c.t1 > c.T_qt)
-    residual_pv<T>(a, c, reinterpret_cast<float*>(buf), Pres, kPresStride,
+    residual_pv<T>(a, c, reinterpret_cast<float*>(buf), Pres, PT,
                    -static_cast<int>(max(c.t0, c.T_qt) - c.T_qt), tot);
   write_partial(a, c, blockIdx.x, reinterpret_cast<float*>(buf), red, tot);
 }
