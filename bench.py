@@ -32,7 +32,7 @@ FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used if ME
 # ncu captures summarised in profiles/decode_mma_kernel_batched_4layers.txt (p = 0) and
 # profiles/decode_stp_kernel_batched_4layers_p02.txt (p > 0): a 4-layer cut of the batched workload,
 # scaled to the launch by the token-heads it processes (traffic is proportional to them).
-NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = {"decode_mma_kernel": 74.95, "decode_stp_kernel": 77.70}
+NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = {"decode_stream_kernel": None, "decode_stp_kernel": None}
 
 
 def algorithmic_decode_bytes(B, L, H_kv, H_q, T_q0, n_flush, n_res, n_prot, elem=2):
@@ -355,7 +355,7 @@ def main():
     q_tokens = n_caches * B * T * L
     kern_bytes = dec_bytes / steps_dec
     kern_gbs = kern_bytes / (kern_avg_ms * 1e-3) / 1e9
-    kernel_name = "decode_stp_kernel" if n_prot > 0 else "decode_mma_kernel"
+    kernel_name = "decode_stp_kernel" if n_prot > 0 else "decode_stream_kernel"
     traffic = NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD.get(kernel_name)
     if traffic is not None:
         traffic = traffic * B * L * H * (T - T % 32)

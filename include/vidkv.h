@@ -283,8 +283,27 @@ vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const void* cache
                                     int32_t layer_begin, int32_t n_layers, const void* q, void* out,
                                     float softmax_scale, void* stream);
 
+/* Test hooks (no counterpart in the paper; the results of a decode call do not depend on them
+ * beyond floating-point summation order).  A decode call is cut into work in one of two ways
+ * (Algorithm 1 "Decoding" leaves the evaluation order of Eq. 3 open):
+ *   - no protected tokens: the quantized tokens of all slabs of the call form one sequence of
+ *     160-token units; every warp of the launch walks a run of `run_units` consecutive units;
+ *   - protected tokens: one thread block per (slab, split of `split_tokens` tokens).
+ * vidkv_debug_set_decode_plan forces split_tokens (160, 320 or 640) and / or run_units (>= 1) for
+ * later vidkv_decode_attention calls on this handle; 0 leaves the choice to the library.  A forced
+ * plan that needs more partial records than the workspace holds makes the decode call return
+ * VIDKV_ERR_CAPACITY.
+ * vidkv_debug_decode_plan (host only) reports the plan for given token counts on a device with
+ * sm_count multiprocessors: plan_out[10] = { stream kernel? , split_tokens, n_splits,
+ * units_per_slab, run_units, n_runs, records per slab, records needed, records the workspace of
+ * `cfg` holds, chunk-table entries }. */
+vidkv_status_t vidkv_debug_set_decode_plan(vidkv_cache_t* handle, int32_t split_tokens, int32_t run_units);
+vidkv_status_t vidkv_debug_decode_plan(const vidkv_config_t* cfg, int64_t n_prefill_quantized, int64_t n_flushed_chunks,
+                                       int32_t n_residual, int64_t n_protected, int32_t n_layers, int32_t sm_count,
+                                       int32_t split_tokens, int32_t run_units, int64_t* plan_out);
+
 /* Profiling aid: record the two CUDA events (cudaEvent_t passed as void*) immediately before
- * and after the split-KV attention kernel of every later vidkv_decode_attention call on this
+ * and after the attention kernel (stream or split kernel) of every later vidkv_decode_attention call on this
  * handle; NULL, NULL switches it off.  The events are the caller's. */
 vidkv_status_t vidkv_set_profile_events(vidkv_cache_t* handle, void* ev_begin, void* ev_end);
 

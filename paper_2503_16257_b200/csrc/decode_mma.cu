@@ -29,158 +29,11 @@
 // softmax pass turns them into binary16 probabilities in place, phase 2 (warps split the channels)
 // accumulates P V.  With protected tokens the probabilities are scattered into stream order and
 // the protected 2-bit groups are read from global memory as they are consumed.
-#include "common.cuh"
-#include "kernels.cuh"
+#include "decode_common.cuh"
 
 namespace vidkv {
 
 namespace {
-
-constexpr int kPrepWords = 24;     // 32-bit words per lane per (slab, chunk)
-constexpr int kThreads = 128;
-
-__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                        uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// d = a b + c with c given separately (no copy into the accumulator beforehand)
-__device__ __forceinline__ void mma_f16_c(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                          uint32_t b1, float c0, float c1, float c2, float c3) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
-      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c0), "f"(c1), "f"(c2), "f"(c3));
-}
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// q . k with the operands in the cache's element type (rows 8-15 of A unused)
-template <typename T> __device__ __forceinline__ void mma_in(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1);
-template <> __device__ __forceinline__ void mma_in<__half>(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  mma_f16(d, a0, 0u, a2, 0u, b0, b1);
-}
-template <> __device__ __forceinline__ void mma_in<__nv_bfloat16>(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0,
-                                                                  uint32_t b1) {
-  mma_bf16(d, a0, 0u, a2, 0u, b0, b1);
-}
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-  const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
-}
-// Copy n16 16-byte pieces from global to shared memory, pieces interleaved over the CTA's threads;
-// unrolled by four so that the offsets are immediates.
-__device__ __forceinline__ void stage_async(uint8_t* dst, const uint8_t* src, int n16, int tid) {
-  constexpr int kStep = 128 * 16;
-  uint8_t* d = dst + tid * 16;
-  const uint8_t* s = src + tid * 16;
-  int i = tid;
-  for (; i + 3 * 128 < n16; i += 4 * 128, d += 4 * kStep, s += 4 * kStep) {
-    cp_async16(d, s);
-    cp_async16(d + kStep, s + kStep);
-    cp_async16(d + 2 * kStep, s + 2 * kStep);
-    cp_async16(d + 3 * kStep, s + 3 * kStep);
-  }
-  for (; i < n16; i += 128, d += kStep, s += kStep) cp_async16(d, s);
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ uint32_t hmul2_u(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-// a * b + c on two binary16 lanes (one rounding)
-__device__ __forceinline__ uint32_t hfma2_u(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-// a * b - c on two binary16 lanes (one rounding)
-__device__ __forceinline__ uint32_t hfms2_u(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("{ .reg .b32 n; neg.f16x2 n, %3; fma.rn.f16x2 %0, %1, %2, n; }" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
-  const __half2 h = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&h);
-}
-// (x & m) | c and (x & m) ^ c as one three-input logic instruction
-__device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t m, uint32_t c) {
-  uint32_t d;
-  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "r"(m), "r"(c));
-  return d;
-}
-__device__ __forceinline__ uint32_t and_xor(uint32_t x, uint32_t m, uint32_t c) {
-  uint32_t d;
-  asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(x), "r"(m), "r"(c));
-  return d;
-}
-// Bit patterns of the code expansion.  They live in constant memory rather than in the
-// instruction stream so that mask and pattern both reach the logic instruction as register
-// operands (an instruction encodes one immediate at most).
-__constant__ uint32_t kExpand[4] = {0x03000300u,   // two-bit field at mantissa bits 8-9 of each binary16 lane
-                                    0x44004400u,   // 4.0 in each lane
-                                    0x80008000u,   // the sign bits
-                                    0xbc00bc00u};  // -1.0 in each lane
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-  uint32_t d;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-  return d;
-}
-
-// 2^k as a float, |k| <= 126
-__device__ __forceinline__ float pow2i(int k) { return __uint_as_float(static_cast<uint32_t>(127 + k) << 23); }
-
-// Query normalisation.  The score operands q_j s_j and Q_f s_f are binary16 numbers, so a large
-// query entry times a large key scale would overflow although the score itself is an ordinary
-// float.  Every query head is therefore multiplied by the power of two 2^(-e - kQShift), e =
-// floor(log2(max_c |q_c|)), which puts its largest entry into [1/8, 1/4): no product of a scaled
-// entry (or of a spectrum coefficient, at most 16 times the largest entry) with a binary16 scale
-// below 16376 leaves the binary16 range.  Scores are linear in q, so the softmax multiplies by the
-// inverse power of two; both factors are exact.  head_exponent returns e (0 for a head that is all
-// zero or holds no finite maximum); the NSUB lanes sub = 0..NSUB-1 share the 128 entries of the row,
-// and all 32 lanes of the warp must call it.
-constexpr int kQShift = 3;
-template <typename T, int NSUB>
-__device__ __forceinline__ int head_exponent(const T* qrow, int sub, bool live) {
-  float m = 0.0f;
-  if (live) {
-    const uint2* p = reinterpret_cast<const uint2*>(qrow + sub * (kD / NSUB));
-#pragma unroll
-    for (int i = 0; i < kD / NSUB / 4; ++i) {
-      const uint2 v = __ldg(p + i);
-      const float2 a = Elem<T>::to_float2(v.x), b = Elem<T>::to_float2(v.y);
-      m = fmaxf(m, fmaxf(fmaxf(fabsf(a.x), fabsf(a.y)), fmaxf(fabsf(b.x), fabsf(b.y))));
-    }
-  }
-#pragma unroll
-  for (int o = NSUB / 2; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  if (!(m > 0.0f) || m > 3.0e38f) return 0;
-  const int e = static_cast<int>(__float_as_uint(m) >> 23) - 127;
-  return max(-100, min(100, e));
-}
-
 }  // namespace
 
 size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks) {
@@ -194,6 +47,8 @@ size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks) {
 //   words  8..15  leading binary16 part of the transformed query Q at the spectrum
 //                 columns (16 r + 2 i, 16 r + 2 i + 1)
 //   words 16..23  binary16 remainder Q - leading part
+//   word  24      float: softmax scale * log2 e * 2^(e + kQShift), which turns a score of this
+//                 normalised query into a base-2 logit
 // for head lane / 4 (zero when that head does not exist) and r = lane % 4, all of the query
 // normalised by its head's power of two (head_exponent).
 // Q_f = sum_c q_c W[c, f] with W the weights with which spectrum column f enters channel c of
@@ -215,7 +70,8 @@ __global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int
                         static_cast<int64_t>(chunk) * kChunkBytes;
   const T* qrow = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(lb) * cv.H_q + h * rep + hd) * kD;
   const bool live = hd < rep;
-  const float qf = pow2i(-head_exponent<T, 4>(qrow, r, live) - kQShift);   // normalised query, see head_exponent
+  const int qe = head_exponent<T, 4>(qrow, r, live);
+  const float qf = pow2i(-qe - kQShift);                                   // normalised query, see head_exponent
   auto q_at = [&](int c) -> float { return live ? Elem<T>::to_float(qrow[c]) * qf : 0.0f; };
   if (chunk == 0 && a.append_row >= 0) {
     // Algorithm 1, Decoding: the step's new key / value row joins the residual (lanes 0-15 copy
@@ -265,6 +121,8 @@ __global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int
     out[(8 + nt) * 32] = pack_half2(__half2float(h0), __half2float(h1));
     out[(16 + nt) * 32] = pack_half2(x0 - __half2float(h0), x1 - __half2float(h1));
   }
+  // factor that turns a score in the normalised units into a base-2 logit
+  out[24 * 32] = __float_as_uint(a.scale * 1.4426950408889634f * pow2i(qe + kQShift));
 }
 
 // ---------------------------------------------------------------------------------
@@ -290,8 +148,8 @@ __device__ __forceinline__ Split make_split(const DecodeArgs& a, int split) {
   c.T_q0 = a.st.T_q0;
   c.T_qt = c.T_q0 + a.st.n_flush * kR;
   const int64_t T_tot = c.T_qt + a.st.n_res;
-  c.t0 = static_cast<int64_t>(c.split) * a.split_tokens;
-  c.t1 = min(c.t0 + a.split_tokens, T_tot);
+  c.t0 = static_cast<int64_t>(c.split) * a.plan.split_tokens;
+  c.t1 = min(c.t0 + a.plan.split_tokens, T_tot);
   c.tq1 = max(min(c.t1, c.T_qt), c.t0);
   c.n_loc = static_cast<int>(c.t1 - c.t0);
   c.nq = static_cast<int>(c.tq1 - c.t0);
@@ -542,11 +400,10 @@ __device__ __forceinline__ void residual_pv(const DecodeArgs& a, const Split& c,
   __syncthreads();
 }
 
-// Write one partial record per query head: (max, sum, unnormalised out[128]).  ml[h] = scaled
-// maximum, ml[8 + h] = sum of the probabilities; O is the staging buffer (free, 4 KB).
+// Write one partial record per query head: (max, sum, unnormalised out[128]).  ml[h] = maximum
+// (base-2 logit), ml[8 + h] = sum of the probabilities; O is the staging buffer (free, 4 KB).
 __device__ __forceinline__ void write_partial(const DecodeArgs& a, const Split& c, int part, float* O, const float* ml,
                                               const float (&tot)[2][4]) {
-  const CacheView& cv = a.cv;
   const int c0 = 32 * c.warp + 4 * c.hd, r = c.r;
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
@@ -560,8 +417,7 @@ __device__ __forceinline__ void write_partial(const DecodeArgs& a, const Split& 
 #pragma unroll
   for (int k = 0; k < kMaxRep; ++k) {
     if (k < c.rep) {
-      const int64_t qh = static_cast<int64_t>(c.lb) * cv.H_q + c.h * c.rep + k;
-      float* pr = a.partials + (qh * a.n_parts + part) * 130;
+      float* pr = a.partials + ((static_cast<int64_t>(c.slab) * a.plan.parts_stride + part) * kMaxRep + k) * kRecordFloats;
       pr[2 + ch] = O[k * kD + ch];
       if (ch == 0) { pr[0] = ml[k]; pr[1] = ml[8 + k]; }
     }
@@ -574,7 +430,7 @@ __device__ __forceinline__ void write_partial(const DecodeArgs& a, const Split& 
 // cleared once its scores are in registers and becomes the ternary-stream row: quantized
 // tokens [0, nq) go to their stream position through `map` (bit 15 = protected stream, row of
 // Pprot), residual tokens [nq, n_loc) to Pres[row][i - nq].
-// red[row] = scaled row maximum, red[8 + row] = sum of the probabilities.  The scores arrive in
+// red[row] = row maximum as a base-2 logit (score * scale * log2 e), red[8 + row] = sum of the probabilities.  The scores arrive in
 // units of the head's query normalisation; the inverse power of two joins the softmax scale.
 template <bool STP, bool FULL = false>     // FULL: the split holds exactly 640 tokens, no bound checks
 __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& c, float* S, int SS, float* red,
@@ -634,7 +490,7 @@ __device__ __forceinline__ void softmax_phase(const DecodeArgs& a, const Split& 
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-    if (lane == 0) { red[row_h] = m * scale_h; red[8 + row_h] = l; }
+    if (lane == 0) { red[row_h] = m * sl2; red[8 + row_h] = l; }
   }
 }
 
@@ -657,94 +513,6 @@ __device__ __forceinline__ void group_sums(const Split& c, const __half* P, int 
     }
     out[i] = factor * (s0 + s1);
   }
-}
-
-// ---------------------------------------------------------------------------------
-// Caches without protected tokens.  Shared memory for a split of ST tokens (a multiple of 160):
-//   kbuf  ST/32 key groups           (reused for the output staging after phase 1)
-//   vbuf  ST/160 ternary supergroups
-//   S     8 rows of ST + 4 floats: scores, then binary16 probabilities in place
-//   psum  [ST/32][8]  -5 * (sum of the rounded probabilities of the group)
-//   red   [16]        row maxima and sums
-//   qexp  [8]         exponents of the query normalisation (head_exponent)
-// ---------------------------------------------------------------------------------
-size_t decode_mma_smem_bytes(int ST) {
-  return static_cast<size_t>(ST / 32) * kKGroupBytes + sizeof(float) * (8 * (ST + 4) + 8 * (ST / 32) + 16 + 8);
-}
-
-template <typename T>
-__global__ void __launch_bounds__(kThreads, 4) decode_mma_kernel(DecodeArgs a, int n_chunks) {
-  extern __shared__ __align__(16) uint8_t smem_raw[];
-  const int ST = a.split_tokens;
-  const int SS = ST + 4;                                  // row stride of S in floats
-  uint8_t* kbuf = smem_raw;                               // keys, then values (ST/160 * 5376 <= ST/32 * 1152)
-  uint8_t* vbuf = kbuf;
-  float* S = reinterpret_cast<float*>(kbuf + (ST / 32) * kKGroupBytes);
-  float* psum = S + 8 * SS;
-  float* red = psum + 8 * (ST / 32);
-  int* qexp = reinterpret_cast<int*>(red + 16);
-  const CacheView& cv = a.cv;
-  // One CTA walks a.splits_per_cta consecutive splits of its slab and keeps a running
-  // (max, sum, out) per head, rescaled as in a streaming softmax; one record leaves at the end.
-  float TOT[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
-  float Mr[2] = {-INFINITY, -INFINITY}, Lr[2] = {0.0f, 0.0f};
-  Split c = make_split(a, blockIdx.x * a.splits_per_cta);
-  query_exponents<T>(a, c, qexp);                           // visible after the first barrier below
-#pragma unroll 1
-  for (int it = 0; it < a.splits_per_cta; ++it) {
-    const int split = blockIdx.x * a.splits_per_cta + it;
-    if (split >= a.n_splits) break;
-    if (it > 0) c = make_split(a, split);
-    const int n_sg = (c.n_kg + kSGGroups - 1) / kSGGroups;   // ternary groups = key groups here
-    {
-      const uint8_t* ksrc = c.slab_ptr + cv.kgroup_offset + c.gk0 * kKGroupBytes;
-      stage_async(kbuf, ksrc, c.n_kg * (kKGroupBytes / 16), c.tid);
-      cp_async_commit();
-    }
-    cp_async_wait<0>();
-    __syncthreads();
-    score_phase<T>(a, n_chunks, c, kbuf, S, SS, qexp);
-    __syncthreads();
-    {
-      // the key groups are spent: the ternary supergroups take their place while the softmax runs
-      const uint8_t* vsrc = c.slab_ptr + cv.tern_offset + (c.t0 / (kG * kSGGroups)) * kSGBytes;
-      stage_async(vbuf, vsrc, n_sg * (kSGBytes / 16), c.tid);
-      cp_async_commit();
-    }
-    if (c.n_loc == 640)
-      softmax_phase<false, true>(a, c, S, SS, red, 640, nullptr, nullptr, 0, nullptr, 0, qexp);
-    else
-      softmax_phase<false>(a, c, S, SS, red, max(n_sg * kSGGroups * kG, (c.n_loc + 1) & ~1), nullptr, nullptr, 0, nullptr, 0, qexp);
-    __syncthreads();
-    group_sums(c, reinterpret_cast<const __half*>(S), 2 * SS, n_sg * kSGGroups, -5.0f, psum);
-    cp_async_wait<0>();
-    __syncthreads();
-    float tot[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
-    ternary_phase<false>(c, vbuf, n_sg, 0, c.n_kg, reinterpret_cast<const uint8_t*>(S + c.hd * SS), psum, tot);
-    __syncthreads();                                        // the staging buffer is the key / value buffer
-    if (c.t1 > c.T_qt)
-      residual_pv<T>(a, c, reinterpret_cast<float*>(kbuf), reinterpret_cast<const __half*>(S), 2 * SS,
-                     static_cast<int>(c.T_qt - c.t0), tot);
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const float m_i = red[2 * c.r + j], l_i = red[8 + 2 * c.r + j];
-      const float m_new = fmaxf(Mr[j], m_i);
-      const float so = __expf(Mr[j] - m_new), si = __expf(m_i - m_new);
-      Lr[j] = Lr[j] * so + l_i * si;
-#pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        TOT[i][j] = TOT[i][j] * so + tot[i][j] * si;
-        TOT[i][2 + j] = TOT[i][2 + j] * so + tot[i][2 + j] * si;
-      }
-      Mr[j] = m_new;
-    }
-    __syncthreads();                                        // red, S and the buffers are rewritten next
-  }
-  if (c.warp == 0 && c.hd == 0) {
-    red[2 * c.r] = Mr[0]; red[2 * c.r + 1] = Mr[1];
-    red[8 + 2 * c.r] = Lr[0]; red[8 + 2 * c.r + 1] = Lr[1];
-  }
-  write_partial(a, c, blockIdx.x, reinterpret_cast<float*>(kbuf), red, TOT);
 }
 
 // ---------------------------------------------------------------------------------
@@ -779,7 +547,7 @@ size_t decode_stp_smem_bytes(int ST) {
 template <typename T>
 __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, int n_chunks) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  const int ST = a.split_tokens;
+  const int ST = a.plan.split_tokens;
   const int SS = stp_row_floats(ST);
   const int PT = 2 * SS;                                   // row stride in binary16 entries
   uint8_t* buf = smem_raw;
@@ -922,48 +690,36 @@ __global__ void __launch_bounds__(kThreads, 4) decode_stp_kernel(DecodeArgs a, i
   write_partial(a, c, blockIdx.x, reinterpret_cast<float*>(buf), red, tot);
 }
 
-cudaError_t launch_decode_mma(const DecodeArgs& a_in, cudaStream_t stream) {
-  DecodeArgs a = a_in;
+cudaError_t launch_decode_prep(DecodeArgs& a, cudaStream_t stream) {
   a.dft = nullptr;
   const int n_slabs = a.n_layers * a.cv.B * a.cv.H_kv;
-  const int n_chunks = static_cast<int>((a.st.T_q0 > 0 ? 1 : 0) + a.st.n_flush);
-  const bool stp = a.n_prot > 0;
-  const size_t smem = stp ? decode_stp_smem_bytes(a.split_tokens) : decode_mma_smem_bytes(a.split_tokens);
-  static size_t attr_smem_dev[64][2] = {};   // function attributes are per device
+  const int n_chunks = a.plan.n_chunks;
+  if (n_chunks < 1) return cudaSuccess;
+  cudaError_t e;
+  if ((e = dft_fragments(&a.dft, stream))) return e;
+  const int n_items = n_slabs * n_chunks;
+  const int pgrid = (n_items + kThreads / 32 - 1) / (kThreads / 32);
+  if (a.in_dtype == VIDKV_F16) decode_prep_kernel<__half><<<pgrid, kThreads, 0, stream>>>(a, n_chunks, n_items);
+  else decode_prep_kernel<__nv_bfloat16><<<pgrid, kThreads, 0, stream>>>(a, n_chunks, n_items);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode_stp(const DecodeArgs& a, cudaStream_t stream) {
+  const int n_slabs = a.n_layers * a.cv.B * a.cv.H_kv;
+  const size_t smem = decode_stp_smem_bytes(a.plan.split_tokens);
+  static size_t attr_smem_dev[64] = {};   // function attributes are per device
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  size_t* attr_smem = attr_smem_dev[dev];
-  if (smem > attr_smem[stp]) {
+  if (smem > attr_smem_dev[dev]) {
     cudaError_t e;
-    if (stp) {
-      if ((e = cudaFuncSetAttribute(decode_stp_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-      if ((e = cudaFuncSetAttribute(decode_stp_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    } else {
-      if ((e = cudaFuncSetAttribute(decode_mma_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-      if ((e = cudaFuncSetAttribute(decode_mma_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
-    }
-    attr_smem[stp] = smem;
+    if ((e = cudaFuncSetAttribute(decode_stp_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    if ((e = cudaFuncSetAttribute(decode_stp_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem))) return e;
+    attr_smem_dev[dev] = smem;
   }
-  const int chunk_stride = n_chunks > 0 ? n_chunks : 1;
-  if (n_chunks > 0) {
-    cudaError_t e;
-    if ((e = dft_fragments(&a.dft, stream))) return e;
-    const int n_items = n_slabs * n_chunks;
-    const int pgrid = (n_items + kThreads / 32 - 1) / (kThreads / 32);
-    if (a.in_dtype == VIDKV_F16) decode_prep_kernel<__half><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride, n_items);
-    else decode_prep_kernel<__nv_bfloat16><<<pgrid, kThreads, 0, stream>>>(a, chunk_stride, n_items);
-    count_launches(1);
-  }
-  const dim3 grid(a.n_parts, n_slabs);
-  if (a.ev_begin) cudaEventRecord(a.ev_begin, stream);
-  if (stp) {
-    if (a.in_dtype == VIDKV_F16) decode_stp_kernel<__half><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
-    else decode_stp_kernel<__nv_bfloat16><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
-  } else {
-    if (a.in_dtype == VIDKV_F16) decode_mma_kernel<__half><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
-    else decode_mma_kernel<__nv_bfloat16><<<grid, kThreads, smem, stream>>>(a, chunk_stride);
-  }
-  if (a.ev_end) cudaEventRecord(a.ev_end, stream);
+  const dim3 grid(a.plan.n_splits, n_slabs);
+  if (a.in_dtype == VIDKV_F16) decode_stp_kernel<__half><<<grid, kThreads, smem, stream>>>(a, a.plan.n_chunks);
+  else decode_stp_kernel<__nv_bfloat16><<<grid, kThreads, smem, stream>>>(a, a.plan.n_chunks);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -1,0 +1,451 @@
+// Decode attention over the packed cache for caches without protected tokens (Algorithm 1
+// "Decoding", Eq. 3): the stream kernel.
+//
+// The quantized tokens of all slabs of a call form one sequence of 160-token units (five
+// 32-token key groups and the ternary supergroup that holds the same tokens' values).  Every
+// warp of the launch owns a contiguous run of units and works through it alone, the way a
+// streaming softmax does:
+//   1. the unit's key groups arrive in the warp's key buffer by one bulk copy
+//      (cp.async.bulk + mbarrier); the scores q . K' of its 160 tokens come out of
+//      mma.sync.m16n8k16 with rows = query heads (exact binary16 pair hi + lo of q_j s_j),
+//      columns = tokens, the codes expanded in registers as the B operand -- the same
+//      arithmetic as in decode_mma.cu;
+//   2. the accumulator fragment of that product (head = lane / 4, tokens 2 r, 2 r + 1) is
+//      exactly the B fragment of the next one, so the probabilities 2^(logit - running maximum)
+//      stay in registers as binary16 pairs; the running maximum only moves (and the
+//      accumulated output is only rescaled) when a unit's maximum exceeds it by more than
+//      kStaleLog2, so probabilities reach 2^kStaleLog2 at most;
+//   3. the unit's ternary supergroup (second bulk copy, in flight during step 1) is peeled digit
+//      by digit into 5 + trit, multiplied with the probabilities into per-group accumulators
+//      that start at -5 sum p (the sums come from a product with a constant matrix, which also
+//      yields the softmax denominator), and the per-(group, channel) scales fold the group
+//      accumulators into the warp's running output for all 128 channels x 8 heads.
+// While a unit is being worked on, the next unit's keys and values are already on their way
+// into the two buffers (a buffer is refilled as soon as its reader is done).  A warp leaves one
+// partial record (maximum, sum, out[128]) per query head for every slab its run touches; the
+// merge kernel combines them and attends to the FP16 / BF16 residual.
+//
+// Nothing is shared between warps: no block-wide barrier, no shared score matrix.
+#include "decode_common.cuh"
+
+namespace vidkv {
+
+namespace {
+
+constexpr int kKBufBytes = kSGGroups * kKGroupBytes;   // 5760: the key groups of one unit
+constexpr int kVBufBytes = kSGBytes;                   // 5376: its ternary supergroup
+constexpr int kTotBytes = 4 * 2 * 32 * 16;             // 4096: the warp's running output (128 channels x 8 heads, float)
+constexpr int kWarpBufBytes = kKBufBytes + kVBufBytes + kTotBytes;   // 15232 per warp
+constexpr uint32_t kWaitLimit = 1u << 16;              // mbarrier polls before a warp gives up
+constexpr float kStaleLog2 = 6.0f;                     // the running maximum may lag a unit's maximum by this much
+constexpr uint32_t kMinus5 = 0xc500c500u;              // binary16 pair (-5.0, -5.0)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+// One bulk copy global -> shared of `bytes` (multiple of 16, both addresses 16-byte aligned),
+// completion counted on `bar`.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  const uint32_t b = smem_u32(bar), d = smem_u32(dst);
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(d),
+               "l"(src), "r"(bytes), "r"(b)
+               : "memory");
+}
+// Bounded wait for the phase with the given parity; false if it never completed.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t b = smem_u32(bar);
+  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(b), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+// Per-lane state of the running softmax of one slab (the running output itself is in shared memory).
+struct Running {
+  float l[2];           // sums of the probabilities of heads 2 r, 2 r + 1
+  float m;              // running maximum (base-2 logit) of head hd
+};
+
+// Scores of one 32-token key group: sc[nt][0..1] = q . K' of head hd and tokens 8 nt + 2 r, + 1,
+// in the units of the normalised query.
+__device__ __forceinline__ void score_group(const uint8_t* kg, int lane, int hd, int r, const uint32_t (&qa)[8],
+                                            const uint32_t (&qha)[8], const uint32_t (&qhb)[8], uint32_t m_field,
+                                            uint32_t c_four, uint32_t m_sign, uint32_t c_neg1, float (&sc)[4][2]) {
+  uint32_t s2[8], z2[8], s1[8];
+  {
+    const uint4 x0 = *reinterpret_cast<const uint4*>(kg + kKG_S2 + 32 * r);
+    const uint4 x1 = *reinterpret_cast<const uint4*>(kg + kKG_S2 + 32 * r + 16);
+    s2[0] = x0.x; s2[1] = x0.y; s2[2] = x0.z; s2[3] = x0.w; s2[4] = x1.x; s2[5] = x1.y; s2[6] = x1.z; s2[7] = x1.w;
+    const uint8_t* zs = kg + ((hd & 1) ? kKG_S2 : kKG_Z2) + 32 * r;   // B operand of the constants: z for even columns, s for odd
+    const uint4 y0 = *reinterpret_cast<const uint4*>(zs);
+    const uint4 y1 = *reinterpret_cast<const uint4*>(zs + 16);
+    z2[0] = y0.x; z2[1] = y0.y; z2[2] = y0.z; z2[3] = y0.w; z2[4] = y1.x; z2[5] = y1.y; z2[6] = y1.z; z2[7] = y1.w;
+    const uint4 w0 = *reinterpret_cast<const uint4*>(kg + kKG_S1 + 32 * r);
+    const uint4 w1 = *reinterpret_cast<const uint4*>(kg + kKG_S1 + 32 * r + 16);
+    s1[0] = w0.x; s1[1] = w0.y; s1[2] = w0.z; s1[3] = w0.w; s1[4] = w1.x; s1[5] = w1.y; s1[6] = w1.z; s1[7] = w1.w;
+  }
+  // constants of the group: column 2 r of the result = sum q z, column 2 r + 1 = sum q s
+  float cst;
+  {
+    float cz[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) mma_f16(cz, qa[2 * ks], 0u, qa[2 * ks + 1], 0u, z2[2 * ks], z2[2 * ks + 1]);
+    cst = cz[0] - 4.0f * cz[1];
+  }
+  const uint4 c2 = *reinterpret_cast<const uint4*>(kg + kKG_Codes2 + lane * 16);
+  const uint2 c1 = *reinterpret_cast<const uint2*>(kg + kKG_Bits1 + lane * 8);
+  const uint32_t w2[4] = {c2.x, c2.y, c2.z, c2.w};
+  const uint32_t h1[4] = {c1.x & 0xffffu, c1.x >> 16, c1.y & 0xffffu, c1.y >> 16};
+  float acc[4][4];
+  // anomalous channels: q s as exact binary16 pairs hi + lo against 4 + code
+  {
+    uint32_t hi2[8], lo2[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      hi2[i] = hmul2_u(qa[i], s2[i]);
+      lo2[i] = hfms2_u(qa[i], s2[i], hi2[i]);
+    }
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      const uint32_t w = w2[nt];
+      uint32_t x[8];
+      x[0] = and_or(w << 8, m_field, c_four);
+      x[1] = and_or(w << 6, m_field, c_four);
+      x[2] = and_or(w << 4, m_field, c_four);
+      x[3] = and_or(w << 2, m_field, c_four);
+      x[4] = and_or(w, m_field, c_four);
+      const uint32_t wh = w >> 6;                           // fields 5-7 through one right shift, then multiplies
+      x[5] = and_or(wh << 4, m_field, c_four);
+      x[6] = and_or(wh << 2, m_field, c_four);
+      x[7] = and_or(wh, m_field, c_four);
+      mma_f16_c(acc[nt], hi2[0], lo2[0], hi2[1], lo2[1], x[0], x[1], cst, cst, 0.0f, 0.0f);
+#pragma unroll
+      for (int ks = 1; ks < 4; ++ks)
+        mma_f16(acc[nt], hi2[2 * ks], lo2[2 * ks], hi2[2 * ks + 1], lo2[2 * ks + 1], x[2 * ks], x[2 * ks + 1]);
+    }
+  }
+  // normal channels in the frequency domain: Q s (leading part + remainder) against +-1
+  {
+    uint32_t hi1[8], lo1[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      hi1[i] = hmul2_u(qha[i], s1[i]);
+      lo1[i] = hfma2_u(qhb[i], s1[i], hfms2_u(qha[i], s1[i], hi1[i]));
+    }
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      // sign bits: low lane <- bit 15 - 2 m, high lane <- bit 14 - 2 m of the half-word
+      const uint32_t X = h1[nt] * 0x00020001u;
+      uint32_t y[8];
+#pragma unroll
+      for (int m = 0; m < 8; ++m) y[m] = and_xor(X << (2 * m), m_sign, c_neg1);
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks)
+        mma_f16(acc[nt], hi1[2 * ks], lo1[2 * ks], hi1[2 * ks + 1], lo1[2 * ks + 1], y[2 * ks], y[2 * ks + 1]);
+      sc[nt][0] = acc[nt][0] + acc[nt][2];
+      sc[nt][1] = acc[nt][1] + acc[nt][3];
+    }
+  }
+}
+
+// Running output of the warp, kept in shared memory: float4 tot[j][lane], j = 2 w + i, holds the
+// accumulator fragment of channels 32 w + 4 hd + 2 i + (e >> 1) and heads 2 r + (e & 1), e = 0..3.
+
+// One unit of NG (1..5) groups: scores, probabilities, P V into the running state.
+// Returns false if a copy never arrived.
+template <int NG>
+__device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float* totbuf, uint64_t* kbar, uint64_t* vbar,
+                                             uint32_t& kpar, uint32_t& vpar, int lane, int hd, int r,
+                                             const uint32_t* prep_slab, int64_t g_first, int64_t g0n, int& cur_chunk,
+                                             uint32_t (&qa)[8], uint32_t (&qha)[8], uint32_t (&qhb)[8], float sl2,
+                                             Running& run, bool more, const uint8_t* next_k, uint32_t next_k_bytes,
+                                             const uint8_t* next_v) {
+  const uint32_t m_field = kExpand[0], c_four = kExpand[1], m_sign = kExpand[2], c_neg1 = kExpand[3];
+  if (!mbar_wait(kbar, kpar)) return false;
+  kpar ^= 1u;
+  // ---- scores, group by group; a group's scores replace its (spent) bytes in the key buffer:
+  // float2 (tokens 8 nt + 2 r, + 1 of head hd) at word pair (nt * 32 + lane) of the group
+  float mx = -INFINITY;
+#pragma unroll 1
+  for (int g = 0; g < NG; ++g) {
+    const int64_t gidx = g_first + g;
+    const int chunk = gidx < g0n ? 0 : 1 + static_cast<int>((gidx - g0n) / (kR / kG));
+    if (chunk != cur_chunk) {
+      cur_chunk = chunk;
+      const uint32_t* pp = prep_slab + static_cast<int64_t>(chunk) * (kPrepWords * 32);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        qa[i] = __ldg(pp + i * 32);
+        qha[i] = __ldg(pp + (8 + i) * 32);
+        qhb[i] = __ldg(pp + (16 + i) * 32);
+      }
+    }
+    float sc[4][2];
+    uint8_t* kg = kbuf + g * kKGroupBytes;
+    score_group(kg, lane, hd, r, qa, qha, qhb, m_field, c_four, m_sign, c_neg1, sc);
+    __syncwarp();                                           // every lane has read the group's bytes
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      reinterpret_cast<float2*>(kg)[nt * 32 + lane] = make_float2(sc[nt][0], sc[nt][1]);
+      mx = fmaxf(mx, fmaxf(sc[nt][0], sc[nt][1]));
+    }
+  }
+  // ---- probabilities against the running maximum
+  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+  {
+    const float mu = mx * sl2;                              // sl2 > 0
+    const bool up = mu > run.m + kStaleLog2;                // always true for the first unit (run.m = -inf)
+    if (__any_sync(0xffffffffu, up)) {
+      const float m_new = up ? mu : run.m;
+      const float f = ex2_approx(run.m - m_new);            // 1 for heads whose maximum stays
+      run.m = m_new;
+      const float fa = __shfl_sync(0xffffffffu, f, 8 * r), fb = __shfl_sync(0xffffffffu, f, 8 * r + 4);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float4* t = reinterpret_cast<float4*>(totbuf) + j * 32 + lane;
+        float4 v = *t;
+        v.x *= fa; v.y *= fb; v.z *= fa; v.w *= fb;
+        *t = v;
+      }
+      run.l[0] *= fa; run.l[1] *= fb;
+    }
+  }
+  uint32_t P[NG][4];
+  float ps[NG][4];
+#pragma unroll
+  for (int g = 0; g < NG; ++g) {
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      const float2 v = reinterpret_cast<const float2*>(kbuf + g * kKGroupBytes)[nt * 32 + lane];
+      P[g][nt] = pack_half2(ex2_approx(fmaf(v.x, sl2, -run.m)), ex2_approx(fmaf(v.y, sl2, -run.m)));
+    }
+    // -5 * (sums of the rounded probabilities) of heads 2 r, 2 r + 1, for rows hd and hd + 8 alike:
+    // a product with a matrix of -5, whose accumulator fragment is the initial value of every
+    // P V accumulator of the group as it stands
+    ps[g][0] = 0.0f; ps[g][1] = 0.0f; ps[g][2] = 0.0f; ps[g][3] = 0.0f;
+    mma_f16(ps[g], kMinus5, kMinus5, kMinus5, kMinus5, P[g][0], P[g][1]);
+    mma_f16(ps[g], kMinus5, kMinus5, kMinus5, kMinus5, P[g][2], P[g][3]);
+    run.l[0] = fmaf(-0.2f, ps[g][0], run.l[0]);
+    run.l[1] = fmaf(-0.2f, ps[g][1], run.l[1]);
+  }
+  __syncwarp();                                             // the scores are in registers: the key buffer is free
+  if (more && lane == 0) {
+    // the buffer was used through ordinary loads and stores; order them before the bulk copy's writes
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    bulk_load(kbuf, next_k, next_k_bytes, kbar);
+  }
+  // ---- P V over the ternary supergroup, 32 channels (two MMA row blocks) at a time: fragment i of
+  // block w covers channels 32 w + 4 hd + 2 i + {0, 1} in rows hd, hd + 8
+  if (!mbar_wait(vbar, vpar)) return false;
+  vpar ^= 1u;
+#pragma unroll 1
+  for (int w = 0; w < 4; ++w) {
+    float acc[NG][2][4];
+#pragma unroll
+    for (int kt = 0; kt < 2; ++kt) {
+      const uint2 wa = *reinterpret_cast<const uint2*>(vbuf + ((((kt * 2 + 0) * 4 + w) * 4 + r) * 8 + hd) * 8);
+      const uint2 wb = *reinterpret_cast<const uint2*>(vbuf + ((((kt * 2 + 1) * 4 + w) * 4 + r) * 8 + hd) * 8);
+      uint32_t W[8];
+      W[0] = prmt(wa.x, 0u, 0x4140u); W[1] = prmt(wa.x, 0u, 0x4342u);
+      W[2] = prmt(wb.x, 0u, 0x4140u); W[3] = prmt(wb.x, 0u, 0x4342u);
+      W[4] = prmt(wa.y, 0u, 0x4140u); W[5] = prmt(wa.y, 0u, 0x4342u);
+      W[6] = prmt(wb.y, 0u, 0x4140u); W[7] = prmt(wb.y, 0u, 0x4342u);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) W[k] = mad_u32(W[k], 3u, 0u);          // 3 * byte per 16-bit lane
+#pragma unroll
+      for (int g = 0; g < NG; ++g) {
+        uint32_t A[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          // W holds 3 * (remaining byte) per 16-bit lane; the digit sits at bits 8-9.
+          // Next W = 3 * (W - digit << 8) = 3 W - 3 A + 3 * 0x4400 (no lane ever borrows).
+          // Half of the lanes take that route (two multiply-adds), the other half mask the digit
+          // away and multiply (one logic, one multiply-add): the two pipes share the work.
+          A[k] = and_or(W[k], m_field, c_four);
+          if (g + 1 < NG) {
+            if (k & 1) W[k] = mad_u32(A[k], 0xfffffffdu, mad_u32(W[k], 3u, 0xcc00cc00u));
+            else W[k] = mad_u32(W[k] & 0x00ff00ffu, 3u, 0u);
+          }
+        }
+        const uint32_t b0 = P[g][2 * kt], b1 = P[g][2 * kt + 1];
+        if (kt == 0) {
+          mma_f16_c(acc[g][0], A[0], A[1], A[2], A[3], b0, b1, ps[g][0], ps[g][1], ps[g][2], ps[g][3]);
+          mma_f16_c(acc[g][1], A[4], A[5], A[6], A[7], b0, b1, ps[g][0], ps[g][1], ps[g][2], ps[g][3]);
+        } else {
+          mma_f16(acc[g][0], A[0], A[1], A[2], A[3], b0, b1);
+          mma_f16(acc[g][1], A[4], A[5], A[6], A[7], b0, b1);
+        }
+      }
+    }
+    float4* tp = reinterpret_cast<float4*>(totbuf) + (2 * w) * 32 + lane;
+    float4 t0 = tp[0], t1 = tp[32];
+#pragma unroll
+    for (int g = 0; g < NG; ++g) {
+      const uint2 sc2 = *reinterpret_cast<const uint2*>(vbuf + kSG_Scales + g * (kD * 2) + (32 * w + 4 * hd) * 2);
+      const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc2.x));
+      const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&sc2.y));
+      t0.x += sa.x * acc[g][0][0]; t0.y += sa.x * acc[g][0][1];
+      t0.z += sa.y * acc[g][0][2]; t0.w += sa.y * acc[g][0][3];
+      t1.x += sb.x * acc[g][1][0]; t1.y += sb.x * acc[g][1][1];
+      t1.z += sb.y * acc[g][1][2]; t1.w += sb.y * acc[g][1][3];
+    }
+    tp[0] = t0;
+    tp[32] = t1;
+  }
+  __syncwarp();
+  if (more && lane == 0) {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    bulk_load(vbuf, next_v, kVBufBytes, vbar);
+  }
+  return true;
+}
+
+__device__ __forceinline__ void write_record(const DecodeArgs& a, int slab, int run_id, int lane, int hd, int r,
+                                             const Running& run, const float* totbuf) {
+  const DecodePlan& pl = a.plan;
+  const int rep = a.cv.rep;
+  const int first = static_cast<int>(static_cast<int64_t>(slab) * pl.units_per_slab / pl.run_units);
+  float* rec = a.partials + (static_cast<int64_t>(slab) * pl.parts_stride + (run_id - first)) * (kMaxRep * kRecordFloats);
+#pragma unroll
+  for (int w = 0; w < 4; ++w)
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const float4 t = reinterpret_cast<const float4*>(totbuf)[(w * 2 + i) * 32 + lane];
+      const int c = 32 * w + 4 * hd + 2 * i;
+      if (2 * r < rep) {
+        rec[(2 * r) * kRecordFloats + 2 + c] = t.x;
+        rec[(2 * r) * kRecordFloats + 2 + c + 1] = t.z;
+      }
+      if (2 * r + 1 < rep) {
+        rec[(2 * r + 1) * kRecordFloats + 2 + c] = t.y;
+        rec[(2 * r + 1) * kRecordFloats + 2 + c + 1] = t.w;
+      }
+    }
+  if (hd == 0) {
+    if (2 * r < rep) rec[(2 * r) * kRecordFloats + 1] = run.l[0];
+    if (2 * r + 1 < rep) rec[(2 * r + 1) * kRecordFloats + 1] = run.l[1];
+  }
+  if (r == 0 && hd < rep) rec[hd * kRecordFloats] = run.m;
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_stream_kernel(DecodeArgs a) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[kStreamWarps][2];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, hd = lane >> 2, r = lane & 3;
+  const DecodePlan& pl = a.plan;
+  const CacheView& cv = a.cv;
+  const int run_id = blockIdx.x * kStreamWarps + warp;
+  const int64_t u_begin = static_cast<int64_t>(run_id) * pl.run_units;
+  const int64_t u_end = min(u_begin + pl.run_units, pl.n_units);
+  if (u_begin >= u_end) return;                            // warps do not wait on one another
+  uint8_t* kbuf = smem_raw + warp * kWarpBufBytes;
+  uint8_t* vbuf = kbuf + kKBufBytes;
+  float* totbuf = reinterpret_cast<float*>(vbuf + kVBufBytes);
+  uint64_t* kbar = &bars[warp][0];
+  uint64_t* vbar = &bars[warp][1];
+  if (lane == 0) {
+    mbar_init(kbar, 1);
+    mbar_init(vbar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  const int S = pl.units_per_slab;
+  const int64_t n_groups = (a.st.T_q0 + a.st.n_flush * kR) / kG;   // key groups = ternary groups per slab
+  const int64_t g0n = a.st.T_q0 / kG;
+  const uint8_t* slab0 = cv.base + cv.slab_offset + static_cast<int64_t>(a.layer0) * cv.B * cv.H_kv * cv.slab_stride;
+  int slab = static_cast<int>(u_begin / S);
+  int k = static_cast<int>(u_begin - static_cast<int64_t>(slab) * S);
+  auto groups_of = [&](int kk) -> int {
+    const int64_t left = n_groups - static_cast<int64_t>(kk) * kSGGroups;
+    return left < kSGGroups ? static_cast<int>(left) : kSGGroups;
+  };
+  auto key_src = [&](int sl, int kk) -> const uint8_t* {
+    return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.kgroup_offset + static_cast<int64_t>(kk) * kKBufBytes;
+  };
+  auto val_src = [&](int sl, int kk) -> const uint8_t* {
+    return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.tern_offset + static_cast<int64_t>(kk) * kVBufBytes;
+  };
+  if (lane == 0) {
+    bulk_load(kbuf, key_src(slab, k), groups_of(k) * kKGroupBytes, kbar);
+    bulk_load(vbuf, val_src(slab, k), kVBufBytes, vbar);
+  }
+  uint32_t kpar = 0u, vpar = 0u;
+  Running run;
+  run.l[0] = 0.0f; run.l[1] = 0.0f; run.m = -INFINITY;
+  uint32_t qa[8], qha[8], qhb[8];
+  int cur_chunk = -1, cur_slab = -1;
+  const uint32_t* prep_slab = nullptr;
+  float sl2 = 0.0f;
+  bool ok = true;
+#pragma unroll 1
+  for (int64_t u = u_begin; u < u_end; ++u) {
+    if (slab != cur_slab) {
+      if (cur_slab >= 0) write_record(a, cur_slab, run_id, lane, hd, r, run, totbuf);
+      cur_slab = slab;
+      cur_chunk = -1;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) reinterpret_cast<float4*>(totbuf)[j * 32 + lane] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      run.l[0] = 0.0f; run.l[1] = 0.0f;
+      run.m = -INFINITY;
+      prep_slab = a.prep + static_cast<int64_t>(slab) * pl.n_chunks * (kPrepWords * 32) + lane;
+      sl2 = __uint_as_float(__ldg(prep_slab + 24 * 32));
+    }
+    const int ng = groups_of(k);
+    int nslab = slab, nk = k + 1;
+    if (nk == S) { nk = 0; ++nslab; }
+    const bool more = u + 1 < u_end;
+    const uint8_t* next_k = more ? key_src(nslab, nk) : nullptr;
+    const uint32_t next_k_bytes = more ? static_cast<uint32_t>(groups_of(nk) * kKGroupBytes) : 0u;
+    const uint8_t* next_v = more ? val_src(nslab, nk) : nullptr;
+#define VIDKV_UNIT(N)                                                                                                \
+  ok = process_unit<N>(kbuf, vbuf, totbuf, kbar, vbar, kpar, vpar, lane, hd, r, prep_slab,                           \
+                       static_cast<int64_t>(k) * kSGGroups, g0n, cur_chunk, qa, qha, qhb, sl2, run, more, next_k,      \
+                       next_k_bytes, next_v)
+    if (ng == 5) VIDKV_UNIT(5);
+    else if (ng == 4) VIDKV_UNIT(4);
+    else if (ng == 3) VIDKV_UNIT(3);
+    else if (ng == 2) VIDKV_UNIT(2);
+    else VIDKV_UNIT(1);
+#undef VIDKV_UNIT
+    if (!ok) break;
+    slab = nslab; k = nk;
+  }
+  if (!ok) {
+    // a copy never arrived: report it and leave (the wait already ran its full course, so nothing
+    // this warp issued can still be expected)
+    if (lane == 0) atomicCAS(reinterpret_cast<int*>(cv.base + kHdrStatus), VIDKV_OK, VIDKV_ERR_TIMEOUT);
+    return;
+  }
+  write_record(a, cur_slab, run_id, lane, hd, r, run, totbuf);
+}
+
+cudaError_t launch_decode_stream(const DecodeArgs& a, cudaStream_t stream) {
+  const size_t smem = static_cast<size_t>(kStreamWarps) * kWarpBufBytes;
+  static bool attr_set[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!attr_set[dev]) {
+    const cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set[dev] = true;
+  }
+  const int grid = (a.plan.n_runs + kStreamWarps - 1) / kStreamWarps;
+  if (grid < 1) return cudaSuccess;
+  decode_stream_kernel<<<grid, kStreamWarps * 32, smem, stream>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+}  // namespace vidkv

@@ -66,37 +66,6 @@ void compute_layout(const vidkv_config_t& c, Layout* out) {
   l.total_bytes = l.slab_offset + l.slab_stride * c.L * c.B * c.H_kv;
 }
 
-// Tokens per split: the largest of {640, 320, 160} that still gives >= 4 CTAs per SM on a
-// 148-SM part, else 160.
-int choose_split_tokens(int64_t T_tot, int64_t n_slabs, bool /*stp*/) {
-  const int cand[3] = {640, 320, 160};
-  for (int s : cand)
-    if (n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
-  return 160;
-}
-
-// Consecutive splits one CTA folds into a single partial record: as many as still leave about
-// eight waves of CTAs (4 per SM, 148 SMs), at most 8; 1 with protected tokens.
-int choose_splits_per_cta(int64_t n_splits, int64_t n_slabs, bool stp) {
-  if (stp) return 1;
-  const int64_t k = n_splits * n_slabs / 4736;
-  return static_cast<int>(k < 1 ? 1 : (k > 8 ? 8 : k));
-}
-
-int64_t max_partial_entries(const vidkv_config_t& c, int64_t T_max) {
-  int64_t best = 0;
-  if (T_max < 1) T_max = 1;
-  for (int n = 1; n <= c.L; ++n) {
-    const int64_t slabs = static_cast<int64_t>(n) * c.B * c.H_kv;
-    for (int stp = 0; stp <= (c.p_ratio > 0.0f ? 1 : 0); ++stp) {
-      const int st = choose_split_tokens(T_max, slabs, stp != 0);
-      const int64_t e = static_cast<int64_t>(n) * c.B * c.H_q * ((T_max + st - 1) / st);
-      if (e > best) best = e;
-    }
-  }
-  return best;
-}
-
 struct WsPlan {
   int64_t minmax_off, partials_off, prep_off, idx_prot_off, idx_rest_off, counts_off, total;
   int64_t partial_entries;
@@ -106,9 +75,9 @@ void plan_workspace(const vidkv_config_t& c, const Layout& L, WsPlan* w) {
   int64_t off = 0;
   w->minmax_off = off;
   off = round_up(off + 2 * static_cast<int64_t>(c.L) * c.B * c.H_kv * 2 * kD * 4, kAlign);   // two alternating buffers
-  w->partial_entries = max_partial_entries(c, L.max_total_tokens);
+  w->partial_entries = max_decode_records(static_cast<int64_t>(c.L) * c.B * c.H_kv, L.max_total_tokens, c.p_ratio > 0.0f);
   w->partials_off = off;
-  off = round_up(off + w->partial_entries * 130 * 4, kAlign);
+  off = round_up(off + w->partial_entries * kRecordFloats * 4, kAlign);
   w->prep_off = off;
   off = round_up(off + static_cast<int64_t>(decode_prep_bytes(static_cast<int64_t>(c.L) * c.B * c.H_kv, L.lay.max_chunks)),
                  kAlign);
@@ -143,6 +112,8 @@ struct vidkv_cache {
   uint8_t* workspace;
   bool sel_set;
   int64_t sel_T, n_prot;
+  int dbg_split_tokens = 0;     // test hook: forced split length of the split kernel (0 = choose)
+  int dbg_run_units = 0;        // test hook: forced run length of the stream kernel (0 = choose)
   int mm_parity = 0;            // which min / max buffer the next key quantization accumulates into
   int64_t mm_dirty[2] = {0, 0}; // words of each buffer written since it was last re-armed
   std::vector<LayerInfo> layers;
@@ -415,7 +386,7 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int dt = h->cfg.in_dtype;
   // the append rides on the query-preparation kernel when there is one (some chunk is quantized)
-  const bool has_chunks = first.T_q0 + first.n_flush > 0;
+  const bool has_chunks = first.T_q0 + first.n_flush * kR > 0;
   if (!has_chunks && launch_append(dt, k_new, v_new, h->cv, layer_begin, n_layers, first.n_res, s) != cudaSuccess)
     return VIDKV_ERR_CUDA;
   DecodeArgs a;
@@ -430,13 +401,9 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   a.scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / std::sqrt(static_cast<float>(kD));
   a.ev_begin = h->ev_begin; a.ev_end = h->ev_end;
   a.st.T_q0 = first.T_q0; a.st.n_flush = first.n_flush; a.st.n_res = first.n_res + 1;
-  const int64_t T_tot = first.T_q0 + first.n_flush * kR + a.st.n_res;
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv;
-  a.split_tokens = choose_split_tokens(T_tot, n_slabs, h->n_prot > 0);
-  a.n_splits = static_cast<int32_t>((T_tot + a.split_tokens - 1) / a.split_tokens);
-  a.splits_per_cta = choose_splits_per_cta(a.n_splits, n_slabs, h->n_prot > 0);
-  a.n_parts = (a.n_splits + a.splits_per_cta - 1) / a.splits_per_cta;
-  if (static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_q * a.n_splits > h->ws.partial_entries) return VIDKV_ERR_CAPACITY;
+  a.plan = plan_decode(a.st, n_slabs, h->n_prot, device_sm_count(), h->dbg_split_tokens, h->dbg_run_units);
+  if (a.plan.records > h->ws.partial_entries) return VIDKV_ERR_CAPACITY;
   if (launch_decode(a, s) != cudaSuccess) return VIDKV_ERR_CUDA;
   const bool flush = a.st.n_res == kR;
   if (flush) {
@@ -461,6 +428,38 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
     if (flush) { li.n_flush += 1; li.n_res = 0; }
     else li.n_res += 1;
   }
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_debug_set_decode_plan(vidkv_cache_t* h, int32_t split_tokens, int32_t run_units) {
+  if (!h) return VIDKV_ERR_INVALID_ARG;
+  if (split_tokens != 0 && split_tokens != 160 && split_tokens != 320 && split_tokens != 640) return VIDKV_ERR_INVALID_ARG;
+  if (run_units < 0) return VIDKV_ERR_INVALID_ARG;
+  h->dbg_split_tokens = split_tokens;
+  h->dbg_run_units = run_units;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_debug_decode_plan(const vidkv_config_t* cfg, int64_t n_prefill_quantized, int64_t n_flushed_chunks,
+                                       int32_t n_residual, int64_t n_protected, int32_t n_layers, int32_t sm_count,
+                                       int32_t split_tokens, int32_t run_units, int64_t* plan_out) {
+  if (!plan_out) return VIDKV_ERR_INVALID_ARG;
+  const vidkv_status_t st = check_config(cfg);
+  if (st != VIDKV_OK) return st;
+  if (n_layers < 1 || n_layers > cfg->L || n_prefill_quantized < 0 || n_prefill_quantized % kG || n_flushed_chunks < 0 ||
+      n_residual < 0 || n_residual > kR || n_protected < 0 || sm_count < 1)
+    return VIDKV_ERR_INVALID_ARG;
+  Layout L;
+  compute_layout(*cfg, &L);
+  WsPlan w;
+  plan_workspace(*cfg, L, &w);
+  LayerState ls;
+  ls.T_q0 = n_prefill_quantized; ls.n_flush = n_flushed_chunks; ls.n_res = n_residual;
+  const DecodePlan p = plan_decode(ls, static_cast<int64_t>(n_layers) * cfg->B * cfg->H_kv, n_protected, sm_count,
+                                   split_tokens, run_units);
+  plan_out[0] = p.stream; plan_out[1] = p.split_tokens; plan_out[2] = p.n_splits; plan_out[3] = p.units_per_slab;
+  plan_out[4] = p.run_units; plan_out[5] = p.n_runs; plan_out[6] = p.parts_stride; plan_out[7] = p.records;
+  plan_out[8] = w.partial_entries; plan_out[9] = p.n_chunks;
   return VIDKV_OK;
 }
 

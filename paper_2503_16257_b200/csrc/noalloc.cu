@@ -37,15 +37,6 @@ vidkv_status_t static_partials(float** out) {
   return VIDKV_OK;
 }
 
-// Tokens per split, by the same rule of thumb as the regular entry point: the largest of
-// {640, 320, 160} that still yields about four CTAs per SM.
-int split_tokens_for(int64_t T_tot, int64_t n_slabs, bool /*stp*/) {
-  const int cand[3] = {640, 320, 160};
-  for (int s : cand)
-    if (n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
-  return 160;
-}
-
 }  // namespace
 
 extern "C" vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const void* cache, int64_t n_prefill_quantized,
@@ -88,16 +79,11 @@ extern "C" vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const 
   a.st.T_q0 = n_prefill_quantized; a.st.n_flush = n_flushed_chunks; a.st.n_res = n_residual;
   a.ev_begin = nullptr; a.ev_end = nullptr;
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * cfg->B * cfg->H_kv;
-  a.split_tokens = split_tokens_for(T_tot, n_slabs, n_protected > 0);
-  a.n_splits = static_cast<int32_t>((T_tot + a.split_tokens - 1) / a.split_tokens);
-  a.splits_per_cta = 1;
   a.append_row = -1;
-  a.n_parts = a.n_splits;
-  const int64_t records = static_cast<int64_t>(n_layers) * cfg->B * cfg->H_q * a.n_splits;
+  a.plan = plan_decode(a.st, n_slabs, n_protected, device_sm_count(), 0, 0);
   // the array holds the partial records, then (256-byte aligned) the per-chunk query images
-  const int64_t prep_at = (records * 130 * 4 + 255) / 256 * 256;
-  const int64_t n_chunks = (n_prefill_quantized > 0 ? 1 : 0) + n_flushed_chunks;
-  const int64_t prep_bytes = static_cast<int64_t>(decode_prep_bytes(n_slabs, n_chunks));
+  const int64_t prep_at = (a.plan.records * kRecordFloats * 4 + 255) / 256 * 256;
+  const int64_t prep_bytes = static_cast<int64_t>(decode_prep_bytes(n_slabs, a.plan.n_chunks));
   if (prep_at + prep_bytes > static_cast<int64_t>(kStaticPartialFloats * sizeof(float))) return VIDKV_ERR_CAPACITY;
   const vidkv_status_t sp = static_partials(&a.partials);
   if (sp != VIDKV_OK) return sp;
