@@ -65,11 +65,12 @@ DecodePlan plan_decode(const LayerState& st, int64_t n_slabs, int64_t n_prot, in
 
 int64_t max_decode_records(int64_t max_slabs, int64_t max_tokens, bool stp) {
   if (max_tokens < 1) max_tokens = 1;
-  // Stream kernel: parts per slab = ceil(S / run) + 1 with run >= max(kMinRunUnits, n_units / warps),
-  // so slabs * parts <= min(slabs * ceil(S / kMinRunUnits), warps + slabs) + slabs for every S.
+  // Stream kernel: parts per slab = ceil(S / run) + 1 with run >= max(1, n_units / warps) (the
+  // chooser never goes below kMinRunUnits, the test hook may force 1), so
+  // slabs * parts <= min(slabs * S, warps + slabs) + slabs for every S.
   const int64_t S = (max_tokens + kStreamUnitTokens - 1) / kStreamUnitTokens;
   const int64_t warps = static_cast<int64_t>(kMaxSMs) * kStreamCtasPerSM * kStreamWarps;
-  int64_t parts = max_slabs * ((S + kMinRunUnits - 1) / kMinRunUnits);
+  int64_t parts = max_slabs * S;
   if (parts > warps + max_slabs) parts = warps + max_slabs;
   parts += max_slabs;
   if (stp) {

@@ -312,7 +312,7 @@ vidkv_status_t vidkv_set_token_mask(vidkv_cache_t* h, const uint8_t* E, int64_t 
 
 static vidkv_status_t check_kv_args(vidkv_cache_t* h, int32_t layer, const void* X, int64_t T, int64_t sb, int64_t sh,
                                     int64_t st) {
-  if (!h || !X || T < 0) return VIDKV_ERR_INVALID_ARG;
+  if (!h || T < 0 || (!X && T > 0)) return VIDKV_ERR_INVALID_ARG;   // an empty prompt may come with a null pointer
   if (layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
   if (sb < 0 || sh < 0 || st < kD) return VIDKV_ERR_INVALID_ARG;
   if (!aligned16(X) || (sb % 8) || (sh % 8) || (st % 8)) return VIDKV_ERR_ALIGNMENT;

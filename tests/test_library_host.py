@@ -140,6 +140,47 @@ def test_channel_metrics_argument_checks_without_a_device(lib):
     assert call(K=ctypes.c_void_p(0x1002)) == -3                                       # misaligned
 
 
+@pytest.mark.parametrize("B,L,T_max,max_new,p", [
+    (4, 1, 24000, 16, 0.2),      # a shorter prompt picks shorter splits and needs about twice the records
+    (1, 1, 100000, 16, 0.2),
+    (4, 1, 24000, 16, 0.0),
+    (16, 28, 12544, 128, 0.2),   # the batched workload
+    (1, 28, 6400, 256, 0.0),
+    (2, 3, 700, 300, 0.5),
+])
+def test_partial_records_fit_the_workspace_for_every_token_count(lib, B, L, T_max, max_new, p):
+    """The workspace is sized once, from the configured maxima; how a decode call is cut into work
+    depends on the live token count and on how many layers the call covers.  Whatever they are,
+    the records the plan needs must fit what was reserved."""
+    cfg = P.VidKVConfig(B=B, L=L, max_prefill_tokens=T_max, max_new_tokens=max_new, p_ratio=p)
+    step = max(32, (T_max // 400) // 32 * 32)
+    tokens = sorted(set(list(range(0, T_max + 1, step)) + [T_max - T_max % 32] +
+                        [t for t in (32, 160, 320, 640, 1280, 18912, 18944, 23008, 23040) if t <= T_max]))
+    worst = 0
+    for n_layers in sorted({1, L, max(1, L // 2)}):
+        for sm in (1, 132, 148, 1000):
+            for T in tokens:
+                T = T - T % 32
+                n_prot = int(p * T) // 2
+                for n_flush, n_res in ((0, 1), (0, 128), (max_new // 128, 77)):
+                    for prot in sorted({0, n_prot}):
+                        pl = P.vidkv_debug_decode_plan(cfg, T, n_flush, n_res, prot, n_layers, sm_count=sm)
+                        assert pl["records"] <= pl["records_capacity"], (n_layers, sm, T, n_flush, n_res, prot, pl)
+                        worst = max(worst, pl["records"])
+                        assert pl["stream"] == (1 if prot == 0 else 0)
+                        if pl["stream"] and T > 0:
+                            assert pl["n_runs"] * pl["run_units"] >= n_layers * B * 4 * pl["units_per_slab"]
+                            assert pl["parts_stride"] >= -(-pl["units_per_slab"] // pl["run_units"]) + 1
+    assert worst > 0
+    # a plan forced through the test hook may need more than was reserved (the decode call then
+    # returns VIDKV_ERR_CAPACITY); on problems with fewer units than the largest launch has warps, one
+    # unit per run still fits
+    T = T_max - T_max % 32
+    if B * L * 4 * (-(-T // 160)) <= 256 * 12:
+        assert P.vidkv_debug_decode_plan(cfg, T, 0, 1, 0, L, run_units=1)["records"] <= \
+            P.vidkv_debug_decode_plan(cfg, T, 0, 1, 0, L)["records_capacity"]
+
+
 def test_missing_library_fails_loudly(monkeypatch):
     import paper_2503_16257_b200.api as api
     monkeypatch.setattr(api, "_LIB", None)
