@@ -23,9 +23,12 @@
  *     and passes the buffers in.  The handle is a small host object.
  *   - All device work is enqueued on the caller's stream (a cudaStream_t passed
  *     as void*) and is asynchronous.  Argument errors are detected on the host
- *     before anything is launched.  One exception: the first key quantization or
- *     decode call on each device fills the tables of DFT coefficients inside the
- *     library (56 KB) and synchronises the stream once.
+ *     before anything is launched.  No call synchronises the stream except
+ *     vidkv_cache_status and vidkv_set_token_mask with n_protected == -1.  The first key
+ *     quantization or decode call on each device fills the tables of DFT coefficients inside
+ *     the library (56 KB) with one extra small kernel on the caller's stream and records an
+ *     event that later calls make their streams wait for; make that first call outside any
+ *     stream capture.
  *   - Fixed in this library: D = 128, G = 32, R = 128, k = 0.5 (64 two-bit and 64
  *     one-bit channels), H_q a multiple of H_kv with H_q / H_kv <= 8.  Other
  *     shapes return VIDKV_ERR_UNSUPPORTED.
@@ -210,8 +213,12 @@ vidkv_status_t vidkv_select_tokens(vidkv_cache_t* handle, const float* saliency,
 
 /* Algorithm 2 takes the mask E as a parameter: the same, from a ready mask
  * E [B, T] (uint8, nonzero = protected; every batch element must protect the same
- * number of tokens, all below T - T % G). */
-vidkv_status_t vidkv_set_token_mask(vidkv_cache_t* handle, const uint8_t* E, int64_t T, void* stream);
+ * number of tokens, all below T - T % G).  n_protected >= 0 states that number: the call is
+ * then asynchronous like the others, and a row of E that protects a different number sets
+ * VIDKV_ERR_INVALID_ARG in the cache's status word (vidkv_cache_status).  n_protected == -1
+ * lets the library count: it then reads the counts back and synchronises the stream once. */
+vidkv_status_t vidkv_set_token_mask(vidkv_cache_t* handle, const uint8_t* E, int64_t T, int64_t n_protected,
+                                    void* stream);
 
 /* Algorithm 1 "Prefill", key half, for one layer: K [B, H_kv, T, D] (in_dtype) with
  * element strides stride_b / stride_h / stride_t (channel stride 1; strides multiples
@@ -255,6 +262,31 @@ vidkv_status_t vidkv_cache_status(vidkv_cache_t* handle, void* stream);
  * one layer to float32, out [B, H_kv, n_quantized, D] contiguous.  DeQuant of Algorithm 1. */
 vidkv_status_t vidkv_dequantize_keys(vidkv_cache_t* handle, int32_t layer, float* out, void* stream);
 vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* handle, int32_t layer, float* out, void* stream);
+
+/* Test and inspection only: the packed codes and metadata of one layer as plain arrays, one
+ * element per code, so that a test need not know the bit layout (Eq. 4, Eq. 5, Eq. 6 codes as
+ * Algorithm 1 stores them).  With ng = n_quantized / 32 key groups, nt ternary stream groups
+ * (ceil((n_prefill_quantized - n_protected) / 32) + 4 per flush) and np = ceil(n_protected / 32)
+ * protected groups, per slab = (b, h) of the layer, all device pointers, any of them may be NULL:
+ *   k2      int8  [B, H_kv, 32 ng, 64]   Eq. 4 codes 0..3 of the 2-bit channels, slot order
+ *                                        (slot j = j-th channel of the chunk's ascending 2-bit list)
+ *   k1bits  uint8 [B, H_kv, 32 ng, 64]   Eq. 5 bits of the spectrum columns (column order of the layout)
+ *   k_s2, k_z2, k_s1  binary16 [B, H_kv, ng, 64]
+ *   v_trits int8  [B, H_kv, 32 nt, 128]  Eq. 6 codes -1, 0, +1 in ternary stream order
+ *   v_s     binary16 [B, H_kv, nt, 128]
+ *   v2      int8  [B, H_kv, 32 np, 128]  Eq. 4 codes of the protected tokens, stream order
+ *   v2_s, v2_z        binary16 [B, H_kv, np, 128]
+ * Positions past the end of a stream hold whatever the cache holds there (zeros after init). */
+vidkv_status_t vidkv_export_codes(vidkv_cache_t* handle, int32_t layer, int8_t* k2, uint8_t* k1bits, void* k_s2,
+                                  void* k_z2, void* k_s1, int8_t* v_trits, void* v_s, int8_t* v2, void* v2_s,
+                                  void* v2_z, void* stream);
+
+/* Test and inspection only: the selections of Algorithm 3 and Algorithm 2 as byte masks.
+ *   dmask uint8 [B, H_kv, 1 + flushes, 128]  1 = 2-bit (anomalous) channel of that chunk (D-mask);
+ *                                            chunk 0 is the prefill, all zero if it is empty
+ *   E     uint8 [B, T]                       1 = protected token (T = the prompt length given at prefill)
+ * Either pointer may be NULL. */
+vidkv_status_t vidkv_get_selection(vidkv_cache_t* handle, int32_t layer, uint8_t* dmask, uint8_t* E, void* stream);
 
 /* For callers that cannot obtain device memory.  (The paper has no counterpart to this
  * entry point; it exists for deployment reasons only.)  Some callers are handed their
@@ -301,6 +333,16 @@ vidkv_status_t vidkv_debug_set_decode_plan(vidkv_cache_t* handle, int32_t split_
 vidkv_status_t vidkv_debug_decode_plan(const vidkv_config_t* cfg, int64_t n_prefill_quantized, int64_t n_flushed_chunks,
                                        int32_t n_residual, int64_t n_protected, int32_t n_layers, int32_t sm_count,
                                        int32_t split_tokens, int32_t run_units, int64_t* plan_out);
+
+/* Test hook for the two bounded device-side waits (no counterpart in the paper).  The key encoder
+ * waits on the barrier its tensor-core products commit to, the stream kernel of the decode call
+ * on the barriers of its bulk copies; both waits give up after a fixed number of polls, record
+ * VIDKV_ERR_TIMEOUT in the cache's status word and leave in order (copies drained, tensor memory
+ * freed).  what = 1 makes the next key quantization withhold the products of every block's first
+ * tile, what = 2 makes the next decode call without protected tokens withhold every warp's first
+ * value copy, so that the waits run out with nothing outstanding; the affected call's results
+ * are garbage by design, the flag clears itself, and later calls are normal.  0 switches it off. */
+vidkv_status_t vidkv_debug_withhold_once(int32_t what);
 
 /* Profiling aid: record the two CUDA events (cudaEvent_t passed as void*) immediately before
  * and after the attention kernel (stream or split kernel) of every later vidkv_decode_attention call on this

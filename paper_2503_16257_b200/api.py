@@ -79,7 +79,7 @@ _SIGNATURES = {
     "vidkv_saliency_scores": (C.c_int32, [C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int64,
                                           C.c_void_p, C.c_void_p, C.c_void_p]),
     "vidkv_select_tokens": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p]),
-    "vidkv_set_token_mask": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]),
+    "vidkv_set_token_mask": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p]),
     "vidkv_quantize_keys": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                         C.c_int64, C.c_void_p]),
     "vidkv_quantize_values": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
@@ -89,9 +89,12 @@ _SIGNATURES = {
     "vidkv_layer_state": (C.c_int32, [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                                       C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "vidkv_cache_status": (C.c_int32, [C.c_void_p, C.c_void_p]),
+    "vidkv_debug_withhold_once": (C.c_int32, [C.c_int32]),
     "vidkv_debug_set_decode_plan": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),
     "vidkv_debug_decode_plan": (C.c_int32, [C.POINTER(_Config), C.c_int64, C.c_int64, C.c_int32, C.c_int64, C.c_int32,
                                             C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]),
+    "vidkv_export_codes": (C.c_int32, [C.c_void_p, C.c_int32] + [C.c_void_p] * 10 + [C.c_void_p]),
+    "vidkv_get_selection": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "vidkv_dequantize_keys": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
     "vidkv_dequantize_values": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
 }
@@ -180,6 +183,12 @@ def vidkv_saliency_scores(x_v, x_t, text_sum=None, saliency=None):
     return saliency
 
 
+def vidkv_debug_withhold_once(what: int):
+    """Test hook: 1 = the next key quantization, 2 = the next decode call without protected tokens
+    lets its bounded device-side wait run out (see include/vidkv.h)."""
+    _check("vidkv_debug_withhold_once", load_library().vidkv_debug_withhold_once(what))
+
+
 _PLAN_FIELDS = ("stream", "split_tokens", "n_splits", "units_per_slab", "run_units", "n_runs", "parts_stride",
                 "records", "records_capacity", "n_chunks")
 
@@ -260,10 +269,12 @@ class VidKVCache:
             assert saliency.is_contiguous() and saliency.dtype.is_floating_point and saliency.element_size() == 4
         _check("vidkv_select_tokens", self.lib.vidkv_select_tokens(self.handle, ptr, vis_begin, l_v, T, _stream_ptr()))
 
-    def set_token_mask(self, E, T: int):
+    def set_token_mask(self, E, T: int, n_protected: int = -1):
+        """n_protected >= 0: asynchronous, a disagreeing row shows in status(); -1: counted by the
+        library (one stream synchronisation)."""
         assert E.is_contiguous() and E.element_size() == 1
         _check("vidkv_set_token_mask", self.lib.vidkv_set_token_mask(self.handle, C.c_void_p(E.data_ptr()), T,
-                                                                     _stream_ptr()))
+                                                                     n_protected, _stream_ptr()))
 
     def quantize_keys(self, layer: int, K):
         sb, sh, st = _strides_bht(K)
@@ -301,6 +312,46 @@ class VidKVCache:
 
     def status(self) -> int:
         return self.lib.vidkv_cache_status(self.handle, _stream_ptr())
+
+    def export_codes(self, layer: int, T: int) -> dict:
+        """Plain arrays of every code and scale of one layer (torch tensors; see vidkv_export_codes);
+        T is the prompt length given at prefill."""
+        import torch
+        st = self.layer_state(layer)
+        B, H = self.cfg.B, self.cfg.H_kv
+        ng = st["n_quantized"] // 32
+        n_prefill_q = T - T % 32
+        n_flush = (st["n_quantized"] - n_prefill_q) // 128
+        nt = (n_prefill_q - st["n_protected"] + 31) // 32 + 4 * n_flush
+        npg = (st["n_protected"] + 31) // 32
+        dev = self.cache.device
+        out = dict(
+            k2=torch.zeros((B, H, 32 * ng, 64), dtype=torch.int8, device=dev),
+            k1bits=torch.zeros((B, H, 32 * ng, 64), dtype=torch.uint8, device=dev),
+            k_s2=torch.zeros((B, H, ng, 64), dtype=torch.float16, device=dev),
+            k_z2=torch.zeros((B, H, ng, 64), dtype=torch.float16, device=dev),
+            k_s1=torch.zeros((B, H, ng, 64), dtype=torch.float16, device=dev),
+            v_trits=torch.zeros((B, H, 32 * nt, 128), dtype=torch.int8, device=dev),
+            v_s=torch.zeros((B, H, nt, 128), dtype=torch.float16, device=dev),
+            v2=torch.zeros((B, H, 32 * npg, 128), dtype=torch.int8, device=dev),
+            v2_s=torch.zeros((B, H, npg, 128), dtype=torch.float16, device=dev),
+            v2_z=torch.zeros((B, H, npg, 128), dtype=torch.float16, device=dev))
+        ptr = [C.c_void_p(out[k].data_ptr() if out[k].numel() else 0)
+               for k in ("k2", "k1bits", "k_s2", "k_z2", "k_s1", "v_trits", "v_s", "v2", "v2_s", "v2_z")]
+        _check("vidkv_export_codes", self.lib.vidkv_export_codes(self.handle, layer, *ptr, _stream_ptr()))
+        return out
+
+    def get_selection(self, layer: int, T: int):
+        """(dmask [B, H_kv, chunks, 128], E [B, T]) as uint8 tensors; see vidkv_get_selection."""
+        import torch
+        st = self.layer_state(layer)
+        n_flush = (st["n_quantized"] - (T - T % 32)) // 128
+        dev = self.cache.device
+        dmask = torch.zeros((self.cfg.B, self.cfg.H_kv, 1 + n_flush, 128), dtype=torch.uint8, device=dev)
+        E = torch.zeros((self.cfg.B, max(T, 1)), dtype=torch.uint8, device=dev)
+        _check("vidkv_get_selection", self.lib.vidkv_get_selection(
+            self.handle, layer, C.c_void_p(dmask.data_ptr()), C.c_void_p(E.data_ptr() if T else 0), _stream_ptr()))
+        return dmask, E[:, :T]
 
     def dequantize_keys(self, layer: int):
         import torch

@@ -246,7 +246,10 @@ __device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float
   }
   // ---- P V over the ternary supergroup, 32 channels (two MMA row blocks) at a time: fragment i of
   // block w covers channels 32 w + 4 hd + 2 i + {0, 1} in rows hd, hd + 8
-  if (!mbar_wait(vbar, vpar)) return false;
+  if (!mbar_wait(vbar, vpar)) {
+    if (more) mbar_wait(kbar, kpar);                        // let the key copy issued above land before leaving
+    return false;
+  }
   vpar ^= 1u;
 #pragma unroll 1
   for (int w = 0; w < 4; ++w) {
@@ -379,7 +382,7 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_st
   };
   if (lane == 0) {
     bulk_load(kbuf, key_src(slab, k), groups_of(k) * kKGroupBytes, kbar);
-    bulk_load(vbuf, val_src(slab, k), kVBufBytes, vbar);
+    if (!a.withhold) bulk_load(vbuf, val_src(slab, k), kVBufBytes, vbar);   // (test hook: see DecodeArgs::withhold)
   }
   uint32_t kpar = 0u, vpar = 0u;
   Running run;
@@ -431,7 +434,9 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_st
   write_record(a, cur_slab, run_id, lane, hd, r, run, totbuf);
 }
 
-cudaError_t launch_decode_stream(const DecodeArgs& a, cudaStream_t stream) {
+cudaError_t launch_decode_stream(const DecodeArgs& a_in, cudaStream_t stream) {
+  DecodeArgs a = a_in;
+  if (g_debug_withhold == 2) { a.withhold = 1; g_debug_withhold = 0; }
   const size_t smem = static_cast<size_t>(kStreamWarps) * kWarpBufBytes;
   static bool attr_set[64] = {};
   int dev = 0;

@@ -100,7 +100,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 }  // namespace
 
-namespace vidkv { unsigned long long g_launch_count = 0; }
+namespace vidkv { unsigned long long g_launch_count = 0; int g_debug_withhold = 0; }
 
 struct vidkv_cache {
   cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
@@ -203,14 +203,13 @@ vidkv_status_t vidkv_cache_init(const vidkv_config_t* cfg, void* cache, size_t c
   h->layers.assign(cfg->L, LayerInfo());
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(h->cache, 0, static_cast<size_t>(l.total_bytes), s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }
+  // the kernel that arms the channel-range accumulators also writes the header words
   if (launch_init_minmax(reinterpret_cast<uint32_t*>(h->workspace + h->ws.minmax_off),
-                         2 * static_cast<int64_t>(cfg->L) * cfg->B * cfg->H_kv * 2 * kD, s) != cudaSuccess) {
+                         2 * static_cast<int64_t>(cfg->L) * cfg->B * cfg->H_kv * 2 * kD, reinterpret_cast<uint32_t*>(h->cache),
+                         static_cast<uint32_t>(vidkv_version()), s) != cudaSuccess) {
     delete h;
     return VIDKV_ERR_CUDA;
   }
-  const uint32_t hdr[3] = {kMagic, static_cast<uint32_t>(vidkv_version()), 0u};
-  if (cudaMemcpyAsync(h->cache, hdr, sizeof(hdr), cudaMemcpyHostToDevice, s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }
-  if (cudaStreamSynchronize(s) != cudaSuccess) { delete h; return VIDKV_ERR_CUDA; }   // hdr is a stack buffer
   *handle = h;
   return VIDKV_OK;
 }
@@ -286,19 +285,27 @@ vidkv_status_t vidkv_select_tokens(vidkv_cache_t* h, const float* saliency, int6
   return VIDKV_OK;
 }
 
-vidkv_status_t vidkv_set_token_mask(vidkv_cache_t* h, const uint8_t* E, int64_t T, void* stream) {
-  if (!h || !E || T < 0) return VIDKV_ERR_INVALID_ARG;
+vidkv_status_t vidkv_set_token_mask(vidkv_cache_t* h, const uint8_t* E, int64_t T, int64_t n_protected, void* stream) {
+  if (!h || !E || T < 0 || n_protected < -1) return VIDKV_ERR_INVALID_ARG;
   if (T > h->cfg.max_prefill_tokens) return VIDKV_ERR_CAPACITY;
   for (const LayerInfo& li : h->layers)
     if (li.v_done) return VIDKV_ERR_STATE;
-  if (h->L.max_prot == 0) return VIDKV_ERR_CAPACITY;
+  if (h->L.max_prot == 0 || n_protected > h->L.max_prot) return VIDKV_ERR_CAPACITY;
   const int64_t T_q = T - T % kG;
+  if (n_protected > T_q) return VIDKV_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int32_t* ip = reinterpret_cast<int32_t*>(h->workspace + h->ws.idx_prot_off);
   int32_t* ir = reinterpret_cast<int32_t*>(h->workspace + h->ws.idx_rest_off);
   int32_t* dc = reinterpret_cast<int32_t*>(h->workspace + h->ws.counts_off);
-  if (launch_mask_to_selection(E, T, T_q, h->cv, ip, ir, h->L.max_prot, h->cfg.max_prefill_tokens, dc, s) != cudaSuccess)
+  if (launch_mask_to_selection(E, T, T_q, h->cv, ip, ir, h->L.max_prot, h->cfg.max_prefill_tokens, dc, n_protected, s) !=
+      cudaSuccess)
     return VIDKV_ERR_CUDA;
+  if (n_protected >= 0) {
+    // the caller stated the count: nothing comes back to the host; a row that disagrees is
+    // reported through the cache's status word
+    h->sel_set = true; h->sel_T = T; h->n_prot = n_protected;
+    return VIDKV_OK;
+  }
   std::vector<int32_t> counts(h->cfg.B);
   if (cudaMemcpyAsync(counts.data(), dc, sizeof(int32_t) * h->cfg.B, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
       cudaStreamSynchronize(s) != cudaSuccess)
@@ -400,6 +407,7 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   a.n_prot = h->n_prot;
   a.scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / std::sqrt(static_cast<float>(kD));
   a.ev_begin = h->ev_begin; a.ev_end = h->ev_end;
+  a.withhold = 0;
   a.st.T_q0 = first.T_q0; a.st.n_flush = first.n_flush; a.st.n_res = first.n_res + 1;
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv;
   a.plan = plan_decode(a.st, n_slabs, h->n_prot, device_sm_count(), h->dbg_split_tokens, h->dbg_run_units);
@@ -428,6 +436,12 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
     if (flush) { li.n_flush += 1; li.n_res = 0; }
     else li.n_res += 1;
   }
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_debug_withhold_once(int32_t what) {
+  if (what < 0 || what > 2) return VIDKV_ERR_INVALID_ARG;
+  g_debug_withhold = what;
   return VIDKV_OK;
 }
 
@@ -482,6 +496,36 @@ vidkv_status_t vidkv_cache_status(vidkv_cache_t* h, void* stream) {
       cudaStreamSynchronize(s) != cudaSuccess)
     return VIDKV_ERR_CUDA;
   return word;
+}
+
+vidkv_status_t vidkv_export_codes(vidkv_cache_t* h, int32_t layer, int8_t* k2, uint8_t* k1bits, void* k_s2, void* k_z2,
+                                  void* k_s1, int8_t* v_trits, void* v_s, int8_t* v2, void* v2_s, void* v2_z,
+                                  void* stream) {
+  if (!h || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  const LayerInfo& li = h->layers[layer];
+  if (!li.k_done || !li.v_done) return VIDKV_ERR_STATE;
+  const int64_t n_kgroups = li.T_q0 / kG + (kR / kG) * li.n_flush;
+  const int64_t n_rest = li.T_q0 - h->n_prot;
+  const int64_t n_tgroups = (n_rest + kG - 1) / kG + (kR / kG) * li.n_flush;
+  const int64_t n_pgroups = (h->n_prot + kG - 1) / kG;
+  if (launch_export_codes(h->cv, layer, n_kgroups, n_tgroups, n_pgroups, k2, k1bits, static_cast<uint16_t*>(k_s2),
+                          static_cast<uint16_t*>(k_z2), static_cast<uint16_t*>(k_s1), v_trits, static_cast<uint16_t*>(v_s),
+                          v2, static_cast<uint16_t*>(v2_s), static_cast<uint16_t*>(v2_z),
+                          static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_get_selection(vidkv_cache_t* h, int32_t layer, uint8_t* dmask, uint8_t* E, void* stream) {
+  if (!h || layer < 0 || layer >= h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  const LayerInfo& li = h->layers[layer];
+  if (dmask && !li.k_done) return VIDKV_ERR_STATE;
+  const int n_chunks = static_cast<int>(1 + li.n_flush);
+  const int64_t T = li.k_done || li.v_done ? li.T : h->sel_T;
+  const int64_t T_sel = h->sel_set && h->n_prot > 0 ? h->sel_T - h->sel_T % kG : 0;
+  if (launch_export_selection(h->cv, layer, n_chunks, dmask, T, T_sel, E, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  return VIDKV_OK;
 }
 
 vidkv_status_t vidkv_dequantize_keys(vidkv_cache_t* h, int32_t layer, float* out, void* stream) {

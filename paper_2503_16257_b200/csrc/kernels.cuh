@@ -31,7 +31,8 @@ struct MinMaxBuffers {
   uint32_t* next;
   int next_dirty_words;
 };
-cudaError_t launch_init_minmax(uint32_t* minmax, int64_t n_words, cudaStream_t stream);
+// Also writes the cache header (magic, version, cleared status word) when `header` is not null.
+cudaError_t launch_init_minmax(uint32_t* minmax, int64_t n_words, uint32_t* header, uint32_t version, cudaStream_t stream);
 
 // Algorithm 3 on `T_tokens` tokens (a multiple of 32) of every slab of layers
 // [layer0, layer0 + n_layers): writes chunk `chunk` of the chunk table and the key groups
@@ -48,7 +49,7 @@ cudaError_t launch_encode_keys(int dtype, const KSrc& src, int64_t T_tokens, con
 // ((ks * 8 + nt) * 32 + lane) * 4 + {0, 1} = leading binary16 pairs, + {2, 3} = remainders, for
 // rows 16 ks + 2 r (+1; +8, +9) and column 16 (n / 2) + 2 nt + (n % 2), lane = 4 n + r; column f
 // holds 1/8, (-1)^c / 8, cos(2 pi k c / 64) / 8 (f = 2k) or -sin(2 pi k c / 64) / 8 (f = 2k + 1).
-// Filled on first use on each device (one small kernel and a stream synchronisation).
+// Filled on first use on each device by one small kernel; later calls order their stream after it with an event.
 cudaError_t dft_fragments(const uint32_t** table, cudaStream_t stream);
 
 // Algorithm 2 on the prefill tokens of one layer.  T_q (multiple of 32) tokens; the
@@ -73,7 +74,7 @@ cudaError_t launch_select_tokens(const float* saliency, int64_t vis_begin, int64
                                  int64_t stride_rest, cudaStream_t stream);
 cudaError_t launch_mask_to_selection(const uint8_t* E, int64_t T, int64_t T_q, const CacheView& cv, int32_t* idx_prot,
                                      int32_t* idx_rest, int64_t stride_prot, int64_t stride_rest, int32_t* counts,
-                                     cudaStream_t stream);
+                                     int64_t expect_count, cudaStream_t stream);
 
 // Token counts the decode kernels need (the same for every layer of one call).
 struct LayerState {
@@ -131,6 +132,7 @@ struct DecodeArgs {
   float scale;
   LayerState st;
   cudaEvent_t ev_begin, ev_end;   // optional: recorded around the attention kernel (profiling)
+  int32_t withhold;    // test hook: the stream kernel does not issue its first value copy
 };
 
 // Eq. 7 scores from hidden states: text_sum [B, d] (scratch) and saliency [B, l_v], both float32.
@@ -140,6 +142,11 @@ cudaError_t launch_saliency(int dtype, const void* x_v, const void* x_t, int64_t
 // Variance / outlier count per (slab, channel) of a key tensor; stats [n_slabs][2][128] float64 scratch.
 cudaError_t launch_channel_metrics(int dtype, const KSrc& src, int64_t n_slabs, int64_t T_tokens, int metric, double M,
                                    double* stats, float* out, cudaStream_t stream);
+
+// Test hook (vidkv_debug_withhold_once): 1 = the next key-encode launch withholds the tensor-core
+// products of every block's first tile, 2 = the next stream-kernel launch withholds every warp's
+// first value copy; the launch that honours it clears it.  0 = off.
+extern int g_debug_withhold;
 
 // Number of kernels launched by this library since it was loaded (host counter).
 extern unsigned long long g_launch_count;
@@ -164,5 +171,12 @@ cudaError_t launch_dequant_keys(const CacheView& cv, int layer, int64_t T_q0, in
                                 cudaStream_t stream);
 cudaError_t launch_dequant_values(const CacheView& cv, int layer, int64_t T_q0, int64_t n_flush, int64_t n_prot,
                                   float* out, cudaStream_t stream);
+
+// Test-only exports: undo the bit packing of one layer into plain arrays (any pointer may be null).
+cudaError_t launch_export_codes(const CacheView& cv, int layer, int64_t n_kgroups, int64_t n_tgroups, int64_t n_pgroups,
+                                int8_t* k2, uint8_t* k1, uint16_t* ks2, uint16_t* kz2, uint16_t* ks1, int8_t* trits,
+                                uint16_t* vs, int8_t* v2, uint16_t* v2s, uint16_t* v2z, cudaStream_t stream);
+cudaError_t launch_export_selection(const CacheView& cv, int layer, int n_chunks, uint8_t* dmask, int64_t T, int64_t T_sel,
+                                    uint8_t* E, cudaStream_t stream);
 
 }  // namespace vidkv

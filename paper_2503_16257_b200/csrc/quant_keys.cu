@@ -150,13 +150,14 @@ static cudaError_t launch_keys_t(const KSrc& src, int64_t T_tokens, const CacheV
   return cudaGetLastError();
 }
 
-__global__ void init_min_kernel(uint32_t* minmax, int n_words) {
+__global__ void init_min_kernel(uint32_t* minmax, int n_words, uint32_t* header, uint32_t version) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n_words) minmax[i] = (i & (2 * kD - 1)) < kD ? 0xffffffffu : 0u;
+  if (header && i == 0) { header[0] = kMagic; header[1] = version; header[2] = 0u; }
 }
 
-cudaError_t launch_init_minmax(uint32_t* minmax, int64_t n_words, cudaStream_t stream) {
-  init_min_kernel<<<static_cast<unsigned>((n_words + 255) / 256), 256, 0, stream>>>(minmax, static_cast<int>(n_words));
+cudaError_t launch_init_minmax(uint32_t* minmax, int64_t n_words, uint32_t* header, uint32_t version, cudaStream_t stream) {
+  init_min_kernel<<<static_cast<unsigned>((n_words + 255) / 256), 256, 0, stream>>>(minmax, static_cast<int>(n_words), header, version);
   count_launches(1);
   return cudaGetLastError();
 }

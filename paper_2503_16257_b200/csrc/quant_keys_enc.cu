@@ -228,7 +228,7 @@ size_t k_encode_smem_bytes(int dtype) { return dtype == VIDKV_F16 ? enc_sm_bytes
 template <typename T>
 __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_tokens, CacheView cv, int layer0,
                                                           int slabs_per_layer, int chunk, int64_t kgroup0,
-                                                          int tiles_per_slab, int total_tiles) {
+                                                          int tiles_per_slab, int total_tiles, int withhold_first) {
   extern __shared__ uint8_t esm_raw[];
   uint8_t* esm = esm_raw + ((1024u - (smem_u32(esm_raw) & 1023u)) & 1023u);
   uint8_t* tile = esm + kSmTile;
@@ -336,7 +336,9 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
     if (*fault) break;
 
     // ---- D[128 rows x 128 tokens] = A (leading) x tile^T; D'[.. x ..] = A (remaining parts) x tile^T
-    if (tid == 0) {
+    // (withhold_first, a test hook: the block's first tile gets neither products nor a commit, so the
+    // wait below runs out with nothing outstanding)
+    if (tid == 0 && !(withhold_first && t == tile_begin)) {
       constexpr uint32_t idesc = (1u << 4) | (static_cast<uint32_t>(Enc<T>::kFmt) << 7) | (static_cast<uint32_t>(Enc<T>::kFmt) << 10) |
                                  ((128u >> 3) << 17) | ((128u >> 4) << 24);
 #pragma unroll
@@ -526,11 +528,14 @@ __global__ void __launch_bounds__(256, 2) k_encode_kernel(KSrc src, int64_t T_to
 // ---------------------------------------------------------------------------------
 // Host launcher of the encode pass
 // ---------------------------------------------------------------------------------
-// The DFT fragments are written once per device, ordered before their first use on `stream`
-// (and, through the synchronisation, before any later use on another stream).
+// The DFT fragments are written once per device by a small kernel on the stream of the first
+// call that needs them, followed by an event; every call makes its stream wait for that event
+// (free once it has completed), so uses on other streams are ordered after the fill without a
+// host-side synchronisation.
 cudaError_t dft_fragments(const uint32_t** table, cudaStream_t stream) {
   static bool done[64] = {};
   static const uint32_t* addr[64] = {};
+  static cudaEvent_t ready[64] = {};
   cudaError_t e;
   int dev = 0;
   if ((e = cudaGetDevice(&dev))) return e;
@@ -538,12 +543,15 @@ cudaError_t dft_fragments(const uint32_t** table, cudaStream_t stream) {
   if (!done[dev]) {
     void* p = nullptr;
     if ((e = cudaGetSymbolAddress(&p, g_dft_frag))) return e;
+    if ((e = cudaEventCreateWithFlags(&ready[dev], cudaEventDisableTiming))) return e;
     dft_table_kernel<<<1, 256, 0, stream>>>();
     if ((e = cudaGetLastError())) return e;
-    if ((e = cudaStreamSynchronize(stream))) return e;
+    if ((e = cudaEventRecord(ready[dev], stream))) return e;
     addr[dev] = static_cast<const uint32_t*>(p);
     done[dev] = true;
     count_launches(1);
+  } else if ((e = cudaStreamWaitEvent(stream, ready[dev], 0))) {
+    return e;
   }
   *table = addr[dev];
   return cudaSuccess;
@@ -569,8 +577,10 @@ static cudaError_t launch_encode_t(const KSrc& src, int64_t T_tokens, const Cach
   if (total <= 0) return cudaSuccess;
   if (total > INT32_MAX) return cudaErrorInvalidValue;
   const int blocks = static_cast<int>(std::min<int64_t>(total, 2 * n_sms[dev]));
+  const int withhold = (g_debug_withhold == 1) ? 1 : 0;
+  if (withhold) g_debug_withhold = 0;
   k_encode_kernel<T><<<blocks, 256, smem, stream>>>(src, T_tokens, cv, layer0, slabs_per_layer, chunk, kgroup0,
-                                                    static_cast<int>(tiles_per_slab), static_cast<int>(total));
+                                                    static_cast<int>(tiles_per_slab), static_cast<int>(total), withhold);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -424,7 +424,8 @@ __global__ void __launch_bounds__(1024) select_tokens_kernel(const float* __rest
                                                              int64_t vis_begin, int64_t l_v, int64_t n_prot,
                                                              int64_t T_q, CacheView cv, int32_t* idx_prot,
                                                              int32_t* idx_rest, int64_t stride_prot,
-                                                             int64_t stride_rest, int32_t* counts) {
+                                                             int64_t stride_rest, int32_t* counts,
+                                                             int64_t expect_count) {
   __shared__ int hist[256];
   __shared__ int s_warp[32];
   __shared__ uint32_t s_prefix, s_need;
@@ -502,6 +503,9 @@ __global__ void __launch_bounds__(1024) select_tokens_kernel(const float* __rest
     e_prefix[W] = static_cast<uint32_t>(prot_carry);
     e_words[W] = 0;
     if (counts) counts[b] = prot_carry;
+    // a mask whose row does not protect the number of tokens the caller stated
+    if (expect_count >= 0 && prot_carry != expect_count)
+      atomicCAS(reinterpret_cast<int*>(cv.base + kHdrStatus), VIDKV_OK, VIDKV_ERR_INVALID_ARG);
   }
 }
 
@@ -591,16 +595,16 @@ cudaError_t launch_select_tokens(const float* saliency, int64_t vis_begin, int64
                                  const CacheView& cv, int32_t* idx_prot, int32_t* idx_rest, int64_t stride_prot,
                                  int64_t stride_rest, cudaStream_t stream) {
   select_tokens_kernel<<<cv.B, 1024, 0, stream>>>(saliency, nullptr, 0, vis_begin, l_v, n_prot, T_q, cv, idx_prot,
-                                                  idx_rest, stride_prot, stride_rest, nullptr);
+                                                  idx_rest, stride_prot, stride_rest, nullptr, -1);
   count_launches(1);
   return cudaGetLastError();
 }
 
 cudaError_t launch_mask_to_selection(const uint8_t* E, int64_t T, int64_t T_q, const CacheView& cv, int32_t* idx_prot,
                                      int32_t* idx_rest, int64_t stride_prot, int64_t stride_rest, int32_t* counts,
-                                     cudaStream_t stream) {
+                                     int64_t expect_count, cudaStream_t stream) {
   select_tokens_kernel<<<cv.B, 1024, 0, stream>>>(nullptr, E, T, 0, 0, 0, T_q, cv, idx_prot, idx_rest, stride_prot,
-                                                  stride_rest, counts);
+                                                  stride_rest, counts, expect_count);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -281,6 +281,52 @@ def test_mixquant_structure_and_dequant():
     assert rel_abn < rel_nom
 
 
+def test_mixquant_dequant_scatters_a_hand_built_chunk_to_its_channels():
+    """DeQuant of a chunk written by hand, against closed forms: the anomalous channels are a constant
+    (s = 0, so every code dequantizes to z), the normal channels hold a spectrum with a single real
+    bin k0 (every other column has scale 0), i.e. a cosine over the normal channels in ascending
+    channel order, which numpy's inverse real FFT gives independently.  Two groups with different
+    amplitudes and per-token signs catch a transposed or mis-scattered result."""
+    T, k0 = 40, 5                                             # one full group and a short one
+    r = rng(77)
+    abn = np.sort(r.permutation(128)[:64])
+    nom = np.setdiff1d(np.arange(128), abn)
+    z2 = np.stack([np.linspace(-3, 3, 64), np.linspace(5, -5, 64)]).astype(np.float16)
+    amp = np.array([2.0, 0.75])
+    s1 = np.zeros((2, 128), dtype=np.float16)
+    s1[:, k0] = amp; s1[:, 64 - k0] = amp                      # Re X[k0] and its mirror bin
+    sign = r.integers(0, 2, size=T)
+    bits1 = np.zeros((T, 128), dtype=np.uint8)
+    bits1[:, k0] = sign; bits1[:, 64 - k0] = sign
+    mq = dict(T=T, abn_idx=abn, nom_idx=nom, codes2=np.zeros((T, 64), dtype=np.int8),
+              s2=np.zeros((2, 64), dtype=np.float16), z2=z2, bits1=bits1, s1=s1)
+    kd = O.mixquant_dequant(mq)
+    assert kd.shape == (T, 128)
+    for t in range(T):
+        g = t // 32
+        assert np.array_equal(kd[t, abn], z2[g].astype(np.float64))
+        spec = np.zeros(33)
+        spec[k0] = (2 * sign[t] - 1) * amp[g]
+        want = np.fft.irfft(spec, n=64, norm="ortho")        # = +-(amp / 4) cos(2 pi k0 n / 64)
+        assert np.allclose(kd[t, nom], want, atol=1e-12)
+        assert np.allclose(want, (2 * sign[t] - 1) * amp[g] / 4 * np.cos(2 * np.pi * k0 * np.arange(64) / 64), atol=1e-12)
+
+
+def test_dequant_1p58_groups_closed_form():
+    """trit * s per (32-token group, channel): hand values, with a short second group."""
+    trits = np.zeros((33, 3), dtype=np.int8)
+    trits[0] = [1, 0, -1]
+    trits[31] = [-1, -1, 1]
+    trits[32] = [1, -1, 0]
+    s = np.array([[2.0, 7.0, 0.5], [3.0, 0.25, 9.0]], dtype=np.float16)
+    out = O.dequant_1p58_groups(trits, s)
+    assert out.shape == (33, 3)
+    assert np.array_equal(out[0], [2.0, 0.0, -0.5])
+    assert np.array_equal(out[31], [-2.0, -7.0, 0.5])
+    assert np.array_equal(out[32], [3.0, -0.25, 0.0])         # the second group's scales
+    assert np.count_nonzero(out[1:31]) == 0
+
+
 def test_mixquant_chunks_do_not_see_each_other():
     k = fp16_values((64, 128), 15)
     k[:32, 5] *= 50            # channel 5 is anomalous only in the first half
