@@ -2,8 +2,9 @@
 // work (plan_decode), the launch sequence, and the last kernel of a step, which merges the
 // partial records of the attention kernels by log-sum-exp and, for caches without protected
 // tokens, attends to the FP16 / BF16 residual itself.
-#include "common.cuh"
-#include "kernels.cuh"
+#include <type_traits>
+
+#include "decode_common.cuh"
 
 namespace vidkv {
 
@@ -84,22 +85,37 @@ int64_t max_decode_records(int64_t max_slabs, int64_t max_tokens, bool stp) {
 }
 
 // ---------------------------------------------------------------------------------
-// One block of 128 threads per slab = (layer, batch element, KV head), serving its query heads.
-// Residual tokens (stream plan): thread t scores token t against every head, a warp per head
-// finds the maximum over the residual scores and the records' maxima and turns the scores into
-// probabilities, thread c accumulates channel c of P V_r; then the records join with their
-// weights 2^(m_record - M).  Scores and maxima are base-2 logits (score * scale * log2 e).
+// One block of 4 warps per slab = (layer, batch element, KV head), serving its query heads.
+// Residual tokens (stream plan): the FP16 / BF16 rows K_r, V_r are staged in shared memory (V_r as
+// binary16; the inputs are representable there), q K_r^T runs on the tensor cores in the input
+// type (rows = heads, columns = tokens; products of two 16-bit values are exact), a warp per head
+// turns the scores and the records' maxima into probabilities (binary16, as in the attention
+// kernels), P V_r runs on the tensor cores with V_r read through transposing matrix loads, and the
+// records join with their weights 2^(m_record - M).  Scores and maxima are base-2 logits.
+// Shared memory for n_pad staged rows (n_res rounded up to 16):
+//   Ks, Vs  n_pad rows of 272 bytes (256 + 16 of padding: conflict-free fragment loads)
+//   S       [8][n_pad] float scores        Ph  [8][n_pad + 8] binary16 probabilities
+//   Mh, Lh  [8] maxima and denominators
 // ---------------------------------------------------------------------------------
+constexpr int kMergeRow = kD * 2 + 16;
+size_t merge_smem_bytes(int n_pad) {
+  return static_cast<size_t>(2) * n_pad * kMergeRow + sizeof(float) * 8 * n_pad + sizeof(__half) * 8 * (n_pad + 8) + 64;
+}
+
 template <typename T>
-__global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int with_residual) {
-  __shared__ float qs[kMaxRep][kD];
-  __shared__ float P[kMaxRep][kR];
-  __shared__ float Mh[kMaxRep], Lh[kMaxRep];
+__global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int n_res, int n_pad) {
+  extern __shared__ __align__(16) uint8_t msm[];
+  uint8_t* Ks = msm;
+  uint8_t* Vs = Ks + n_pad * kMergeRow;
+  float* S = reinterpret_cast<float*>(Vs + n_pad * kMergeRow);
+  __half* Ph = reinterpret_cast<__half*>(S + 8 * n_pad);
+  const int PS = n_pad + 8;
+  float* Mh = reinterpret_cast<float*>(Ph + 8 * PS);
+  float* Lh = Mh + 8;
   const CacheView& cv = a.cv;
-  const int slab = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int slab = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, hd = lane >> 2, r = lane & 3;
   const int h = slab % cv.H_kv, lb = slab / cv.H_kv, rep = cv.rep;
   const uint8_t* slab_ptr = cv.base + cv.slab_offset + (static_cast<int64_t>(a.layer0) * cv.B * cv.H_kv + slab) * cv.slab_stride;
-  const int n_res = with_residual ? a.st.n_res : 0;
   int n_parts;
   {
     const DecodePlan& pl = a.plan;
@@ -112,87 +128,107 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int with
   }
   const float* rec = a.partials + static_cast<int64_t>(slab) * a.plan.parts_stride * (kMaxRep * kRecordFloats);
   const int64_t q0 = (static_cast<int64_t>(lb) * cv.H_q + h * rep) * kD;
-  if (n_res > 0) {
-    const T* qp = reinterpret_cast<const T*>(a.q) + q0;
-    for (int k = 0; k < rep; ++k) qs[k][tid] = Elem<T>::to_float(qp[k * kD + tid]);
-    __syncthreads();
-    if (tid < n_res) {
-      const uint4* kr = reinterpret_cast<const uint4*>(slab_ptr + cv.kres_offset) + tid * (kD / 8);
-      float acc[kMaxRep];
+  if (n_pad > 0) {
+    // ---- stage the residual rows (16-byte pieces, all loads of a thread independent)
+    const uint4* ksrc = reinterpret_cast<const uint4*>(slab_ptr + cv.kres_offset);
+    const uint4* vsrc = reinterpret_cast<const uint4*>(slab_ptr + cv.vres_offset);
+    for (int i = tid; i < n_pad * 16; i += kD) {
+      const int row = i >> 4, col = i & 15;
+      uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
+      if (row < n_res) {
+        kv = __ldg(ksrc + i);
+        vv = __ldg(vsrc + i);
+        if (sizeof(T) == 2 && !std::is_same<T, __half>::value) {      // bfloat16 values -> binary16 (exact for the admitted inputs)
+          uint32_t* w = &vv.x;
 #pragma unroll
-      for (int k = 0; k < kMaxRep; ++k) acc[k] = 0.0f;
-      for (int c8 = 0; c8 < kD / 8; ++c8) {
-        const uint4 v = __ldg(kr + c8);
-        const float2 x0 = Elem<T>::to_float2(v.x), x1 = Elem<T>::to_float2(v.y);
-        const float2 x2 = Elem<T>::to_float2(v.z), x3 = Elem<T>::to_float2(v.w);
-#pragma unroll
-        for (int k = 0; k < kMaxRep; ++k) {
-          if (k < rep) {
-            const float4 qa = *reinterpret_cast<const float4*>(&qs[k][c8 * 8]);
-            const float4 qb = *reinterpret_cast<const float4*>(&qs[k][c8 * 8 + 4]);
-            acc[k] += qa.x * x0.x + qa.y * x0.y + qa.z * x1.x + qa.w * x1.y + qb.x * x2.x + qb.y * x2.y + qb.z * x3.x +
-                      qb.w * x3.y;
+          for (int j = 0; j < 4; ++j) {
+            const float2 f = Elem<T>::to_float2(w[j]);
+            const __half2 hh = __floats2half2_rn(f.x, f.y);
+            w[j] = *reinterpret_cast<const uint32_t*>(&hh);
           }
         }
       }
-      const float sl2 = a.scale * 1.4426950408889634f;
+      *reinterpret_cast<uint4*>(Ks + row * kMergeRow + col * 16) = kv;
+      *reinterpret_cast<uint4*>(Vs + row * kMergeRow + col * 16) = vv;
+    }
+    // ---- q fragments: rows 0-7 = this slab's heads (zero beyond rep), rows 8-15 unused
+    const T* qp = reinterpret_cast<const T*>(a.q) + q0;
+    uint32_t qn[16];
 #pragma unroll
-      for (int k = 0; k < kMaxRep; ++k)
-        if (k < rep) P[k][tid] = acc[k] * sl2;
+    for (int i = 0; i < 16; ++i)
+      qn[i] = hd < rep ? __ldg(reinterpret_cast<const uint32_t*>(qp + hd * kD + 8 * i + 2 * r)) : 0u;
+    __syncthreads();
+    const float sl2 = a.scale * 1.4426950408889634f;
+    for (int tile = warp; tile < n_pad / 8; tile += kD / 32) {
+      const uint32_t* kr = reinterpret_cast<const uint32_t*>(Ks + (tile * 8 + hd) * kMergeRow) + r;
+      float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) mma_in<T>(acc, qn[2 * ks], qn[2 * ks + 1], kr[ks * 8], kr[ks * 8 + 4]);
+      *reinterpret_cast<float2*>(S + hd * n_pad + tile * 8 + 2 * r) = make_float2(acc[0] * sl2, acc[1] * sl2);
     }
     __syncthreads();
   }
-  // maxima and denominators: warp w takes heads w and w + 4
-  for (int k = warp; k < rep; k += kD / 32) {
+  // ---- maxima and denominators: warp w takes heads w and w + 4
+  for (int k = warp; k < kMaxRep; k += kD / 32) {
     float m = -INFINITY;
-    for (int t = lane; t < n_res; t += 32) m = fmaxf(m, P[k][t]);
-    for (int j = lane; j < n_parts; j += 32) m = fmaxf(m, rec[(j * kMaxRep + k) * kRecordFloats]);
+    if (k < rep) {
+      for (int t = lane; t < n_res; t += 32) m = fmaxf(m, S[k * n_pad + t]);
+      for (int j = lane; j < n_parts; j += 32) m = fmaxf(m, rec[(j * kMaxRep + k) * kRecordFloats]);
+    }
 #pragma unroll
     for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     float l = 0.0f;
-    for (int t = lane; t < n_res; t += 32) {
-      const float p = exp2f(P[k][t] - m);
-      P[k][t] = p;
-      l += p;
+    for (int t = lane; t < n_pad; t += 32) {
+      __half ph = __float2half_rn(0.0f);
+      if (k < rep && t < n_res) ph = __float2half_rn(exp2f(S[k * n_pad + t] - m));
+      Ph[k * PS + t] = ph;
+      l += __half2float(ph);
     }
-    for (int j = lane; j < n_parts; j += 32) {
-      const float* pr = rec + (j * kMaxRep + k) * kRecordFloats;
-      l += pr[1] * exp2f(pr[0] - m);
-    }
+    if (k < rep)
+      for (int j = lane; j < n_parts; j += 32) {
+        const float* pr = rec + (j * kMaxRep + k) * kRecordFloats;
+        l += pr[1] * exp2f(pr[0] - m);
+      }
 #pragma unroll
     for (int o = 16; o; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
     if (lane == 0) { Mh[k] = m; Lh[k] = l; }
   }
   __syncthreads();
-  float o[kMaxRep];
+  // ---- P V_r: warp w owns channels 32 w .. 32 w + 31 as four 8-channel tiles
+  float acc[4][4];
 #pragma unroll
-  for (int k = 0; k < kMaxRep; ++k) o[k] = 0.0f;
-  if (n_res > 0) {
-    const T* vres = reinterpret_cast<const T*>(slab_ptr + cv.vres_offset) + tid;
-    for (int t = 0; t < n_res; ++t) {
-      const float v = Elem<T>::to_float(vres[t * kD]);
+  for (int j = 0; j < 4; ++j) { acc[j][0] = 0.0f; acc[j][1] = 0.0f; acc[j][2] = 0.0f; acc[j][3] = 0.0f; }
+  for (int kt = 0; kt < n_pad / 16; ++kt) {
+    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(Ph + hd * PS + 16 * kt + 2 * r);
+    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(Ph + hd * PS + 16 * kt + 2 * r + 8);
+    const uint32_t vrow = static_cast<uint32_t>(__cvta_generic_to_shared(Vs + (16 * kt + (lane & 15)) * kMergeRow + 64 * warp));
 #pragma unroll
-      for (int k = 0; k < kMaxRep; ++k)
-        if (k < rep) o[k] += P[k][t] * v;
+    for (int j = 0; j < 4; ++j) {
+      uint32_t b0, b1;
+      asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(vrow + 16 * j));
+      mma_f16(acc[j], a0, 0u, a2, 0u, b0, b1);
     }
   }
-  for (int j = 0; j < n_parts; ++j) {
+  // ---- join the records: lane (hd, r) holds head hd, channels 32 w + 8 j + 2 r, + 1
+  if (hd < rep) {
+    const float M = Mh[hd], inv = 1.0f / Lh[hd];
+    for (int jp = 0; jp < n_parts; ++jp) {
+      const float* pr = rec + (jp * kMaxRep + hd) * kRecordFloats;
+      const float wgt = exp2f(pr[0] - M);
 #pragma unroll
-    for (int k = 0; k < kMaxRep; ++k) {
-      if (k < rep) {
-        const float* pr = rec + (j * kMaxRep + k) * kRecordFloats;
-        o[k] += exp2f(pr[0] - Mh[k]) * pr[2 + tid];
+      for (int j = 0; j < 4; ++j) {
+        const float2 o = *reinterpret_cast<const float2*>(pr + 2 + 32 * warp + 8 * j + 2 * r);
+        acc[j][0] += wgt * o.x;
+        acc[j][1] += wgt * o.y;
       }
     }
-  }
 #pragma unroll
-  for (int k = 0; k < kMaxRep; ++k) {
-    if (k < rep) {
-      const float v = o[k] / Lh[k];
-      const int64_t i = q0 + k * kD + tid;
-      if (a.out_dtype == VIDKV_F32) reinterpret_cast<float*>(a.out)[i] = v;
-      else if (a.out_dtype == VIDKV_F16) reinterpret_cast<__half*>(a.out)[i] = __float2half_rn(v);
-      else reinterpret_cast<__nv_bfloat16*>(a.out)[i] = __float2bfloat16_rn(v);
+    for (int j = 0; j < 4; ++j) {
+      const float v0 = acc[j][0] * inv, v1 = acc[j][1] * inv;
+      const int64_t i = q0 + hd * kD + 32 * warp + 8 * j + 2 * r;
+      if (a.out_dtype == VIDKV_F32) *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.out) + i) = make_float2(v0, v1);
+      else if (a.out_dtype == VIDKV_F16) *reinterpret_cast<__half2*>(reinterpret_cast<__half*>(a.out) + i) = __floats2half2_rn(v0, v1);
+      else *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(a.out) + i) = __floats2bfloat162_rn(v0, v1);
     }
   }
 }
@@ -209,9 +245,20 @@ cudaError_t launch_decode(const DecodeArgs& a_in, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
   }
   count_launches(1);
-  const int with_residual = a.plan.stream;
-  if (a.in_dtype == VIDKV_F16) decode_merge_kernel<__half><<<n_slabs, kD, 0, stream>>>(a, with_residual);
-  else decode_merge_kernel<__nv_bfloat16><<<n_slabs, kD, 0, stream>>>(a, with_residual);
+  const int n_res = a.plan.stream ? a.st.n_res : 0;       // the split kernel attends to the residual itself
+  const int n_pad = (n_res + 15) / 16 * 16;
+  const size_t smem = merge_smem_bytes(n_pad);
+  static bool attr_set[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!attr_set[dev]) {
+    const int most = static_cast<int>(merge_smem_bytes(kR));
+    if ((e = cudaFuncSetAttribute(decode_merge_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, most))) return e;
+    if ((e = cudaFuncSetAttribute(decode_merge_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, most))) return e;
+    attr_set[dev] = true;
+  }
+  if (a.in_dtype == VIDKV_F16) decode_merge_kernel<__half><<<n_slabs, kD, smem, stream>>>(a, n_res, n_pad);
+  else decode_merge_kernel<__nv_bfloat16><<<n_slabs, kD, smem, stream>>>(a, n_res, n_pad);
   return cudaGetLastError();
 }
 

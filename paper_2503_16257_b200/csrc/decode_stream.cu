@@ -75,11 +75,15 @@ struct Running {
   float m;              // running maximum (base-2 logit) of head hd
 };
 
-// Scores of one 32-token key group: sc[nt][0..1] = q . K' of head hd and tokens 8 nt + 2 r, + 1,
-// in the units of the normalised query.
+// Raw scores of one 32-token key group: sc[nt][0..1] = q . K' of head hd and tokens 8 nt + 2 r, + 1
+// without the group's constant, which is returned in cst (the same for the 32 tokens), all in the
+// units of the normalised query.  Consecutive products go to different accumulators (the four
+// 8-token tiles, and the chain of the constants in between), so that no product waits for the
+// one issued just before it.
 __device__ __forceinline__ void score_group(const uint8_t* kg, int lane, int hd, int r, const uint32_t (&qa)[8],
                                             const uint32_t (&qha)[8], const uint32_t (&qhb)[8], uint32_t m_field,
-                                            uint32_t c_four, uint32_t m_sign, uint32_t c_neg1, float (&sc)[4][2]) {
+                                            uint32_t c_four, uint32_t m_sign, uint32_t c_neg1, float (&sc)[4][2],
+                                            float& cst) {
   uint32_t s2[8], z2[8], s1[8];
   {
     const uint4 x0 = *reinterpret_cast<const uint4*>(kg + kKG_S2 + 32 * r);
@@ -93,19 +97,18 @@ __device__ __forceinline__ void score_group(const uint8_t* kg, int lane, int hd,
     const uint4 w1 = *reinterpret_cast<const uint4*>(kg + kKG_S1 + 32 * r + 16);
     s1[0] = w0.x; s1[1] = w0.y; s1[2] = w0.z; s1[3] = w0.w; s1[4] = w1.x; s1[5] = w1.y; s1[6] = w1.z; s1[7] = w1.w;
   }
-  // constants of the group: column 2 r of the result = sum q z, column 2 r + 1 = sum q s
-  float cst;
-  {
-    float cz[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-    for (int ks = 0; ks < 4; ++ks) mma_f16(cz, qa[2 * ks], 0u, qa[2 * ks + 1], 0u, z2[2 * ks], z2[2 * ks + 1]);
-    cst = cz[0] - 4.0f * cz[1];
-  }
   const uint4 c2 = *reinterpret_cast<const uint4*>(kg + kKG_Codes2 + lane * 16);
   const uint2 c1 = *reinterpret_cast<const uint2*>(kg + kKG_Bits1 + lane * 8);
   const uint32_t w2[4] = {c2.x, c2.y, c2.z, c2.w};
-  const uint32_t h1[4] = {c1.x & 0xffffu, c1.x >> 16, c1.y & 0xffffu, c1.y >> 16};
+  const uint32_t wh[4] = {c2.x >> 6, c2.y >> 6, c2.z >> 6, c2.w >> 6};   // fields 5-7 come from one right shift
+  // sign bits: low lane <- bit 15 - 2 m, high lane <- bit 14 - 2 m of the token's half-word
+  const uint32_t X[4] = {(c1.x & 0xffffu) * 0x00020001u, (c1.x >> 16) * 0x00020001u, (c1.y & 0xffffu) * 0x00020001u,
+                         (c1.y >> 16) * 0x00020001u};
   float acc[4][4];
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) { acc[nt][0] = 0.0f; acc[nt][1] = 0.0f; acc[nt][2] = 0.0f; acc[nt][3] = 0.0f; }
+  // constants of the group: column 2 r of the result = sum q z, column 2 r + 1 = sum q s
+  float cz[4] = {0.0f, 0.0f, 0.0f, 0.0f};
   // anomalous channels: q s as exact binary16 pairs hi + lo against 4 + code
   {
     uint32_t hi2[8], lo2[8];
@@ -115,22 +118,16 @@ __device__ __forceinline__ void score_group(const uint8_t* kg, int lane, int hd,
       lo2[i] = hfms2_u(qa[i], s2[i], hi2[i]);
     }
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      const uint32_t w = w2[nt];
-      uint32_t x[8];
-      x[0] = and_or(w << 8, m_field, c_four);
-      x[1] = and_or(w << 6, m_field, c_four);
-      x[2] = and_or(w << 4, m_field, c_four);
-      x[3] = and_or(w << 2, m_field, c_four);
-      x[4] = and_or(w, m_field, c_four);
-      const uint32_t wh = w >> 6;                           // fields 5-7 through one right shift, then multiplies
-      x[5] = and_or(wh << 4, m_field, c_four);
-      x[6] = and_or(wh << 2, m_field, c_four);
-      x[7] = and_or(wh, m_field, c_four);
-      mma_f16_c(acc[nt], hi2[0], lo2[0], hi2[1], lo2[1], x[0], x[1], cst, cst, 0.0f, 0.0f);
+    for (int ks = 0; ks < 4; ++ks) {
+      mma_f16(cz, qa[2 * ks], 0u, qa[2 * ks + 1], 0u, z2[2 * ks], z2[2 * ks + 1]);
 #pragma unroll
-      for (int ks = 1; ks < 4; ++ks)
-        mma_f16(acc[nt], hi2[2 * ks], lo2[2 * ks], hi2[2 * ks + 1], lo2[2 * ks + 1], x[2 * ks], x[2 * ks + 1]);
+      for (int nt = 0; nt < 4; ++nt) {
+        // fields 2 ks and 2 ks + 1 of the word: shifts by 8 - 4 ks and 6 - 4 ks bits
+        const uint32_t f0 = ks == 0 ? w2[nt] << 8 : ks == 1 ? w2[nt] << 4 : ks == 2 ? w2[nt] : wh[nt] << 2;
+        const uint32_t f1 = ks == 0 ? w2[nt] << 6 : ks == 1 ? w2[nt] << 2 : ks == 2 ? wh[nt] << 4 : wh[nt];
+        mma_f16(acc[nt], hi2[2 * ks], lo2[2 * ks], hi2[2 * ks + 1], lo2[2 * ks + 1], and_or(f0, m_field, c_four),
+                and_or(f1, m_field, c_four));
+      }
     }
   }
   // normal channels in the frequency domain: Q s (leading part + remainder) against +-1
@@ -142,18 +139,18 @@ __device__ __forceinline__ void score_group(const uint8_t* kg, int lane, int hd,
       lo1[i] = hfma2_u(qhb[i], s1[i], hfms2_u(qha[i], s1[i], hi1[i]));
     }
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-      // sign bits: low lane <- bit 15 - 2 m, high lane <- bit 14 - 2 m of the half-word
-      const uint32_t X = h1[nt] * 0x00020001u;
-      uint32_t y[8];
+    for (int ks = 0; ks < 4; ++ks) {
 #pragma unroll
-      for (int m = 0; m < 8; ++m) y[m] = and_xor(X << (2 * m), m_sign, c_neg1);
-#pragma unroll
-      for (int ks = 0; ks < 4; ++ks)
-        mma_f16(acc[nt], hi1[2 * ks], lo1[2 * ks], hi1[2 * ks + 1], lo1[2 * ks + 1], y[2 * ks], y[2 * ks + 1]);
-      sc[nt][0] = acc[nt][0] + acc[nt][2];
-      sc[nt][1] = acc[nt][1] + acc[nt][3];
+      for (int nt = 0; nt < 4; ++nt)
+        mma_f16(acc[nt], hi1[2 * ks], lo1[2 * ks], hi1[2 * ks + 1], lo1[2 * ks + 1],
+                and_xor(X[nt] << (4 * ks), m_sign, c_neg1), and_xor(X[nt] << (4 * ks + 2), m_sign, c_neg1));
     }
+  }
+  cst = cz[0] - 4.0f * cz[1];
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) {
+    sc[nt][0] = acc[nt][0] + acc[nt][2];
+    sc[nt][1] = acc[nt][1] + acc[nt][3];
   }
 }
 
@@ -173,7 +170,8 @@ __device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float
   if (!mbar_wait(kbar, kpar)) return false;
   kpar ^= 1u;
   // ---- scores, group by group; a group's scores replace its (spent) bytes in the key buffer:
-  // float2 (tokens 8 nt + 2 r, + 1 of head hd) at word pair (nt * 32 + lane) of the group
+  // float2 (tokens 8 nt + 2 r, + 1 of head hd) at word pair (nt * 32 + lane) of the group, the
+  // group's additive constant at word 256 + lane
   float mx = -INFINITY;
 #pragma unroll 1
   for (int g = 0; g < NG; ++g) {
@@ -189,15 +187,18 @@ __device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float
         qhb[i] = __ldg(pp + (16 + i) * 32);
       }
     }
-    float sc[4][2];
+    float sc[4][2], cst;
     uint8_t* kg = kbuf + g * kKGroupBytes;
-    score_group(kg, lane, hd, r, qa, qha, qhb, m_field, c_four, m_sign, c_neg1, sc);
+    score_group(kg, lane, hd, r, qa, qha, qhb, m_field, c_four, m_sign, c_neg1, sc, cst);
     __syncwarp();                                           // every lane has read the group's bytes
+    float gm = fmaxf(sc[0][0], sc[0][1]);
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
       reinterpret_cast<float2*>(kg)[nt * 32 + lane] = make_float2(sc[nt][0], sc[nt][1]);
-      mx = fmaxf(mx, fmaxf(sc[nt][0], sc[nt][1]));
+      gm = fmaxf(gm, fmaxf(sc[nt][0], sc[nt][1]));
     }
+    reinterpret_cast<float*>(kg)[256 + lane] = cst;         // the group's constant joins in the exponent
+    mx = fmaxf(mx, gm + cst);
   }
   // ---- probabilities against the running maximum
   mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
@@ -224,10 +225,11 @@ __device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float
   float ps[NG][4];
 #pragma unroll
   for (int g = 0; g < NG; ++g) {
+    const float off = fmaf(reinterpret_cast<const float*>(kbuf + g * kKGroupBytes)[256 + lane], sl2, -run.m);
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
       const float2 v = reinterpret_cast<const float2*>(kbuf + g * kKGroupBytes)[nt * 32 + lane];
-      P[g][nt] = pack_half2(ex2_approx(fmaf(v.x, sl2, -run.m)), ex2_approx(fmaf(v.y, sl2, -run.m)));
+      P[g][nt] = pack_half2(ex2_approx(fmaf(v.x, sl2, off)), ex2_approx(fmaf(v.y, sl2, off)));
     }
     // -5 * (sums of the rounded probabilities) of heads 2 r, 2 r + 1, for rows hd and hd + 8 alike:
     // a product with a matrix of -5, whose accumulator fragment is the initial value of every
