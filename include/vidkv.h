@@ -316,30 +316,29 @@ vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const void* cache
                                     float softmax_scale, void* stream);
 
 /* Test hooks (no counterpart in the paper; the results of a decode call do not depend on them
- * beyond floating-point summation order).  A decode call is cut into work in one of two ways
- * (Algorithm 1 "Decoding" leaves the evaluation order of Eq. 3 open):
- *   - no protected tokens: the quantized tokens of all slabs of the call form one sequence of
- *     160-token units; every warp of the launch walks a run of `run_units` consecutive units;
- *   - protected tokens: one thread block per (slab, split of `split_tokens` tokens).
- * vidkv_debug_set_decode_plan forces split_tokens (160, 320 or 640) and / or run_units (>= 1) for
- * later vidkv_decode_attention calls on this handle; 0 leaves the choice to the library.  A forced
- * plan that needs more partial records than the workspace holds makes the decode call return
- * VIDKV_ERR_CAPACITY.
+ * beyond floating-point summation order).  Algorithm 1 "Decoding" leaves the evaluation order of
+ * Eq. 3 open; the library cuts a decode call into work like this: the quantized tokens of all
+ * slabs of the call form one sequence of 160-token units, and every warp of the launch walks a
+ * run of `run_units` consecutive units (crossing slab boundaries where its run does) and leaves
+ * one partial result per slab it touches.
+ * vidkv_debug_set_decode_plan forces run_units (>= 1) for later vidkv_decode_attention calls on
+ * this handle; 0 leaves the choice to the library.  A forced plan that needs more partial records
+ * than the workspace holds makes the decode call return VIDKV_ERR_CAPACITY.
  * vidkv_debug_decode_plan (host only) reports the plan for given token counts on a device with
- * sm_count multiprocessors: plan_out[10] = { stream kernel? , split_tokens, n_splits,
- * units_per_slab, run_units, n_runs, records per slab, records needed, records the workspace of
- * `cfg` holds, chunk-table entries }. */
-vidkv_status_t vidkv_debug_set_decode_plan(vidkv_cache_t* handle, int32_t split_tokens, int32_t run_units);
+ * sm_count multiprocessors: plan_out[8] = { units per slab, run_units, runs (= warps),
+ * records per slab, records needed, records the workspace of `cfg` holds, chunk-table entries,
+ * units in all }. */
+vidkv_status_t vidkv_debug_set_decode_plan(vidkv_cache_t* handle, int32_t run_units);
 vidkv_status_t vidkv_debug_decode_plan(const vidkv_config_t* cfg, int64_t n_prefill_quantized, int64_t n_flushed_chunks,
                                        int32_t n_residual, int64_t n_protected, int32_t n_layers, int32_t sm_count,
-                                       int32_t split_tokens, int32_t run_units, int64_t* plan_out);
+                                       int32_t run_units, int64_t* plan_out);
 
 /* Test hook for the two bounded device-side waits (no counterpart in the paper).  The key encoder
  * waits on the barrier its tensor-core products commit to, the stream kernel of the decode call
  * on the barriers of its bulk copies; both waits give up after a fixed number of polls, record
  * VIDKV_ERR_TIMEOUT in the cache's status word and leave in order (copies drained, tensor memory
  * freed).  what = 1 makes the next key quantization withhold the products of every block's first
- * tile, what = 2 makes the next decode call without protected tokens withhold every warp's first
+ * tile, what = 2 makes the next decode call (on a cache without protected tokens) withhold every warp's first
  * value copy, so that the waits run out with nothing outstanding; the affected call's results
  * are garbage by design, the flag clears itself, and later calls are normal.  0 switches it off. */
 vidkv_status_t vidkv_debug_withhold_once(int32_t what);

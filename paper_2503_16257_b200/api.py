@@ -90,9 +90,9 @@ _SIGNATURES = {
                                       C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "vidkv_cache_status": (C.c_int32, [C.c_void_p, C.c_void_p]),
     "vidkv_debug_withhold_once": (C.c_int32, [C.c_int32]),
-    "vidkv_debug_set_decode_plan": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),
+    "vidkv_debug_set_decode_plan": (C.c_int32, [C.c_void_p, C.c_int32]),
     "vidkv_debug_decode_plan": (C.c_int32, [C.POINTER(_Config), C.c_int64, C.c_int64, C.c_int32, C.c_int64, C.c_int32,
-                                            C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]),
+                                            C.c_int32, C.c_int32, C.POINTER(C.c_int64)]),
     "vidkv_export_codes": (C.c_int32, [C.c_void_p, C.c_int32] + [C.c_void_p] * 10 + [C.c_void_p]),
     "vidkv_get_selection": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "vidkv_dequantize_keys": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]),
@@ -189,19 +189,17 @@ def vidkv_debug_withhold_once(what: int):
     _check("vidkv_debug_withhold_once", load_library().vidkv_debug_withhold_once(what))
 
 
-_PLAN_FIELDS = ("stream", "split_tokens", "n_splits", "units_per_slab", "run_units", "n_runs", "parts_stride",
-                "records", "records_capacity", "n_chunks")
+_PLAN_FIELDS = ("units_per_slab", "run_units", "n_runs", "parts_stride", "records", "records_capacity", "n_chunks",
+                "n_units")
 
 
 def vidkv_debug_decode_plan(cfg: VidKVConfig, n_prefill_quantized: int, n_flushed_chunks: int, n_residual: int,
-                            n_protected: int, n_layers: int, sm_count: int = 148, split_tokens: int = 0,
-                            run_units: int = 0) -> dict:
+                            n_protected: int, n_layers: int, sm_count: int = 148, run_units: int = 0) -> dict:
     """How a decode call with these token counts would be cut into work (host only, no device)."""
     out = (C.c_int64 * len(_PLAN_FIELDS))()
     c = cfg.to_c()
     _check("vidkv_debug_decode_plan", load_library().vidkv_debug_decode_plan(
-        C.byref(c), n_prefill_quantized, n_flushed_chunks, n_residual, n_protected, n_layers, sm_count, split_tokens,
-        run_units, out))
+        C.byref(c), n_prefill_quantized, n_flushed_chunks, n_residual, n_protected, n_layers, sm_count, run_units, out))
     return dict(zip(_PLAN_FIELDS, [int(v) for v in out]))
 
 
@@ -305,10 +303,9 @@ class VidKVCache:
         b = C.c_void_p(ev_end.cuda_event) if ev_end is not None else C.c_void_p(0)
         _check("vidkv_set_profile_events", self.lib.vidkv_set_profile_events(self.handle, a, b))
 
-    def debug_set_decode_plan(self, split_tokens: int = 0, run_units: int = 0):
-        """Test hook: force the split length (160 / 320 / 640) of the split kernel and the run length
-        (160-token units per warp) of the stream kernel for later decode calls; 0 = choose."""
-        _check("vidkv_debug_set_decode_plan", self.lib.vidkv_debug_set_decode_plan(self.handle, split_tokens, run_units))
+    def debug_set_decode_plan(self, run_units: int = 0):
+        """Test hook: force the run length (160-token units per warp) of later decode calls; 0 = choose."""
+        _check("vidkv_debug_set_decode_plan", self.lib.vidkv_debug_set_decode_plan(self.handle, run_units))
 
     def status(self) -> int:
         return self.lib.vidkv_cache_status(self.handle, _stream_ptr())

@@ -13,15 +13,6 @@ namespace {
 constexpr int kMaxSMs = 256;        // multiprocessor count the sizing formulas assume at most
 constexpr int kMinRunUnits = 2;     // a warp's run is never shorter (one record per 320 tokens at worst)
 
-// Tokens per split of the split kernel: the largest of {640, 320, 160} that still gives
-// >= 4 CTAs per SM on a 148-SM part, else 160.
-int choose_split_tokens(int64_t T_tot, int64_t n_slabs) {
-  const int cand[3] = {640, 320, 160};
-  for (int s : cand)
-    if (n_slabs * ((T_tot + s - 1) / s) >= 592) return s;
-  return 160;
-}
-
 }  // namespace
 
 int device_sm_count() {
@@ -36,57 +27,40 @@ int device_sm_count() {
   return sm_of_device[dev];
 }
 
-DecodePlan plan_decode(const LayerState& st, int64_t n_slabs, int64_t n_prot, int sm_count, int force_split_tokens,
-                       int force_run_units) {
+DecodePlan plan_decode(const LayerState& st, int64_t n_slabs, bool stp, int sm_count, int force_run_units) {
   DecodePlan p = {};
   const int64_t T_qt = st.T_q0 + st.n_flush * kR;
   p.n_chunks = T_qt > 0 ? 1 + static_cast<int32_t>(st.n_flush) : 0;
-  if (n_prot > 0) {
-    const int64_t T_tot = T_qt + st.n_res;
-    p.stream = 0;
-    p.split_tokens = force_split_tokens > 0 ? force_split_tokens : choose_split_tokens(T_tot, n_slabs);
-    p.n_splits = static_cast<int32_t>((T_tot + p.split_tokens - 1) / p.split_tokens);
-    p.parts_stride = p.n_splits;
-  } else {
-    p.stream = 1;
-    p.units_per_slab = static_cast<int32_t>((T_qt + kStreamUnitTokens - 1) / kStreamUnitTokens);
-    p.n_units = n_slabs * p.units_per_slab;
-    const int sms = sm_count < 1 ? 1 : (sm_count > kMaxSMs ? kMaxSMs : sm_count);
-    const int64_t warps = static_cast<int64_t>(sms) * kStreamCtasPerSM * kStreamWarps;
-    int64_t run = (p.n_units + warps - 1) / warps;
-    if (run < kMinRunUnits) run = kMinRunUnits;
-    if (force_run_units > 0) run = force_run_units;
-    p.run_units = static_cast<int32_t>(run);
-    p.n_runs = static_cast<int32_t>((p.n_units + run - 1) / run);
-    p.parts_stride = p.units_per_slab > 0 ? static_cast<int32_t>((p.units_per_slab + run - 1) / run) + 1 : 1;
-  }
+  p.units_per_slab = static_cast<int32_t>((T_qt + kStreamUnitTokens - 1) / kStreamUnitTokens);
+  p.n_units = n_slabs * p.units_per_slab;
+  const int sms = sm_count < 1 ? 1 : (sm_count > kMaxSMs ? kMaxSMs : sm_count);
+  const int64_t warps = static_cast<int64_t>(sms) * (stp ? kStreamStpCtasPerSM : kStreamCtasPerSM) * kStreamWarps;
+  int64_t run = (p.n_units + warps - 1) / warps;
+  if (run < kMinRunUnits) run = kMinRunUnits;
+  if (force_run_units > 0) run = force_run_units;
+  p.run_units = static_cast<int32_t>(run);
+  p.n_runs = static_cast<int32_t>((p.n_units + run - 1) / run);
+  p.parts_stride = p.units_per_slab > 0 ? static_cast<int32_t>((p.units_per_slab + run - 1) / run) + 1 : 1;
   p.records = n_slabs * p.parts_stride * kMaxRep;
   return p;
 }
 
-int64_t max_decode_records(int64_t max_slabs, int64_t max_tokens, bool stp) {
+int64_t max_decode_records(int64_t max_slabs, int64_t max_tokens) {
   if (max_tokens < 1) max_tokens = 1;
-  // Stream kernel: parts per slab = ceil(S / run) + 1 with run >= max(1, n_units / warps) (the
-  // chooser never goes below kMinRunUnits, the test hook may force 1), so
+  // parts per slab = ceil(S / run) + 1 with run >= max(1, n_units / warps) (the chooser never goes
+  // below kMinRunUnits, the test hook may force 1), warps >= 8 per multiprocessor, so
   // slabs * parts <= min(slabs * S, warps + slabs) + slabs for every S.
   const int64_t S = (max_tokens + kStreamUnitTokens - 1) / kStreamUnitTokens;
   const int64_t warps = static_cast<int64_t>(kMaxSMs) * kStreamCtasPerSM * kStreamWarps;
   int64_t parts = max_slabs * S;
   if (parts > warps + max_slabs) parts = warps + max_slabs;
   parts += max_slabs;
-  if (stp) {
-    // Split kernel: 640-token splits give slabs * ceil(T / 640) records; 320- and 160-token splits
-    // are only chosen while the coarser size yields fewer than 592 CTAs, i.e. below 1184 of them.
-    int64_t sp = max_slabs * ((max_tokens + 639) / 640);
-    if (sp < 1184) sp = 1184;
-    if (sp > parts) parts = sp;
-  }
   return parts * kMaxRep;
 }
 
 // ---------------------------------------------------------------------------------
 // One block of 4 warps per slab = (layer, batch element, KV head), serving its query heads.
-// Residual tokens (stream plan): the FP16 / BF16 rows K_r, V_r are staged in shared memory (V_r as
+// Residual tokens: the FP16 / BF16 rows K_r, V_r are staged in shared memory (V_r as
 // binary16; the inputs are representable there), q K_r^T runs on the tensor cores in the input
 // type (rows = heads, columns = tokens; products of two 16-bit values are exact), a warp per head
 // turns the scores and the records' maxima into probabilities (binary16, as in the attention
@@ -119,8 +93,7 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int n_re
   int n_parts;
   {
     const DecodePlan& pl = a.plan;
-    if (!pl.stream) n_parts = pl.n_splits;
-    else if (pl.units_per_slab == 0) n_parts = 0;
+    if (pl.units_per_slab == 0) n_parts = 0;
     else {
       const int64_t u0 = static_cast<int64_t>(slab) * pl.units_per_slab;
       n_parts = static_cast<int>((u0 + pl.units_per_slab - 1) / pl.run_units - u0 / pl.run_units) + 1;
@@ -240,12 +213,12 @@ cudaError_t launch_decode(const DecodeArgs& a_in, cudaStream_t stream) {
   if (a.plan.n_chunks > 0) {
     if ((e = launch_decode_prep(a, stream)) != cudaSuccess) return e;
     if (a.ev_begin) cudaEventRecord(a.ev_begin, stream);
-    e = a.plan.stream ? launch_decode_stream(a, stream) : launch_decode_stp(a, stream);
+    e = a.n_prot > 0 ? launch_decode_stream_stp(a, stream) : launch_decode_stream(a, stream);
     if (a.ev_end) cudaEventRecord(a.ev_end, stream);
     if (e != cudaSuccess) return e;
   }
   count_launches(1);
-  const int n_res = a.plan.stream ? a.st.n_res : 0;       // the split kernel attends to the residual itself
+  const int n_res = a.st.n_res;
   const int n_pad = (n_res + 15) / 16 * 16;
   const size_t smem = merge_smem_bytes(n_pad);
   static bool attr_set[64] = {};

@@ -157,6 +157,71 @@ __device__ __forceinline__ void score_group(const uint8_t* kg, int lane, int hd,
 // Running output of the warp, kept in shared memory: float4 tot[j][lane], j = 2 w + i, holds the
 // accumulator fragment of channels 32 w + 4 hd + 2 i + (e >> 1) and heads 2 r + (e & 1), e = 0..3.
 
+// P V of one staged ternary supergroup: for NG of its groups, P[g][nt] holds the probabilities of
+// head hd at stream tokens 32 g + 8 nt + 2 r, + 1 (binary16 pairs) and ps[g] the accumulator
+// fragment -5 * (sum of those probabilities) of heads 2 r, 2 r + 1.  32 channels (two MMA row
+// blocks) at a time: fragment i of block w covers channels 32 w + 4 hd + 2 i + {0, 1} in rows hd,
+// hd + 8.  Adds into the warp's running output.
+template <int NG>
+__device__ __forceinline__ void pv_ternary(const uint8_t* vbuf, float* totbuf, const uint32_t (&P)[NG][4],
+                                           const float (&ps)[NG][4], int lane, int hd, int r, uint32_t m_field,
+                                           uint32_t c_four) {
+#pragma unroll 1
+  for (int w = 0; w < 4; ++w) {
+    float acc[NG][2][4];
+#pragma unroll
+    for (int kt = 0; kt < 2; ++kt) {
+      const uint2 wa = *reinterpret_cast<const uint2*>(vbuf + ((((kt * 2 + 0) * 4 + w) * 4 + r) * 8 + hd) * 8);
+      const uint2 wb = *reinterpret_cast<const uint2*>(vbuf + ((((kt * 2 + 1) * 4 + w) * 4 + r) * 8 + hd) * 8);
+      uint32_t W[8];
+      W[0] = prmt(wa.x, 0u, 0x4140u); W[1] = prmt(wa.x, 0u, 0x4342u);
+      W[2] = prmt(wb.x, 0u, 0x4140u); W[3] = prmt(wb.x, 0u, 0x4342u);
+      W[4] = prmt(wa.y, 0u, 0x4140u); W[5] = prmt(wa.y, 0u, 0x4342u);
+      W[6] = prmt(wb.y, 0u, 0x4140u); W[7] = prmt(wb.y, 0u, 0x4342u);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) W[k] = mad_u32(W[k], 3u, 0u);          // 3 * byte per 16-bit lane
+#pragma unroll
+      for (int g = 0; g < NG; ++g) {
+        uint32_t A[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          // W holds 3 * (remaining byte) per 16-bit lane; the digit sits at bits 8-9.
+          // Next W = 3 * (W - digit << 8) = 3 W - 3 A + 3 * 0x4400 (no lane ever borrows).
+          // Half of the lanes take that route (two multiply-adds), the other half mask the digit
+          // away and multiply (one logic, one multiply-add): the two pipes share the work.
+          A[k] = and_or(W[k], m_field, c_four);
+          if (g + 1 < NG) {
+            if (k & 1) W[k] = mad_u32(A[k], 0xfffffffdu, mad_u32(W[k], 3u, 0xcc00cc00u));
+            else W[k] = mad_u32(W[k] & 0x00ff00ffu, 3u, 0u);
+          }
+        }
+        const uint32_t b0 = P[g][2 * kt], b1 = P[g][2 * kt + 1];
+        if (kt == 0) {
+          mma_f16_c(acc[g][0], A[0], A[1], A[2], A[3], b0, b1, ps[g][0], ps[g][1], ps[g][2], ps[g][3]);
+          mma_f16_c(acc[g][1], A[4], A[5], A[6], A[7], b0, b1, ps[g][0], ps[g][1], ps[g][2], ps[g][3]);
+        } else {
+          mma_f16(acc[g][0], A[0], A[1], A[2], A[3], b0, b1);
+          mma_f16(acc[g][1], A[4], A[5], A[6], A[7], b0, b1);
+        }
+      }
+    }
+    float4* tp = reinterpret_cast<float4*>(totbuf) + (2 * w) * 32 + lane;
+    float4 t0 = tp[0], t1 = tp[32];
+#pragma unroll
+    for (int g = 0; g < NG; ++g) {
+      const uint2 sc2 = *reinterpret_cast<const uint2*>(vbuf + kSG_Scales + g * (kD * 2) + (32 * w + 4 * hd) * 2);
+      const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc2.x));
+      const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&sc2.y));
+      t0.x += sa.x * acc[g][0][0]; t0.y += sa.x * acc[g][0][1];
+      t0.z += sa.y * acc[g][0][2]; t0.w += sa.y * acc[g][0][3];
+      t1.x += sb.x * acc[g][1][0]; t1.y += sb.x * acc[g][1][1];
+      t1.z += sb.y * acc[g][1][2]; t1.w += sb.y * acc[g][1][3];
+    }
+    tp[0] = t0;
+    tp[32] = t1;
+  }
+}
+
 // One unit of NG (1..5) groups: scores, probabilities, P V into the running state.
 // Returns false if a copy never arrived.
 template <int NG>
@@ -246,67 +311,13 @@ __device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     bulk_load(kbuf, next_k, next_k_bytes, kbar);
   }
-  // ---- P V over the ternary supergroup, 32 channels (two MMA row blocks) at a time: fragment i of
-  // block w covers channels 32 w + 4 hd + 2 i + {0, 1} in rows hd, hd + 8
+  // ---- P V over the ternary supergroup
   if (!mbar_wait(vbar, vpar)) {
     if (more) mbar_wait(kbar, kpar);                        // let the key copy issued above land before leaving
     return false;
   }
   vpar ^= 1u;
-#pragma unroll 1
-  for (int w = 0; w < 4; ++w) {
-    float acc[NG][2][4];
-#pragma unroll
-    for (int kt = 0; kt < 2; ++kt) {
-      const uint2 wa = *reinterpret_cast<const uint2*>(vbuf + ((((kt * 2 + 0) * 4 + w) * 4 + r) * 8 + hd) * 8);
-      const uint2 wb = *reinterpret_cast<const uint2*>(vbuf + ((((kt * 2 + 1) * 4 + w) * 4 + r) * 8 + hd) * 8);
-      uint32_t W[8];
-      W[0] = prmt(wa.x, 0u, 0x4140u); W[1] = prmt(wa.x, 0u, 0x4342u);
-      W[2] = prmt(wb.x, 0u, 0x4140u); W[3] = prmt(wb.x, 0u, 0x4342u);
-      W[4] = prmt(wa.y, 0u, 0x4140u); W[5] = prmt(wa.y, 0u, 0x4342u);
-      W[6] = prmt(wb.y, 0u, 0x4140u); W[7] = prmt(wb.y, 0u, 0x4342u);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) W[k] = mad_u32(W[k], 3u, 0u);          // 3 * byte per 16-bit lane
-#pragma unroll
-      for (int g = 0; g < NG; ++g) {
-        uint32_t A[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          // W holds 3 * (remaining byte) per 16-bit lane; the digit sits at bits 8-9.
-          // Next W = 3 * (W - digit << 8) = 3 W - 3 A + 3 * 0x4400 (no lane ever borrows).
-          // Half of the lanes take that route (two multiply-adds), the other half mask the digit
-          // away and multiply (one logic, one multiply-add): the two pipes share the work.
-          A[k] = and_or(W[k], m_field, c_four);
-          if (g + 1 < NG) {
-            if (k & 1) W[k] = mad_u32(A[k], 0xfffffffdu, mad_u32(W[k], 3u, 0xcc00cc00u));
-            else W[k] = mad_u32(W[k] & 0x00ff00ffu, 3u, 0u);
-          }
-        }
-        const uint32_t b0 = P[g][2 * kt], b1 = P[g][2 * kt + 1];
-        if (kt == 0) {
-          mma_f16_c(acc[g][0], A[0], A[1], A[2], A[3], b0, b1, ps[g][0], ps[g][1], ps[g][2], ps[g][3]);
-          mma_f16_c(acc[g][1], A[4], A[5], A[6], A[7], b0, b1, ps[g][0], ps[g][1], ps[g][2], ps[g][3]);
-        } else {
-          mma_f16(acc[g][0], A[0], A[1], A[2], A[3], b0, b1);
-          mma_f16(acc[g][1], A[4], A[5], A[6], A[7], b0, b1);
-        }
-      }
-    }
-    float4* tp = reinterpret_cast<float4*>(totbuf) + (2 * w) * 32 + lane;
-    float4 t0 = tp[0], t1 = tp[32];
-#pragma unroll
-    for (int g = 0; g < NG; ++g) {
-      const uint2 sc2 = *reinterpret_cast<const uint2*>(vbuf + kSG_Scales + g * (kD * 2) + (32 * w + 4 * hd) * 2);
-      const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc2.x));
-      const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&sc2.y));
-      t0.x += sa.x * acc[g][0][0]; t0.y += sa.x * acc[g][0][1];
-      t0.z += sa.y * acc[g][0][2]; t0.w += sa.y * acc[g][0][3];
-      t1.x += sb.x * acc[g][1][0]; t1.y += sb.x * acc[g][1][1];
-      t1.z += sb.y * acc[g][1][2]; t1.w += sb.y * acc[g][1][3];
-    }
-    tp[0] = t0;
-    tp[32] = t1;
-  }
+  pv_ternary<NG>(vbuf, totbuf, P, ps, lane, hd, r, m_field, c_four);
   __syncwarp();
   if (more && lane == 0) {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -434,6 +445,389 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_st
     return;
   }
   write_record(a, cur_slab, run_id, lane, hd, r, run, totbuf);
+}
+
+// ---------------------------------------------------------------------------------
+// Caches with protected tokens (STPQuant, Algorithm 2): the same walk over 160-token key units,
+// but the values of a unit's tokens sit in two streams whose order differs from the key order:
+// unprotected tokens in the ternary stream (position = token - protected tokens before it;
+// flushed tokens follow from the next group boundary), protected ones in 2-bit groups of 32.
+// The probabilities of a unit are therefore scattered (as binary16) into two per-warp rings in
+// stream order, one row per head, and a ternary supergroup (160 stream positions) or protected
+// group (32) is multiplied as soon as all of its positions have been written.  Positions of a
+// supergroup or group that belong to a neighbouring run stay zero; the neighbour multiplies the
+// same bytes with its own probabilities.  The running maximum is kept integral (base-2), so that
+// probabilities waiting in the rings are rescaled exactly when it moves.
+// Per-warp shared memory: key buffer, ternary supergroup buffer, protected group buffer, running
+// output, ternary ring [8 heads][320 positions], protected ring [8 heads][192 positions].
+// ---------------------------------------------------------------------------------
+namespace {
+
+constexpr int kTRing = 2 * kStreamUnitTokens;          // ternary ring: an unfinished supergroup plus one unit
+constexpr int kPRing = 6 * kG;                         // protected ring: an unfinished group plus one unit
+constexpr int kTRingRow = kTRing * 2 + 16;             // bytes per head row (rows start in different banks)
+constexpr int kPRingRow = kPRing * 2 + 16;
+constexpr int kStpWarpBytes = kKBufBytes + kVBufBytes + kPGBytes + kTotBytes + 8 * kTRingRow + 8 * kPRingRow;
+constexpr uint32_t kMinus4 = 0xc400c400u;              // binary16 pair (-4.0, -4.0)
+
+// P V of one protected group (Eq. 4 codes as 4 + code): P4[nt] = probabilities of head hd at
+// the group's tokens 8 nt + 2 r, + 1.  out += s * (sum (4 + code) p - 4 sum p) + z * sum p.
+__device__ __forceinline__ void pv_protected(const uint8_t* pg, float* totbuf, const uint32_t (&P4)[4], float (&l)[2],
+                                             int lane, int hd, int r, uint32_t m_field, uint32_t c_four) {
+  float cq[4] = {0.0f, 0.0f, 0.0f, 0.0f};               // -4 * (sum of the probabilities) of heads 2 r, 2 r + 1
+  mma_f16(cq, kMinus4, kMinus4, kMinus4, kMinus4, P4[0], P4[1]);
+  mma_f16(cq, kMinus4, kMinus4, kMinus4, kMinus4, P4[2], P4[3]);
+  const float sp0 = -0.25f * cq[0], sp1 = -0.25f * cq[1];
+  l[0] += sp0; l[1] += sp1;
+#pragma unroll 1
+  for (int w = 0; w < 4; ++w) {
+    const int w_off = (((w * 4) + r) * 8 + hd) * 4, m_off = (32 * w + 4 * hd) * 2;
+    const uint32_t wk[2] = {*reinterpret_cast<const uint32_t*>(pg + w_off), *reinterpret_cast<const uint32_t*>(pg + 512 + w_off)};
+    const uint2 sc = *reinterpret_cast<const uint2*>(pg + kPG_S + m_off);
+    const uint2 zc = *reinterpret_cast<const uint2*>(pg + kPG_Z + m_off);
+    float acc[2][4];
+#pragma unroll
+    for (int kt = 0; kt < 2; ++kt) {
+      const uint32_t wd = wk[kt], wh = wd >> 6;
+      uint32_t x[8];
+      x[0] = and_or(wd << 8, m_field, c_four);
+      x[1] = and_or(wd << 6, m_field, c_four);
+      x[2] = and_or(wd << 4, m_field, c_four);
+      x[3] = and_or(wd << 2, m_field, c_four);
+      x[4] = and_or(wd, m_field, c_four);
+      x[5] = and_or(wh << 4, m_field, c_four);
+      x[6] = and_or(wh << 2, m_field, c_four);
+      x[7] = and_or(wh, m_field, c_four);
+      const uint32_t b0 = P4[2 * kt], b1 = P4[2 * kt + 1];
+      if (kt == 0) {
+        mma_f16_c(acc[0], x[0], x[1], x[4], x[5], b0, b1, cq[0], cq[1], cq[2], cq[3]);
+        mma_f16_c(acc[1], x[2], x[3], x[6], x[7], b0, b1, cq[0], cq[1], cq[2], cq[3]);
+      } else {
+        mma_f16(acc[0], x[0], x[1], x[4], x[5], b0, b1);
+        mma_f16(acc[1], x[2], x[3], x[6], x[7], b0, b1);
+      }
+    }
+    const float2 sa = __half22float2(*reinterpret_cast<const __half2*>(&sc.x));
+    const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&sc.y));
+    const float2 za = __half22float2(*reinterpret_cast<const __half2*>(&zc.x));
+    const float2 zb = __half22float2(*reinterpret_cast<const __half2*>(&zc.y));
+    float4* tp = reinterpret_cast<float4*>(totbuf) + (2 * w) * 32 + lane;
+    float4 t0 = tp[0], t1 = tp[32];
+    t0.x += sa.x * acc[0][0] + za.x * sp0; t0.y += sa.x * acc[0][1] + za.x * sp1;
+    t0.z += sa.y * acc[0][2] + za.y * sp0; t0.w += sa.y * acc[0][3] + za.y * sp1;
+    t1.x += sb.x * acc[1][0] + zb.x * sp0; t1.y += sb.x * acc[1][1] + zb.x * sp1;
+    t1.z += sb.y * acc[1][2] + zb.y * sp0; t1.w += sb.y * acc[1][3] + zb.y * sp1;
+    tp[0] = t0;
+    tp[32] = t1;
+  }
+}
+
+__device__ __forceinline__ void zero_ring_range(uint8_t* ring, int row_bytes, int ring_len, int64_t pos_begin, int64_t pos_end,
+                                                int lane) {
+  for (int64_t pos = pos_begin + lane; pos < pos_end; pos += 32) {
+    const int idx = static_cast<int>(pos % ring_len);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) *reinterpret_cast<uint16_t*>(ring + k * row_bytes + idx * 2) = 0;
+  }
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode_stream_stp_kernel(DecodeArgs a) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[kStreamWarps][3];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, hd = lane >> 2, r = lane & 3;
+  const DecodePlan& pl = a.plan;
+  const CacheView& cv = a.cv;
+  const int run_id = blockIdx.x * kStreamWarps + warp;
+  const int64_t u_begin = static_cast<int64_t>(run_id) * pl.run_units;
+  const int64_t u_end = min(u_begin + pl.run_units, pl.n_units);
+  if (u_begin >= u_end) return;
+  uint8_t* kbuf = smem_raw + warp * kStpWarpBytes;
+  uint8_t* vbuf = kbuf + kKBufBytes;
+  uint8_t* pbuf = vbuf + kVBufBytes;
+  float* totbuf = reinterpret_cast<float*>(pbuf + kPGBytes);
+  uint8_t* tring = reinterpret_cast<uint8_t*>(totbuf) + kTotBytes;
+  uint8_t* pring = tring + 8 * kTRingRow;
+  uint64_t* kbar = &bars[warp][0];
+  uint64_t* vbar = &bars[warp][1];
+  uint64_t* pbar = &bars[warp][2];
+  if (lane == 0) {
+    mbar_init(kbar, 1);
+    mbar_init(vbar, 1);
+    mbar_init(pbar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  const uint32_t m_field = kExpand[0], c_four = kExpand[1], m_sign = kExpand[2], c_neg1 = kExpand[3];
+  const int S = pl.units_per_slab;
+  const int64_t T_q0 = a.st.T_q0, T_qt = T_q0 + a.st.n_flush * kR;
+  const int64_t n_groups = T_qt / kG, g0n = T_q0 / kG;
+  const int64_t n_prot = a.n_prot, n_rest = T_q0 - n_prot;
+  const int64_t u_fl0 = (n_rest + kG - 1) / kG * kG;                                  // flushed tokens start here
+  const int64_t tg_total = (n_rest + kG - 1) / kG + (kR / kG) * a.st.n_flush;         // ternary groups that exist
+  const int64_t sg_total = (tg_total + kSGGroups - 1) / kSGGroups;
+  const int64_t pg_total = (n_prot + kG - 1) / kG;
+  const int64_t u_total = tg_total > 0 ? (a.st.n_flush > 0 ? u_fl0 + a.st.n_flush * kR : n_rest) : 0;   // ternary positions in use
+  const uint8_t* slab0 = cv.base + cv.slab_offset + static_cast<int64_t>(a.layer0) * cv.B * cv.H_kv * cv.slab_stride;
+  int slab = static_cast<int>(u_begin / S);
+  int k = static_cast<int>(u_begin - static_cast<int64_t>(slab) * S);
+  auto groups_of = [&](int kk) -> int {
+    const int64_t left = n_groups - static_cast<int64_t>(kk) * kSGGroups;
+    return left < kSGGroups ? static_cast<int>(left) : kSGGroups;
+  };
+  auto key_src = [&](int sl, int kk) -> const uint8_t* {
+    return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.kgroup_offset + static_cast<int64_t>(kk) * kKBufBytes;
+  };
+  if (lane == 0) bulk_load(kbuf, key_src(slab, k), groups_of(k) * kKGroupBytes, kbar);
+  uint32_t kpar = 0u, vpar = 0u, ppar = 0u;
+  bool v_pending = false, p_pending = false;               // a copy into vbuf / pbuf has been issued and not yet waited for
+  Running run;
+  run.l[0] = 0.0f; run.l[1] = 0.0f; run.m = -INFINITY;
+  uint32_t qa[8], qha[8], qhb[8];
+  int cur_chunk = -1, cur_slab = -1;
+  const uint32_t* prep_slab = nullptr;
+  const uint32_t* ew = nullptr;
+  const uint32_t* ep = nullptr;
+  const uint8_t* slab_ptr = nullptr;
+  int64_t sg_next = 0, pg_next = 0;
+  float sl2 = 0.0f;
+  bool ok = true;
+#pragma unroll 1
+  for (int64_t u = u_begin; u < u_end && ok; ++u) {
+    const int64_t t_unit = static_cast<int64_t>(k) * kStreamUnitTokens;
+    if (slab != cur_slab) {
+      if (cur_slab >= 0) write_record(a, cur_slab, run_id, lane, hd, r, run, totbuf);
+      cur_slab = slab;
+      cur_chunk = -1;
+      slab_ptr = slab0 + static_cast<int64_t>(slab) * cv.slab_stride;
+      const int b = (slab / cv.H_kv) % cv.B;
+      ew = cv.e_words(b);
+      ep = cv.e_prefix(b);
+      // zero the running output and both rings
+      for (int i = lane; i < (kTotBytes + 8 * kTRingRow + 8 * kPRingRow) / 16; i += 32)
+        reinterpret_cast<uint4*>(totbuf)[i] = make_uint4(0u, 0u, 0u, 0u);
+      run.l[0] = 0.0f; run.l[1] = 0.0f;
+      run.m = -INFINITY;
+      prep_slab = a.prep + static_cast<int64_t>(slab) * pl.n_chunks * (kPrepWords * 32) + lane;
+      sl2 = __uint_as_float(__ldg(prep_slab + 24 * 32));
+      // where the run enters the two value streams
+      int64_t pp0, uu0;
+      if (t_unit <= T_q0) { pp0 = __ldg(ep + t_unit / kG); uu0 = t_unit - pp0; }
+      else { pp0 = n_prot; uu0 = u_fl0 + (t_unit - T_q0); }
+      sg_next = uu0 / kStreamUnitTokens;
+      pg_next = pp0 / kG;
+      __syncwarp();
+      if (lane == 0) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (sg_next < sg_total) bulk_load(vbuf, slab_ptr + cv.tern_offset + sg_next * kVBufBytes, kVBufBytes, vbar);
+        if (pg_next < pg_total) bulk_load(pbuf, slab_ptr + cv.prot_offset + pg_next * kPGBytes, kPGBytes, pbar);
+      }
+      v_pending = sg_next < sg_total;
+      p_pending = pg_next < pg_total;
+    }
+    const int ng = groups_of(k);
+    int nslab = slab, nk = k + 1;
+    if (nk == S) { nk = 0; ++nslab; }
+    const bool more = u + 1 < u_end;
+    const bool last_of_slab = !more || nslab != slab;      // the run leaves this slab after this unit
+    // ---- scores of the unit's groups into the key buffer (raw scores, then the group's constant)
+    if (!mbar_wait(kbar, kpar)) { ok = false; break; }
+    kpar ^= 1u;
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int g = 0; g < ng; ++g) {
+      const int64_t gidx = static_cast<int64_t>(k) * kSGGroups + g;
+      const int chunk = gidx < g0n ? 0 : 1 + static_cast<int>((gidx - g0n) / (kR / kG));
+      if (chunk != cur_chunk) {
+        cur_chunk = chunk;
+        const uint32_t* pp = prep_slab + static_cast<int64_t>(chunk) * (kPrepWords * 32);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          qa[i] = __ldg(pp + i * 32);
+          qha[i] = __ldg(pp + (8 + i) * 32);
+          qhb[i] = __ldg(pp + (16 + i) * 32);
+        }
+      }
+      float sc[4][2], cst;
+      uint8_t* kg = kbuf + g * kKGroupBytes;
+      score_group(kg, lane, hd, r, qa, qha, qhb, m_field, c_four, m_sign, c_neg1, sc, cst);
+      __syncwarp();
+      float gm = fmaxf(sc[0][0], sc[0][1]);
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) {
+        reinterpret_cast<float2*>(kg)[nt * 32 + lane] = make_float2(sc[nt][0], sc[nt][1]);
+        gm = fmaxf(gm, fmaxf(sc[nt][0], sc[nt][1]));
+      }
+      reinterpret_cast<float*>(kg)[256 + lane] = cst;
+      mx = fmaxf(mx, gm + cst);
+    }
+    // ---- running maximum (integral), exact rescale of everything that is kept in its units
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    {
+      const float mu = mx * sl2;
+      const bool up = mu > run.m + kStaleLog2;
+      if (__any_sync(0xffffffffu, up)) {
+        const float m_new = up ? ceilf(mu) : run.m;
+        const float f = ex2_approx(run.m - m_new);          // a power of two (0 on the first unit)
+        run.m = m_new;
+        const float fa = __shfl_sync(0xffffffffu, f, 8 * r), fb = __shfl_sync(0xffffffffu, f, 8 * r + 4);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float4* t = reinterpret_cast<float4*>(totbuf) + j * 32 + lane;
+          float4 v = *t;
+          v.x *= fa; v.y *= fb; v.z *= fa; v.w *= fb;
+          *t = v;
+        }
+        run.l[0] *= fa; run.l[1] *= fb;
+        // probabilities waiting in the rings: row hd belongs to this lane's head, its four lanes share the row
+        const __half2 f2 = __float2half2_rn(f);
+        for (int i = r; i < kTRingRow / 4; i += 4) {
+          __half2* q = reinterpret_cast<__half2*>(tring + hd * kTRingRow) + i;
+          *q = __hmul2(*q, f2);
+        }
+        for (int i = r; i < kPRingRow / 4; i += 4) {
+          __half2* q = reinterpret_cast<__half2*>(pring + hd * kPRingRow) + i;
+          *q = __hmul2(*q, f2);
+        }
+        __syncwarp();
+      }
+    }
+    // ---- probabilities, scattered into stream order
+#pragma unroll 1
+    for (int g = 0; g < ng; ++g) {
+      const uint8_t* kg = kbuf + g * kKGroupBytes;
+      const float off = fmaf(reinterpret_cast<const float*>(kg)[256 + lane], sl2, -run.m);
+      const int64_t tg = t_unit + g * kG;
+      uint8_t* trow = tring + hd * kTRingRow;
+      uint8_t* prow = pring + hd * kPRingRow;
+      if (tg < T_q0) {
+        const uint32_t word = __ldg(ew + tg / kG);
+        const int64_t base = __ldg(ep + tg / kG);             // protected tokens before the group
+        const int tmod = static_cast<int>((tg - base) % kTRing), pmod = static_cast<int>(base % kPRing);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          const float2 v = reinterpret_cast<const float2*>(kg)[nt * 32 + lane];
+          const __half2 ph = __floats2half2_rn(ex2_approx(fmaf(v.x, sl2, off)), ex2_approx(fmaf(v.y, sl2, off)));
+          const int i = 8 * nt + 2 * r;
+          const int below = __popc(word & ((1u << i) - 1u));
+          const uint32_t e0 = (word >> i) & 1u, e1 = (word >> (i + 1)) & 1u;
+          int d0 = e0 ? pmod + below : tmod + i - below;
+          const int below1 = below + static_cast<int>(e0);
+          int d1 = e1 ? pmod + below1 : tmod + i + 1 - below1;
+          d0 -= e0 ? (d0 >= kPRing ? kPRing : 0) : (d0 >= kTRing ? kTRing : 0);
+          d1 -= e1 ? (d1 >= kPRing ? kPRing : 0) : (d1 >= kTRing ? kTRing : 0);
+          *reinterpret_cast<__half*>((e0 ? prow : trow) + d0 * 2) = __low2half(ph);
+          *reinterpret_cast<__half*>((e1 ? prow : trow) + d1 * 2) = __high2half(ph);
+        }
+      } else {
+        if (tg == T_q0 && u_fl0 > n_rest) zero_ring_range(tring, kTRingRow, kTRing, n_rest, u_fl0, lane);   // the gap before the flushed tokens
+        const int tmod = static_cast<int>((u_fl0 + (tg - T_q0)) % kTRing);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          const float2 v = reinterpret_cast<const float2*>(kg)[nt * 32 + lane];
+          *reinterpret_cast<__half2*>(trow + (tmod + 8 * nt + 2 * r) * 2) =
+              __floats2half2_rn(ex2_approx(fmaf(v.x, sl2, off)), ex2_approx(fmaf(v.y, sl2, off)));
+        }
+      }
+    }
+    __syncwarp();
+    if (more && lane == 0) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      bulk_load(kbuf, key_src(nslab, nk), groups_of(nk) * kKGroupBytes, kbar);
+    }
+    // ---- how far the two streams are complete now
+    const int64_t t_end = t_unit + static_cast<int64_t>(ng) * kG;
+    int64_t pp_hi, u_hi;
+    if (t_end <= T_q0) { pp_hi = __ldg(ep + t_end / kG); u_hi = t_end - pp_hi; }
+    else { pp_hi = n_prot; u_hi = u_fl0 + (t_end - T_q0); }
+    if (last_of_slab) {
+      // what is left of the last supergroup / group belongs to a neighbour (or to nobody): zeros
+      const int64_t sg_end = (u_hi + kStreamUnitTokens - 1) / kStreamUnitTokens * kStreamUnitTokens;
+      zero_ring_range(tring, kTRingRow, kTRing, u_hi, sg_end, lane);
+      zero_ring_range(pring, kPRingRow, kPRing, pp_hi, (pp_hi + kG - 1) / kG * kG, lane);
+      __syncwarp();
+    }
+    // ---- ternary supergroups whose positions are all written
+    while (ok && (last_of_slab ? sg_next * kStreamUnitTokens < u_hi : (sg_next + 1) * kStreamUnitTokens <= u_hi)) {
+      if (!mbar_wait(vbar, vpar)) { ok = false; break; }
+      vpar ^= 1u;
+      v_pending = false;
+      uint32_t P[kSGGroups][4];
+      float ps[kSGGroups][4];
+      const uint8_t* rp = tring + hd * kTRingRow + (static_cast<int>(sg_next & 1) * kStreamUnitTokens + 2 * r) * 2;
+#pragma unroll
+      for (int g = 0; g < kSGGroups; ++g) {
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) P[g][nt] = *reinterpret_cast<const uint32_t*>(rp + (g * kG + 8 * nt) * 2);
+        ps[g][0] = 0.0f; ps[g][1] = 0.0f; ps[g][2] = 0.0f; ps[g][3] = 0.0f;
+        mma_f16(ps[g], kMinus5, kMinus5, kMinus5, kMinus5, P[g][0], P[g][1]);
+        mma_f16(ps[g], kMinus5, kMinus5, kMinus5, kMinus5, P[g][2], P[g][3]);
+        run.l[0] = fmaf(-0.2f, ps[g][0], run.l[0]);
+        run.l[1] = fmaf(-0.2f, ps[g][1], run.l[1]);
+      }
+      pv_ternary<kSGGroups>(vbuf, totbuf, P, ps, lane, hd, r, m_field, c_four);
+      ++sg_next;
+      __syncwarp();
+      if (sg_next < sg_total) {
+        if (lane == 0) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          bulk_load(vbuf, slab_ptr + cv.tern_offset + sg_next * kVBufBytes, kVBufBytes, vbar);
+        }
+        v_pending = true;
+      }
+    }
+    // ---- protected groups whose positions are all written
+    while (ok && (last_of_slab ? pg_next * kG < pp_hi : (pg_next + 1) * kG <= pp_hi)) {
+      if (!mbar_wait(pbar, ppar)) { ok = false; break; }
+      ppar ^= 1u;
+      p_pending = false;
+      uint32_t P4[4];
+      const uint8_t* rp = pring + hd * kPRingRow + (static_cast<int>(pg_next % 6) * kG + 2 * r) * 2;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) P4[nt] = *reinterpret_cast<const uint32_t*>(rp + 8 * nt * 2);
+      pv_protected(pbuf, totbuf, P4, run.l, lane, hd, r, m_field, c_four);
+      ++pg_next;
+      __syncwarp();
+      if (pg_next < pg_total) {
+        if (lane == 0) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          bulk_load(pbuf, slab_ptr + cv.prot_offset + pg_next * kPGBytes, kPGBytes, pbar);
+        }
+        p_pending = true;
+      }
+    }
+    if (last_of_slab && ok) {
+      // copies fetched ahead for a neighbour's part of the streams: let them land, the buffers are reused
+      if (v_pending) { ok = mbar_wait(vbar, vpar); vpar ^= 1u; v_pending = false; }
+      if (ok && p_pending) { ok = mbar_wait(pbar, ppar); ppar ^= 1u; p_pending = false; }
+    }
+    slab = nslab; k = nk;
+  }
+  if (!ok) {
+    if (lane == 0) atomicCAS(reinterpret_cast<int*>(cv.base + kHdrStatus), VIDKV_OK, VIDKV_ERR_TIMEOUT);
+    return;
+  }
+  (void)u_total;
+  write_record(a, cur_slab, run_id, lane, hd, r, run, totbuf);
+}
+
+cudaError_t launch_decode_stream_stp(const DecodeArgs& a, cudaStream_t stream) {
+  const size_t smem = static_cast<size_t>(kStreamWarps) * kStpWarpBytes;
+  static bool attr_set[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!attr_set[dev]) {
+    const cudaError_t e = cudaFuncSetAttribute(decode_stream_stp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set[dev] = true;
+  }
+  const int grid = (a.plan.n_runs + kStreamWarps - 1) / kStreamWarps;
+  if (grid < 1) return cudaSuccess;
+  decode_stream_stp_kernel<<<grid, kStreamWarps * 32, smem, stream>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_decode_stream(const DecodeArgs& a_in, cudaStream_t stream) {

@@ -75,7 +75,7 @@ void plan_workspace(const vidkv_config_t& c, const Layout& L, WsPlan* w) {
   int64_t off = 0;
   w->minmax_off = off;
   off = round_up(off + 2 * static_cast<int64_t>(c.L) * c.B * c.H_kv * 2 * kD * 4, kAlign);   // two alternating buffers
-  w->partial_entries = max_decode_records(static_cast<int64_t>(c.L) * c.B * c.H_kv, L.max_total_tokens, c.p_ratio > 0.0f);
+  w->partial_entries = max_decode_records(static_cast<int64_t>(c.L) * c.B * c.H_kv, L.max_total_tokens);
   w->partials_off = off;
   off = round_up(off + w->partial_entries * kRecordFloats * 4, kAlign);
   w->prep_off = off;
@@ -112,8 +112,7 @@ struct vidkv_cache {
   uint8_t* workspace;
   bool sel_set;
   int64_t sel_T, n_prot;
-  int dbg_split_tokens = 0;     // test hook: forced split length of the split kernel (0 = choose)
-  int dbg_run_units = 0;        // test hook: forced run length of the stream kernel (0 = choose)
+  int dbg_run_units = 0;        // test hook: forced run length of the stream kernels (0 = choose)
   int mm_parity = 0;            // which min / max buffer the next key quantization accumulates into
   int64_t mm_dirty[2] = {0, 0}; // words of each buffer written since it was last re-armed
   std::vector<LayerInfo> layers;
@@ -410,7 +409,7 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
   a.withhold = 0;
   a.st.T_q0 = first.T_q0; a.st.n_flush = first.n_flush; a.st.n_res = first.n_res + 1;
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv;
-  a.plan = plan_decode(a.st, n_slabs, h->n_prot, device_sm_count(), h->dbg_split_tokens, h->dbg_run_units);
+  a.plan = plan_decode(a.st, n_slabs, h->n_prot > 0, device_sm_count(), h->dbg_run_units);
   if (a.plan.records > h->ws.partial_entries) return VIDKV_ERR_CAPACITY;
   if (launch_decode(a, s) != cudaSuccess) return VIDKV_ERR_CUDA;
   const bool flush = a.st.n_res == kR;
@@ -445,23 +444,20 @@ vidkv_status_t vidkv_debug_withhold_once(int32_t what) {
   return VIDKV_OK;
 }
 
-vidkv_status_t vidkv_debug_set_decode_plan(vidkv_cache_t* h, int32_t split_tokens, int32_t run_units) {
-  if (!h) return VIDKV_ERR_INVALID_ARG;
-  if (split_tokens != 0 && split_tokens != 160 && split_tokens != 320 && split_tokens != 640) return VIDKV_ERR_INVALID_ARG;
-  if (run_units < 0) return VIDKV_ERR_INVALID_ARG;
-  h->dbg_split_tokens = split_tokens;
+vidkv_status_t vidkv_debug_set_decode_plan(vidkv_cache_t* h, int32_t run_units) {
+  if (!h || run_units < 0) return VIDKV_ERR_INVALID_ARG;
   h->dbg_run_units = run_units;
   return VIDKV_OK;
 }
 
 vidkv_status_t vidkv_debug_decode_plan(const vidkv_config_t* cfg, int64_t n_prefill_quantized, int64_t n_flushed_chunks,
                                        int32_t n_residual, int64_t n_protected, int32_t n_layers, int32_t sm_count,
-                                       int32_t split_tokens, int32_t run_units, int64_t* plan_out) {
+                                       int32_t run_units, int64_t* plan_out) {
   if (!plan_out) return VIDKV_ERR_INVALID_ARG;
   const vidkv_status_t st = check_config(cfg);
   if (st != VIDKV_OK) return st;
   if (n_layers < 1 || n_layers > cfg->L || n_prefill_quantized < 0 || n_prefill_quantized % kG || n_flushed_chunks < 0 ||
-      n_residual < 0 || n_residual > kR || n_protected < 0 || sm_count < 1)
+      n_residual < 0 || n_residual > kR || n_protected < 0 || sm_count < 1 || run_units < 0)
     return VIDKV_ERR_INVALID_ARG;
   Layout L;
   compute_layout(*cfg, &L);
@@ -469,11 +465,9 @@ vidkv_status_t vidkv_debug_decode_plan(const vidkv_config_t* cfg, int64_t n_pref
   plan_workspace(*cfg, L, &w);
   LayerState ls;
   ls.T_q0 = n_prefill_quantized; ls.n_flush = n_flushed_chunks; ls.n_res = n_residual;
-  const DecodePlan p = plan_decode(ls, static_cast<int64_t>(n_layers) * cfg->B * cfg->H_kv, n_protected, sm_count,
-                                   split_tokens, run_units);
-  plan_out[0] = p.stream; plan_out[1] = p.split_tokens; plan_out[2] = p.n_splits; plan_out[3] = p.units_per_slab;
-  plan_out[4] = p.run_units; plan_out[5] = p.n_runs; plan_out[6] = p.parts_stride; plan_out[7] = p.records;
-  plan_out[8] = w.partial_entries; plan_out[9] = p.n_chunks;
+  const DecodePlan p = plan_decode(ls, static_cast<int64_t>(n_layers) * cfg->B * cfg->H_kv, n_protected > 0, sm_count, run_units);
+  plan_out[0] = p.units_per_slab; plan_out[1] = p.run_units; plan_out[2] = p.n_runs; plan_out[3] = p.parts_stride;
+  plan_out[4] = p.records; plan_out[5] = w.partial_entries; plan_out[6] = p.n_chunks; plan_out[7] = p.n_units;
   return VIDKV_OK;
 }
 

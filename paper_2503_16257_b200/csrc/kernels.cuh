@@ -86,32 +86,28 @@ struct LayerState {
 constexpr int kStreamUnitTokens = 160;  // one unit of the stream kernel: 5 key groups = 1 ternary supergroup
 constexpr int kStreamWarps = 4;         // warps per CTA of the stream kernel
 constexpr int kStreamCtasPerSM = 3;     // its CTAs per multiprocessor (register bound)
+constexpr int kStreamStpCtasPerSM = 2;  // the same for the variant with protected tokens (shared-memory bound)
 constexpr int kPrepWords = 25;     // 32-bit words per lane per (slab, chunk) of prepared query
 constexpr int kRecordFloats = 130; // one partial record: running maximum (base-2 logits), sum, out[128]
 
-// How one attention call over n_slabs slabs is cut into work (host side, decode.cu).
-//   Caches without protected tokens: the stream kernel.  The quantized tokens of all slabs form
-//   one sequence of 160-token units (units_per_slab each); warp number w of the launch walks the
-//   units [w * run_units, (w + 1) * run_units) and leaves one partial record per slab it touches,
-//   record (slab, w - first warp of the slab).
-//   Caches with protected tokens: one CTA per (slab, split of split_tokens tokens), record
-//   (slab, split).
+// How one attention call over n_slabs slabs is cut into work (host side, decode.cu): the
+// quantized tokens of all slabs form one sequence of 160-token units (units_per_slab each); warp
+// number w of the launch walks the units [w * run_units, (w + 1) * run_units) and leaves one
+// partial record per slab it touches, record (slab, w - first warp of the slab).
 // parts_stride = records reserved per slab; the partials buffer holds n_slabs * parts_stride * 8
 // records of kRecordFloats floats.
 struct DecodePlan {
-  int32_t stream;          // 1: stream kernel, 0: split kernel
-  int32_t split_tokens, n_splits;
   int32_t units_per_slab, run_units, n_runs;
   int64_t n_units;
   int32_t parts_stride;
   int32_t n_chunks;        // chunk-table entries the query preparation covers (0: nothing quantized)
   int64_t records;         // n_slabs * parts_stride * 8
 };
-// force_split_tokens / force_run_units: 0 = choose; otherwise the test hook's values.
-DecodePlan plan_decode(const LayerState& st, int64_t n_slabs, int64_t n_prot, int sm_count,
-                       int force_split_tokens, int force_run_units);
+// stp: the cache holds protected tokens (the kernel for them keeps fewer warps per multiprocessor).
+// force_run_units: 0 = choose; otherwise the test hook's value.
+DecodePlan plan_decode(const LayerState& st, int64_t n_slabs, bool stp, int sm_count, int force_run_units);
 // Largest `records` any call on at most max_slabs slabs and max_tokens tokens can plan.
-int64_t max_decode_records(int64_t max_slabs, int64_t max_tokens, bool stp);
+int64_t max_decode_records(int64_t max_slabs, int64_t max_tokens);
 // Multiprocessors of the current device (cached per device); 0 on error.
 int device_sm_count();
 
@@ -123,7 +119,7 @@ struct DecodeArgs {
   void* out;
   float* partials;     // [n_slabs][parts_stride][8 heads][kRecordFloats]
   uint32_t* prep;      // per (slab, chunk) query images of the tensor-core path (decode_prep_bytes)
-  const uint32_t* dft; // DFT matrix fragments (dft_fragments), set by launch_decode_mma
+  const uint32_t* dft; // DFT matrix fragments (dft_fragments), set by launch_decode_prep
   int32_t append_row;  // >= 0: the preparation kernel also writes k_new / v_new into this residual row
   int32_t layer0, n_layers;
   int32_t in_dtype, out_dtype;
@@ -152,15 +148,14 @@ extern int g_debug_withhold;
 extern unsigned long long g_launch_count;
 inline void count_launches(int n) { g_launch_count += static_cast<unsigned long long>(n); }
 
-// Attention over the packed cache + residual: query preparation, the stream or split kernel,
-// then the merge of the partial records (which also attends to the residual for the stream kernel).
+// Attention over the packed cache + residual: query preparation, the stream kernel, then the merge
+// of the partial records, which also attends to the residual.
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
 // Query preparation (and the step's append) for a.plan.n_chunks chunk-table entries per slab.
 cudaError_t launch_decode_prep(DecodeArgs& a, cudaStream_t stream);
-// Caches with protected tokens: one CTA per (slab, split).
-cudaError_t launch_decode_stp(const DecodeArgs& a, cudaStream_t stream);
-// Caches without protected tokens: persistent warps over 160-token units.
+// Persistent warps over 160-token units: caches without / with protected tokens.
 cudaError_t launch_decode_stream(const DecodeArgs& a, cudaStream_t stream);
+cudaError_t launch_decode_stream_stp(const DecodeArgs& a, cudaStream_t stream);
 size_t decode_prep_bytes(int64_t n_slabs, int64_t n_chunks);
 // Write k_new / v_new [n_layers, B, H_kv, D] into row `row` of the residual rings.
 cudaError_t launch_append(int dtype, const void* k_new, const void* v_new, const CacheView& cv, int layer0,

@@ -81,7 +81,7 @@ extern "C" vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const 
   a.withhold = 0;
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * cfg->B * cfg->H_kv;
   a.append_row = -1;
-  a.plan = plan_decode(a.st, n_slabs, n_protected, device_sm_count(), 0, 0);
+  a.plan = plan_decode(a.st, n_slabs, n_protected > 0, device_sm_count(), 0);
   // the array holds the partial records, then (256-byte aligned) the per-chunk query images
   const int64_t prep_at = (a.plan.records * kRecordFloats * 4 + 255) / 256 * 256;
   const int64_t prep_bytes = static_cast<int64_t>(decode_prep_bytes(n_slabs, a.plan.n_chunks));

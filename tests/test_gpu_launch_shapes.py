@@ -1,8 +1,8 @@
 """GPU parity at the launch shapes the benchmark times and at every way a decode call can be cut
 into work: the named workloads at their full sizes (the oracle recomputes sampled slabs), and
-small inputs on which every slab is checked while the test hook forces each split length of the
-split kernel (protected tokens) and several run lengths of the stream kernel (no protected
-tokens), including runs that cross slab boundaries and steps after a residual flush."""
+small inputs on which every slab is checked while the test hook forces several run lengths of the
+stream kernels (without and with protected tokens), including runs that end inside slabs, on slab
+boundaries and span several slabs, and steps after a residual flush."""
 import numpy as np
 import pytest
 import torch
@@ -87,18 +87,15 @@ def _plan(run: SampledRun, n_residual):
 @pytest.mark.parametrize("L,p,steps", [
     (8, 0.0, 2),       # runs of about 23 units: three to four runs per slab
     (28, 0.0, 2),      # the launch bench.py times: runs of 80 units, every run crosses a slab boundary
-    (28, 0.2, 2),      # the launch bench.py --p 0.2 times: 640-token splits of the split kernel
+    (28, 0.2, 2),      # the launch bench.py --p 0.2 times: runs of 120 units (two thirds of the warps)
 ])
 def test_batched_workload_at_the_timed_launch_shape(L, p, steps):
     wl = CONFIGS["batched"]
     samples = [(0, 0, 0), (L // 2, 7, 2), (L - 1, 15, 3), (L - 1, 3, 1)]
     run = SampledRun("batched", L, wl.batch, wl.T, p, steps, samples)
     plan = _plan(run, 1)
-    if p == 0:
-        sm = torch.cuda.get_device_properties(0).multi_processor_count
-        assert plan["stream"] == 1 and plan["run_units"] == -(-(L * 64 * 79) // (sm * 12))      # 80 at L = 28 on 148 SMs
-    else:
-        assert plan["stream"] == 0 and plan["split_tokens"] == 640
+    sm = torch.cuda.get_device_properties(0).multi_processor_count
+    assert plan["run_units"] == -(-(L * 64 * 79) // (sm * (12 if p == 0 else 8)))      # 80 / 120 at L = 28 on 148 SMs
     for _ in range(steps):
         run.decode()
     assert run.cache.status() == 0
@@ -107,13 +104,11 @@ def test_batched_workload_at_the_timed_launch_shape(L, p, steps):
 @pytest.mark.parametrize("p", [0.0, 0.2])
 def test_batched_shape_through_the_flush(p):
     """Two layers at batch 16 (128 slabs): 129 steps, so the 128-token residual is flushed and the step
-    after it attends to the flushed chunk.  With p = 0.2 the split kernel runs 640-token splits
-    (128 slabs x 20 splits), and with 2508 protected tokens per sequence split boundaries fall
-    inside protected groups."""
+    after it attends to the flushed chunk.  With p = 0.2 (2508 protected tokens per sequence) unit and
+    run boundaries fall inside ternary supergroups and protected groups."""
     wl = CONFIGS["batched"]
     run = SampledRun("batched", 2, wl.batch, wl.T, p, 130, [(0, 0, 0), (1, 9, 2)])
-    plan = _plan(run, 1)
-    assert (plan["split_tokens"] == 640) if p > 0 else (plan["stream"] == 1)
+    assert _plan(run, 1)["run_units"] > 2
     for s in range(129):
         run.decode(check=(s < 2 or s >= 126))
     assert run.cache.layer_state(1) == dict(n_quantized=wl.T + 128, n_residual=1, n_chunks=2,
@@ -146,24 +141,27 @@ def test_stress_length_slab(p):
 
 
 # ------------------------------------------------------------------ every plan on small inputs, all slabs checked
-@pytest.mark.parametrize("split_tokens", [160, 320, 640])
+@pytest.mark.parametrize("run_units", [1, 2, 3, 5, 13, 40])
 @pytest.mark.parametrize("name,T,B,L,p", [
-    ("tiny", 2000, 2, 2, 0.2),       # 1984 quantized tokens: 12.4 / 6.2 / 3.1 splits, the last one ragged, 16 residual tokens
+    ("tiny", 2000, 2, 2, 0.2),       # 1984 quantized tokens = 12.4 units per slab, 16 residual tokens
     ("qwen", 1311, 1, 1, 0.5),       # bfloat16, half the visual tokens protected
+    ("tiny", 1632, 1, 1, 0.9),       # long protected stream, short ternary one
 ])
-def test_split_kernel_at_every_split_length(split_tokens, name, T, B, L, p):
+def test_stream_kernel_with_protected_tokens_at_every_run_length(run_units, name, T, B, L, p):
+    """Runs of 1 .. 40 units over caches with protected tokens: runs end inside ternary supergroups and
+    protected groups, which both neighbours then multiply with their own probabilities."""
     pair = Pair(CONFIGS[name], T, B=B, L=L, p=p, max_new=4).prefill()
-    pair.cache.debug_set_decode_plan(split_tokens=split_tokens)
+    pair.cache.debug_set_decode_plan(run_units=run_units)
     for _ in range(3):
         out, ref = pair.decode()
         assert np.abs(out - ref).max() <= _rel_tol(ref)
     assert pair.cache.status() == 0
 
 
-@pytest.mark.parametrize("split_tokens", [320, 640])
-def test_split_kernel_across_a_flush(split_tokens):
+@pytest.mark.parametrize("run_units", [1, 3])
+def test_stream_kernel_with_protected_tokens_across_a_flush(run_units):
     pair = Pair(CONFIGS["tiny"], 1000, B=1, L=1, p=0.2, max_new=125).prefill()    # 992 + 8; flush at step 120
-    pair.cache.debug_set_decode_plan(split_tokens=split_tokens)
+    pair.cache.debug_set_decode_plan(run_units=run_units)
     for s in range(123):
         out, ref = pair.decode()
         assert np.abs(out - ref).max() <= _rel_tol(ref), s

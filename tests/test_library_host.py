@@ -167,9 +167,9 @@ def test_partial_records_fit_the_workspace_for_every_token_count(lib, B, L, T_ma
                         pl = P.vidkv_debug_decode_plan(cfg, T, n_flush, n_res, prot, n_layers, sm_count=sm)
                         assert pl["records"] <= pl["records_capacity"], (n_layers, sm, T, n_flush, n_res, prot, pl)
                         worst = max(worst, pl["records"])
-                        assert pl["stream"] == (1 if prot == 0 else 0)
-                        if pl["stream"] and T > 0:
-                            assert pl["n_runs"] * pl["run_units"] >= n_layers * B * 4 * pl["units_per_slab"]
+                        if T > 0:
+                            assert pl["n_units"] == n_layers * B * 4 * pl["units_per_slab"]
+                            assert pl["n_runs"] * pl["run_units"] >= pl["n_units"]
                             assert pl["parts_stride"] >= -(-pl["units_per_slab"] // pl["run_units"]) + 1
     assert worst > 0
     # a plan forced through the test hook may need more than was reserved (the decode call then
