@@ -459,15 +459,15 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_st
 // same bytes with its own probabilities.  The running maximum is kept integral (base-2), so that
 // probabilities waiting in the rings are rescaled exactly when it moves.
 // Per-warp shared memory: key buffer, ternary supergroup buffer, protected group buffer, running
-// output, ternary ring [8 heads][320 positions], protected ring [8 heads][192 positions].
+// output, and the rings: one row per head with 320 ternary and 192 protected positions.
 // ---------------------------------------------------------------------------------
 namespace {
 
 constexpr int kTRing = 2 * kStreamUnitTokens;          // ternary ring: an unfinished supergroup plus one unit
 constexpr int kPRing = 6 * kG;                         // protected ring: an unfinished group plus one unit
-constexpr int kTRingRow = kTRing * 2 + 16;             // bytes per head row (rows start in different banks)
-constexpr int kPRingRow = kPRing * 2 + 16;
-constexpr int kStpWarpBytes = kKBufBytes + kVBufBytes + kPGBytes + kTotBytes + 8 * kTRingRow + 8 * kPRingRow;
+constexpr int kPRingAt = kTRing * 2;                   // a head's row: 320 ternary entries, then 192 protected ones,
+constexpr int kRingRow = (kTRing + kPRing) * 2 + 48;   // then padding: 1072 bytes, rows start in different banks
+constexpr int kStpWarpBytes = kKBufBytes + kVBufBytes + kPGBytes + kTotBytes + 8 * kRingRow;
 constexpr uint32_t kMinus4 = 0xc400c400u;              // binary16 pair (-4.0, -4.0)
 
 // P V of one protected group (Eq. 4 codes as 4 + code): P4[nt] = probabilities of head hd at
@@ -522,12 +522,13 @@ __device__ __forceinline__ void pv_protected(const uint8_t* pg, float* totbuf, c
   }
 }
 
-__device__ __forceinline__ void zero_ring_range(uint8_t* ring, int row_bytes, int ring_len, int64_t pos_begin, int64_t pos_end,
-                                                int lane) {
-  for (int64_t pos = pos_begin + lane; pos < pos_end; pos += 32) {
-    const int idx = static_cast<int>(pos % ring_len);
+// Zero the entries of stream positions [pos_begin, pos_end) in every head's row; `ring` points at
+// entry 0 of the stream's part of row 0, ring_len is the stream's ring length.
+__device__ __forceinline__ void zero_ring_range(uint8_t* ring, int ring_len, int pos_begin, int pos_end, int lane) {
+  for (int pos = pos_begin + lane; pos < pos_end; pos += 32) {
+    const int idx = pos % ring_len;
 #pragma unroll
-    for (int k = 0; k < 8; ++k) *reinterpret_cast<uint16_t*>(ring + k * row_bytes + idx * 2) = 0;
+    for (int k = 0; k < 8; ++k) *reinterpret_cast<uint16_t*>(ring + k * kRingRow + idx * 2) = 0;
   }
 }
 
@@ -547,8 +548,8 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
   uint8_t* vbuf = kbuf + kKBufBytes;
   uint8_t* pbuf = vbuf + kVBufBytes;
   float* totbuf = reinterpret_cast<float*>(pbuf + kPGBytes);
-  uint8_t* tring = reinterpret_cast<uint8_t*>(totbuf) + kTotBytes;
-  uint8_t* pring = tring + 8 * kTRingRow;
+  uint8_t* rings = reinterpret_cast<uint8_t*>(totbuf) + kTotBytes;
+  uint8_t* myrow = rings + hd * kRingRow;                  // the row of this lane's head
   uint64_t* kbar = &bars[warp][0];
   uint64_t* vbar = &bars[warp][1];
   uint64_t* pbar = &bars[warp][2];
@@ -561,25 +562,26 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
   __syncwarp();
   const uint32_t m_field = kExpand[0], c_four = kExpand[1], m_sign = kExpand[2], c_neg1 = kExpand[3];
   const int S = pl.units_per_slab;
-  const int64_t T_q0 = a.st.T_q0, T_qt = T_q0 + a.st.n_flush * kR;
-  const int64_t n_groups = T_qt / kG, g0n = T_q0 / kG;
-  const int64_t n_prot = a.n_prot, n_rest = T_q0 - n_prot;
-  const int64_t u_fl0 = (n_rest + kG - 1) / kG * kG;                                  // flushed tokens start here
-  const int64_t tg_total = (n_rest + kG - 1) / kG + (kR / kG) * a.st.n_flush;         // ternary groups that exist
-  const int64_t sg_total = (tg_total + kSGGroups - 1) / kSGGroups;
-  const int64_t pg_total = (n_prot + kG - 1) / kG;
-  const int64_t u_total = tg_total > 0 ? (a.st.n_flush > 0 ? u_fl0 + a.st.n_flush * kR : n_rest) : 0;   // ternary positions in use
+  // token and stream positions fit 32 bits (the layout's group counts do)
+  const int T_q0 = static_cast<int>(a.st.T_q0), T_qt = T_q0 + static_cast<int>(a.st.n_flush) * kR;
+  const int n_groups = T_qt / kG, g0n = T_q0 / kG;
+  const int n_prot = static_cast<int>(a.n_prot), n_rest = T_q0 - n_prot;
+  const int u_fl0 = (n_rest + kG - 1) / kG * kG;                                          // flushed tokens start here
+  const int tg_total = (n_rest + kG - 1) / kG + (kR / kG) * static_cast<int>(a.st.n_flush);   // ternary groups that exist
+  const int sg_total = (tg_total + kSGGroups - 1) / kSGGroups;
+  const int pg_total = (n_prot + kG - 1) / kG;
   const uint8_t* slab0 = cv.base + cv.slab_offset + static_cast<int64_t>(a.layer0) * cv.B * cv.H_kv * cv.slab_stride;
   int slab = static_cast<int>(u_begin / S);
   int k = static_cast<int>(u_begin - static_cast<int64_t>(slab) * S);
   auto groups_of = [&](int kk) -> int {
-    const int64_t left = n_groups - static_cast<int64_t>(kk) * kSGGroups;
-    return left < kSGGroups ? static_cast<int>(left) : kSGGroups;
+    const int left = n_groups - kk * kSGGroups;
+    return left < kSGGroups ? left : kSGGroups;
   };
   auto key_src = [&](int sl, int kk) -> const uint8_t* {
     return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.kgroup_offset + static_cast<int64_t>(kk) * kKBufBytes;
   };
   if (lane == 0) bulk_load(kbuf, key_src(slab, k), groups_of(k) * kKGroupBytes, kbar);
+  const uint32_t lt_mask = (1u << lane) - 1u;              // lanes (= tokens of a group) before this one
   uint32_t kpar = 0u, vpar = 0u, ppar = 0u;
   bool v_pending = false, p_pending = false;               // a copy into vbuf / pbuf has been issued and not yet waited for
   Running run;
@@ -590,12 +592,12 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
   const uint32_t* ew = nullptr;
   const uint32_t* ep = nullptr;
   const uint8_t* slab_ptr = nullptr;
-  int64_t sg_next = 0, pg_next = 0;
+  int sg_next = 0, pg_next = 0;
   float sl2 = 0.0f;
   bool ok = true;
 #pragma unroll 1
   for (int64_t u = u_begin; u < u_end && ok; ++u) {
-    const int64_t t_unit = static_cast<int64_t>(k) * kStreamUnitTokens;
+    const int t_unit = k * kStreamUnitTokens;
     if (slab != cur_slab) {
       if (cur_slab >= 0) write_record(a, cur_slab, run_id, lane, hd, r, run, totbuf);
       cur_slab = slab;
@@ -605,23 +607,23 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
       ew = cv.e_words(b);
       ep = cv.e_prefix(b);
       // zero the running output and both rings
-      for (int i = lane; i < (kTotBytes + 8 * kTRingRow + 8 * kPRingRow) / 16; i += 32)
+      for (int i = lane; i < (kTotBytes + 8 * kRingRow) / 16; i += 32)
         reinterpret_cast<uint4*>(totbuf)[i] = make_uint4(0u, 0u, 0u, 0u);
       run.l[0] = 0.0f; run.l[1] = 0.0f;
       run.m = -INFINITY;
       prep_slab = a.prep + static_cast<int64_t>(slab) * pl.n_chunks * (kPrepWords * 32) + lane;
       sl2 = __uint_as_float(__ldg(prep_slab + 24 * 32));
       // where the run enters the two value streams
-      int64_t pp0, uu0;
-      if (t_unit <= T_q0) { pp0 = __ldg(ep + t_unit / kG); uu0 = t_unit - pp0; }
+      int pp0, uu0;
+      if (t_unit <= T_q0) { pp0 = static_cast<int>(__ldg(ep + t_unit / kG)); uu0 = t_unit - pp0; }
       else { pp0 = n_prot; uu0 = u_fl0 + (t_unit - T_q0); }
       sg_next = uu0 / kStreamUnitTokens;
       pg_next = pp0 / kG;
       __syncwarp();
       if (lane == 0) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (sg_next < sg_total) bulk_load(vbuf, slab_ptr + cv.tern_offset + sg_next * kVBufBytes, kVBufBytes, vbar);
-        if (pg_next < pg_total) bulk_load(pbuf, slab_ptr + cv.prot_offset + pg_next * kPGBytes, kPGBytes, pbar);
+        if (sg_next < sg_total) bulk_load(vbuf, slab_ptr + cv.tern_offset + static_cast<int64_t>(sg_next) * kVBufBytes, kVBufBytes, vbar);
+        if (pg_next < pg_total) bulk_load(pbuf, slab_ptr + cv.prot_offset + static_cast<int64_t>(pg_next) * kPGBytes, kPGBytes, pbar);
       }
       v_pending = sg_next < sg_total;
       p_pending = pg_next < pg_total;
@@ -637,8 +639,8 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
     float mx = -INFINITY;
 #pragma unroll 1
     for (int g = 0; g < ng; ++g) {
-      const int64_t gidx = static_cast<int64_t>(k) * kSGGroups + g;
-      const int chunk = gidx < g0n ? 0 : 1 + static_cast<int>((gidx - g0n) / (kR / kG));
+      const int gidx = k * kSGGroups + g;
+      const int chunk = gidx < g0n ? 0 : 1 + (gidx - g0n) / (kR / kG);
       if (chunk != cur_chunk) {
         cur_chunk = chunk;
         const uint32_t* pp = prep_slab + static_cast<int64_t>(chunk) * (kPrepWords * 32);
@@ -683,51 +685,45 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
         run.l[0] *= fa; run.l[1] *= fb;
         // probabilities waiting in the rings: row hd belongs to this lane's head, its four lanes share the row
         const __half2 f2 = __float2half2_rn(f);
-        for (int i = r; i < kTRingRow / 4; i += 4) {
-          __half2* q = reinterpret_cast<__half2*>(tring + hd * kTRingRow) + i;
-          *q = __hmul2(*q, f2);
-        }
-        for (int i = r; i < kPRingRow / 4; i += 4) {
-          __half2* q = reinterpret_cast<__half2*>(pring + hd * kPRingRow) + i;
+        for (int i = r; i < kRingRow / 4; i += 4) {
+          __half2* q = reinterpret_cast<__half2*>(myrow) + i;
           *q = __hmul2(*q, f2);
         }
         __syncwarp();
       }
     }
-    // ---- probabilities, scattered into stream order
+    // ---- probabilities, scattered into stream order.  Where a token goes depends on the token
+    // alone, so lane j works out the destination of the group's token j (byte offset inside a
+    // head's row: 2 * ternary ring index, or kPRingAt + 2 * protected ring index) and the lanes
+    // pick up the destinations of their own four token pairs with shuffles.
 #pragma unroll 1
     for (int g = 0; g < ng; ++g) {
       const uint8_t* kg = kbuf + g * kKGroupBytes;
       const float off = fmaf(reinterpret_cast<const float*>(kg)[256 + lane], sl2, -run.m);
-      const int64_t tg = t_unit + g * kG;
-      uint8_t* trow = tring + hd * kTRingRow;
-      uint8_t* prow = pring + hd * kPRingRow;
+      const int tg = t_unit + g * kG;
       if (tg < T_q0) {
         const uint32_t word = __ldg(ew + tg / kG);
-        const int64_t base = __ldg(ep + tg / kG);             // protected tokens before the group
-        const int tmod = static_cast<int>((tg - base) % kTRing), pmod = static_cast<int>(base % kPRing);
+        const int base = static_cast<int>(__ldg(ep + tg / kG));   // protected tokens before the group
+        const int below = __popc(word & lt_mask);
+        const bool prot = (word >> lane) & 1u;
+        int idx = prot ? (base + below) % kPRing : (tg - base + lane - below) % kTRing;
+        uint32_t dst = static_cast<uint32_t>(prot ? kPRingAt + 2 * idx : 2 * idx);
+        dst |= __shfl_down_sync(0xffffffffu, dst, 1) << 16;   // even lanes: this token and the next
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
           const float2 v = reinterpret_cast<const float2*>(kg)[nt * 32 + lane];
           const __half2 ph = __floats2half2_rn(ex2_approx(fmaf(v.x, sl2, off)), ex2_approx(fmaf(v.y, sl2, off)));
-          const int i = 8 * nt + 2 * r;
-          const int below = __popc(word & ((1u << i) - 1u));
-          const uint32_t e0 = (word >> i) & 1u, e1 = (word >> (i + 1)) & 1u;
-          int d0 = e0 ? pmod + below : tmod + i - below;
-          const int below1 = below + static_cast<int>(e0);
-          int d1 = e1 ? pmod + below1 : tmod + i + 1 - below1;
-          d0 -= e0 ? (d0 >= kPRing ? kPRing : 0) : (d0 >= kTRing ? kTRing : 0);
-          d1 -= e1 ? (d1 >= kPRing ? kPRing : 0) : (d1 >= kTRing ? kTRing : 0);
-          *reinterpret_cast<__half*>((e0 ? prow : trow) + d0 * 2) = __low2half(ph);
-          *reinterpret_cast<__half*>((e1 ? prow : trow) + d1 * 2) = __high2half(ph);
+          const uint32_t d = __shfl_sync(0xffffffffu, dst, 8 * nt + 2 * r);
+          *reinterpret_cast<__half*>(myrow + (d & 0xffffu)) = __low2half(ph);
+          *reinterpret_cast<__half*>(myrow + (d >> 16)) = __high2half(ph);
         }
       } else {
-        if (tg == T_q0 && u_fl0 > n_rest) zero_ring_range(tring, kTRingRow, kTRing, n_rest, u_fl0, lane);   // the gap before the flushed tokens
-        const int tmod = static_cast<int>((u_fl0 + (tg - T_q0)) % kTRing);
+        if (tg == T_q0 && u_fl0 > n_rest) zero_ring_range(rings, kTRing, n_rest, u_fl0, lane);   // the gap before the flushed tokens
+        const int tmod = (u_fl0 + (tg - T_q0)) % kTRing;
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
           const float2 v = reinterpret_cast<const float2*>(kg)[nt * 32 + lane];
-          *reinterpret_cast<__half2*>(trow + (tmod + 8 * nt + 2 * r) * 2) =
+          *reinterpret_cast<__half2*>(myrow + (tmod + 8 * nt + 2 * r) * 2) =
               __floats2half2_rn(ex2_approx(fmaf(v.x, sl2, off)), ex2_approx(fmaf(v.y, sl2, off)));
         }
       }
@@ -738,15 +734,15 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
       bulk_load(kbuf, key_src(nslab, nk), groups_of(nk) * kKGroupBytes, kbar);
     }
     // ---- how far the two streams are complete now
-    const int64_t t_end = t_unit + static_cast<int64_t>(ng) * kG;
-    int64_t pp_hi, u_hi;
-    if (t_end <= T_q0) { pp_hi = __ldg(ep + t_end / kG); u_hi = t_end - pp_hi; }
+    const int t_end = t_unit + ng * kG;
+    int pp_hi, u_hi;
+    if (t_end <= T_q0) { pp_hi = static_cast<int>(__ldg(ep + t_end / kG)); u_hi = t_end - pp_hi; }
     else { pp_hi = n_prot; u_hi = u_fl0 + (t_end - T_q0); }
     if (last_of_slab) {
       // what is left of the last supergroup / group belongs to a neighbour (or to nobody): zeros
-      const int64_t sg_end = (u_hi + kStreamUnitTokens - 1) / kStreamUnitTokens * kStreamUnitTokens;
-      zero_ring_range(tring, kTRingRow, kTRing, u_hi, sg_end, lane);
-      zero_ring_range(pring, kPRingRow, kPRing, pp_hi, (pp_hi + kG - 1) / kG * kG, lane);
+      const int sg_end = (u_hi + kStreamUnitTokens - 1) / kStreamUnitTokens * kStreamUnitTokens;
+      zero_ring_range(rings, kTRing, u_hi, sg_end, lane);
+      zero_ring_range(rings + kPRingAt, kPRing, pp_hi, (pp_hi + kG - 1) / kG * kG, lane);
       __syncwarp();
     }
     // ---- ternary supergroups whose positions are all written
@@ -756,7 +752,7 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
       v_pending = false;
       uint32_t P[kSGGroups][4];
       float ps[kSGGroups][4];
-      const uint8_t* rp = tring + hd * kTRingRow + (static_cast<int>(sg_next & 1) * kStreamUnitTokens + 2 * r) * 2;
+      const uint8_t* rp = myrow + ((sg_next & 1) * kStreamUnitTokens + 2 * r) * 2;
 #pragma unroll
       for (int g = 0; g < kSGGroups; ++g) {
 #pragma unroll
@@ -773,7 +769,7 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
       if (sg_next < sg_total) {
         if (lane == 0) {
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          bulk_load(vbuf, slab_ptr + cv.tern_offset + sg_next * kVBufBytes, kVBufBytes, vbar);
+          bulk_load(vbuf, slab_ptr + cv.tern_offset + static_cast<int64_t>(sg_next) * kVBufBytes, kVBufBytes, vbar);
         }
         v_pending = true;
       }
@@ -784,7 +780,7 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
       ppar ^= 1u;
       p_pending = false;
       uint32_t P4[4];
-      const uint8_t* rp = pring + hd * kPRingRow + (static_cast<int>(pg_next % 6) * kG + 2 * r) * 2;
+      const uint8_t* rp = myrow + kPRingAt + ((pg_next % 6) * kG + 2 * r) * 2;
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) P4[nt] = *reinterpret_cast<const uint32_t*>(rp + 8 * nt * 2);
       pv_protected(pbuf, totbuf, P4, run.l, lane, hd, r, m_field, c_four);
@@ -793,7 +789,7 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
       if (pg_next < pg_total) {
         if (lane == 0) {
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          bulk_load(pbuf, slab_ptr + cv.prot_offset + pg_next * kPGBytes, kPGBytes, pbar);
+          bulk_load(pbuf, slab_ptr + cv.prot_offset + static_cast<int64_t>(pg_next) * kPGBytes, kPGBytes, pbar);
         }
         p_pending = true;
       }
@@ -809,7 +805,6 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
     if (lane == 0) atomicCAS(reinterpret_cast<int*>(cv.base + kHdrStatus), VIDKV_OK, VIDKV_ERR_TIMEOUT);
     return;
   }
-  (void)u_total;
   write_record(a, cur_slab, run_id, lane, hd, r, run, totbuf);
 }
 
