@@ -28,11 +28,12 @@ if ROOT not in sys.path:
 
 NOMINAL_HBM_GBS = 8000.0          # the 8 TB/s the targets are quoted against
 FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used if MEASURED_PEAKS.json is absent
-# DRAM bytes per cached token per KV head moved by one launch of the split-KV decode kernel, from the
-# ncu captures summarised in profiles/decode_mma_kernel_batched_4layers.txt (p = 0) and
-# profiles/decode_stp_kernel_batched_4layers_p02.txt (p > 0): a 4-layer cut of the batched workload,
-# scaled to the launch by the token-heads it processes (traffic is proportional to them).
-NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = {"decode_stream_kernel": None, "decode_stp_kernel": None}
+# DRAM bytes per cached token per KV head moved by one launch of the decode attention kernel, from the
+# ncu captures summarised in profiles/decode_stream_kernel_batched_4layers.txt (p = 0) and
+# profiles/decode_stream_stp_kernel_batched_4layers_p02.txt (p > 0): a 4-layer cut of the batched workload
+# (3 211 264 cached token-heads per launch), scaled to the launch by the token-heads it processes
+# (traffic is proportional to them).
+NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = {"decode_stream_kernel": 72.15, "decode_stream_stp_kernel": 79.28}
 
 
 def algorithmic_decode_bytes(B, L, H_kv, H_q, T_q0, n_flush, n_res, n_prot, elem=2):
@@ -122,7 +123,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample(wl, p, device_tensors=None):
+def oracle_sample(wl, p, device_tensors=None, max_batch=8, n_steps=8):
     """Time the CPU oracle, as it stands, on a bounded sample of the workload (about ten seconds of
     host time on the batched shape): layer 0, up to 8 batch elements, all KV heads, full T, K+V
     quantize once and 8 decode steps."""
@@ -135,7 +136,7 @@ def oracle_sample(wl, p, device_tensors=None):
     except Exception:
         threads = os.cpu_count() or 1
     T = min(wl.T, 12544)
-    nb = min(wl.batch, 8)
+    nb = min(wl.batch, max_batch)
     if device_tensors is not None:
         K, V = device_tensors
         K, V = K[:nb, :, :T].float().cpu(), V[:nb, :, :T].float().cpu()
@@ -157,7 +158,6 @@ def oracle_sample(wl, p, device_tensors=None):
             sc.prefill(K[b, h].float().numpy(), V[b, h].float().numpy(), E[b] if E is not None else None)
             slabs.append(sc)
     t_quant = time.perf_counter() - t0
-    n_steps = 8
     rep = 7   # query heads per KV head in every workload
     t0 = time.perf_counter()
     for s in range(n_steps):
@@ -224,6 +224,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-token-scores", action="store_true", help="skip the stand-alone timing of vidkv_saliency_scores")
+    ap.add_argument("--no-variants", action="store_true", help="skip the warm / cold and per-layer-launch figures of "
+                    "the workloads whose packed cache fits L2")
     args = ap.parse_args()
 
     from dataclasses import replace
@@ -355,7 +357,7 @@ def main():
     q_tokens = n_caches * B * T * L
     kern_bytes = dec_bytes / steps_dec
     kern_gbs = kern_bytes / (kern_avg_ms * 1e-3) / 1e9
-    kernel_name = "decode_stp_kernel" if n_prot > 0 else "decode_stream_kernel"
+    kernel_name = "decode_stream_stp_kernel" if n_prot > 0 else "decode_stream_kernel"
     traffic = NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD.get(kernel_name)
     if traffic is not None:
         traffic = traffic * B * L * H * (T - T % 32)
@@ -378,6 +380,14 @@ def main():
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
+    # what the packed cache saves: FP16 K and V of the prompt against the bytes the layout holds for it
+    fp16_bytes = 2 * 2 * 128 * H * B * L * T
+    packed_bytes = B * L * H * ((T // 32) * 1152 + ((T - T % 32 - n_prot + 31) // 32) * (5376 / 5) + ((n_prot + 31) // 32) * 1536
+                                + (T % 32) * 512)
+    line["memory"] = {"fp16_kv_bytes": fp16_bytes, "packed_kv_bytes": packed_bytes,
+                      "bytes_saved_vs_fp16": fp16_bytes - packed_bytes, "saved_frac": 1.0 - packed_bytes / fp16_bytes}
+    if rank == 0 and world == 1 and one_cache < 400e6 and not args.no_variants:
+        line["l2_sized_variants"] = run_variants(P, torch, wl, cfg, caches, qs, ks, vs, out, n_prot, quantize)
 
     if rank == 0 and not args.no_e2e:
         line["e2e"] = run_e2e(P, torch, wl, cfg, caches[0], Ks, Vs, qs, ks, vs, sal, out, n_prot, dev, world)
@@ -386,6 +396,15 @@ def main():
         line["cpu_baseline"] = {"value": res["decode_gbs"], "unit": "GB/s", "cores": res["cores"], "kind": "oracle",
                                 "sample": res["sample"], "quantize_tokens_per_s": res["quantize_tokens_per_s"],
                                 "seconds": res["seconds"]}
+        try:                                           # the same oracle on one thread, on a quarter of the sample
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                one = oracle_sample(wl, args.p, device_tensors=(Ks[0], Vs[0]), max_batch=2, n_steps=4)
+            line["cpu_baseline"]["single_thread"] = {"value": one["decode_gbs"], "unit": "GB/s", "cores": 1,
+                                                     "quantize_tokens_per_s": one["quantize_tokens_per_s"],
+                                                     "seconds": one["seconds"], "sample": one["sample"]}
+        except Exception as e:                         # threadpoolctl missing: say so instead of guessing
+            line["cpu_baseline"]["single_thread"] = {"unavailable": repr(e)}
     if rank == 0 and not args.no_token_scores:
         line["token_scores"] = run_token_scores(P, torch, wl, dev, peak)
         line["channel_metrics"] = run_channel_metrics(P, torch, Ks, peak)
@@ -393,6 +412,43 @@ def main():
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_variants(P, torch, wl, cfg, caches, qs, ks, vs, out, n_prot, quantize):
+    """Workloads whose packed cache fits the 126 MB L2 (tiny, LLaVA-shaped, Qwen-shaped): decode GB/s of
+    algorithmic bytes with the cache cold (rotating over copies larger than L2 in sum) and warm (the same
+    cache every step), and with one library call per decode step for all layers or one call per layer."""
+    L, B, T, H, HQ = wl.layers, wl.batch, wl.T, 4, 28
+    n_steps = min(32, wl.steps)
+    res = {}
+    for cold in (True, False):
+        for per_layer in (False, True):
+            use = caches if cold else caches[:1]
+            for c in use:
+                quantize(c)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            nbytes = 0.0
+            e0.record()
+            for s in range(n_steps * len(use)):
+                c = use[s % len(use)]
+                st = c.layer_state(0)
+                i = s // len(use)
+                if per_layer:
+                    for layer in range(L):
+                        c.decode_attention(layer, 1, qs[i][layer:layer + 1], ks[i][layer:layer + 1], vs[i][layer:layer + 1],
+                                           out[layer:layer + 1])
+                else:
+                    c.decode_attention(0, L, qs[i], ks[i], vs[i], out)
+                nbytes += algorithmic_decode_bytes(B, L, H, HQ, T - T % 32, 0, st["n_residual"] + 1, n_prot)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            res[("cold" if cold else "warm") + ("_per_layer_calls" if per_layer else "_one_call")] = {
+                "GBps": nbytes / (ms * 1e-3) / 1e9, "us_per_decode_step": 1e3 * ms / (n_steps * len(use))}
+    res["note"] = ("cold: every step reads a cache that is not in L2 (rotation over %d copies); warm: one cache, L2-resident; "
+                   "per_layer_calls: %d library calls per decode step instead of one" % (len(caches), L))
+    return res
 
 
 def run_channel_metrics(P, torch, Ks, peak):
@@ -499,8 +555,12 @@ def run_e2e(P, torch, wl, cfg, cache, Ks, Vs, qs, ks, vs, sal, out, n_prot, dev,
         t1.record()
         torch.cuda.synchronize()
         dms += e_mid.elapsed_time(t1); tot += t0.elapsed_time(t1)
-    return {"value": world * dec_bytes / (dms / n * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": int(h2d),
-            "d2h_bytes_per_step": int(d2h), "ms_per_step": tot / n, "decode_ms_per_step": dms / n, "steps": n,
+    return {"value": world * dec_bytes / (dms / n * 1e-3) / 1e9, "unit": "GB/s",
+            "scope": "decode part of the step: per decode step H2D of q, k_new, v_new, the attention call, D2H of the output "
+                     "and a stream synchronisation; the H2D of the prompt's K and V sits in the quantize part",
+            "whole_step_value": world * dec_bytes / (tot / n * 1e-3) / 1e9,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": tot / n,
+            "decode_ms_per_step": dms / n, "steps": n,
             "quantize_tokens_per_s": world * B * T * L / ((tot - dms) / n * 1e-3)}
 
 

@@ -101,28 +101,56 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int n_re
   }
   const float* rec = a.partials + static_cast<int64_t>(slab) * a.plan.parts_stride * (kMaxRep * kRecordFloats);
   const int64_t q0 = (static_cast<int64_t>(lb) * cv.H_q + h * rep) * kD;
+  // ---- the records' maxima, sums and this lane's output fragments are fetched first, so that their
+  // latency passes behind the staging of the residual (the first kRecAhead records; more are read later)
+  constexpr int kRecAhead = 3;
+  float rec_m[kRecAhead], rec_l[kRecAhead];
+  float2 rec_o[kRecAhead][4];
+#pragma unroll
+  for (int jp = 0; jp < kRecAhead; ++jp) {
+    rec_m[jp] = -INFINITY; rec_l[jp] = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) rec_o[jp][j] = make_float2(0.0f, 0.0f);
+    if (jp < n_parts && hd < rep) {
+      const float* pr = rec + (jp * kMaxRep + hd) * kRecordFloats;
+      rec_m[jp] = __ldg(pr);
+      rec_l[jp] = __ldg(pr + 1);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) rec_o[jp][j] = __ldg(reinterpret_cast<const float2*>(pr + 2 + 32 * warp + 8 * j + 2 * r));
+    }
+  }
+  (void)rec_l;
   if (n_pad > 0) {
     // ---- stage the residual rows (16-byte pieces, all loads of a thread independent)
     const uint4* ksrc = reinterpret_cast<const uint4*>(slab_ptr + cv.kres_offset);
     const uint4* vsrc = reinterpret_cast<const uint4*>(slab_ptr + cv.vres_offset);
+    constexpr bool kConvert = !std::is_same<T, __half>::value;          // bfloat16 values -> binary16 (exact for the admitted inputs)
     for (int i = tid; i < n_pad * 16; i += kD) {
       const int row = i >> 4, col = i & 15;
-      uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
+      uint8_t* kd = Ks + row * kMergeRow + col * 16;
+      uint8_t* vd = Vs + row * kMergeRow + col * 16;
       if (row < n_res) {
-        kv = __ldg(ksrc + i);
-        vv = __ldg(vsrc + i);
-        if (sizeof(T) == 2 && !std::is_same<T, __half>::value) {      // bfloat16 values -> binary16 (exact for the admitted inputs)
-          uint32_t* w = &vv.x;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const float2 f = Elem<T>::to_float2(w[j]);
-            const __half2 hh = __floats2half2_rn(f.x, f.y);
-            w[j] = *reinterpret_cast<const uint32_t*>(&hh);
-          }
-        }
+        cp_async16(kd, ksrc + i);
+        if (!kConvert) cp_async16(vd, vsrc + i);
+      } else {
+        *reinterpret_cast<uint4*>(kd) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(vd) = make_uint4(0u, 0u, 0u, 0u);
       }
-      *reinterpret_cast<uint4*>(Ks + row * kMergeRow + col * 16) = kv;
-      *reinterpret_cast<uint4*>(Vs + row * kMergeRow + col * 16) = vv;
+    }
+    cp_async_commit();
+    if (kConvert) {
+#pragma unroll 4
+      for (int i = tid; i < n_res * 16; i += kD) {
+        uint4 vv = __ldg(vsrc + i);
+        uint32_t* w = &vv.x;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 f = Elem<T>::to_float2(w[j]);
+          const __half2 hh = __floats2half2_rn(f.x, f.y);
+          w[j] = *reinterpret_cast<const uint32_t*>(&hh);
+        }
+        *reinterpret_cast<uint4*>(Vs + (i >> 4) * kMergeRow + (i & 15) * 16) = vv;
+      }
     }
     // ---- q fragments: rows 0-7 = this slab's heads (zero beyond rep), rows 8-15 unused
     const T* qp = reinterpret_cast<const T*>(a.q) + q0;
@@ -130,6 +158,7 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int n_re
 #pragma unroll
     for (int i = 0; i < 16; ++i)
       qn[i] = hd < rep ? __ldg(reinterpret_cast<const uint32_t*>(qp + hd * kD + 8 * i + 2 * r)) : 0u;
+    cp_async_wait<0>();
     __syncthreads();
     const float sl2 = a.scale * 1.4426950408889634f;
     for (int tile = warp; tile < n_pad / 8; tile += kD / 32) {
@@ -146,7 +175,7 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int n_re
     float m = -INFINITY;
     if (k < rep) {
       for (int t = lane; t < n_res; t += 32) m = fmaxf(m, S[k * n_pad + t]);
-      for (int j = lane; j < n_parts; j += 32) m = fmaxf(m, rec[(j * kMaxRep + k) * kRecordFloats]);
+      for (int j = lane; j < n_parts; j += 32) m = fmaxf(m, __ldg(rec + (j * kMaxRep + k) * kRecordFloats));
     }
 #pragma unroll
     for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -185,7 +214,16 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int n_re
   // ---- join the records: lane (hd, r) holds head hd, channels 32 w + 8 j + 2 r, + 1
   if (hd < rep) {
     const float M = Mh[hd], inv = 1.0f / Lh[hd];
-    for (int jp = 0; jp < n_parts; ++jp) {
+#pragma unroll
+    for (int jp = 0; jp < kRecAhead; ++jp) {
+      const float wgt = exp2f(rec_m[jp] - M);                // 0 for a record that does not exist
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        acc[j][0] += wgt * rec_o[jp][j].x;
+        acc[j][1] += wgt * rec_o[jp][j].y;
+      }
+    }
+    for (int jp = kRecAhead; jp < n_parts; ++jp) {
       const float* pr = rec + (jp * kMaxRep + hd) * kRecordFloats;
       const float wgt = exp2f(pr[0] - M);
 #pragma unroll
