@@ -155,7 +155,7 @@ typedef struct {
 typedef struct vidkv_cache vidkv_cache_t;
 
 /* Sizes (host only).  cache_bytes / workspace_bytes are what vidkv_cache_init wants.
- * The workspace holds split-KV partial results, prepared queries, channel ranges and
+ * The workspace holds partial attention results, prepared queries, channel ranges and
  * the gather lists of the token selection.  Between calls it carries the gather lists,
  * which vidkv_quantize_values reads, and the armed channel-range accumulators that
  * vidkv_cache_init sets up: it belongs to one handle and must not be overwritten while
@@ -299,11 +299,11 @@ vidkv_status_t vidkv_get_selection(vidkv_cache_t* handle, int32_t layer, uint8_t
  * (no append, no flush), the cache having been filled through a handle built on the same
  * `cfg`.  The caller states the token counts that vidkv_layer_state reports for the layers:
  * n_prefill_quantized (a multiple of G), n_flushed_chunks, n_residual (0..R) and n_protected.
- * The split-KV scratch lives in a 16 MiB array inside the library, which every GPU that
- * loads the library keeps until the process exits.  It must hold 520 bytes per (query head,
- * split) record, n_layers * B * H_q * ceil(tokens / split) of them with split = 160, 320 or
- * 640 tokens, plus 3072 bytes per (layer, batch element,
- * KV head, chunk) -- larger problems return VIDKV_ERR_CAPACITY (use fewer layers per call).
+ * The scratch for partial results lives in a 16 MiB array inside the library, which every GPU
+ * that loads the library keeps until the process exits.  It must hold 520 bytes per (query
+ * head, partial record) -- about 8 * (warps resident on the device + 2 * n_layers * B * H_kv)
+ * records at most -- plus 3200 bytes per (layer, batch element, KV head, chunk); larger
+ * problems return VIDKV_ERR_CAPACITY (use fewer layers per call).
  * Nothing is allocated or freed.  The first call on each device looks up the array's device
  * address, so make that first call outside any stream capture.  All calls share the array:
  * two calls whose kernels may overlap on the GPU (different streams, no ordering) race on it;
@@ -344,7 +344,7 @@ vidkv_status_t vidkv_debug_decode_plan(const vidkv_config_t* cfg, int64_t n_pref
 vidkv_status_t vidkv_debug_withhold_once(int32_t what);
 
 /* Profiling aid: record the two CUDA events (cudaEvent_t passed as void*) immediately before
- * and after the attention kernel (stream or split kernel) of every later vidkv_decode_attention call on this
+ * and after the attention kernel (the stream kernel) of every later vidkv_decode_attention call on this
  * handle; NULL, NULL switches it off.  The events are the caller's. */
 vidkv_status_t vidkv_set_profile_events(vidkv_cache_t* handle, void* ev_begin, void* ev_end);
 

@@ -141,7 +141,7 @@ def vidkv_launch_count() -> int:
 def vidkv_attend_noalloc(cfg: VidKVConfig, cache, n_prefill_quantized: int, n_flushed_chunks: int, n_residual: int,
                          n_protected: int, layer_begin: int, n_layers: int, q, out, softmax_scale: float = 0.0):
     """Attention of q over the packed cache tensor `cache` as it stands, for callers that cannot
-    provide workspace memory: the split-KV scratch is a fixed array inside the library.  Same
+    provide workspace memory: the scratch for partial results is a fixed array inside the library.  Same
     arguments as the C function; raises VidKVError (CAPACITY when the problem needs more than the
     array holds)."""
     c = cfg.to_c()

@@ -1,4 +1,4 @@
-// Device helpers shared by the decode attention kernels (decode_mma.cu, decode_stream.cu):
+// Device helpers shared by the decode attention kernels (decode_prep.cu, decode_stream.cu, decode.cu):
 // mma.sync wrappers, the logic / multiply-add forms of the code expansion, and the query
 // normalisation.
 #pragma once

@@ -8,8 +8,8 @@
 //   1. the unit's key groups arrive in the warp's key buffer by one bulk copy
 //      (cp.async.bulk + mbarrier); the scores q . K' of its 160 tokens come out of
 //      mma.sync.m16n8k16 with rows = query heads (exact binary16 pair hi + lo of q_j s_j),
-//      columns = tokens, the codes expanded in registers as the B operand -- the same
-//      arithmetic as in decode_mma.cu;
+//      columns = tokens, the codes expanded in registers as the B operand:
+//      shifts and masks are all they need;
 //   2. the accumulator fragment of that product (head = lane / 4, tokens 2 r, 2 r + 1) is
 //      exactly the B fragment of the next one, so the probabilities 2^(logit - running maximum)
 //      stay in registers as binary16 pairs; the running maximum only moves (and the

@@ -1,5 +1,5 @@
 // vidkv_attend_noalloc: attention of a query over a packed cache as it stands, with the
-// split-KV partial results kept in a fixed device array that is part of this library
+// partial attention results kept in a fixed device array that is part of this library
 // instead of in caller-provided workspace memory.
 //
 // Who this is for.  Some callers are handed device tensors by a host framework and have no
@@ -14,7 +14,7 @@
 
 namespace {
 
-// 16 MiB of scratch: the split-KV partials ((query head, split) records of 130 floats) and
+// 16 MiB of scratch: the partial records (130 floats per query head and warp run) and
 // 3 KiB of prepared query per (slab, chunk).  Every GPU
 // that loads this library holds the array until the process exits.
 constexpr size_t kStaticPartialFloats = 4u * 1024u * 1024u;
