@@ -233,6 +233,15 @@ vidkv_status_t vidkv_quantize_keys(vidkv_cache_t* handle, int32_t layer, const v
 vidkv_status_t vidkv_quantize_values(vidkv_cache_t* handle, int32_t layer, const void* V, int64_t T,
                                      int64_t stride_b, int64_t stride_h, int64_t stride_t, void* stream);
 
+/* The same for n_layers consecutive layers in one call (fewer launches where a layer's tensors are
+ * small): K / V [n_layers, B, H_kv, T, D] with the layers stride_b * B elements apart, i.e.
+ * source slab (layer, b, h) starts at ((layer - layer_begin) * B + b) * stride_b + h * stride_h.
+ * Every layer gets its own channel split and scales, exactly as with one call per layer. */
+vidkv_status_t vidkv_quantize_keys_layers(vidkv_cache_t* handle, int32_t layer_begin, int32_t n_layers, const void* K,
+                                          int64_t T, int64_t stride_b, int64_t stride_h, int64_t stride_t, void* stream);
+vidkv_status_t vidkv_quantize_values_layers(vidkv_cache_t* handle, int32_t layer_begin, int32_t n_layers, const void* V,
+                                            int64_t T, int64_t stride_b, int64_t stride_h, int64_t stride_t, void* stream);
+
 /* Algorithm 1 "Decoding" for n_layers independent layers in one call:
  *   q      [n_layers, B, H_q,  D]  (in_dtype)
  *   k_new  [n_layers, B, H_kv, D]  (in_dtype)    appended to the residual first

@@ -84,6 +84,10 @@ _SIGNATURES = {
                                         C.c_int64, C.c_void_p]),
     "vidkv_quantize_values": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                           C.c_int64, C.c_void_p]),
+    "vidkv_quantize_keys_layers": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                               C.c_int64, C.c_void_p]),
+    "vidkv_quantize_values_layers": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                                 C.c_int64, C.c_void_p]),
     "vidkv_decode_attention": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_float, C.c_void_p]),
     "vidkv_layer_state": (C.c_int32, [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
@@ -283,6 +287,21 @@ class VidKVCache:
         sb, sh, st = _strides_bht(V)
         _check("vidkv_quantize_values", self.lib.vidkv_quantize_values(
             self.handle, layer, C.c_void_p(V.data_ptr()), V.shape[2], sb, sh, st, _stream_ptr()))
+
+    def _layers_args(self, X):
+        assert X.dim() == 5 and X.stride(4) == 1, "expected [n_layers, B, H, T, D] with unit channel stride"
+        assert X.stride(0) == X.shape[1] * X.stride(1), "layers must be stride_b * B elements apart"
+        return X.shape[0], X.shape[3], X.stride(1), X.stride(2), X.stride(3)
+
+    def quantize_keys_layers(self, layer_begin: int, K):
+        n, T, sb, sh, st = self._layers_args(K)
+        _check("vidkv_quantize_keys_layers", self.lib.vidkv_quantize_keys_layers(
+            self.handle, layer_begin, n, C.c_void_p(K.data_ptr()), T, sb, sh, st, _stream_ptr()))
+
+    def quantize_values_layers(self, layer_begin: int, V):
+        n, T, sb, sh, st = self._layers_args(V)
+        _check("vidkv_quantize_values_layers", self.lib.vidkv_quantize_values_layers(
+            self.handle, layer_begin, n, C.c_void_p(V.data_ptr()), T, sb, sh, st, _stream_ptr()))
 
     def decode_attention(self, layer_begin: int, n_layers: int, q, k_new, v_new, out, softmax_scale: float = 0.0):
         for t in (q, k_new, v_new, out):

@@ -326,33 +326,49 @@ static vidkv_status_t check_kv_args(vidkv_cache_t* h, int32_t layer, const void*
   return VIDKV_OK;
 }
 
-vidkv_status_t vidkv_quantize_keys(vidkv_cache_t* h, int32_t layer, const void* K, int64_t T, int64_t stride_b,
-                                   int64_t stride_h, int64_t stride_t, void* stream) {
-  vidkv_status_t st = check_kv_args(h, layer, K, T, stride_b, stride_h, stride_t);
+vidkv_status_t vidkv_quantize_keys_layers(vidkv_cache_t* h, int32_t layer_begin, int32_t n_layers, const void* K, int64_t T,
+                                          int64_t stride_b, int64_t stride_h, int64_t stride_t, void* stream) {
+  vidkv_status_t st = check_kv_args(h, layer_begin, K, T, stride_b, stride_h, stride_t);
   if (st != VIDKV_OK) return st;
-  LayerInfo& li = h->layers[layer];
-  if (li.k_done) return VIDKV_ERR_STATE;
-  if (li.v_done && li.T != T) return VIDKV_ERR_STATE;
+  if (n_layers < 1 || layer_begin + n_layers > h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  for (int l = layer_begin; l < layer_begin + n_layers; ++l) {
+    const LayerInfo& li = h->layers[l];
+    if (li.k_done) return VIDKV_ERR_STATE;
+    if (li.v_done && li.T != T) return VIDKV_ERR_STATE;
+  }
   const int64_t T_q = T - T % kG;
   const int r = static_cast<int>(T % kG);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   KSrc src{K, stride_b, stride_h, stride_t, h->cfg.H_kv};
   if (T_q > 0) {
-    const MinMaxBuffers mm = next_minmax(h, static_cast<int64_t>(h->cfg.B) * h->cfg.H_kv);
-    if (launch_quantize_keys(h->cfg.in_dtype, src, T_q, h->cv, layer, 1, 0, 0, mm, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+    const MinMaxBuffers mm = next_minmax(h, static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv);
+    if (launch_quantize_keys(h->cfg.in_dtype, src, T_q, h->cv, layer_begin, n_layers, 0, 0, mm, s) != cudaSuccess)
+      return VIDKV_ERR_CUDA;
   }
-  if (launch_copy_to_residual(h->cfg.in_dtype, src, T_q, r, h->cv, layer, false, 0, s) != cudaSuccess) return VIDKV_ERR_CUDA;
-  li.k_done = true; li.T = T; li.T_q0 = T_q; li.n_res = r; li.n_flush = 0;
+  if (launch_copy_to_residual(h->cfg.in_dtype, src, T_q, r, h->cv, layer_begin, n_layers, false, 0, s) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  for (int l = layer_begin; l < layer_begin + n_layers; ++l) {
+    LayerInfo& li = h->layers[l];
+    li.k_done = true; li.T = T; li.T_q0 = T_q; li.n_res = r; li.n_flush = 0;
+  }
   return VIDKV_OK;
 }
 
-vidkv_status_t vidkv_quantize_values(vidkv_cache_t* h, int32_t layer, const void* V, int64_t T, int64_t stride_b,
-                                     int64_t stride_h, int64_t stride_t, void* stream) {
-  vidkv_status_t st = check_kv_args(h, layer, V, T, stride_b, stride_h, stride_t);
+vidkv_status_t vidkv_quantize_keys(vidkv_cache_t* h, int32_t layer, const void* K, int64_t T, int64_t stride_b,
+                                   int64_t stride_h, int64_t stride_t, void* stream) {
+  return vidkv_quantize_keys_layers(h, layer, 1, K, T, stride_b, stride_h, stride_t, stream);
+}
+
+vidkv_status_t vidkv_quantize_values_layers(vidkv_cache_t* h, int32_t layer_begin, int32_t n_layers, const void* V, int64_t T,
+                                            int64_t stride_b, int64_t stride_h, int64_t stride_t, void* stream) {
+  vidkv_status_t st = check_kv_args(h, layer_begin, V, T, stride_b, stride_h, stride_t);
   if (st != VIDKV_OK) return st;
-  LayerInfo& li = h->layers[layer];
-  if (li.v_done) return VIDKV_ERR_STATE;
-  if (li.k_done && li.T != T) return VIDKV_ERR_STATE;
+  if (n_layers < 1 || layer_begin + n_layers > h->cfg.L) return VIDKV_ERR_INVALID_ARG;
+  for (int l = layer_begin; l < layer_begin + n_layers; ++l) {
+    const LayerInfo& li = h->layers[l];
+    if (li.v_done) return VIDKV_ERR_STATE;
+    if (li.k_done && li.T != T) return VIDKV_ERR_STATE;
+  }
   if (h->cfg.p_ratio > 0.0f && !h->sel_set) return VIDKV_ERR_STATE;
   if (h->sel_set && h->n_prot > 0 && h->sel_T != T) return VIDKV_ERR_STATE;
   const int64_t T_q = T - T % kG;
@@ -367,12 +383,21 @@ vidkv_status_t vidkv_quantize_values(vidkv_cache_t* h, int32_t layer, const void
     sel.stride_rest = h->cfg.max_prefill_tokens;
     sel.n_prot = h->n_prot;
   }
-  if (T_q > 0 && launch_quantize_values(h->cfg.in_dtype, src, T_q, h->cv, layer, sel, h->cfg.gamma,
+  if (T_q > 0 && launch_quantize_values(h->cfg.in_dtype, src, T_q, h->cv, layer_begin, n_layers, sel, h->cfg.gamma,
                                         h->cfg.ternary_scale == VIDKV_TERNARY_SCALE_NONZERO_MEAN, s) != cudaSuccess)
     return VIDKV_ERR_CUDA;
-  if (launch_copy_to_residual(h->cfg.in_dtype, src, T_q, r, h->cv, layer, true, 0, s) != cudaSuccess) return VIDKV_ERR_CUDA;
-  li.v_done = true; li.T = T; li.T_q0 = T_q; li.n_res = r; li.n_flush = 0;
+  if (launch_copy_to_residual(h->cfg.in_dtype, src, T_q, r, h->cv, layer_begin, n_layers, true, 0, s) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
+  for (int l = layer_begin; l < layer_begin + n_layers; ++l) {
+    LayerInfo& li = h->layers[l];
+    li.v_done = true; li.T = T; li.T_q0 = T_q; li.n_res = r; li.n_flush = 0;
+  }
   return VIDKV_OK;
+}
+
+vidkv_status_t vidkv_quantize_values(vidkv_cache_t* h, int32_t layer, const void* V, int64_t T, int64_t stride_b,
+                                     int64_t stride_h, int64_t stride_t, void* stream) {
+  return vidkv_quantize_values_layers(h, layer, 1, V, T, stride_b, stride_h, stride_t, stream);
 }
 
 vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int32_t n_layers, const void* q,

@@ -52,9 +52,9 @@ cudaError_t launch_encode_keys(int dtype, const KSrc& src, int64_t T_tokens, con
 // Filled on first use on each device by one small kernel; later calls order their stream after it with an event.
 cudaError_t dft_fragments(const uint32_t** table, cudaStream_t stream);
 
-// Algorithm 2 on the prefill tokens of one layer.  T_q (multiple of 32) tokens; the
+// Algorithm 2 on the prefill tokens of n_layers layers (source slabs run over layers, then b, then h).  T_q (multiple of 32) tokens; the
 // unprotected ones go to ternary stream positions 0.., the protected ones to 2-bit groups.
-cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer,
+cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer, int n_layers,
                                    const SelView& sel, float gamma, bool nonzero_mean_scale, cudaStream_t stream);
 
 // 1.58Quant of a full 128-token residual of every slab of the given layers, appended at
@@ -63,9 +63,9 @@ cudaError_t launch_flush_values(int dtype, const KSrc& src, const CacheView& cv,
                                 int64_t tgroup0, float gamma, bool nonzero_mean_scale, cudaStream_t stream);
 
 // Copy `n_tok` tokens starting at token t_begin of every slab of one layer into the
-// residual rings (rows r0 .. r0 + n_tok - 1).
+// residual rings (rows r0 .. r0 + n_tok - 1); n_layers layers from `layer` on.
 cudaError_t launch_copy_to_residual(int dtype, const KSrc& src, int64_t t_begin, int n_tok, const CacheView& cv,
-                                    int layer, bool is_value, int r0, cudaStream_t stream);
+                                    int layer, int n_layers, bool is_value, int r0, cudaStream_t stream);
 
 // Token selection (Sec. 3.3(2)): top-n by saliency, E words + prefix counts into the cache,
 // gather lists into the workspace.

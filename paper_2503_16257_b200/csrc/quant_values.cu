@@ -62,7 +62,7 @@ __device__ __forceinline__ void cp_async16_v(void* smem_dst, const void* gmem_sr
 // NZ: the stored scale is the mean of |v| over the non-zero codes instead of Mean |v| (one more
 // sweep over the staged tile; needs kSGGroups * 4 * kD more floats of shared memory).
 template <typename T, bool NZ>
-__global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest, CacheView cv, int layer,
+__global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest, CacheView cv, int layer0,
                                                         SelView sel, float gamma) {
   extern __shared__ __align__(16) uint8_t vsm[];
   uint8_t* tile = vsm;                                                         // [160][288]
@@ -71,9 +71,10 @@ __global__ void __launch_bounds__(256) v_ternary_kernel(KSrc src, int64_t n_rest
   uint8_t* lut = reinterpret_cast<uint8_t*>(thr + kSGGroups * 64);             // [256]
   float* cnt = reinterpret_cast<float*>(lut + 256);                            // [5][4][128], NZ only
   const int tid = threadIdx.x;
-  const int slab = blockIdx.y;
-  const int b = slab / cv.H_kv, h = slab % cv.H_kv;
-  const T* base = reinterpret_cast<const T*>(src.ptr) + b * src.stride_b + h * src.stride_h;
+  const int slab = blockIdx.y;                              // over the layers of the call, then b, then h
+  const int lb = slab / cv.H_kv, h = slab % cv.H_kv;
+  const int b = lb % cv.B, layer = layer0 + lb / cv.B;
+  const T* base = reinterpret_cast<const T*>(src.ptr) + static_cast<int64_t>(lb) * src.stride_b + h * src.stride_h;
   const int64_t u0 = static_cast<int64_t>(blockIdx.x) * kSGTokens;
   const int n_rows = static_cast<int>(min(static_cast<int64_t>(kSGTokens), n_rest - u0));
   const int32_t* idx = sel.idx_rest ? sel.idx_rest + b * sel.stride_rest : nullptr;
@@ -262,12 +263,13 @@ __device__ __forceinline__ float code_threshold(float s, float z, int k) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(128) v_protect_kernel(KSrc src, CacheView cv, int layer, SelView sel) {
+__global__ void __launch_bounds__(128) v_protect_kernel(KSrc src, CacheView cv, int layer0, SelView sel) {
   __shared__ __align__(16) uint16_t tile[kG * kD];
   __shared__ float s_thr[3][kD];
   const int slab = blockIdx.y;
-  const int b = slab / cv.H_kv, h = slab % cv.H_kv;
-  const T* base = reinterpret_cast<const T*>(src.ptr) + b * src.stride_b + h * src.stride_h;
+  const int lb = slab / cv.H_kv, h = slab % cv.H_kv;
+  const int b = lb % cv.B, layer = layer0 + lb / cv.B;
+  const T* base = reinterpret_cast<const T*>(src.ptr) + static_cast<int64_t>(lb) * src.stride_b + h * src.stride_h;
   const int64_t p0 = static_cast<int64_t>(blockIdx.x) * kG;
   const int n_rows = static_cast<int>(min(static_cast<int64_t>(kG), sel.n_prot - p0));
   const int32_t* idx = sel.idx_prot + b * sel.stride_prot;
@@ -361,11 +363,12 @@ __global__ void __launch_bounds__(kD) v_flush_kernel(KSrc src, CacheView cv, int
 // Residual copies (Algorithm 1: X_r = X[l - r:], and the per-step append).
 // ---------------------------------------------------------------------------------
 template <typename T>
-__global__ void copy_to_residual_kernel(KSrc src, int64_t t_begin, int n_tok, CacheView cv, int layer,
+__global__ void copy_to_residual_kernel(KSrc src, int64_t t_begin, int n_tok, CacheView cv, int layer0,
                                         int64_t res_offset, int r0) {
   const int slab = blockIdx.x;
-  const int b = slab / cv.H_kv, h = slab % cv.H_kv;
-  const T* base = reinterpret_cast<const T*>(src.ptr) + b * src.stride_b + h * src.stride_h;
+  const int lb = slab / cv.H_kv, h = slab % cv.H_kv;
+  const int b = lb % cv.B, layer = layer0 + lb / cv.B;
+  const T* base = reinterpret_cast<const T*>(src.ptr) + static_cast<int64_t>(lb) * src.stride_b + h * src.stride_h;
   uint4* dst = reinterpret_cast<uint4*>(cv.slab(layer, b, h) + res_offset);
   for (int i = threadIdx.x; i < n_tok * 16; i += blockDim.x) {
     const int r = i >> 4, l = i & 15;
@@ -513,9 +516,9 @@ __global__ void __launch_bounds__(1024) select_tokens_kernel(const float* __rest
 // Host launchers
 // ---------------------------------------------------------------------------------
 template <typename T, bool NZ>
-static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheView& cv, int layer, const SelView& sel,
-                                     float gamma, cudaStream_t stream) {
-  const int n_slabs = cv.B * cv.H_kv;
+static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheView& cv, int layer, int n_layers,
+                                     const SelView& sel, float gamma, cudaStream_t stream) {
+  const int n_slabs = n_layers * cv.B * cv.H_kv;
   const int64_t n_rest = T_q - sel.n_prot;
   if (n_rest > 0) {
     const int64_t sgs = (n_rest + kSGTokens - 1) / kSGTokens;
@@ -541,13 +544,13 @@ static cudaError_t quantize_values_t(const KSrc& src, int64_t T_q, const CacheVi
   return cudaGetLastError();
 }
 
-cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer,
+cudaError_t launch_quantize_values(int dtype, const KSrc& src, int64_t T_q, const CacheView& cv, int layer, int n_layers,
                                    const SelView& sel, float gamma, bool nonzero_mean_scale, cudaStream_t stream) {
   if (dtype == VIDKV_F16)
-    return nonzero_mean_scale ? quantize_values_t<__half, true>(src, T_q, cv, layer, sel, gamma, stream)
-                              : quantize_values_t<__half, false>(src, T_q, cv, layer, sel, gamma, stream);
-  return nonzero_mean_scale ? quantize_values_t<__nv_bfloat16, true>(src, T_q, cv, layer, sel, gamma, stream)
-                            : quantize_values_t<__nv_bfloat16, false>(src, T_q, cv, layer, sel, gamma, stream);
+    return nonzero_mean_scale ? quantize_values_t<__half, true>(src, T_q, cv, layer, n_layers, sel, gamma, stream)
+                              : quantize_values_t<__half, false>(src, T_q, cv, layer, n_layers, sel, gamma, stream);
+  return nonzero_mean_scale ? quantize_values_t<__nv_bfloat16, true>(src, T_q, cv, layer, n_layers, sel, gamma, stream)
+                            : quantize_values_t<__nv_bfloat16, false>(src, T_q, cv, layer, n_layers, sel, gamma, stream);
 }
 
 template <typename T, bool NZ>
@@ -571,12 +574,12 @@ cudaError_t launch_flush_values(int dtype, const KSrc& src, const CacheView& cv,
 }
 
 cudaError_t launch_copy_to_residual(int dtype, const KSrc& src, int64_t t_begin, int n_tok, const CacheView& cv,
-                                    int layer, bool is_value, int r0, cudaStream_t stream) {
+                                    int layer, int n_layers, bool is_value, int r0, cudaStream_t stream) {
   if (n_tok <= 0) return cudaSuccess;
   const int64_t off = is_value ? cv.vres_offset : cv.kres_offset;
   // 16-bit elements either way: the copy is type-agnostic
   (void)dtype;
-  copy_to_residual_kernel<__half><<<cv.B * cv.H_kv, 256, 0, stream>>>(src, t_begin, n_tok, cv, layer, off, r0);
+  copy_to_residual_kernel<__half><<<n_layers * cv.B * cv.H_kv, 256, 0, stream>>>(src, t_begin, n_tok, cv, layer, off, r0);
   count_launches(1);
   return cudaGetLastError();
 }

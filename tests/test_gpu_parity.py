@@ -531,6 +531,36 @@ def test_strided_inputs_give_the_same_cache(name, p):
     assert np.array_equal(caches[0], caches[1])
 
 
+@pytest.mark.parametrize("name,T,p", [("tiny", 1003, 0.2), ("qwen", 640, 0.0)])
+def test_layer_range_quantization_gives_the_same_cache(name, T, p):
+    """vidkv_quantize_keys_layers / vidkv_quantize_values_layers on [n_layers, B, H, T, D] tensors pack
+    the same bytes as one call per layer (each layer keeps its own channel split and scales)."""
+    import paper_2503_16257_b200 as P
+    wl = CONFIGS[name]
+    B, L = 2, 3
+    in_dt = P.VIDKV_F16 if wl.dtype == "fp16" else P.VIDKV_BF16
+    cfg = P.VidKVConfig(B=B, L=L, max_prefill_tokens=T, max_new_tokens=1, p_ratio=p, in_dtype=in_dt, out_dtype=P.VIDKV_F32)
+    KV = [make_layer_kv(wl, layer, "cuda", T=T, B=B) for layer in range(L)]
+    sal = make_saliency(wl, "cuda", l_v=T - T % 32, B=B) if p > 0 else None
+    caches = []
+    for ranged in (False, True):
+        c = P.VidKVCache(cfg, device="cuda")
+        if sal is not None:
+            c.select_tokens(sal, 0, T - T % 32, T)
+        if ranged:
+            c.quantize_keys_layers(0, torch.stack([kv[0] for kv in KV]))
+            c.quantize_values_layers(1, torch.stack([kv[1] for kv in KV[1:]]))      # a range that starts at layer 1
+            c.quantize_values_layers(0, KV[0][1][None])
+        else:
+            for layer in range(L):
+                c.quantize_keys(layer, KV[layer][0])
+                c.quantize_values(layer, KV[layer][1])
+        torch.cuda.synchronize()
+        assert c.status() == 0 and c.layer_state(2)["n_quantized"] == T - T % 32
+        caches.append(c.cache.cpu().numpy())
+    assert np.array_equal(caches[0], caches[1])
+
+
 def test_two_caches_on_two_streams():
     """Two caches worked on from two streams at once (prefill and decode interleaved) end up exactly
     as when each runs alone: the library keeps no per-call state outside the handle."""

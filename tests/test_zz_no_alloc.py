@@ -61,3 +61,25 @@ def test_attend_noalloc_rejects_what_does_not_fit():
     with pytest.raises(P.VidKVError) as e:
         P.vidkv_attend_noalloc(cfg, cache, 100, 0, 1, 0, 0, 1, q, out)     # not a multiple of G
     assert e.value.status == -1
+
+
+@pytest.mark.parametrize("p", [0.0, 0.2])
+def test_attend_noalloc_matches_the_oracle(p):
+    """The workspace-free call against the oracle itself (not only against the regular call): after a
+    regular step the cache holds that step's token, so the same query through the workspace-free call
+    must reproduce the oracle's output of that step.  Without and with protected tokens."""
+    import paper_2503_16257_b200 as P
+    from tests.helpers import Pair, TOL_ABS
+    from workloads import CONFIGS, make_step_inputs
+
+    wl = CONFIGS["tiny"]
+    T, B, L = 1000, 2, 2
+    pair = Pair(wl, T, B=B, L=L, p=p, max_new=3).prefill()
+    for step in range(2):
+        _, ref = pair.decode()
+        q = torch.stack([make_step_inputs(wl, layer, step, "cpu", T=T, B=B)[0] for layer in range(L)]).cuda()
+        st = pair.cache.layer_state(0)
+        out = torch.full((L, B, 28, 128), float("nan"), dtype=torch.float32, device="cuda")
+        P.vidkv_attend_noalloc(pair.cfg, pair.cache.cache, 992, 0, st["n_residual"], st["n_protected"], 0, L, q, out)
+        torch.cuda.synchronize()
+        assert np.abs(out.cpu().numpy().astype(np.float64) - ref).max() <= TOL_ABS
