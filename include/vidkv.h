@@ -259,6 +259,28 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* handle, int32_t layer_begin
                                       const void* q, const void* k_new, const void* v_new, void* out,
                                       float softmax_scale, void* stream);
 
+/* Caches beyond one device (the 1000-frame case of Sec. 1): the token axis of Eq. 3 can be cut into
+ * shards, each held by its own cache (its own device), because Softmax(q K^T) V over the whole
+ * sequence follows from per-shard (maximum, sum, unnormalised output) triples.
+ * vidkv_decode_attention_partial is vidkv_decode_attention for one shard:
+ *   partial [n_layers, B, H_q, 130] float32 device: per query head the largest base-2 logit
+ *           m = max_t (q . k_t) * softmax_scale * log2(e), l = sum_t 2^(logit_t - m) and
+ *           o[128] = sum_t 2^(logit_t - m) v_t over the shard's tokens (packed cache + residual);
+ *   k_new, v_new: the shard that owns the newest token passes them (appended first, residual
+ *           flushed when full, exactly as in vidkv_decode_attention); the other shards pass NULL
+ *           for both and are attended to as they stand (STATE if such a shard holds no token).
+ * The caller moves the triples between devices (e.g. an all-gather of 130 floats per query head
+ * and shard into its own memory) and vidkv_merge_partials combines them:
+ *   partials [n_parts, n_rows, 130] float32 device, n_rows = n_layers * B * H_q;
+ *   out [n_rows, 128] in out_dtype:  sum_p 2^(m_p - M) o_p / sum_p 2^(m_p - M) l_p, M = max_p m_p.
+ * Every shard quantizes its own tokens (its own chunks and channel splits, Algorithm 3 applied to
+ * the tokens it holds). */
+vidkv_status_t vidkv_decode_attention_partial(vidkv_cache_t* handle, int32_t layer_begin, int32_t n_layers,
+                                              const void* q, const void* k_new, const void* v_new, float* partial,
+                                              float softmax_scale, void* stream);
+vidkv_status_t vidkv_merge_partials(const float* partials, int64_t n_parts, int64_t n_rows, void* out,
+                                    int32_t out_dtype, void* stream);
+
 /* Host view of a layer's token counts (any pointer may be NULL). */
 vidkv_status_t vidkv_layer_state(const vidkv_cache_t* handle, int32_t layer, int64_t* n_quantized,
                                  int64_t* n_residual, int64_t* n_chunks, int64_t* n_protected);

@@ -376,6 +376,30 @@ def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float) -> np.n
     return w @ np.asarray(V, np.float64)
 
 
+def attention_partial(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float):
+    """Eq. 3 restricted to a shard of the token axis, left unnormalised: per query row the largest
+    logit m (natural units, -inf for an empty shard), l = sum_t exp(logit_t - m) and
+    o = sum_t exp(logit_t - m) V_t.  Softmax(q K^T) V over the union of shards follows from these
+    triples alone (merge_partials)."""
+    q = np.asarray(q, np.float64)
+    K = np.asarray(K, np.float64)
+    V = np.asarray(V, np.float64)
+    if K.shape[0] == 0:
+        return np.full(q.shape[0], -np.inf), np.zeros(q.shape[0]), np.zeros((q.shape[0], V.shape[1]))
+    logits = (q @ K.T) * scale
+    m = logits.max(axis=-1)
+    w = np.exp(logits - m[:, None])
+    return m, w.sum(axis=-1), w @ V
+
+
+def merge_partials(parts):
+    """Combine (m, l, o) triples of disjoint token shards: out = sum_p e^(m_p - M) o_p / sum_p e^(m_p - M) l_p."""
+    M = np.max(np.stack([p[0] for p in parts]), axis=0)
+    num = sum(np.where(np.isfinite(p[0]), np.exp(p[0] - M), 0.0)[:, None] * p[2] for p in parts)
+    den = sum(np.where(np.isfinite(p[0]), np.exp(p[0] - M), 0.0) * p[1] for p in parts)
+    return num / den[:, None]
+
+
 # --------------------------------------------------------------------------
 # Algorithm 1 : Prefill / Decoding for one (layer, batch element, KV head)
 # --------------------------------------------------------------------------

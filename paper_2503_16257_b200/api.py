@@ -90,6 +90,9 @@ _SIGNATURES = {
                                                  C.c_int64, C.c_void_p]),
     "vidkv_decode_attention": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_float, C.c_void_p]),
+    "vidkv_decode_attention_partial": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                   C.c_void_p, C.c_float, C.c_void_p]),
+    "vidkv_merge_partials": (C.c_int32, [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_int32, C.c_void_p]),
     "vidkv_layer_state": (C.c_int32, [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                                       C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "vidkv_cache_status": (C.c_int32, [C.c_void_p, C.c_void_p]),
@@ -185,6 +188,18 @@ def vidkv_saliency_scores(x_v, x_t, text_sum=None, saliency=None):
         dtype, C.c_void_p(x_v.data_ptr()), C.c_void_p(x_t.data_ptr()), B, l_v, l_t, d,
         C.c_void_p(text_sum.data_ptr()), C.c_void_p(saliency.data_ptr()), _stream_ptr()))
     return saliency
+
+
+def vidkv_merge_partials(partials, out):
+    """partials [n_parts, ..., 130] float32 (device) -> out [..., 128]: log-sum-exp merge of per-shard triples."""
+    import torch
+    assert partials.is_contiguous() and out.is_contiguous() and partials.dtype == torch.float32
+    n_parts = partials.shape[0]
+    n_rows = partials.numel() // (n_parts * 130)
+    dt = {torch.float32: VIDKV_F32, torch.float16: VIDKV_F16, torch.bfloat16: VIDKV_BF16}[out.dtype]
+    _check("vidkv_merge_partials", load_library().vidkv_merge_partials(
+        C.c_void_p(partials.data_ptr()), n_parts, n_rows, C.c_void_p(out.data_ptr()), dt, _stream_ptr()))
+    return out
 
 
 def vidkv_debug_withhold_once(what: int):
@@ -309,6 +324,14 @@ class VidKVCache:
         _check("vidkv_decode_attention", self.lib.vidkv_decode_attention(
             self.handle, layer_begin, n_layers, C.c_void_p(q.data_ptr()), C.c_void_p(k_new.data_ptr()),
             C.c_void_p(v_new.data_ptr()), C.c_void_p(out.data_ptr()), softmax_scale, _stream_ptr()))
+
+    def decode_attention_partial(self, layer_begin: int, n_layers: int, q, k_new, v_new, partial, softmax_scale: float = 0.0):
+        """One token shard's (maximum, sum, unnormalised out) triples; k_new = v_new = None: attend as it stands."""
+        kp = C.c_void_p(k_new.data_ptr()) if k_new is not None else C.c_void_p(0)
+        vp = C.c_void_p(v_new.data_ptr()) if v_new is not None else C.c_void_p(0)
+        _check("vidkv_decode_attention_partial", self.lib.vidkv_decode_attention_partial(
+            self.handle, layer_begin, n_layers, C.c_void_p(q.data_ptr()), kp, vp, C.c_void_p(partial.data_ptr()),
+            softmax_scale, _stream_ptr()))
 
     def layer_state(self, layer: int) -> dict:
         a, b, c, d = C.c_int64(), C.c_int64(), C.c_int64(), C.c_int64()

@@ -11,7 +11,7 @@ namespace vidkv {
 namespace {
 
 constexpr int kMaxSMs = 256;        // multiprocessor count the sizing formulas assume at most
-constexpr int kMinRunUnits = 2;     // a warp's run is never shorter (one record per 320 tokens at worst)
+constexpr int kMinRunUnits = 1;     // with fewer units than warps every unit gets its own warp (shortest critical path)
 
 }  // namespace
 
@@ -233,6 +233,14 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int n_re
         acc[j][1] += wgt * o.y;
       }
     }
+    if (a.partial_out) {
+      // a token shard of a longer sequence: leave (maximum, sum, unnormalised out) for the caller's exchange
+      float* pr = a.partial_out + (q0 / kD + hd) * kRecordFloats;
+      if (warp == 0 && r == 0) { pr[0] = M; pr[1] = Lh[hd]; }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) *reinterpret_cast<float2*>(pr + 2 + 32 * warp + 8 * j + 2 * r) = make_float2(acc[j][0], acc[j][1]);
+      return;
+    }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float v0 = acc[j][0] * inv, v1 = acc[j][1] * inv;
@@ -242,6 +250,34 @@ __global__ void __launch_bounds__(kD) decode_merge_kernel(DecodeArgs a, int n_re
       else *reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(a.out) + i) = __floats2bfloat162_rn(v0, v1);
     }
   }
+}
+
+// out[row][c] = sum_p 2^(m_p - M) o_p[c] / sum_p 2^(m_p - M) l_p over n_parts partial sets of n_rows rows each
+// (M = max_p m_p); a set that saw no token has l = 0 and m = -inf.
+__global__ void __launch_bounds__(kD) merge_partials_kernel(const float* __restrict__ parts, int64_t n_parts, int64_t n_rows,
+                                                           void* __restrict__ out, int out_dtype) {
+  const int64_t row = blockIdx.x;
+  const int c = threadIdx.x;
+  float M = -INFINITY;
+  for (int64_t p = 0; p < n_parts; ++p) M = fmaxf(M, parts[(p * n_rows + row) * kRecordFloats]);
+  float num = 0.0f, den = 0.0f;
+  for (int64_t p = 0; p < n_parts; ++p) {
+    const float* pr = parts + (p * n_rows + row) * kRecordFloats;
+    const float w = pr[1] > 0.0f ? exp2f(pr[0] - M) : 0.0f;
+    num += w * pr[2 + c];
+    den += w * pr[1];
+  }
+  const float v = num / den;
+  if (out_dtype == VIDKV_F32) reinterpret_cast<float*>(out)[row * kD + c] = v;
+  else if (out_dtype == VIDKV_F16) reinterpret_cast<__half*>(out)[row * kD + c] = __float2half_rn(v);
+  else reinterpret_cast<__nv_bfloat16*>(out)[row * kD + c] = __float2bfloat16_rn(v);
+}
+
+cudaError_t launch_merge_partials(const float* parts, int64_t n_parts, int64_t n_rows, void* out, int out_dtype,
+                                  cudaStream_t stream) {
+  merge_partials_kernel<<<static_cast<unsigned>(n_rows), kD, 0, stream>>>(parts, n_parts, n_rows, out, out_dtype);
+  count_launches(1);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_decode(const DecodeArgs& a_in, cudaStream_t stream) {

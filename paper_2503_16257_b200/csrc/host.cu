@@ -400,43 +400,51 @@ vidkv_status_t vidkv_quantize_values(vidkv_cache_t* h, int32_t layer, const void
   return vidkv_quantize_values_layers(h, layer, 1, V, T, stride_b, stride_h, stride_t, stream);
 }
 
-vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int32_t n_layers, const void* q,
-                                      const void* k_new, const void* v_new, void* out, float softmax_scale,
-                                      void* stream) {
-  if (!h || !q || !k_new || !v_new || !out) return VIDKV_ERR_INVALID_ARG;
+}  // extern "C"
+
+// Algorithm 1 "Decoding" for a layer range.  append: k_new / v_new join the residual first (and a full
+// residual is flushed afterwards); without it the cache is attended to as it stands.  partial: leave
+// (maximum, sum, unnormalised out) per query head instead of the normalised output.
+static vidkv_status_t decode_impl(vidkv_cache_t* h, int32_t layer_begin, int32_t n_layers, const void* q, const void* k_new,
+                                  const void* v_new, void* out, float* partial, float softmax_scale, void* stream) {
+  const bool append = k_new != nullptr;
+  if (!h || !q || (k_new == nullptr) != (v_new == nullptr) || (!out && !partial)) return VIDKV_ERR_INVALID_ARG;
   if (layer_begin < 0 || n_layers < 1 || layer_begin + n_layers > h->cfg.L) return VIDKV_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return VIDKV_ERR_ALIGNMENT;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out) || !aligned16(partial)) return VIDKV_ERR_ALIGNMENT;
   if (!std::isfinite(softmax_scale)) return VIDKV_ERR_INVALID_ARG;
   const LayerInfo& first = h->layers[layer_begin];
   for (int l = layer_begin; l < layer_begin + n_layers; ++l) {
     const LayerInfo& li = h->layers[l];
     if (!li.k_done || !li.v_done) return VIDKV_ERR_STATE;
     if (li.T_q0 != first.T_q0 || li.n_flush != first.n_flush || li.n_res != first.n_res) return VIDKV_ERR_STATE;
-    if (li.new_tokens + 1 > h->cfg.max_new_tokens) return VIDKV_ERR_CAPACITY;
+    if (append && li.new_tokens + 1 > h->cfg.max_new_tokens) return VIDKV_ERR_CAPACITY;
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int dt = h->cfg.in_dtype;
   // the append rides on the query-preparation kernel when there is one (some chunk is quantized)
   const bool has_chunks = first.T_q0 + first.n_flush * kR > 0;
-  if (!has_chunks && launch_append(dt, k_new, v_new, h->cv, layer_begin, n_layers, first.n_res, s) != cudaSuccess)
+  if (!append && !has_chunks && first.n_res == 0) return VIDKV_ERR_STATE;       // nothing to attend to
+  if (append && !has_chunks && launch_append(dt, k_new, v_new, h->cv, layer_begin, n_layers, first.n_res, s) != cudaSuccess)
     return VIDKV_ERR_CUDA;
   DecodeArgs a;
   a.cv = h->cv;
   a.q = q; a.k_new = k_new; a.v_new = v_new; a.out = out;
   a.partials = reinterpret_cast<float*>(h->workspace + h->ws.partials_off);
   a.prep = reinterpret_cast<uint32_t*>(h->workspace + h->ws.prep_off);
-  a.append_row = has_chunks ? first.n_res : -1;
+  a.append_row = append && has_chunks ? first.n_res : -1;
+  a.partial_out = partial;
   a.layer0 = layer_begin; a.n_layers = n_layers;
   a.in_dtype = dt; a.out_dtype = h->cfg.out_dtype;
   a.n_prot = h->n_prot;
   a.scale = softmax_scale > 0.0f ? softmax_scale : 1.0f / std::sqrt(static_cast<float>(kD));
   a.ev_begin = h->ev_begin; a.ev_end = h->ev_end;
   a.withhold = 0;
-  a.st.T_q0 = first.T_q0; a.st.n_flush = first.n_flush; a.st.n_res = first.n_res + 1;
+  a.st.T_q0 = first.T_q0; a.st.n_flush = first.n_flush; a.st.n_res = first.n_res + (append ? 1 : 0);
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * h->cfg.B * h->cfg.H_kv;
   a.plan = plan_decode(a.st, n_slabs, h->n_prot > 0, device_sm_count(), h->dbg_run_units);
   if (a.plan.records > h->ws.partial_entries) return VIDKV_ERR_CAPACITY;
   if (launch_decode(a, s) != cudaSuccess) return VIDKV_ERR_CUDA;
+  if (!append) return VIDKV_OK;
   const bool flush = a.st.n_res == kR;
   if (flush) {
     const int64_t es = h->cv.slab_stride / 2;    // slab stride in 16-bit elements
@@ -460,6 +468,34 @@ vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int
     if (flush) { li.n_flush += 1; li.n_res = 0; }
     else li.n_res += 1;
   }
+  return VIDKV_OK;
+}
+
+extern "C" {
+
+vidkv_status_t vidkv_decode_attention(vidkv_cache_t* h, int32_t layer_begin, int32_t n_layers, const void* q,
+                                      const void* k_new, const void* v_new, void* out, float softmax_scale,
+                                      void* stream) {
+  if (!k_new || !v_new || !out) return VIDKV_ERR_INVALID_ARG;
+  return decode_impl(h, layer_begin, n_layers, q, k_new, v_new, out, nullptr, softmax_scale, stream);
+}
+
+vidkv_status_t vidkv_decode_attention_partial(vidkv_cache_t* h, int32_t layer_begin, int32_t n_layers, const void* q,
+                                              const void* k_new, const void* v_new, float* partial, float softmax_scale,
+                                              void* stream) {
+  if (!partial) return VIDKV_ERR_INVALID_ARG;
+  return decode_impl(h, layer_begin, n_layers, q, k_new, v_new, nullptr, partial, softmax_scale, stream);
+}
+
+vidkv_status_t vidkv_merge_partials(const float* partials, int64_t n_parts, int64_t n_rows, void* out, int32_t out_dtype,
+                                    void* stream) {
+  if (!partials || !out || n_parts < 1 || n_rows < 0) return VIDKV_ERR_INVALID_ARG;
+  if (out_dtype != VIDKV_F16 && out_dtype != VIDKV_BF16 && out_dtype != VIDKV_F32) return VIDKV_ERR_INVALID_ARG;
+  if (!aligned16(partials) || !aligned16(out)) return VIDKV_ERR_ALIGNMENT;
+  if (n_rows == 0) return VIDKV_OK;
+  if (n_rows > 0x7fffffff) return VIDKV_ERR_UNSUPPORTED;
+  if (launch_merge_partials(partials, n_parts, n_rows, out, out_dtype, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return VIDKV_ERR_CUDA;
   return VIDKV_OK;
 }
 

@@ -129,6 +129,7 @@ struct DecodeArgs {
   LayerState st;
   cudaEvent_t ev_begin, ev_end;   // optional: recorded around the attention kernel (profiling)
   int32_t withhold;    // test hook: the stream kernel does not issue its first value copy
+  float* partial_out;  // not null: leave [n_layers * B * H_q][kRecordFloats] (max, sum, unnormalised out) instead of `out`
 };
 
 // Eq. 7 scores from hidden states: text_sum [B, d] (scratch) and saliency [B, l_v], both float32.
@@ -151,6 +152,9 @@ inline void count_launches(int n) { g_launch_count += static_cast<unsigned long 
 // Attention over the packed cache + residual: query preparation, the stream kernel, then the merge
 // of the partial records, which also attends to the residual.
 cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t stream);
+// Log-sum-exp merge of n_parts partial sets [n_parts][n_rows][kRecordFloats] into out [n_rows][128].
+cudaError_t launch_merge_partials(const float* parts, int64_t n_parts, int64_t n_rows, void* out, int out_dtype,
+                                  cudaStream_t stream);
 // Query preparation (and the step's append) for a.plan.n_chunks chunk-table entries per slab.
 cudaError_t launch_decode_prep(DecodeArgs& a, cudaStream_t stream);
 // Persistent warps over 160-token units: caches without / with protected tokens.

@@ -79,6 +79,7 @@ extern "C" vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const 
   a.st.T_q0 = n_prefill_quantized; a.st.n_flush = n_flushed_chunks; a.st.n_res = n_residual;
   a.ev_begin = nullptr; a.ev_end = nullptr;
   a.withhold = 0;
+  a.partial_out = nullptr;
   const int64_t n_slabs = static_cast<int64_t>(n_layers) * cfg->B * cfg->H_kv;
   a.append_row = -1;
   a.plan = plan_decode(a.st, n_slabs, n_protected > 0, device_sm_count(), 0);

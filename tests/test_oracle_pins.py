@@ -586,3 +586,25 @@ def test_fft_smooths_one_bit_error_direction():
     plain = np.sign(x) * np.abs(x).mean(0)[None]
     err_plain = ((plain - x) ** 2).mean()
     assert err_fft < err_plain
+
+
+def test_attention_over_token_shards_merges_to_the_whole():
+    """Pins attention_partial / merge_partials to the plain definition: any cut of the token axis into
+    shards (an empty one included) merges to Softmax(q K^T) V of the whole, and to torch's
+    scaled_dot_product_attention."""
+    import torch
+    r = rng(91)
+    q = r.standard_normal((7, 128)) * 2
+    K = r.standard_normal((300, 128)) * 3          # logits spread over tens of units: the maxima matter
+    V = r.standard_normal((300, 128))
+    scale = 1.0 / np.sqrt(128.0)
+    whole = O.attention(q, K, V, scale)
+    for cuts in ([0, 300], [0, 1, 300], [0, 130, 130, 300], [0, 64, 200, 299, 300]):
+        parts = [O.attention_partial(q, K[a:b], V[a:b], scale) for a, b in zip(cuts[:-1], cuts[1:])]
+        assert np.allclose(O.merge_partials(parts), whole, rtol=1e-12, atol=1e-13)
+    ref = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(q)[None], torch.from_numpy(K)[None],
+                                                           torch.from_numpy(V)[None])[0].numpy()
+    assert np.allclose(whole, ref, atol=1e-10)
+    m, l, o = O.attention_partial(q, K[:0], V[:0], scale)
+    assert np.isneginf(m).all() and (l == 0).all() and (o == 0).all()
+
