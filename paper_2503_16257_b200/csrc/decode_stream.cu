@@ -36,7 +36,7 @@ constexpr int kKBufBytes = kSGGroups * kKGroupBytes;   // 5760: the key groups o
 constexpr int kVBufBytes = kSGBytes;                   // 5376: its ternary supergroup
 constexpr int kTotBytes = 4 * 2 * 32 * 16;             // 4096: the warp's running output (128 channels x 8 heads, float)
 constexpr int kWarpBufBytes = kKBufBytes + kVBufBytes + kTotBytes;   // 15232 per warp
-constexpr uint32_t kWaitLimit = 1u << 20;              // mbarrier polls before a warp gives up (tens of milliseconds)
+constexpr uint32_t kWaitLimit = 1u << 19;              // mbarrier polls before a warp gives up (about a second)
 constexpr float kStaleLog2 = 6.0f;                     // the running maximum may lag a unit's maximum by this much
 constexpr uint32_t kMinus5 = 0xc500c500u;              // binary16 pair (-5.0, -5.0)
 
