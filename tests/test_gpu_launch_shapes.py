@@ -192,6 +192,30 @@ def test_stream_kernel_across_two_flushes(run_units):
     assert pair.cache.layer_state(0)["n_chunks"] == 3 and pair.cache.status() == 0
 
 
+def _random_plans(n, seed):
+    r = np.random.default_rng(seed)
+    cases = []
+    for _ in range(n):
+        name = ["tiny", "llava", "qwen"][int(r.integers(0, 3))]
+        T = int(r.integers(33, 2600))
+        steps = int(r.integers(1, 4)) if r.random() < 0.75 else 128 - T % 32 + int(r.integers(1, 4))
+        cases.append((name, T, int(r.integers(1, 3)), int(r.integers(1, 3)), [0.0, 0.05, 0.2, 0.5, 0.97][int(r.integers(0, 5))],
+                      [1, 2, 3, 7, 19][int(r.integers(0, 5))], steps))
+    return cases
+
+
+@pytest.mark.parametrize("name,T,B,L,p,run_units,steps", _random_plans(14, 20250317))
+def test_seeded_random_shapes_and_run_lengths(name, T, B, L, p, run_units, steps):
+    """Shapes, protection ratios and run lengths nobody picked by hand (a quarter of the cases decode
+    across a residual flush), every slab against the oracle."""
+    pair = Pair(CONFIGS[name], T, B=B, L=L, p=p, max_new=steps + 1).prefill()
+    pair.cache.debug_set_decode_plan(run_units=run_units)
+    for s in range(steps):
+        out, ref = pair.decode()
+        assert np.abs(out - ref).max() <= _rel_tol(ref), s
+    assert pair.cache.status() == 0
+
+
 # ------------------------------------------------------------------ prompts shorter than one group
 @pytest.mark.parametrize("T", [31, 0])
 def test_flushes_after_a_prompt_with_nothing_to_quantize(T):
