@@ -11,7 +11,8 @@ What follows the paper, step by step, in its notation:
 * ``dft64`` / ``idft64``        the discrete Fourier transform written out as
                                  its defining matrix (no FFT routine)
 * ``fft_1bit``          Eq. 5   sign code + mean-|.| scale in the frequency domain
-* ``mixquant``          Algorithm 3 MixQuant (k = 0.5 : 64 two-bit + 64 one-bit)
+* ``mixquant``          Algorithm 3 MixQuant (k = 0.5 : 64 two-bit + 64 one-bit; other k and the
+                        plain min/max 1-bit code of 1BitQuant's other branch as parameters)
 * ``quant_1p58``        Eq. 6 / Algorithm 2 "1.58Quant" (ternary, gamma = 0.7)
 * ``stp_saliency``      Eq. 7   cross-modal scores I = X_v X_t^T, summed over the text tokens
 * ``select_tokens``     Eq. 7 / Sec. 3.3(2): top n = floor(p * l_v) visual tokens
@@ -233,23 +234,40 @@ def hermitian_pack_columns(n: int = N_FFT) -> np.ndarray:
 # --------------------------------------------------------------------------
 # Algorithm 3 : MixQuant
 # --------------------------------------------------------------------------
-def mixquant(k: np.ndarray, ratio: float = 0.5):
+def one_bit_mode(ratio: float) -> str:
+    """Algorithm 3, 1BitQuant, and Sec. 4.1 (Implementation Details): the normal channels go through
+    the FFT only at k = 0.5 and k = 0.75; every other k uses the plain 1-bit quantizer."""
+    return "fft" if ratio in (0.5, 0.75) else "minmax"
+
+
+def mixquant(k: np.ndarray, ratio: float = 0.5, one_bit: str = "auto"):
     """Algorithm 3 MixQuant on one chunk k [T, D] (T a multiple of G or not).
 
-    Returns a dict: abn_idx, nom_idx, codes2 [T, n_abn], s2, z2 [ng, n_abn],
-    bits1 [T, 2*n_nom] (full complex columns), s1 [ng, 2*n_nom]."""
+    one_bit: "fft" = Eq. 5 on the transformed normal channels, "minmax" = GQuant(bit=1) (Eq. 4 with
+    n = 1) on the normal channels as they are, "auto" = the paper's choice for this k
+    (``one_bit_mode``).  k = 1 leaves no normal channel.
+
+    Returns a dict: abn_idx, nom_idx, codes2 [T, n_abn], s2, z2 [ng, n_abn], mode, and for "fft"
+    bits1 [T, 2*n_nom] (full complex columns), s1 [ng, 2*n_nom]; for "minmax" codes1 [T, n_nom],
+    s1 and z1 [ng, n_nom]."""
     k = np.asarray(k, dtype=np.float32)
     T = k.shape[0]
+    mode = one_bit_mode(ratio) if one_bit == "auto" else one_bit
     abn, nom = select_channels(k, ratio)
     codes2, s2, z2 = gquant_groups(k[:, abn], 2)          # GQuant(X_abn, bit=2)
     ng = (T + G - 1) // G
+    out = dict(abn_idx=abn, nom_idx=nom, codes2=codes2, s2=s2, z2=z2, T=T, mode=mode)
+    if mode == "minmax":                                   # 1BitQuant without the transform
+        out["codes1"], out["s1"], out["z1"] = gquant_groups(k[:, nom], 1)
+        return out
     bits1 = np.zeros((T, 2 * len(nom)), dtype=np.uint8)
     s1 = np.zeros((ng, 2 * len(nom)), dtype=np.float16)
     for g in range(ng):                                    # 1BitQuant(X_nom)
         sl = slice(g * G, min((g + 1) * G, T))
-        bits1[sl], s1[g] = fft_1bit(k[sl][:, nom])
-    return dict(abn_idx=abn, nom_idx=nom, codes2=codes2, s2=s2, z2=z2,
-                bits1=bits1, s1=s1, T=T)
+        if len(nom):
+            bits1[sl], s1[g] = fft_1bit(k[sl][:, nom])
+    out["bits1"], out["s1"] = bits1, s1
+    return out
 
 
 def mixquant_dequant(mq) -> np.ndarray:
@@ -258,6 +276,11 @@ def mixquant_dequant(mq) -> np.ndarray:
     d = len(mq["abn_idx"]) + len(mq["nom_idx"])
     out = np.zeros((T, d), dtype=np.float64)
     out[:, mq["abn_idx"]] = gdequant_groups(mq["codes2"], mq["s2"], mq["z2"])
+    if len(mq["nom_idx"]) == 0:
+        return out
+    if mq.get("mode", "fft") == "minmax":
+        out[:, mq["nom_idx"]] = gdequant_groups(mq["codes1"], mq["s1"], mq["z1"])
+        return out
     for g in range(mq["s1"].shape[0]):
         sl = slice(g * G, min((g + 1) * G, T))
         xr, _ = fft_1bit_dequant(mq["bits1"][sl], mq["s1"][g])
@@ -408,8 +431,9 @@ class SlabCache:
     Algorithm 1, Q(X_Kq), X_Kr, Q(X_Vq), X_Vr, with the key part kept as a list
     of independently MixQuant-ed chunks (prefill chunk, then one per flush)."""
 
-    def __init__(self, ratio: float = 0.5, gamma=GAMMA, ternary_scale: str = "mean_abs"):
+    def __init__(self, ratio: float = 0.5, gamma=GAMMA, ternary_scale: str = "mean_abs", one_bit: str = "auto"):
         self.ratio = ratio
+        self.one_bit = one_bit
         self.gamma = gamma
         self.ternary_scale = ternary_scale
         self.k_chunks = []        # list of mixquant dicts
@@ -429,7 +453,7 @@ class SlabCache:
         if E is None:
             E = np.zeros(l, dtype=bool)
         self.v_prefill = stpquant(vq, np.asarray(E[:l - r], dtype=bool), self.gamma, self.ternary_scale)
-        self.k_chunks = [mixquant(kq, self.ratio)] if l - r > 0 else []
+        self.k_chunks = [mixquant(kq, self.ratio, self.one_bit)] if l - r > 0 else []
 
     def dequant_k(self) -> np.ndarray:
         """DeQuant(Q(X_Kq)); each chunk's result is kept once computed."""
@@ -466,7 +490,7 @@ class SlabCache:
         out = attention(q, K, V, scale)
         if self.v_res.shape[0] == R:                      # residual flush
             self.v_flush.append(quant_1p58_groups(self.v_res, self.gamma, self.ternary_scale))
-            self.k_chunks.append(mixquant(self.k_res, self.ratio))
+            self.k_chunks.append(mixquant(self.k_res, self.ratio, self.one_bit))
             self.k_res = np.zeros((0, d), dtype=np.float32)
             self.v_res = np.zeros((0, d), dtype=np.float32)
         return out

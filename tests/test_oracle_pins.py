@@ -608,3 +608,100 @@ def test_attention_over_token_shards_merges_to_the_whole():
     m, l, o = O.attention_partial(q, K[:0], V[:0], scale)
     assert np.isneginf(m).all() and (l == 0).all() and (o == 0).all()
 
+
+
+# ------------------------------------------------------------------ other bit widths (Algorithm 3 with other k)
+def test_bit_accounting_of_the_other_ratios():
+    k = fp16_values((64, 128), 11)
+    for ratio, key in ((0.25, "key_bits_at_k_0p25"), (1.0, "key_bits_at_k_1p0")):
+        abn, nom = O.select_channels(k, ratio)
+        assert len(abn) + len(nom) == 128 and not set(abn) & set(nom)
+        assert (2 * len(abn) + len(nom)) / 128 == GOLD[key]["value"]
+    for ratio in (0.25, 0.5, 0.75, 1.0):
+        assert (O.one_bit_mode(ratio) == "fft") == (ratio in GOLD["fft_one_bit_ratios"]["value"])
+
+
+def test_one_bit_minmax_is_the_two_level_code():
+    # GQuant with n = 1 (Eq. 4): levels z = min and z + s = max; every element goes to the nearer one
+    x = fp16_values((32, 24), 12, scale=3.0)
+    q, s, z = O.gquant(x, 1)
+    assert set(np.unique(q)) == {0, 1}
+    s32, z32 = s.astype(np.float64), z.astype(np.float64)
+    for c in range(x.shape[1]):
+        col = x[:, c].astype(np.float64)
+        assert q[col.argmin(), c] == 0 and q[col.argmax(), c] == 1
+        nearer = (np.abs(col - (z32[c] + s32[c])) < np.abs(col - z32[c])).astype(np.int8)
+        undecided = np.abs(np.abs(col - (z32[c] + s32[c])) - np.abs(col - z32[c])) < 1e-3 * s32[c]
+        assert np.array_equal(q[:, c][~undecided], nearer[~undecided])
+    d = O.gdequant(q, s, z)
+    assert np.all(np.abs(d - x) <= 0.5 * s32 + np.abs(x) * 2.0 ** -10 + 1e-6)
+
+
+@pytest.mark.parametrize("ratio,n_abn", [(0.25, 32), (0.5, 64), (0.75, 96)])
+def test_mixquant_minmax_mode(ratio, n_abn):
+    cfg = CONFIGS["tiny"]
+    K, _ = make_layer_kv(cfg, 0, T=96)
+    k = K[0, 2].float().numpy()
+    mq = O.mixquant(k, ratio, one_bit="minmax")
+    assert mq["mode"] == "minmax" and len(mq["abn_idx"]) == n_abn and len(mq["nom_idx"]) == 128 - n_abn
+    assert mq["codes1"].shape == (96, 128 - n_abn) and mq["s1"].shape == (3, 128 - n_abn) == mq["z1"].shape
+    kd = O.mixquant_dequant(mq)
+    nom, abn = mq["nom_idx"], mq["abn_idx"]
+    # normal channels: every dequantized element is one of the group's two levels, which are the
+    # binary16 roundings of the group's minimum and of minimum + (maximum - minimum)
+    for g in range(3):
+        blk = k[32 * g:32 * g + 32][:, nom]
+        lo = blk.min(axis=0).astype(np.float16).astype(np.float64)
+        rng_h = (blk.max(axis=0) - blk.min(axis=0)).astype(np.float16).astype(np.float64)
+        got = kd[32 * g:32 * g + 32][:, nom]
+        assert np.all((got == lo) | (got == lo + rng_h))
+        assert np.all(np.abs(got - blk) <= 0.5 * rng_h + np.abs(blk) * 2.0 ** -10 + 1e-6)
+    # anomalous channels are untouched by the mode
+    ref = O.mixquant(k, ratio, one_bit="fft")
+    assert np.array_equal(ref["abn_idx"], abn) and np.array_equal(ref["codes2"], mq["codes2"])
+    assert np.array_equal(kd[:, abn], O.mixquant_dequant(ref)[:, abn])
+
+
+def test_mixquant_all_channels_two_bit():
+    k = fp16_values((64, 128), 13, scale=2.0)
+    mq = O.mixquant(k, 1.0)
+    assert len(mq["nom_idx"]) == 0 and np.array_equal(mq["abn_idx"], np.arange(128))
+    kd = O.mixquant_dequant(mq)
+    c, s, z = O.gquant_groups(k, 2)
+    assert np.array_equal(kd, O.gdequant_groups(c, s, z))
+    s_tok = np.repeat(s.astype(np.float64), 32, axis=0)
+    assert np.all(np.abs(kd - k) <= 0.5 * s_tok + np.abs(k) * 2.0 ** -10 + 1e-6)
+
+
+def test_mixquant_fft_on_32_normal_channels():
+    # k = 0.75: the transform runs over the 32 normal channels; a chunk whose normal channels hold one
+    # cosine of the channel position has a single spectral line, so the sign code keeps its phase
+    T = 32
+    k = np.zeros((T, 128), dtype=np.float32)
+    k[:, :96] = (np.arange(96) % 7 + 1.0) * 4.0 * np.where(np.arange(T)[:, None] % 2, 1.0, -1.0)   # wide range: anomalous
+    pos = np.arange(32)
+    k[:, 96:] = np.cos(2 * np.pi * 3 * pos / 32)[None, :].astype(np.float16)
+    mq = O.mixquant(k, 0.75)
+    assert mq["mode"] == "fft" and np.array_equal(mq["nom_idx"], np.arange(96, 128))
+    assert mq["bits1"].shape == (T, 64) and mq["s1"].shape == (1, 64)
+    # the library transform of the same rows: the code's scales are the mean magnitudes of its parts
+    spec = np.fft.fft(k[:, 96:].astype(np.float64), axis=1, norm="ortho")
+    assert np.allclose(mq["s1"][0, :32].astype(np.float64), np.abs(spec.real).mean(axis=0), rtol=2e-3, atol=1e-4)
+    assert np.allclose(mq["s1"][0, 32:].astype(np.float64), np.abs(spec.imag).mean(axis=0), rtol=2e-3, atol=1e-4)
+    kd = O.mixquant_dequant(mq)[:, 96:]
+    # bins 3 and 29 dominate the reconstruction: it correlates strongly with the input
+    corr = (kd * k[:, 96:]).sum() / np.sqrt((kd ** 2).sum() * (k[:, 96:] ** 2).sum())
+    assert corr > 0.9
+
+
+def test_slabcache_carries_ratio_and_mode_through_a_flush():
+    cfg = CONFIGS["tiny"]
+    K, V = make_layer_kv(cfg, 0, T=64 + O.R)
+    k, v = K[0, 0].float().numpy(), V[0, 0].float().numpy()
+    sc = O.SlabCache(ratio=0.25, one_bit="auto")
+    sc.prefill(k[:64], v[:64])
+    q = fp16_values((7, 128), 14)
+    for t in range(O.R):
+        sc.decode_step(q, k[64 + t], v[64 + t])
+    assert len(sc.k_chunks) == 2 and all(c["mode"] == "minmax" and len(c["abn_idx"]) == 32 for c in sc.k_chunks)
+    assert sc.dequant_k().shape == (64 + O.R, 128)
