@@ -102,7 +102,13 @@ enum {
 };
 
 enum { VIDKV_F16 = 0, VIDKV_BF16 = 1, VIDKV_F32 = 2 };
-enum { VIDKV_KEY1BIT_FFT_SIGN = 0 };
+/* Algorithm 3, 1BitQuant: how the normal (1-bit) key channels are coded.
+ *   VIDKV_KEY1BIT_FFT_SIGN      Eq. 5: orthonormal DFT over the normal channels of a token, then sign bit and
+ *                               per-(group, column) mean magnitude; k_ratio 0.5 or 0.75 (as in Sec. 4.1)
+ *   VIDKV_KEY1BIT_PLAIN_MINMAX  the other branch: Eq. 4 with n = 1 on the channels as they are (levels
+ *                               min and max of the group); k_ratio 0.25, 0.5 or 0.75
+ * With k_ratio = 1 every channel is 2-bit and the mode has no effect. */
+enum { VIDKV_KEY1BIT_FFT_SIGN = 0, VIDKV_KEY1BIT_PLAIN_MINMAX = 1 };
 /* Channel metrics of Sec. 4.1(1) other than the range (which the method uses and computes itself). */
 enum { VIDKV_METRIC_VARIANCE = 1, VIDKV_METRIC_OUTLIERS = 2 };
 /* Scale stored with the ternary codes of Eq. 6 (the paper gives the codes only): the Mean |v|
@@ -120,12 +126,12 @@ typedef struct {
   int32_t D;                  /* head dimension (128) */
   int32_t G;                  /* group size (32) */
   int32_t R;                  /* residual length (128) */
-  float k_ratio;              /* fraction of key channels kept at 2 bits (0.5) */
+  float k_ratio;              /* fraction of key channels kept at 2 bits: 0.25, 0.5 (default), 0.75 or 1 */
   float p_ratio;              /* fraction of visual tokens protected at 2 bits, in [0, 1] */
   float gamma;                /* ternary threshold factor (0.7) */
   int32_t in_dtype;           /* VIDKV_F16 | VIDKV_BF16 */
   int32_t out_dtype;          /* VIDKV_F16 | VIDKV_BF16 | VIDKV_F32 */
-  int32_t key_1bit_mode;      /* VIDKV_KEY1BIT_FFT_SIGN */
+  int32_t key_1bit_mode;      /* VIDKV_KEY1BIT_FFT_SIGN | VIDKV_KEY1BIT_PLAIN_MINMAX */
   int32_t ternary_scale;      /* VIDKV_TERNARY_SCALE_MEAN_ABS (default) | VIDKV_TERNARY_SCALE_NONZERO_MEAN */
   int64_t max_prefill_tokens; /* largest T passed to vidkv_quantize_* */
   int64_t max_new_tokens;     /* decode steps the cache must be able to absorb */

@@ -10,5 +10,5 @@ from .api import (  # noqa: F401
     vidkv_cache_bytes, vidkv_cache_layout, vidkv_version, vidkv_launch_count, vidkv_attend_noalloc, vidkv_saliency_scores, vidkv_channel_metrics,
     vidkv_debug_decode_plan, vidkv_debug_withhold_once, vidkv_merge_partials,
     STATUS_NAMES,
-    VIDKV_F16, VIDKV_BF16, VIDKV_F32, VIDKV_TERNARY_SCALE_MEAN_ABS, VIDKV_TERNARY_SCALE_NONZERO_MEAN, VIDKV_METRIC_VARIANCE, VIDKV_METRIC_OUTLIERS,
+    VIDKV_F16, VIDKV_BF16, VIDKV_F32, VIDKV_TERNARY_SCALE_MEAN_ABS, VIDKV_TERNARY_SCALE_NONZERO_MEAN, VIDKV_METRIC_VARIANCE, VIDKV_METRIC_OUTLIERS, VIDKV_KEY1BIT_FFT_SIGN, VIDKV_KEY1BIT_PLAIN_MINMAX,
 )

@@ -7,6 +7,7 @@ from dataclasses import dataclass
 
 VIDKV_F16, VIDKV_BF16, VIDKV_F32 = 0, 1, 2
 VIDKV_TERNARY_SCALE_MEAN_ABS, VIDKV_TERNARY_SCALE_NONZERO_MEAN = 0, 1
+VIDKV_KEY1BIT_FFT_SIGN, VIDKV_KEY1BIT_PLAIN_MINMAX = 0, 1
 VIDKV_METRIC_VARIANCE, VIDKV_METRIC_OUTLIERS = 1, 2
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "UNSUPPORTED", -3: "ALIGNMENT", -4: "CAPACITY",
                 -5: "STATE", -6: "CUDA", -7: "TIMEOUT"}
@@ -364,12 +365,16 @@ class VidKVCache:
         nt = (n_prefill_q - st["n_protected"] + 31) // 32 + 4 * n_flush
         npg = (st["n_protected"] + 31) // 32
         dev = self.cache.device
+        n2 = int(round(self.cfg.k_ratio * 128))
+        n1 = 128 - n2
+        plain = n1 > 0 and self.cfg.key_1bit_mode == VIDKV_KEY1BIT_PLAIN_MINMAX
         out = dict(
-            k2=torch.zeros((B, H, 32 * ng, 64), dtype=torch.int8, device=dev),
-            k1bits=torch.zeros((B, H, 32 * ng, 64), dtype=torch.uint8, device=dev),
-            k_s2=torch.zeros((B, H, ng, 64), dtype=torch.float16, device=dev),
-            k_z2=torch.zeros((B, H, ng, 64), dtype=torch.float16, device=dev),
-            k_s1=torch.zeros((B, H, ng, 64), dtype=torch.float16, device=dev),
+            k2=torch.zeros((B, H, 32 * ng, n2), dtype=torch.int8, device=dev),
+            k1bits=torch.zeros((B, H, 32 * ng, n1), dtype=torch.uint8, device=dev),
+            k_s2=torch.zeros((B, H, ng, n2), dtype=torch.float16, device=dev),
+            k_z2=torch.zeros((B, H, ng, n2), dtype=torch.float16, device=dev),
+            # plain min/max mode: per group the n1 scales, then the n1 zero points
+            k_s1=torch.zeros((B, H, ng, 2, n1) if plain else (B, H, ng, n1), dtype=torch.float16, device=dev),
             v_trits=torch.zeros((B, H, 32 * nt, 128), dtype=torch.int8, device=dev),
             v_s=torch.zeros((B, H, nt, 128), dtype=torch.float16, device=dev),
             v2=torch.zeros((B, H, 32 * npg, 128), dtype=torch.int8, device=dev),

@@ -11,7 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvidkv.so")
-SOURCES = ["host.cu", "quant_keys.cu", "quant_keys_enc.cu", "quant_values.cu", "decode.cu", "decode_prep.cu", "decode_stream.cu", "dequant.cu", "export.cu", "noalloc.cu", "saliency.cu", "chan_metrics.cu"]
+SOURCES = ["host.cu", "quant_keys.cu", "quant_keys_enc.cu", "quant_keys_general.cu", "quant_values.cu", "decode.cu", "decode_prep.cu", "decode_stream.cu", "dequant.cu", "export.cu", "noalloc.cu", "saliency.cu", "chan_metrics.cu"]
 HEADERS = ["common.cuh", "kernels.cuh", "decode_common.cuh", os.path.join("..", "..", "include", "vidkv.h")]
 
 

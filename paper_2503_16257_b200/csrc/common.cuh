@@ -31,9 +31,64 @@ constexpr int kHdrStatus = 8;      // byte offset of the device status word
 
 constexpr uint32_t kMagic = 0x564b4456u;  // "VDKV"
 
+// Key-group format of a cache (Algorithm 3 with its parameter k and the 1-bit mode).  The default
+// (64 two-bit channels, Eq. 5 on the other 64) has the fixed layout above and its own kernels; every
+// other combination uses the general layout, built from blocks of 32 channels:
+//   [0, 256 n2b)            2-bit codes, block by block: lane l = 4 tl + r of a warp owns the 8 bytes
+//                           8 l .. 8 l + 7 of a block = four 16-bit half-words, one per 8-token tile
+//                           nt; the half-word of token t = 8 nt + tl holds the block's slots
+//                           8 r + e: even e in the low byte, odd e in the high byte, at bits 2 (e / 2);
+//   then 128 n1b bytes      1-bit codes, block by block: lane l owns the 32-bit word l of a block,
+//                           byte nt of it holds columns 8 r + e of token 8 nt + tl at bit 7 - e;
+//   then s (binary16) and z (binary16) of the n2 two-bit slots;
+//   then s of the n1 one-bit columns (Eq. 5: spectrum columns of the orthonormal n1-point DFT of the
+//   normal channels in Hermitian order; plain mode: the normal channels), and in plain mode their z.
+struct KeyFmt {
+  int32_t n2;            // two-bit (anomalous) channels: 32, 64, 96 or 128
+  int32_t plain;         // 1: the one-bit channels carry the plain min/max code (Eq. 4 with n = 1), 0: Eq. 5
+  int32_t general;       // 0: the default format with its fixed layout
+  int32_t group_bytes;   // bytes of one 32-token key group
+  int32_t off_bits1, off_s2, off_z2, off_s1, off_z1;   // general layout: byte offsets inside a group
+  __host__ __device__ int n1() const { return kD - n2; }
+};
+inline KeyFmt make_key_fmt(int n2, int plain) {
+  KeyFmt f;
+  f.n2 = n2; f.plain = plain;
+  f.general = !(n2 == kNA && !plain);
+  if (!f.general) {
+    f.group_bytes = kKGroupBytes;
+    f.off_bits1 = kKG_Bits1; f.off_s2 = kKG_S2; f.off_z2 = kKG_Z2; f.off_s1 = kKG_S1; f.off_z1 = kKGroupBytes;
+    return f;
+  }
+  const int n1 = kD - n2;
+  f.off_bits1 = n2 * 8;
+  f.off_s2 = f.off_bits1 + n1 * 4;
+  f.off_z2 = f.off_s2 + n2 * 2;
+  f.off_s1 = f.off_z2 + n2 * 2;
+  f.off_z1 = f.off_s1 + n1 * 2;
+  f.group_bytes = f.off_z1 + (plain ? n1 * 2 : 0);
+  return f;
+}
+// The key format a configuration asks for (k_ratio and key_1bit_mode already validated).
+inline KeyFmt key_fmt_of_config(const vidkv_config_t& c) {
+  const int n2 = static_cast<int>(c.k_ratio * kD + 0.5f);
+  return make_key_fmt(n2, (n2 < kD && c.key_1bit_mode == VIDKV_KEY1BIT_PLAIN_MINMAX) ? 1 : 0);
+}
+constexpr int kMaxKGroupBytes = 1536;   // the largest general key group (all channels at two bits)
+// General layout: where slot j (of the n2 two-bit slots) / column f (of the n1 one-bit columns) of token t sits.
+__host__ __device__ __forceinline__ int gk2_byte(int t, int j) {
+  return (j >> 5) * 256 + ((t & 7) * 4 + ((j >> 3) & 3)) * 8 + (t >> 3) * 2 + (j & 1);
+}
+__host__ __device__ __forceinline__ int gk2_bit(int j) { return 2 * ((j & 7) >> 1); }
+__host__ __device__ __forceinline__ int gk1_byte(int t, int f) {
+  return (f >> 5) * 128 + ((t & 7) * 4 + ((f >> 3) & 3)) * 4 + (t >> 3);
+}
+__host__ __device__ __forceinline__ int gk1_bit(int f) { return 7 - (f & 7); }
+
 // Device-side view of one cache: everything a kernel needs to find a slab region.
 struct CacheView {
   uint8_t* base;
+  KeyFmt kf;
   int64_t sel_offset, sel_stride_b, sel_words;
   int64_t slab_offset, slab_stride;
   int64_t chunk_table_offset, kgroup_offset, tern_offset, prot_offset, kres_offset, vres_offset;

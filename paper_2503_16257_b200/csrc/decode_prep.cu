@@ -100,15 +100,90 @@ __global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int
   out[24 * 32] = __float_as_uint(a.scale * 1.4426950408889634f * pow2i(qe + kQShift));
 }
 
+// ---------------------------------------------------------------------------------
+// The same for the general key formats (KeyFmt): one warp per (chunk, slab); per lane (head hd = lane / 4,
+// r = lane % 4), all of the normalised query:
+//   words 0 .. n2/8 - 1         binary16 pairs of q at the two-bit slots 32 (w / 4) + 8 r + 2 (w % 4), + 1
+//   then n1/8 words             plain mode: pairs of q at the one-bit channels with the same index rule;
+//                               Eq. 5: leading binary16 part of the transformed query Q at those columns,
+//   then (Eq. 5) n1/8 words     binary16 remainder Q - leading part
+//   word 24                     the factor that turns a score into a base-2 logit
+// Q_f = sum_c q_c W[c, f], W = the weights with which column f of the Hermitian half spectrum enters
+// normal channel c under the inverse orthonormal n1-point transform (columns >= 2 count twice).
+// ---------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads) decode_prep_general_kernel(DecodeArgs a, int n_chunks, int n_items) {
+  const CacheView& cv = a.cv;
+  const int lane = threadIdx.x & 31;
+  const int item = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+  if (item >= n_items) return;
+  const int chunk = item % n_chunks, slab = item / n_chunks;
+  const int hd = lane >> 2, r = lane & 3;
+  const int h = slab % cv.H_kv, lb = slab / cv.H_kv;
+  const int rep = cv.rep;
+  const int n2 = cv.kf.n2, n1 = kD - n2;
+  const uint8_t* perm = cv.slab(a.layer0 + lb / cv.B, lb % cv.B, h) + cv.chunk_table_offset +
+                        static_cast<int64_t>(chunk) * kChunkBytes;
+  const T* qrow = reinterpret_cast<const T*>(a.q) + (static_cast<int64_t>(lb) * cv.H_q + h * rep + hd) * kD;
+  const bool live = hd < rep;
+  const int qe = head_exponent<T, 4>(qrow, r, live);
+  const float qf = pow2i(-qe - kQShift);
+  auto q_at = [&](int c) -> float { return live ? Elem<T>::to_float(qrow[c]) * qf : 0.0f; };
+  if (chunk == 0 && a.append_row >= 0) {
+    uint8_t* sp = cv.slab(a.layer0 + lb / cv.B, lb % cv.B, h);
+    const uint4* srcp = reinterpret_cast<const uint4*>(lane < 16 ? a.k_new : a.v_new) + static_cast<int64_t>(slab) * 16 + (lane & 15);
+    reinterpret_cast<uint4*>(sp + (lane < 16 ? cv.kres_offset : cv.vres_offset))[a.append_row * 16 + (lane & 15)] = __ldg(srcp);
+  }
+  uint32_t* out = a.prep + (static_cast<int64_t>(slab) * n_chunks + chunk) * (kPrepWords * 32) + lane;
+  for (int w = 0; w < n2 / 8; ++w) {
+    const int j = 32 * (w >> 2) + 8 * r + 2 * (w & 3);
+    out[w * 32] = pack_half2(q_at(perm[j]), q_at(perm[j + 1]));
+  }
+  const int w1 = n2 / 8;
+  if (cv.kf.plain) {
+    for (int w = 0; w < n1 / 8; ++w) {
+      const int i = 32 * (w >> 2) + 8 * r + 2 * (w & 3);
+      out[(w1 + w) * 32] = pack_half2(q_at(perm[n2 + i]), q_at(perm[n2 + i + 1]));
+    }
+  } else {
+    const float norm = rsqrtf(static_cast<float>(n1));
+    for (int w = 0; w < n1 / 8; ++w) {
+      float x[2];
+      for (int e = 0; e < 2; ++e) {
+        const int f = 32 * (w >> 2) + 8 * r + 2 * (w & 3) + e;
+        const int k = f < 2 ? (f == 0 ? 0 : n1 / 2) : f >> 1;
+        const bool imag = f >= 2 && (f & 1);
+        float acc = 0.0f;
+        for (int c = 0; c < n1; ++c) {
+          float sn, cs;
+          sincospif(2.0f * static_cast<float>((k * c) % n1) / static_cast<float>(n1), &sn, &cs);
+          acc = fmaf(q_at(perm[n2 + c]), imag ? -sn : cs, acc);
+        }
+        x[e] = acc * norm * (f < 2 ? 1.0f : 2.0f);
+      }
+      const __half h0 = __float2half_rn(x[0]), h1 = __float2half_rn(x[1]);
+      out[(w1 + w) * 32] = pack_half2(__half2float(h0), __half2float(h1));
+      out[(w1 + n1 / 8 + w) * 32] = pack_half2(x[0] - __half2float(h0), x[1] - __half2float(h1));
+    }
+  }
+  out[24 * 32] = __float_as_uint(a.scale * 1.4426950408889634f * pow2i(qe + kQShift));
+}
+
 cudaError_t launch_decode_prep(DecodeArgs& a, cudaStream_t stream) {
   a.dft = nullptr;
   const int n_slabs = a.n_layers * a.cv.B * a.cv.H_kv;
   const int n_chunks = a.plan.n_chunks;
   if (n_chunks < 1) return cudaSuccess;
   cudaError_t e;
-  if ((e = dft_fragments(&a.dft, stream))) return e;
   const int n_items = n_slabs * n_chunks;
   const int pgrid = (n_items + kThreads / 32 - 1) / (kThreads / 32);
+  if (a.cv.kf.general) {
+    if (a.in_dtype == VIDKV_F16) decode_prep_general_kernel<__half><<<pgrid, kThreads, 0, stream>>>(a, n_chunks, n_items);
+    else decode_prep_general_kernel<__nv_bfloat16><<<pgrid, kThreads, 0, stream>>>(a, n_chunks, n_items);
+    count_launches(1);
+    return cudaGetLastError();
+  }
+  if ((e = dft_fragments(&a.dft, stream))) return e;
   if (a.in_dtype == VIDKV_F16) decode_prep_kernel<__half><<<pgrid, kThreads, 0, stream>>>(a, n_chunks, n_items);
   else decode_prep_kernel<__nv_bfloat16><<<pgrid, kThreads, 0, stream>>>(a, n_chunks, n_items);
   count_launches(1);

@@ -36,6 +36,7 @@ constexpr int kKBufBytes = kSGGroups * kKGroupBytes;   // 5760: the key groups o
 constexpr int kVBufBytes = kSGBytes;                   // 5376: its ternary supergroup
 constexpr int kTotBytes = 4 * 2 * 32 * 16;             // 4096: the warp's running output (128 channels x 8 heads, float)
 constexpr int kWarpBufBytes = kKBufBytes + kVBufBytes + kTotBytes;   // 15232 per warp
+constexpr int kGenKBufBytes = kSGGroups * kMaxKGroupBytes;           // key buffer of the general key formats
 constexpr uint32_t kWaitLimit = 1u << 19;              // mbarrier polls before a warp gives up (about a second)
 constexpr float kStaleLog2 = 6.0f;                     // the running maximum may lag a unit's maximum by this much
 constexpr uint32_t kMinus5 = 0xc500c500u;              // binary16 pair (-5.0, -5.0)
@@ -154,6 +155,92 @@ __device__ __forceinline__ void score_group(const uint8_t* kg, int lane, int hd,
   }
 }
 
+// The same for a key group in the general layout (KeyFmt): blocks of 32 two-bit slots, then blocks of
+// 32 one-bit columns.  pp points at this lane's prepared query words of the group's chunk (32 words
+// apart).  Two-bit slots as above (q s as hi + lo against 4 + code).  One-bit columns: Eq. 5 as above
+// with the transformed query; in plain mode the value is code s + z = (+-1) s / 2 + (z + s / 2), so q s
+// (hi + lo) meets +-1, the products are halved at the end and the constant takes sum q z + sum q s / 2.
+__device__ __forceinline__ void score_group_general(const uint8_t* kg, const KeyFmt& kf, int lane, int hd, int r,
+                                                    const uint32_t* pp, uint32_t m_field, uint32_t c_four, uint32_t m_sign,
+                                                    uint32_t c_neg1, float (&sc)[4][2], float& cst) {
+  float acc[4][4], acc1[4][4];
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { acc[nt][i] = 0.0f; acc1[nt][i] = 0.0f; }
+  }
+  float cz[4] = {0.0f, 0.0f, 0.0f, 0.0f}, cz1[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+  const int n2b = kf.n2 >> 5, n1b = (kD - kf.n2) >> 5;
+#pragma unroll 1
+  for (int b = 0; b < n2b; ++b) {
+    uint32_t qa[4], hi[4], lo[4];
+    const uint4 sv = *reinterpret_cast<const uint4*>(kg + kf.off_s2 + 64 * b + 16 * r);
+    const uint4 zv = *reinterpret_cast<const uint4*>(kg + ((hd & 1) ? kf.off_s2 : kf.off_z2) + 64 * b + 16 * r);
+    const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w}, zw[4] = {zv.x, zv.y, zv.z, zv.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      qa[j] = __ldg(pp + (4 * b + j) * 32);
+      hi[j] = hmul2_u(qa[j], sw[j]);
+      lo[j] = hfms2_u(qa[j], sw[j], hi[j]);
+    }
+    const uint2 cw = *reinterpret_cast<const uint2*>(kg + 256 * b + lane * 8);
+    uint32_t W[4];
+    W[0] = prmt(cw.x, 0u, 0x1404u); W[1] = prmt(cw.x, 0u, 0x3424u);
+    W[2] = prmt(cw.y, 0u, 0x1404u); W[3] = prmt(cw.y, 0u, 0x3424u);
+#pragma unroll
+    for (int kp = 0; kp < 2; ++kp) {
+      mma_f16(cz, qa[2 * kp], 0u, qa[2 * kp + 1], 0u, zw[2 * kp], zw[2 * kp + 1]);
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt)
+        mma_f16(acc[nt], hi[2 * kp], lo[2 * kp], hi[2 * kp + 1], lo[2 * kp + 1], and_or(W[nt] >> (4 * kp), m_field, c_four),
+                and_or(W[nt] >> (4 * kp + 2), m_field, c_four));
+    }
+  }
+  const int w1 = kf.n2 >> 3, nw1 = (kD - kf.n2) >> 3;
+#pragma unroll 1
+  for (int b = 0; b < n1b; ++b) {
+    uint32_t hi[4], lo[4];
+    const uint4 sv = *reinterpret_cast<const uint4*>(kg + kf.off_s1 + 64 * b + 16 * r);
+    const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
+    if (kf.plain) {
+      const uint4 zv = *reinterpret_cast<const uint4*>(kg + ((hd & 1) ? kf.off_s1 : kf.off_z1) + 64 * b + 16 * r);
+      const uint32_t zw[4] = {zv.x, zv.y, zv.z, zv.w};
+      uint32_t qb[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        qb[j] = __ldg(pp + (w1 + 4 * b + j) * 32);
+        hi[j] = hmul2_u(qb[j], sw[j]);
+        lo[j] = hfms2_u(qb[j], sw[j], hi[j]);
+      }
+      mma_f16(cz1, qb[0], 0u, qb[1], 0u, zw[0], zw[1]);
+      mma_f16(cz1, qb[2], 0u, qb[3], 0u, zw[2], zw[3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t qh = __ldg(pp + (w1 + 4 * b + j) * 32), ql = __ldg(pp + (w1 + nw1 + 4 * b + j) * 32);
+        hi[j] = hmul2_u(qh, sw[j]);
+        lo[j] = hfma2_u(ql, sw[j], hfms2_u(qh, sw[j], hi[j]));
+      }
+    }
+    const uint32_t cw = *reinterpret_cast<const uint32_t*>(kg + kf.off_bits1 + 128 * b + lane * 4);
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      const uint32_t X = ((cw >> (8 * nt)) & 0xffu) * 0x02000100u;   // low lane: bit 7 at the sign, high lane: bit 6
+#pragma unroll
+      for (int kp = 0; kp < 2; ++kp)
+        mma_f16(acc1[nt], hi[2 * kp], lo[2 * kp], hi[2 * kp + 1], lo[2 * kp + 1], and_xor(X << (4 * kp), m_sign, c_neg1),
+                and_xor(X << (4 * kp + 2), m_sign, c_neg1));
+    }
+  }
+  const float f1 = kf.plain ? 0.5f : 1.0f;
+  cst = cz[0] - 4.0f * cz[1] + (kf.plain ? cz1[0] + 0.5f * cz1[1] : 0.0f);
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) {
+    sc[nt][0] = acc[nt][0] + acc[nt][2] + f1 * (acc1[nt][0] + acc1[nt][2]);
+    sc[nt][1] = acc[nt][1] + acc[nt][3] + f1 * (acc1[nt][1] + acc1[nt][3]);
+  }
+}
+
 // Running output of the warp, kept in shared memory: float4 tot[j][lane], j = 2 w + i, holds the
 // accumulator fragment of channels 32 w + 4 hd + 2 i + (e >> 1) and heads 2 r + (e & 1), e = 0..3.
 
@@ -224,14 +311,15 @@ __device__ __forceinline__ void pv_ternary(const uint8_t* vbuf, float* totbuf, c
 
 // One unit of NG (1..5) groups: scores, probabilities, P V into the running state.
 // Returns false if a copy never arrived.
-template <int NG>
-__device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float* totbuf, uint64_t* kbar, uint64_t* vbar,
+template <int NG, bool GEN>
+__device__ __forceinline__ bool process_unit(const KeyFmt& kf, const uint32_t*& ppc, uint8_t* kbuf, uint8_t* vbuf, float* totbuf, uint64_t* kbar, uint64_t* vbar,
                                              uint32_t& kpar, uint32_t& vpar, int lane, int hd, int r,
                                              const uint32_t* prep_slab, int64_t g_first, int64_t g0n, int& cur_chunk,
                                              uint32_t (&qa)[8], uint32_t (&qha)[8], uint32_t (&qhb)[8], float sl2,
                                              Running& run, bool more, const uint8_t* next_k, uint32_t next_k_bytes,
                                              const uint8_t* next_v) {
   const uint32_t m_field = kExpand[0], c_four = kExpand[1], m_sign = kExpand[2], c_neg1 = kExpand[3];
+  const int kgb = GEN ? kf.group_bytes : kKGroupBytes;      // bytes of one key group
   if (!mbar_wait(kbar, kpar)) return false;
   kpar ^= 1u;
   // ---- scores, group by group; a group's scores replace its (spent) bytes in the key buffer:
@@ -245,16 +333,20 @@ __device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float
     if (chunk != cur_chunk) {
       cur_chunk = chunk;
       const uint32_t* pp = prep_slab + static_cast<int64_t>(chunk) * (kPrepWords * 32);
+      ppc = pp;
+      if (!GEN) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        qa[i] = __ldg(pp + i * 32);
-        qha[i] = __ldg(pp + (8 + i) * 32);
-        qhb[i] = __ldg(pp + (16 + i) * 32);
+        for (int i = 0; i < 8; ++i) {
+          qa[i] = __ldg(pp + i * 32);
+          qha[i] = __ldg(pp + (8 + i) * 32);
+          qhb[i] = __ldg(pp + (16 + i) * 32);
+        }
       }
     }
     float sc[4][2], cst;
-    uint8_t* kg = kbuf + g * kKGroupBytes;
-    score_group(kg, lane, hd, r, qa, qha, qhb, m_field, c_four, m_sign, c_neg1, sc, cst);
+    uint8_t* kg = kbuf + g * kgb;
+    if (GEN) score_group_general(kg, kf, lane, hd, r, ppc, m_field, c_four, m_sign, c_neg1, sc, cst);
+    else score_group(kg, lane, hd, r, qa, qha, qhb, m_field, c_four, m_sign, c_neg1, sc, cst);
     __syncwarp();                                           // every lane has read the group's bytes
     float gm = fmaxf(sc[0][0], sc[0][1]);
 #pragma unroll
@@ -290,10 +382,10 @@ __device__ __forceinline__ bool process_unit(uint8_t* kbuf, uint8_t* vbuf, float
   float ps[NG][4];
 #pragma unroll
   for (int g = 0; g < NG; ++g) {
-    const float off = fmaf(reinterpret_cast<const float*>(kbuf + g * kKGroupBytes)[256 + lane], sl2, -run.m);
+    const float off = fmaf(reinterpret_cast<const float*>(kbuf + g * kgb)[256 + lane], sl2, -run.m);
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
-      const float2 v = reinterpret_cast<const float2*>(kbuf + g * kKGroupBytes)[nt * 32 + lane];
+      const float2 v = reinterpret_cast<const float2*>(kbuf + g * kgb)[nt * 32 + lane];
       P[g][nt] = pack_half2(ex2_approx(fmaf(v.x, sl2, off)), ex2_approx(fmaf(v.y, sl2, off)));
     }
     // -5 * (sums of the rounded probabilities) of heads 2 r, 2 r + 1, for rows hd and hd + 8 alike:
@@ -356,6 +448,7 @@ __device__ __forceinline__ void write_record(const DecodeArgs& a, int slab, int 
 
 }  // namespace
 
+template <bool GEN>
 __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_stream_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[kStreamWarps][2];
@@ -366,8 +459,11 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_st
   const int64_t u_begin = static_cast<int64_t>(run_id) * pl.run_units;
   const int64_t u_end = min(u_begin + pl.run_units, pl.n_units);
   if (u_begin >= u_end) return;                            // warps do not wait on one another
-  uint8_t* kbuf = smem_raw + warp * kWarpBufBytes;
-  uint8_t* vbuf = kbuf + kKBufBytes;
+  const KeyFmt& kf = a.cv.kf;
+  const int kgb = GEN ? kf.group_bytes : kKGroupBytes;
+  constexpr int kbuf_bytes = GEN ? kGenKBufBytes : kKBufBytes;
+  uint8_t* kbuf = smem_raw + warp * (kbuf_bytes + kVBufBytes + kTotBytes);
+  uint8_t* vbuf = kbuf + kbuf_bytes;
   float* totbuf = reinterpret_cast<float*>(vbuf + kVBufBytes);
   uint64_t* kbar = &bars[warp][0];
   uint64_t* vbar = &bars[warp][1];
@@ -388,19 +484,20 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_st
     return left < kSGGroups ? static_cast<int>(left) : kSGGroups;
   };
   auto key_src = [&](int sl, int kk) -> const uint8_t* {
-    return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.kgroup_offset + static_cast<int64_t>(kk) * kKBufBytes;
+    return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.kgroup_offset + static_cast<int64_t>(kk) * (kSGGroups * kgb);
   };
   auto val_src = [&](int sl, int kk) -> const uint8_t* {
     return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.tern_offset + static_cast<int64_t>(kk) * kVBufBytes;
   };
   if (lane == 0) {
-    bulk_load(kbuf, key_src(slab, k), groups_of(k) * kKGroupBytes, kbar);
+    bulk_load(kbuf, key_src(slab, k), groups_of(k) * kgb, kbar);
     if (!a.withhold) bulk_load(vbuf, val_src(slab, k), kVBufBytes, vbar);   // (test hook: see DecodeArgs::withhold)
   }
   uint32_t kpar = 0u, vpar = 0u;
   Running run;
   run.l[0] = 0.0f; run.l[1] = 0.0f; run.m = -INFINITY;
   uint32_t qa[8], qha[8], qhb[8];
+  const uint32_t* ppc = nullptr;
   int cur_chunk = -1, cur_slab = -1;
   const uint32_t* prep_slab = nullptr;
   float sl2 = 0.0f;
@@ -423,10 +520,10 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_st
     if (nk == S) { nk = 0; ++nslab; }
     const bool more = u + 1 < u_end;
     const uint8_t* next_k = more ? key_src(nslab, nk) : nullptr;
-    const uint32_t next_k_bytes = more ? static_cast<uint32_t>(groups_of(nk) * kKGroupBytes) : 0u;
+    const uint32_t next_k_bytes = more ? static_cast<uint32_t>(groups_of(nk) * kgb) : 0u;
     const uint8_t* next_v = more ? val_src(nslab, nk) : nullptr;
 #define VIDKV_UNIT(N)                                                                                                \
-  ok = process_unit<N>(kbuf, vbuf, totbuf, kbar, vbar, kpar, vpar, lane, hd, r, prep_slab,                           \
+  ok = process_unit<N, GEN>(kf, ppc, kbuf, vbuf, totbuf, kbar, vbar, kpar, vpar, lane, hd, r, prep_slab,                           \
                        static_cast<int64_t>(k) * kSGGroups, g0n, cur_chunk, qa, qha, qhb, sl2, run, more, next_k,      \
                        next_k_bytes, next_v)
     if (ng == 5) VIDKV_UNIT(5);
@@ -534,6 +631,7 @@ __device__ __forceinline__ void zero_ring_range(uint8_t* ring, int ring_len, int
 
 }  // namespace
 
+template <bool GEN>
 __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode_stream_stp_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[kStreamWarps][3];
@@ -544,8 +642,11 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
   const int64_t u_begin = static_cast<int64_t>(run_id) * pl.run_units;
   const int64_t u_end = min(u_begin + pl.run_units, pl.n_units);
   if (u_begin >= u_end) return;
-  uint8_t* kbuf = smem_raw + warp * kStpWarpBytes;
-  uint8_t* vbuf = kbuf + kKBufBytes;
+  const KeyFmt& kf = a.cv.kf;
+  const int kgb = GEN ? kf.group_bytes : kKGroupBytes;
+  constexpr int kbuf_bytes = GEN ? kGenKBufBytes : kKBufBytes;
+  uint8_t* kbuf = smem_raw + warp * (kStpWarpBytes - kKBufBytes + kbuf_bytes);
+  uint8_t* vbuf = kbuf + kbuf_bytes;
   uint8_t* pbuf = vbuf + kVBufBytes;
   float* totbuf = reinterpret_cast<float*>(pbuf + kPGBytes);
   uint8_t* rings = reinterpret_cast<uint8_t*>(totbuf) + kTotBytes;
@@ -578,15 +679,16 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
     return left < kSGGroups ? left : kSGGroups;
   };
   auto key_src = [&](int sl, int kk) -> const uint8_t* {
-    return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.kgroup_offset + static_cast<int64_t>(kk) * kKBufBytes;
+    return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.kgroup_offset + static_cast<int64_t>(kk) * (kSGGroups * kgb);
   };
-  if (lane == 0) bulk_load(kbuf, key_src(slab, k), groups_of(k) * kKGroupBytes, kbar);
+  if (lane == 0) bulk_load(kbuf, key_src(slab, k), groups_of(k) * kgb, kbar);
   const uint32_t lt_mask = (1u << lane) - 1u;              // lanes (= tokens of a group) before this one
   uint32_t kpar = 0u, vpar = 0u, ppar = 0u;
   bool v_pending = false, p_pending = false;               // a copy into vbuf / pbuf has been issued and not yet waited for
   Running run;
   run.l[0] = 0.0f; run.l[1] = 0.0f; run.m = -INFINITY;
   uint32_t qa[8], qha[8], qhb[8];
+  const uint32_t* ppc = nullptr;
   int cur_chunk = -1, cur_slab = -1;
   const uint32_t* prep_slab = nullptr;
   const uint32_t* ew = nullptr;
@@ -644,16 +746,20 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
       if (chunk != cur_chunk) {
         cur_chunk = chunk;
         const uint32_t* pp = prep_slab + static_cast<int64_t>(chunk) * (kPrepWords * 32);
+        ppc = pp;
+        if (!GEN) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          qa[i] = __ldg(pp + i * 32);
-          qha[i] = __ldg(pp + (8 + i) * 32);
-          qhb[i] = __ldg(pp + (16 + i) * 32);
+          for (int i = 0; i < 8; ++i) {
+            qa[i] = __ldg(pp + i * 32);
+            qha[i] = __ldg(pp + (8 + i) * 32);
+            qhb[i] = __ldg(pp + (16 + i) * 32);
+          }
         }
       }
       float sc[4][2], cst;
-      uint8_t* kg = kbuf + g * kKGroupBytes;
-      score_group(kg, lane, hd, r, qa, qha, qhb, m_field, c_four, m_sign, c_neg1, sc, cst);
+      uint8_t* kg = kbuf + g * kgb;
+      if (GEN) score_group_general(kg, kf, lane, hd, r, ppc, m_field, c_four, m_sign, c_neg1, sc, cst);
+      else score_group(kg, lane, hd, r, qa, qha, qhb, m_field, c_four, m_sign, c_neg1, sc, cst);
       __syncwarp();
       float gm = fmaxf(sc[0][0], sc[0][1]);
 #pragma unroll
@@ -698,7 +804,7 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
     // pick up the destinations of their own four token pairs with shuffles.
 #pragma unroll 1
     for (int g = 0; g < ng; ++g) {
-      const uint8_t* kg = kbuf + g * kKGroupBytes;
+      const uint8_t* kg = kbuf + g * kgb;
       const float off = fmaf(reinterpret_cast<const float*>(kg)[256 + lane], sl2, -run.m);
       const int tg = t_unit + g * kG;
       if (tg < T_q0) {
@@ -731,7 +837,7 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
     __syncwarp();
     if (more && lane == 0) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      bulk_load(kbuf, key_src(nslab, nk), groups_of(nk) * kKGroupBytes, kbar);
+      bulk_load(kbuf, key_src(nslab, nk), groups_of(nk) * kgb, kbar);
     }
     // ---- how far the two streams are complete now
     const int t_end = t_unit + ng * kG;
@@ -809,18 +915,21 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
 }
 
 cudaError_t launch_decode_stream_stp(const DecodeArgs& a, cudaStream_t stream) {
-  const size_t smem = static_cast<size_t>(kStreamWarps) * kStpWarpBytes;
-  static bool attr_set[64] = {};
+  const bool gen = a.cv.kf.general != 0;
+  const size_t smem = static_cast<size_t>(kStreamWarps) * (kStpWarpBytes + (gen ? kGenKBufBytes - kKBufBytes : 0));
+  static bool attr_set[64][2] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!attr_set[dev]) {
-    const cudaError_t e = cudaFuncSetAttribute(decode_stream_stp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (!attr_set[dev][gen]) {
+    const cudaError_t e = gen ? cudaFuncSetAttribute(decode_stream_stp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                              : cudaFuncSetAttribute(decode_stream_stp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_set[dev] = true;
+    attr_set[dev][gen] = true;
   }
   const int grid = (a.plan.n_runs + kStreamWarps - 1) / kStreamWarps;
   if (grid < 1) return cudaSuccess;
-  decode_stream_stp_kernel<<<grid, kStreamWarps * 32, smem, stream>>>(a);
+  if (gen) decode_stream_stp_kernel<true><<<grid, kStreamWarps * 32, smem, stream>>>(a);
+  else decode_stream_stp_kernel<false><<<grid, kStreamWarps * 32, smem, stream>>>(a);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -828,18 +937,21 @@ cudaError_t launch_decode_stream_stp(const DecodeArgs& a, cudaStream_t stream) {
 cudaError_t launch_decode_stream(const DecodeArgs& a_in, cudaStream_t stream) {
   DecodeArgs a = a_in;
   if (g_debug_withhold == 2) { a.withhold = 1; g_debug_withhold = 0; }
-  const size_t smem = static_cast<size_t>(kStreamWarps) * kWarpBufBytes;
-  static bool attr_set[64] = {};
+  const bool gen = a.cv.kf.general != 0;
+  const size_t smem = static_cast<size_t>(kStreamWarps) * (kWarpBufBytes + (gen ? kGenKBufBytes - kKBufBytes : 0));
+  static bool attr_set[64][2] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (!attr_set[dev]) {
-    const cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (!attr_set[dev][gen]) {
+    const cudaError_t e = gen ? cudaFuncSetAttribute(decode_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                              : cudaFuncSetAttribute(decode_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_set[dev] = true;
+    attr_set[dev][gen] = true;
   }
   const int grid = (a.plan.n_runs + kStreamWarps - 1) / kStreamWarps;
   if (grid < 1) return cudaSuccess;
-  decode_stream_kernel<<<grid, kStreamWarps * 32, smem, stream>>>(a);
+  if (gen) decode_stream_kernel<true><<<grid, kStreamWarps * 32, smem, stream>>>(a);
+  else decode_stream_kernel<false><<<grid, kStreamWarps * 32, smem, stream>>>(a);
   count_launches(1);
   return cudaGetLastError();
 }

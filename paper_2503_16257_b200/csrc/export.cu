@@ -34,6 +34,35 @@ __global__ void __launch_bounds__(128) export_keys_kernel(CacheView cv, int laye
   }
 }
 
+// The same for the general key formats: thread = slot (tid < n2) or one-bit column / channel.
+// ks1 holds per group n1 scales, in plain mode followed by the n1 zero points.
+__global__ void __launch_bounds__(128) export_keys_general_kernel(CacheView cv, int layer, int64_t n_groups, int8_t* k2,
+                                                                  uint8_t* k1, uint16_t* ks2, uint16_t* kz2, uint16_t* ks1) {
+  const int slab = blockIdx.y, tid = threadIdx.x;
+  const int64_t g = blockIdx.x;
+  const KeyFmt kf = cv.kf;
+  const int n2 = kf.n2, n1 = kD - n2;
+  const uint8_t* kg = cv.slab(layer, slab / cv.H_kv, slab % cv.H_kv) + cv.kgroup_offset + g * kf.group_bytes;
+  const int64_t grp = static_cast<int64_t>(slab) * n_groups + g;
+  if (tid < n2) {
+    const int j = tid;
+    if (k2)
+      for (int t = 0; t < kG; ++t) k2[(grp * kG + t) * n2 + j] = static_cast<int8_t>((kg[gk2_byte(t, j)] >> gk2_bit(j)) & 3u);
+    if (ks2) ks2[grp * n2 + j] = reinterpret_cast<const uint16_t*>(kg + kf.off_s2)[j];
+    if (kz2) kz2[grp * n2 + j] = reinterpret_cast<const uint16_t*>(kg + kf.off_z2)[j];
+  } else {
+    const int f = tid - n2;
+    if (k1)
+      for (int t = 0; t < kG; ++t)
+        k1[(grp * kG + t) * n1 + f] = static_cast<uint8_t>((kg[kf.off_bits1 + gk1_byte(t, f)] >> gk1_bit(f)) & 1u);
+    if (ks1) {
+      const int per = kf.plain ? 2 * n1 : n1;
+      ks1[grp * per + f] = reinterpret_cast<const uint16_t*>(kg + kf.off_s1)[f];
+      if (kf.plain) ks1[grp * per + n1 + f] = reinterpret_cast<const uint16_t*>(kg + kf.off_z1)[f];
+    }
+  }
+}
+
 // grid = (ternary stream groups, slabs); 128 threads = channels.
 __global__ void __launch_bounds__(128) export_ternary_kernel(CacheView cv, int layer, int64_t n_groups, int8_t* trits,
                                                              uint16_t* vs) {
@@ -72,7 +101,7 @@ __global__ void __launch_bounds__(128) export_dmask_kernel(CacheView cv, int lay
   uint8_t* out = dmask + (static_cast<int64_t>(slab) * n_chunks + chunk) * kD;
   out[tid] = 0;
   __syncthreads();
-  if (tid < kNA) out[perm[tid]] = 1;
+  if (tid < cv.kf.n2) out[perm[tid]] = 1;
 }
 
 __global__ void export_mask_kernel(CacheView cv, int64_t T, int64_t T_sel, uint8_t* E) {
@@ -89,7 +118,10 @@ cudaError_t launch_export_codes(const CacheView& cv, int layer, int64_t n_kgroup
                                 uint16_t* vs, int8_t* v2, uint16_t* v2s, uint16_t* v2z, cudaStream_t stream) {
   const int slabs = cv.B * cv.H_kv;
   if (n_kgroups > 0 && (k2 || k1 || ks2 || kz2 || ks1)) {
-    export_keys_kernel<<<dim3(static_cast<unsigned>(n_kgroups), slabs), 128, 0, stream>>>(cv, layer, n_kgroups, k2, k1, ks2, kz2, ks1);
+    if (cv.kf.general)
+      export_keys_general_kernel<<<dim3(static_cast<unsigned>(n_kgroups), slabs), 128, 0, stream>>>(cv, layer, n_kgroups, k2, k1, ks2, kz2, ks1);
+    else
+      export_keys_kernel<<<dim3(static_cast<unsigned>(n_kgroups), slabs), 128, 0, stream>>>(cv, layer, n_kgroups, k2, k1, ks2, kz2, ks1);
     count_launches(1);
   }
   if (n_tgroups > 0 && (trits || vs)) {

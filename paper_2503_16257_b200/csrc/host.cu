@@ -32,8 +32,10 @@ vidkv_status_t check_config(const vidkv_config_t* c) {
   if (c->ternary_scale != VIDKV_TERNARY_SCALE_MEAN_ABS && c->ternary_scale != VIDKV_TERNARY_SCALE_NONZERO_MEAN)
     return VIDKV_ERR_INVALID_ARG;
   if (c->D != kD || c->G != kG || c->R != kR) return VIDKV_ERR_UNSUPPORTED;
-  if (c->k_ratio != 0.5f) return VIDKV_ERR_UNSUPPORTED;
-  if (c->key_1bit_mode != VIDKV_KEY1BIT_FFT_SIGN) return VIDKV_ERR_UNSUPPORTED;
+  if (c->key_1bit_mode != VIDKV_KEY1BIT_FFT_SIGN && c->key_1bit_mode != VIDKV_KEY1BIT_PLAIN_MINMAX) return VIDKV_ERR_INVALID_ARG;
+  if (c->k_ratio != 0.25f && c->k_ratio != 0.5f && c->k_ratio != 0.75f && c->k_ratio != 1.0f) return VIDKV_ERR_UNSUPPORTED;
+  // Eq. 5 needs the transform over the normal channels; the paper applies it at k = 0.5 and 0.75 only
+  if (c->key_1bit_mode == VIDKV_KEY1BIT_FFT_SIGN && c->k_ratio == 0.25f) return VIDKV_ERR_UNSUPPORTED;
   if (c->H_q % c->H_kv != 0 || c->H_q / c->H_kv > kMaxRep) return VIDKV_ERR_UNSUPPORTED;
   if (static_cast<int64_t>(c->L) * c->B * c->H_kv > 65535) return VIDKV_ERR_UNSUPPORTED;
   return VIDKV_OK;
@@ -57,7 +59,7 @@ void compute_layout(const vidkv_config_t& c, Layout* out) {
   l.max_pgroups = (out->max_prot + kG - 1) / kG;
   int64_t off = 0;
   l.chunk_table_offset = off; off = round_up(off + l.max_chunks * kChunkBytes, kAlign);
-  l.kgroup_offset = off;      off = round_up(off + l.max_kgroups * kKGroupBytes, kAlign);
+  l.kgroup_offset = off;      off = round_up(off + l.max_kgroups * key_fmt_of_config(c).group_bytes, kAlign);
   l.tern_offset = off;        off = round_up(off + l.max_supergroups * kSGBytes, kAlign);
   l.prot_offset = off;        off = round_up(off + l.max_pgroups * kPGBytes, kAlign);
   l.kres_offset = off;        off += kResBytes;
@@ -192,6 +194,7 @@ vidkv_status_t vidkv_cache_init(const vidkv_config_t* cfg, void* cache, size_t c
   const vidkv_layout_t& l = h->L.lay;
   CacheView& cv = h->cv;
   cv.base = h->cache;
+  cv.kf = key_fmt_of_config(*cfg);
   cv.sel_offset = l.sel_offset; cv.sel_stride_b = l.sel_stride_b; cv.sel_words = l.sel_words;
   cv.slab_offset = l.slab_offset; cv.slab_stride = l.slab_stride;
   cv.chunk_table_offset = l.chunk_table_offset; cv.kgroup_offset = l.kgroup_offset;

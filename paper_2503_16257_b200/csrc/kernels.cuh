@@ -45,6 +45,10 @@ cudaError_t launch_quantize_keys(int dtype, const KSrc& src, int64_t T_tokens, c
 cudaError_t launch_encode_keys(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0, int n_slabs,
                                int slabs_per_layer, int chunk, int64_t kgroup0, cudaStream_t stream);
 
+// The same for the general key formats (other k, plain 1-bit code): one block per 32-token group.
+cudaError_t launch_encode_keys_general(int dtype, const KSrc& src, int64_t T_tokens, const CacheView& cv, int layer0,
+                                       int n_slabs, int slabs_per_layer, int chunk, int64_t kgroup0, cudaStream_t stream);
+
 // Device address of the 64-point DFT matrix in MMA B-fragment order: word
 // ((ks * 8 + nt) * 32 + lane) * 4 + {0, 1} = leading binary16 pairs, + {2, 3} = remainders, for
 // rows 16 ks + 2 r (+1; +8, +9) and column 16 (n / 2) + 2 nt + (n % 2), lane = 4 n + r; column f

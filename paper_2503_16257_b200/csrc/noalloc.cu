@@ -65,6 +65,7 @@ extern "C" vidkv_status_t vidkv_attend_noalloc(const vidkv_config_t* cfg, const 
   DecodeArgs a;
   CacheView& cv = a.cv;
   cv.base = const_cast<uint8_t*>(static_cast<const uint8_t*>(cache));
+  cv.kf = key_fmt_of_config(*cfg);
   cv.sel_offset = lay.sel_offset; cv.sel_stride_b = lay.sel_stride_b; cv.sel_words = lay.sel_words;
   cv.slab_offset = lay.slab_offset; cv.slab_stride = lay.slab_stride;
   cv.chunk_table_offset = lay.chunk_table_offset; cv.kgroup_offset = lay.kgroup_offset;

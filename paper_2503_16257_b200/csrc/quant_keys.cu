@@ -116,7 +116,8 @@ __global__ void __launch_bounds__(kD) k_select_kernel(const uint32_t* __restrict
     const float ro = s_range[o];
     rank += (ro > r) || (ro == r && o < c);
   }
-  const int is_abn = rank < kNA;
+  const int n2 = cv.kf.n2;                 // Algorithm 3: D-mask = the top k D channels by range
+  const int is_abn = rank < n2;
   s_abn[c] = is_abn;
   __syncthreads();
   int before = 0;
@@ -124,7 +125,7 @@ __global__ void __launch_bounds__(kD) k_select_kernel(const uint32_t* __restrict
   uint8_t* entry = cv.slab(layer, bh / cv.H_kv, bh % cv.H_kv) + cv.chunk_table_offset +
                    static_cast<int64_t>(chunk) * kChunkBytes;
   if (is_abn) entry[before] = static_cast<uint8_t>(c);
-  else entry[kNA + (c - before)] = static_cast<uint8_t>(c);
+  else entry[n2 + (c - before)] = static_cast<uint8_t>(c);
 }
 
 // ---------------------------------------------------------------------------------
@@ -143,8 +144,9 @@ static cudaError_t launch_keys_t(const KSrc& src, int64_t T_tokens, const CacheV
   k_range_kernel<T><<<dim3(static_cast<unsigned>(splits), n_slabs), 256, 0, stream>>>(src, T_tokens, tokens_per_block,
                                                                                        minmax);
   k_select_kernel<<<n_slabs, kD, 0, stream>>>(minmax, cv, layer0, slabs_per_layer, chunk, mm.next, mm.next_dirty_words);
-  if ((e = launch_encode_keys(std::is_same<T, __half>::value ? VIDKV_F16 : VIDKV_BF16, src, T_tokens, cv,
-                              layer0, n_slabs, slabs_per_layer, chunk, kgroup0, stream)))
+  const int dt = std::is_same<T, __half>::value ? VIDKV_F16 : VIDKV_BF16;
+  if ((e = cv.kf.general ? launch_encode_keys_general(dt, src, T_tokens, cv, layer0, n_slabs, slabs_per_layer, chunk, kgroup0, stream)
+                         : launch_encode_keys(dt, src, T_tokens, cv, layer0, n_slabs, slabs_per_layer, chunk, kgroup0, stream)))
     return e;
   count_launches(2);
   return cudaGetLastError();

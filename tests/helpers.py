@@ -28,7 +28,8 @@ def to_np(x: torch.Tensor) -> np.ndarray:
 class Pair:
     """One configuration run through both implementations (all layers, all slabs)."""
 
-    def __init__(self, wl, T, B=None, L=None, p=0.0, max_new=16, device="cuda", ternary_scale="mean_abs"):
+    def __init__(self, wl, T, B=None, L=None, p=0.0, max_new=16, device="cuda", ternary_scale="mean_abs",
+                 k_ratio=0.5, one_bit="fft"):
         import paper_2503_16257_b200 as P
         self.P = P
         self.wl, self.T, self.p = wl, T, p
@@ -37,10 +38,12 @@ class Pair:
         self.device = device
         in_dt = P.VIDKV_F16 if wl.dtype == "fp16" else P.VIDKV_BF16
         self.cfg = P.VidKVConfig(B=self.B, L=self.L, max_prefill_tokens=T, max_new_tokens=max_new, p_ratio=p,
-                                 in_dtype=in_dt, out_dtype=P.VIDKV_F32,
+                                 in_dtype=in_dt, out_dtype=P.VIDKV_F32, k_ratio=k_ratio,
+                                 key_1bit_mode=P.VIDKV_KEY1BIT_PLAIN_MINMAX if one_bit == "minmax" else P.VIDKV_KEY1BIT_FFT_SIGN,
                                  ternary_scale=P.VIDKV_TERNARY_SCALE_NONZERO_MEAN if ternary_scale == "nonzero_mean"
                                  else P.VIDKV_TERNARY_SCALE_MEAN_ABS)
         self.ternary_scale = ternary_scale
+        self.k_ratio, self.one_bit = k_ratio, one_bit
         self.cache = P.VidKVCache(self.cfg, device=device)
         self.lay = self.cache.layout
         self.l_v = min(wl.l_v, T - T % 32)
@@ -67,7 +70,7 @@ class Pair:
             self.cache.quantize_values(layer, Vd)
             for b in range(self.B):
                 for h in range(self.cfg.H_kv):
-                    sc = O.SlabCache(ternary_scale=self.ternary_scale)
+                    sc = O.SlabCache(ratio=self.k_ratio, ternary_scale=self.ternary_scale, one_bit=self.one_bit)
                     E = None
                     if self.E is not None:
                         E = np.zeros(self.T, dtype=bool)

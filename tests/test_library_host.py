@@ -82,8 +82,8 @@ def test_layout_regions_do_not_overlap(lib):
 
 
 @pytest.mark.parametrize("kw,status", [
-    (dict(D=64), -2), (dict(G=64), -2), (dict(R=64), -2), (dict(k_ratio=0.75), -2),
-    (dict(H_q=30), -2), (dict(H_q=64), -2), (dict(key_1bit_mode=1), -2),
+    (dict(D=64), -2), (dict(G=64), -2), (dict(R=64), -2), (dict(k_ratio=0.6), -2),
+    (dict(H_q=30), -2), (dict(H_q=64), -2), (dict(key_1bit_mode=2), -1), (dict(k_ratio=0.25, key_1bit_mode=0), -2),
     (dict(B=0), -1), (dict(p_ratio=1.5), -1), (dict(p_ratio=-0.1), -1), (dict(in_dtype=2), -1),
     (dict(out_dtype=7), -1), (dict(max_new_tokens=-1), -1), (dict(gamma=float("nan")), -1),
     (dict(ternary_scale=2), -1),
@@ -94,6 +94,20 @@ def test_config_validation(lib, kw, status):
     with pytest.raises(P.VidKVError) as e:
         P.vidkv_cache_bytes(P.VidKVConfig(**base))
     assert e.value.status == status
+
+
+@pytest.mark.parametrize("k_ratio,mode,group_bytes", [
+    (0.5, 0, 1152), (0.25, 1, 1152), (0.5, 1, 1280), (0.75, 1, 1408), (0.75, 0, 1344), (1.0, 0, 1536), (1.0, 1, 1536)])
+def test_key_group_bytes_follow_the_key_format(lib, k_ratio, mode, group_bytes):
+    """2 bits per anomalous channel, 1 bit per normal one, a binary16 (s, z) pair per two-bit channel,
+    one binary16 scale per spectrum column or an (s, z) pair per plain one-bit channel, per 32 tokens."""
+    n2 = int(k_ratio * 128)
+    n1 = 128 - n2
+    assert group_bytes == (2 * n2 + n1) * 32 // 8 + 4 * n2 + (4 if mode == 1 else 2) * n1
+    cfg = P.VidKVConfig(B=1, L=1, max_prefill_tokens=320, max_new_tokens=0, k_ratio=k_ratio, key_1bit_mode=mode)
+    lay = P.vidkv_cache_layout(cfg)
+    assert lay["max_kgroups"] == 10
+    assert lay["tern_offset"] - lay["kgroup_offset"] == -(-10 * group_bytes // 256) * 256
 
 
 def test_null_arguments_are_rejected_without_a_device(lib):

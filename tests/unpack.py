@@ -107,3 +107,51 @@ def selection_mask(cache: np.ndarray, lay: dict, b: int, T_q: int):
     t = np.arange(T_q)
     E = ((words[t // 32] >> (t % 32)) & 1).astype(bool)
     return E, prefix
+
+
+def general_key_group_bytes(n2: int, plain: bool) -> int:
+    """Bytes of one 32-token key group in the general layout (other k, plain 1-bit code)."""
+    n1 = D - n2
+    return n2 * 8 + n1 * 4 + n2 * 4 + n1 * 2 * (2 if plain else 1)
+
+
+def chunk_perm_general(slab: np.ndarray, lay: dict, chunk: int, n2: int):
+    e = slab[lay["chunk_table_offset"] + chunk * CHUNK_BYTES:][:CHUNK_BYTES]
+    return e[:n2].astype(np.int64), e[n2:].astype(np.int64)
+
+
+def key_groups_general(slab: np.ndarray, lay: dict, g_begin: int, n_groups: int, n2: int, plain: bool):
+    """General key layout -> codes2 [32n, n2], bits1 [32n, n1], s2, z2 [n, n2], s1 [n, n1], z1 [n, n1] or None.
+
+    Blocks of 32 channels.  Two-bit region: byte (block, lane = 4 (t % 8) + (j % 32) // 8, tile t // 8,
+    parity j % 2) at block * 256 + lane * 8 + tile * 2 + parity, field (j % 8) // 2.  One-bit region:
+    byte (block, lane, tile) at block * 128 + lane * 4 + tile, column j % 8 at bit 7 - j % 8."""
+    n1 = D - n2
+    gb = general_key_group_bytes(n2, plain)
+    t = np.arange(G)[:, None]
+    j2 = np.arange(n2)[None, :]
+    off2 = (j2 // 32) * 256 + ((t % 8) * 4 + (j2 % 32) // 8) * 8 + (t // 8) * 2 + j2 % 2
+    sh2 = 2 * ((j2 % 8) // 2)
+    j1 = np.arange(n1)[None, :]
+    off1 = (j1 // 32) * 128 + ((t % 8) * 4 + (j1 % 32) // 8) * 4 + t // 8
+    sh1 = 7 - j1 % 8
+    o_b1 = n2 * 8
+    o_s2 = o_b1 + n1 * 4
+    o_z2 = o_s2 + n2 * 2
+    o_s1 = o_z2 + n2 * 2
+    o_z1 = o_s1 + n1 * 2
+    codes2 = np.zeros((n_groups * G, n2), np.int8)
+    bits1 = np.zeros((n_groups * G, n1), np.uint8)
+    s2 = np.zeros((n_groups, n2), np.float16); z2 = np.zeros((n_groups, n2), np.float16)
+    s1 = np.zeros((n_groups, n1), np.float16); z1 = np.zeros((n_groups, n1), np.float16) if plain else None
+    for g in range(n_groups):
+        rec = slab[lay["kgroup_offset"] + (g_begin + g) * gb:][:gb]
+        codes2[g * G:(g + 1) * G] = (rec[off2].astype(np.int64) >> sh2) & 3
+        if n1:
+            bits1[g * G:(g + 1) * G] = (rec[o_b1:][off1].astype(np.int64) >> sh1) & 1
+        s2[g] = rec[o_s2:o_z2].view("<f2")
+        z2[g] = rec[o_z2:o_s1].view("<f2")
+        s1[g] = rec[o_s1:o_z1].view("<f2")
+        if plain:
+            z1[g] = rec[o_z1:o_z1 + n1 * 2].view("<f2")
+    return codes2, bits1, s2, z2, s1, z1
