@@ -36,13 +36,25 @@ FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used if ME
 NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = {"decode_stream_kernel": 72.15, "decode_stream_stp_kernel": 79.28}
 
 
+KG_BYTES = 1152      # bytes of one 32-token key group; follows --k-ratio / --key-1bit (set in main)
+KEY_FORMAT = {"k_ratio": 0.5, "one_bit": "fft"}
+
+
+def key_group_bytes(k_ratio, one_bit):
+    """2 bits per anomalous channel and 1 per normal one for 32 tokens, a binary16 (s, z) pair per 2-bit channel,
+    a binary16 scale per spectrum column or an (s, z) pair per plain 1-bit channel."""
+    n2 = int(round(k_ratio * 128))
+    n1 = 128 - n2
+    return (2 * n2 + n1) * 4 + 4 * n2 + (4 if one_bit == "minmax" else 2) * n1
+
+
 def algorithmic_decode_bytes(B, L, H_kv, H_q, T_q0, n_flush, n_res, n_prot, elem=2):
     """Bytes one decode step must read/write per the packed layout (all layers)."""
     kgroups = T_q0 // 32 + 4 * n_flush
     n_rest = T_q0 - n_prot
     tgroups = (n_rest + 31) // 32 + 4 * n_flush
     pgroups = (n_prot + 31) // 32
-    per_slab = kgroups * 1152 + tgroups * (5376 / 5) + pgroups * 1536 + n_res * 128 * elem * 2 \
+    per_slab = kgroups * KG_BYTES + tgroups * (5376 / 5) + pgroups * 1536 + n_res * 128 * elem * 2 \
         + (1 + n_flush) * 128
     io = H_q * 128 * (elem + 4) + 2 * H_kv * 128 * elem
     return L * B * (H_kv * per_slab + io)
@@ -51,7 +63,7 @@ def algorithmic_decode_bytes(B, L, H_kv, H_q, T_q0, n_flush, n_res, n_prot, elem
 def algorithmic_quantize_bytes(B, L, H_kv, T, n_prot, elem=2):
     T_q = T - T % 32
     read = 2 * T * 128 * elem
-    write = (T_q // 32) * 1152 + ((T_q - n_prot + 31) // 32) * (5376 / 5) + ((n_prot + 31) // 32) * 1536
+    write = (T_q // 32) * KG_BYTES + ((T_q - n_prot + 31) // 32) * (5376 / 5) + ((n_prot + 31) // 32) * 1536
     return L * B * H_kv * (read + write)
 
 
@@ -154,7 +166,7 @@ def oracle_sample(wl, p, device_tensors=None, max_batch=8, n_steps=8):
     slabs = []
     for b in range(nb):
         for h in range(H):
-            sc = O.SlabCache()
+            sc = O.SlabCache(ratio=KEY_FORMAT["k_ratio"], one_bit=KEY_FORMAT["one_bit"])
             sc.prefill(K[b, h].float().numpy(), V[b, h].float().numpy(), E[b] if E is not None else None)
             slabs.append(sc)
     t_quant = time.perf_counter() - t0
@@ -207,6 +219,7 @@ def run_reference(args, wl):
 def workload_config(wl, p):
     return {"workload": wl.name, "layers": wl.layers, "batch_per_gpu": wl.batch, "tokens": wl.T, "kv_heads": 4,
             "query_heads": 28, "head_dim": 128, "decode_steps": wl.steps, "dtype": wl.dtype, "p": p,
+            "k_ratio": KEY_FORMAT["k_ratio"], "key_1bit": KEY_FORMAT["one_bit"],
             "cache": "inputs larger than L2 (no flush needed)" if wl.name in ("batched", "stress")
             else "packed cache fits L2: rotated over copies larger than L2"}
 
@@ -219,6 +232,10 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="batched")
     ap.add_argument("--p", type=float, default=0.0, help="fraction of visual tokens protected at 2 bits")
+    ap.add_argument("--k-ratio", type=float, default=0.5, choices=[0.25, 0.5, 0.75, 1.0],
+                    help="fraction of key channels at 2 bits (Algorithm 3's k)")
+    ap.add_argument("--key-1bit", default=None, choices=["fft", "minmax"],
+                    help="1-bit code of the normal key channels; default: the paper's choice for the k (Sec. 4.1)")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (profiling captures)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the decode steps per bench step")
     ap.add_argument("--no-e2e", action="store_true")
@@ -227,6 +244,12 @@ def main():
     ap.add_argument("--no-variants", action="store_true", help="skip the warm / cold and per-layer-launch figures of "
                     "the workloads whose packed cache fits L2")
     args = ap.parse_args()
+    global KG_BYTES
+    one_bit = args.key_1bit or ("fft" if args.k_ratio in (0.5, 0.75) else "minmax")
+    if one_bit == "fft" and args.k_ratio == 0.25:
+        ap.error("the FFT 1-bit code is built for k = 0.5 and 0.75 (Sec. 4.1); use --key-1bit minmax")
+    KEY_FORMAT.update(k_ratio=args.k_ratio, one_bit=one_bit)
+    KG_BYTES = key_group_bytes(args.k_ratio, one_bit)
 
     from dataclasses import replace
     from workloads import CONFIGS
@@ -259,7 +282,8 @@ def main():
     steps_dec = wl.steps
     in_dt = P.VIDKV_F16 if wl.dtype == "fp16" else P.VIDKV_BF16
     cfg = P.VidKVConfig(B=B, L=L, max_prefill_tokens=T, max_new_tokens=steps_dec, p_ratio=args.p,
-                        in_dtype=in_dt, out_dtype=P.VIDKV_F32)
+                        in_dtype=in_dt, out_dtype=P.VIDKV_F32, k_ratio=args.k_ratio,
+                        key_1bit_mode=P.VIDKV_KEY1BIT_PLAIN_MINMAX if KEY_FORMAT["one_bit"] == "minmax" else P.VIDKV_KEY1BIT_FFT_SIGN)
     # Small workloads: rotate over enough independent caches that one decode step never finds its
     # cache in L2 (126 MB); large ones exceed L2 by themselves.
     one_cache = algorithmic_decode_bytes(B, L, H, HQ, T - T % 32, 0, 1, 0)
@@ -368,7 +392,10 @@ def main():
     kern_bytes = dec_bytes / steps_dec
     kern_gbs = kern_bytes / (kern_avg_ms * 1e-3) / 1e9
     kernel_name = "decode_stream_stp_kernel" if n_prot > 0 else "decode_stream_kernel"
-    traffic = NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD.get(kernel_name)
+    general_fmt = not (KEY_FORMAT["k_ratio"] == 0.5 and KEY_FORMAT["one_bit"] == "fft")
+    if general_fmt:
+        kernel_name += "<general key format>"          # the same kernel, instantiated for the general key layout
+    traffic = NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD.get(kernel_name)   # counters exist for the default format only
     if traffic is not None:
         traffic = traffic * B * L * H * (T - T % 32)
 
@@ -393,7 +420,7 @@ def main():
     }
     # what the packed cache saves: FP16 K and V of the prompt against the bytes the layout holds for it
     fp16_bytes = 2 * 2 * 128 * H * B * L * T
-    packed_bytes = B * L * H * ((T // 32) * 1152 + ((T - T % 32 - n_prot + 31) // 32) * (5376 / 5) + ((n_prot + 31) // 32) * 1536
+    packed_bytes = B * L * H * ((T // 32) * KG_BYTES + ((T - T % 32 - n_prot + 31) // 32) * (5376 / 5) + ((n_prot + 31) // 32) * 1536
                                 + (T % 32) * 512)
     line["memory"] = {"fp16_kv_bytes": fp16_bytes, "packed_kv_bytes": packed_bytes,
                       "bytes_saved_vs_fp16": fp16_bytes - packed_bytes, "saved_frac": 1.0 - packed_bytes / fp16_bytes}

@@ -29,9 +29,12 @@
  *     the library (56 KB) with one extra small kernel on the caller's stream and records an
  *     event that later calls make their streams wait for; make that first call outside any
  *     stream capture.
- *   - Fixed in this library: D = 128, G = 32, R = 128, k = 0.5 (64 two-bit and 64
- *     one-bit channels), H_q a multiple of H_kv with H_q / H_kv <= 8.  Other
- *     shapes return VIDKV_ERR_UNSUPPORTED.
+ *   - Fixed in this library: D = 128, G = 32, R = 128, H_q a multiple of H_kv with
+ *     H_q / H_kv <= 8; k_ratio one of 0.25, 0.5, 0.75, 1 (32, 64, 96 or 128 two-bit key
+ *     channels; Table 2's 1.25-, 1.5-, 1.75- and 2-bit key rows).  Other shapes return
+ *     VIDKV_ERR_UNSUPPORTED.  k_ratio = 0.5 with VIDKV_KEY1BIT_FFT_SIGN (the default) has the
+ *     key-group layout below and the fastest kernels; every other combination uses the
+ *     general key-group layout described after it.
  *   - Element types: VIDKV_F16 / VIDKV_BF16 for K, V, q, k_new, v_new (in_dtype);
  *     VIDKV_F16 / VIDKV_BF16 / VIDKV_F32 for the attention output (out_dtype).
  *     Input values must be finite and representable in binary16.
@@ -77,6 +80,22 @@
  *     residual     : K_r and V_r, 128 x 128 elements each, in in_dtype.
  *   per batch element: the protection mask E as bit words plus, per word, the
  *   number of protected tokens before it.
+ *
+ * General key-group layout (every k_ratio / key_1bit_mode other than the default), with n2 two-bit
+ * slots and n1 = 128 - n2 one-bit columns, both taken in blocks of 32:
+ *     chunk table  : per chunk 128 bytes: n2 ascending anomalous channel ids, then the n1 normal ones.
+ *     key groups   : per 32 tokens 8 n2 + 4 n1 + 4 n2 + 2 n1 (Eq. 5) or 4 n1 (plain) bytes
+ *                    (token t = 8 nt + tl; lane = 4 tl + r, r = (index within the block) / 8):
+ *                    2-bit codes : block b of 32 slots is 256 bytes; byte b * 256 + lane * 8 + nt * 2 + par
+ *                               holds the slots 32 b + 8 r + e with e % 2 == par of token t, slot e at
+ *                               bits 2 (e / 2);
+ *                    1-bit codes : block b of 32 columns is 128 bytes; byte b * 128 + lane * 4 + nt holds
+ *                               the columns 32 b + 8 r + e of token t, column e at bit 7 - e;
+ *                    then s (binary16) [n2], z (binary16) [n2] of the two-bit slots;
+ *                    then s (binary16) [n1] of the one-bit columns -- Eq. 5: columns of the orthonormal
+ *                    n1-point DFT of the normal channels in the Hermitian order given above (column 1 =
+ *                    Re X[n1 / 2]); plain mode: the normal channels in ascending order, code 0 / 1 with
+ *                    value code * s + z -- and, in plain mode only, their z (binary16) [n1].
  */
 #ifndef VIDKV_H_
 #define VIDKV_H_
@@ -304,11 +323,14 @@ vidkv_status_t vidkv_dequantize_values(vidkv_cache_t* handle, int32_t layer, flo
  * element per code, so that a test need not know the bit layout (Eq. 4, Eq. 5, Eq. 6 codes as
  * Algorithm 1 stores them).  With ng = n_quantized / 32 key groups, nt ternary stream groups
  * (ceil((n_prefill_quantized - n_protected) / 32) + 4 per flush) and np = ceil(n_protected / 32)
- * protected groups, per slab = (b, h) of the layer, all device pointers, any of them may be NULL:
- *   k2      int8  [B, H_kv, 32 ng, 64]   Eq. 4 codes 0..3 of the 2-bit channels, slot order
+ * protected groups, per slab = (b, h) of the layer, all device pointers, any of them may be NULL
+ * (n2 = 128 k_ratio two-bit channels, n1 = 128 - n2; 64 and 64 by default):
+ *   k2      int8  [B, H_kv, 32 ng, n2]   Eq. 4 codes 0..3 of the 2-bit channels, slot order
  *                                        (slot j = j-th channel of the chunk's ascending 2-bit list)
- *   k1bits  uint8 [B, H_kv, 32 ng, 64]   Eq. 5 bits of the spectrum columns (column order of the layout)
- *   k_s2, k_z2, k_s1  binary16 [B, H_kv, ng, 64]
+ *   k1bits  uint8 [B, H_kv, 32 ng, n1]   Eq. 5 bits of the spectrum columns (column order of the layout),
+ *                                        or the plain 1-bit codes of the normal channels (ascending)
+ *   k_s2, k_z2  binary16 [B, H_kv, ng, n2]
+ *   k_s1    binary16 [B, H_kv, ng, n1]; in plain min/max mode [B, H_kv, ng, 2, n1]: scales, then zero points
  *   v_trits int8  [B, H_kv, 32 nt, 128]  Eq. 6 codes -1, 0, +1 in ternary stream order
  *   v_s     binary16 [B, H_kv, nt, 128]
  *   v2      int8  [B, H_kv, 32 np, 128]  Eq. 4 codes of the protected tokens, stream order

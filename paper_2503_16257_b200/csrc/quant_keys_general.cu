@@ -18,13 +18,16 @@ namespace vidkv {
 
 namespace {
 
+constexpr int kMaxFftChannels = 32;   // Eq. 5 comes here for k = 0.75 only (k = 0.5 has the default format's encoder)
+
 template <typename T>
 __global__ void __launch_bounds__(kD) k_encode_general_kernel(KSrc src, CacheView cv, int layer0, int slabs_per_layer,
                                                               int chunk, int64_t kgroup0) {
-  __shared__ float x[kG][kD + 1];            // the group's tile, token major (padded against bank conflicts)
+  __shared__ __align__(16) float x[kG][kD + 4];   // the group's tile, token major
   __shared__ uint8_t code[kG][kD];           // one code per (token, slot / column), packed afterwards
   __shared__ uint8_t perm[kD];
   __shared__ double tw_cos[kD], tw_sin[kD];  // cos / sin of 2 pi m / n1
+  __shared__ double mag[kG][kMaxFftChannels];   // |X| per (token, spectrum column)
   const int tid = threadIdx.x;
   const int slab = blockIdx.y;
   const int64_t g = blockIdx.x;
@@ -36,7 +39,14 @@ __global__ void __launch_bounds__(kD) k_encode_general_kernel(KSrc src, CacheVie
   perm[tid] = slab_ptr[cv.chunk_table_offset + static_cast<int64_t>(chunk) * kChunkBytes + tid];
   const T* base = reinterpret_cast<const T*>(src.ptr) + (slab / src.H) * src.stride_b + (slab % src.H) * src.stride_h +
                   g * kG * src.stride_t;
-  for (int t = 0; t < kG; ++t) x[t][tid] = Elem<T>::to_float(base[t * src.stride_t + tid]);
+  // 16 bytes (8 channels) per thread and step: 16 threads per token row, 8 rows per step
+  for (int t = tid >> 4; t < kG; t += kD / 16) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(base + t * src.stride_t) + (tid & 15));
+    const float2 f0 = Elem<T>::to_float2(v.x), f1 = Elem<T>::to_float2(v.y), f2 = Elem<T>::to_float2(v.z), f3 = Elem<T>::to_float2(v.w);
+    float4* dst = reinterpret_cast<float4*>(&x[t][(tid & 15) * 8]);
+    dst[0] = make_float4(f0.x, f0.y, f1.x, f1.y);
+    dst[1] = make_float4(f2.x, f2.y, f3.x, f3.y);
+  }
   if (!kf.plain && tid < n1) sincospi(2.0 * static_cast<double>(tid) / static_cast<double>(n1), &tw_sin[tid], &tw_cos[tid]);
   __syncthreads();
   uint8_t* kg = slab_ptr + cv.kgroup_offset + (kgroup0 + g) * kf.group_bytes;
@@ -63,24 +73,31 @@ __global__ void __launch_bounds__(kD) k_encode_general_kernel(KSrc src, CacheVie
       reinterpret_cast<uint16_t*>(kg + kf.off_s1)[tid - n2] = sh;
       reinterpret_cast<uint16_t*>(kg + kf.off_z1)[tid - n2] = zh;
     }
-  } else {
-    // Eq. 5: spectrum column f of every token of the group
-    const int f = tid - n2;
-    const int k = f < 2 ? (f == 0 ? 0 : n1 / 2) : f >> 1;
-    const bool imag = f >= 2 && (f & 1);
+  }
+  if (!kf.plain && n1 > 0) {
+    // Eq. 5: the (token, spectrum column) pairs of the group are shared out over all threads; the
+    // magnitudes wait in shared memory and one thread per column adds them up in token order
     const double norm = 1.0 / sqrt(static_cast<double>(n1));
-    double sum = 0.0;
-    for (int t = 0; t < kG; ++t) {
+    const int mask = n1 - 1;                  // Eq. 5 is offered for n1 = 32 (a power of two)
+    for (int idx = tid; idx < n1 * kG; idx += kD) {
+      const int f = idx & mask, t = idx / n1;
+      const int k = f < 2 ? (f == 0 ? 0 : n1 / 2) : f >> 1;
+      const bool imag = f >= 2 && (f & 1);
       double acc = 0.0;
       for (int i = 0; i < n1; ++i) {
-        const int m = (k * i) % n1;
+        const int m = (k * i) & mask;
         acc += static_cast<double>(x[t][perm[n2 + i]]) * (imag ? -tw_sin[m] : tw_cos[m]);
       }
       acc *= norm;
-      sum += fabs(acc);
-      code[t][tid] = acc >= 0.0 ? 1 : 0;
+      mag[t][f] = fabs(acc);
+      code[t][n2 + f] = acc >= 0.0 ? 1 : 0;
     }
-    reinterpret_cast<uint16_t*>(kg + kf.off_s1)[f] = __half_as_ushort(__double2half(sum / kG));
+    __syncthreads();
+    if (tid < n1) {
+      double sum = 0.0;
+      for (int t = 0; t < kG; ++t) sum += mag[t][tid];
+      reinterpret_cast<uint16_t*>(kg + kf.off_s1)[tid] = __half_as_ushort(__double2half(sum / kG));
+    }
   }
   __syncthreads();
   // pack: every output byte of the two code regions is put together by one thread
