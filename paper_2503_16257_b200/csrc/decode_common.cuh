@@ -109,6 +109,12 @@ __device__ __forceinline__ uint32_t and_xor(uint32_t x, uint32_t m, uint32_t c) 
   asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(x), "r"(m), "r"(c));
   return d;
 }
+// (~x & m) ^ c: with m the sign bits, c comes out negated where x has a 0 bit
+__device__ __forceinline__ uint32_t nand_xor(uint32_t x, uint32_t m, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xA6;" : "=r"(d) : "r"(x), "r"(m), "r"(c));
+  return d;
+}
 // Bit patterns of the code expansion.  They live in constant memory rather than in the
 // instruction stream so that mask and pattern both reach the logic instruction as register
 // operands (an instruction encodes one immediate at most).

@@ -131,20 +131,16 @@ __device__ __forceinline__ void score_group(const uint8_t* kg, int lane, int hd,
       }
     }
   }
-  // normal channels in the frequency domain: Q s (leading part + remainder) against +-1
+  // normal channels in the frequency domain: Q (leading part + remainder, rows hd and hd + 8) against
+  // +-s: the scale takes the sign inside the one logic instruction that used to make +-1, and the
+  // products Q s are formed exactly by the tensor core
   {
-    uint32_t hi1[8], lo1[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      hi1[i] = hmul2_u(qha[i], s1[i]);
-      lo1[i] = hfma2_u(qhb[i], s1[i], hfms2_u(qha[i], s1[i], hi1[i]));
-    }
 #pragma unroll
     for (int ks = 0; ks < 4; ++ks) {
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt)
-        mma_f16(acc[nt], hi1[2 * ks], lo1[2 * ks], hi1[2 * ks + 1], lo1[2 * ks + 1],
-                and_xor(X[nt] << (4 * ks), m_sign, c_neg1), and_xor(X[nt] << (4 * ks + 2), m_sign, c_neg1));
+        mma_f16(acc[nt], qha[2 * ks], qhb[2 * ks], qha[2 * ks + 1], qhb[2 * ks + 1],
+                nand_xor(X[nt] << (4 * ks), m_sign, s1[2 * ks]), nand_xor(X[nt] << (4 * ks + 2), m_sign, s1[2 * ks + 1]));
     }
   }
   cst = cz[0] - 4.0f * cz[1];
