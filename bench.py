@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used if ME
 # profiles/decode_stream_stp_kernel_batched_4layers_p02.txt (p > 0): a 4-layer cut of the batched workload
 # (3 211 264 cached token-heads per launch), scaled to the launch by the token-heads it processes
 # (traffic is proportional to them).
-NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = {"decode_stream_kernel": 72.15, "decode_stream_stp_kernel": 79.28}
+NCU_TRAFFIC_BYTES_PER_TOKEN_HEAD = {"decode_stream_kernel": 71.75, "decode_stream_stp_kernel": 79.28}
 
 
 KG_BYTES = 1152      # bytes of one 32-token key group; follows --k-ratio / --key-1bit (set in main)
@@ -460,7 +460,7 @@ def run_variants(P, torch, wl, cfg, caches, qs, ks, vs, out, n_prot, quantize):
     n_steps = min(32, wl.steps)
     res = {}
     # per-layer views made once, outside the timed loops (slicing a tensor costs microseconds of host time)
-    per_layer = [[(qs[i][l:l + 1], ks[i][l:l + 1], vs[i][l:l + 1], out[l:l + 1]) for l in range(L)] for i in range(n_steps)]
+    layer_args = [[(qs[i][l:l + 1], ks[i][l:l + 1], vs[i][l:l + 1], out[l:l + 1]) for l in range(L)] for i in range(n_steps)]
     for cold in (True, False):
         for per_layer in (False, True):
             use = caches if cold else caches[:1]
@@ -476,7 +476,7 @@ def run_variants(P, torch, wl, cfg, caches, qs, ks, vs, out, n_prot, quantize):
                 i = s // len(use)
                 if per_layer:
                     for layer in range(L):
-                        c.decode_attention(layer, 1, *per_layer[i][layer])
+                        c.decode_attention(layer, 1, *layer_args[i][layer])
                 else:
                     c.decode_attention(0, L, qs[i], ks[i], vs[i], out)
                 nbytes += algorithmic_decode_bytes(B, L, H, HQ, T - T % 32, 0, st["n_residual"] + 1, n_prot)
