@@ -115,6 +115,23 @@ __device__ __forceinline__ uint32_t nand_xor(uint32_t x, uint32_t m, uint32_t c)
   asm("lop3.b32 %0, %1, %2, %3, 0xA6;" : "=r"(d) : "r"(x), "r"(m), "r"(c));
   return d;
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start
+// while the kernel before it still runs; pdl_wait() returns once that kernel has completed and its
+// writes are visible (a no-op for an ordinary launch), pdl_release() lets the kernel after this one start.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// Launch `kernel` so that it may overlap the tail of the previous kernel on `stream` (it must call pdl_wait()
+// before touching anything that kernel writes).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 // Bit patterns of the code expansion.  They live in constant memory rather than in the
 // instruction stream so that mask and pattern both reach the logic instruction as register
 // operands (an instruction encodes one immediate at most).

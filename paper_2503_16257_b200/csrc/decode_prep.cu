@@ -36,6 +36,7 @@ __global__ void __launch_bounds__(kThreads) decode_prep_kernel(DecodeArgs a, int
   const CacheView& cv = a.cv;
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+  pdl_release();                                           // the attention kernel may start its first copies now
   if (item >= n_items) return;
   const int chunk = item % n_chunks, slab = item / n_chunks;
   const int hd = lane >> 2, r = lane & 3;
@@ -116,6 +117,7 @@ __global__ void __launch_bounds__(kThreads) decode_prep_general_kernel(DecodeArg
   const CacheView& cv = a.cv;
   const int lane = threadIdx.x & 31;
   const int item = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+  pdl_release();                                           // the attention kernel may start its first copies now
   if (item >= n_items) return;
   const int chunk = item % n_chunks, slab = item / n_chunks;
   const int hd = lane >> 2, r = lane & 3;

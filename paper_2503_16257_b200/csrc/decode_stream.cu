@@ -489,6 +489,10 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamCtasPerSM) decode_st
     bulk_load(kbuf, key_src(slab, k), groups_of(k) * kgb, kbar);
     if (!a.withhold) bulk_load(vbuf, val_src(slab, k), kVBufBytes, vbar);   // (test hook: see DecodeArgs::withhold)
   }
+  // the packed cache is not written by the query preparation, so the copies above may start while
+  // it still runs; the prepared query is read from here on
+  pdl_wait();
+  pdl_release();
   uint32_t kpar = 0u, vpar = 0u;
   Running run;
   run.l[0] = 0.0f; run.l[1] = 0.0f; run.m = -INFINITY;
@@ -678,6 +682,8 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
     return slab0 + static_cast<int64_t>(sl) * cv.slab_stride + cv.kgroup_offset + static_cast<int64_t>(kk) * (kSGGroups * kgb);
   };
   if (lane == 0) bulk_load(kbuf, key_src(slab, k), groups_of(k) * kgb, kbar);
+  pdl_wait();                                              // the prepared query (and nothing else so far) comes from the kernel before
+  pdl_release();
   const uint32_t lt_mask = (1u << lane) - 1u;              // lanes (= tokens of a group) before this one
   uint32_t kpar = 0u, vpar = 0u, ppar = 0u;
   bool v_pending = false, p_pending = false;               // a copy into vbuf / pbuf has been issued and not yet waited for
@@ -924,10 +930,18 @@ cudaError_t launch_decode_stream_stp(const DecodeArgs& a, cudaStream_t stream) {
   }
   const int grid = (a.plan.n_runs + kStreamWarps - 1) / kStreamWarps;
   if (grid < 1) return cudaSuccess;
-  if (gen) decode_stream_stp_kernel<true><<<grid, kStreamWarps * 32, smem, stream>>>(a);
-  else decode_stream_stp_kernel<false><<<grid, kStreamWarps * 32, smem, stream>>>(a);
+  // with profiling events around the launch the kernel starts after the event, as an ordinary launch
+  cudaError_t le;
+  if (a.ev_begin) {
+    if (gen) decode_stream_stp_kernel<true><<<grid, kStreamWarps * 32, smem, stream>>>(a);
+    else decode_stream_stp_kernel<false><<<grid, kStreamWarps * 32, smem, stream>>>(a);
+    le = cudaGetLastError();
+  } else {
+    le = gen ? launch_dependent(decode_stream_stp_kernel<true>, dim3(grid), dim3(kStreamWarps * 32), smem, stream, a)
+             : launch_dependent(decode_stream_stp_kernel<false>, dim3(grid), dim3(kStreamWarps * 32), smem, stream, a);
+  }
   count_launches(1);
-  return cudaGetLastError();
+  return le;
 }
 
 cudaError_t launch_decode_stream(const DecodeArgs& a_in, cudaStream_t stream) {
@@ -946,10 +960,17 @@ cudaError_t launch_decode_stream(const DecodeArgs& a_in, cudaStream_t stream) {
   }
   const int grid = (a.plan.n_runs + kStreamWarps - 1) / kStreamWarps;
   if (grid < 1) return cudaSuccess;
-  if (gen) decode_stream_kernel<true><<<grid, kStreamWarps * 32, smem, stream>>>(a);
-  else decode_stream_kernel<false><<<grid, kStreamWarps * 32, smem, stream>>>(a);
+  cudaError_t le;
+  if (a.ev_begin) {
+    if (gen) decode_stream_kernel<true><<<grid, kStreamWarps * 32, smem, stream>>>(a);
+    else decode_stream_kernel<false><<<grid, kStreamWarps * 32, smem, stream>>>(a);
+    le = cudaGetLastError();
+  } else {
+    le = gen ? launch_dependent(decode_stream_kernel<true>, dim3(grid), dim3(kStreamWarps * 32), smem, stream, a)
+             : launch_dependent(decode_stream_kernel<false>, dim3(grid), dim3(kStreamWarps * 32), smem, stream, a);
+  }
   count_launches(1);
-  return cudaGetLastError();
+  return le;
 }
 
 }  // namespace vidkv
