@@ -737,6 +737,17 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
     if (nk == S) { nk = 0; ++nslab; }
     const bool more = u + 1 < u_end;
     const bool last_of_slab = !more || nslab != slab;      // the run leaves this slab after this unit
+    // the E words and prefix counts of the unit's groups (lane g: group g; lane ng: the prefix count at the
+    // unit's end) are fetched now and picked up with shuffles after the scores, their latency hidden behind them
+    uint32_t e_word_l = 0u;
+    int e_base_l = 0;
+    {
+      const int gl = t_unit / kG + lane;
+      if (lane <= ng && gl * kG <= T_q0) {
+        e_base_l = static_cast<int>(__ldg(ep + gl));
+        if (lane < ng && gl * kG < T_q0) e_word_l = __ldg(ew + gl);
+      }
+    }
     // ---- scores of the unit's groups into the key buffer (raw scores, then the group's constant)
     if (!mbar_wait(kbar, kpar)) { ok = false; break; }
     kpar ^= 1u;
@@ -809,9 +820,9 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
       const uint8_t* kg = kbuf + g * kgb;
       const float off = fmaf(reinterpret_cast<const float*>(kg)[256 + lane], sl2, -run.m);
       const int tg = t_unit + g * kG;
+      const uint32_t word = __shfl_sync(0xffffffffu, e_word_l, g);
+      const int base = __shfl_sync(0xffffffffu, e_base_l, g);   // protected tokens before the group
       if (tg < T_q0) {
-        const uint32_t word = __ldg(ew + tg / kG);
-        const int base = static_cast<int>(__ldg(ep + tg / kG));   // protected tokens before the group
         const int below = __popc(word & lt_mask);
         const bool prot = (word >> lane) & 1u;
         int idx = prot ? (base + below) % kPRing : (tg - base + lane - below) % kTRing;
@@ -844,7 +855,7 @@ __global__ void __launch_bounds__(kStreamWarps * 32, kStreamStpCtasPerSM) decode
     // ---- how far the two streams are complete now
     const int t_end = t_unit + ng * kG;
     int pp_hi, u_hi;
-    if (t_end <= T_q0) { pp_hi = static_cast<int>(__ldg(ep + t_end / kG)); u_hi = t_end - pp_hi; }
+    if (t_end <= T_q0) { pp_hi = __shfl_sync(0xffffffffu, e_base_l, ng); u_hi = t_end - pp_hi; }
     else { pp_hi = n_prot; u_hi = u_fl0 + (t_end - T_q0); }
     if (last_of_slab) {
       // what is left of the last supergroup / group belongs to a neighbour (or to nobody): zeros
