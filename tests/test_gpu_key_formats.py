@@ -154,3 +154,34 @@ def test_workspace_free_attention_on_another_key_format():
             want = O.attention(to_np(q[0, b, h * rep:(h + 1) * rep]), K, V, 1.0 / np.sqrt(128.0))
             got = o1[0, b, h * rep:(h + 1) * rep].cpu().numpy()
             assert np.abs(got - want).max() <= TOL_ABS * max(1.0, np.abs(want).max())
+
+
+def _random_cases(n, seed):
+    r = np.random.default_rng(seed)
+    cases = []
+    for _ in range(n):
+        fmt = FORMATS[int(r.integers(0, len(FORMATS)))]
+        name = ["tiny", "llava", "qwen"][int(r.integers(0, 3))]
+        cases.append((fmt, name, int(r.integers(1, 1500)), int(r.integers(1, 3)), int(r.integers(1, 3)),
+                      [0.0, 0.0, 0.1, 0.5][int(r.integers(0, 4))], int(r.integers(1, 4))))
+    return cases
+
+
+@pytest.mark.parametrize("fmt,name,T,B,L,p,steps", _random_cases(12, 20250317),
+                         ids=lambda v: _fmt_id(v) if isinstance(v, tuple) else str(v))
+def test_seeded_random_shapes(fmt, name, T, B, L, p, steps):
+    """Shapes nobody picked by hand: any token count below 1500 (any remainder modulo 32 and 160), one or two
+    sequences and layers, with and without protected tokens, every key format."""
+    wl = CONFIGS[name]
+    if min(wl.l_v, T - T % 32) < 1:
+        p = 0.0
+    pair = Pair(wl, T, B=B, L=L, p=p, max_new=steps, k_ratio=fmt[0], one_bit=fmt[1])
+    pair.flushed_chunks = {}
+    pair.prefill()
+    if T >= 32:
+        for layer in range(L):
+            _check_layer(pair, layer)
+    for _ in range(steps):
+        out, ref = pair.decode()
+        assert np.abs(out - ref).max() <= TOL_ABS * max(1.0, np.abs(ref).max())
+    assert pair.cache.status() == 0
