@@ -41,6 +41,10 @@
  *   - One handle must not be used from two host threads at once, and calls on
  *     one handle must be issued on one stream (or on streams the caller orders).
  *     Different handles may be worked on from different streams at the same time.
+ *     One exception on one handle: vidkv_quantize_keys and vidkv_quantize_values (and their _layers
+ *     forms) write disjoint parts of the cache and workspace, so the values may be quantized on a
+ *     second stream while the keys are, provided the token selection was enqueued before both and
+ *     both streams are joined before the first decode call.
  *     The one-time set-up per device (tables, kernel attributes) is not guarded
  *     against concurrent host threads: make the first call on a device from one thread.
  *

@@ -8,7 +8,7 @@ from oracle import vidkv_oracle as O
 from tests import unpack as U
 from tests.helpers import (Pair, TOL_ABS, check_stats, compare_key_chunk, compare_ternary, f16_ulp_distance,
                            new_stats, to_np)
-from workloads import CONFIGS, make_layer_kv, make_saliency
+from workloads import CONFIGS, make_layer_kv, make_saliency, make_step_inputs
 
 pytestmark = pytest.mark.gpu
 
@@ -731,3 +731,41 @@ def test_saliency_ties_take_lower_index():
     E, _ = U.selection_mask(c.cache.cpu().numpy(), c.layout, 0, T)
     ref = O.select_tokens(sal[0].numpy(), 0.1875, 0, T)
     assert (E == ref).all() and E.sum() == 12 and E[0] and not E[2]
+
+
+@pytest.mark.parametrize("name,p", [("tiny", 0.2), ("qwen", 0.0)])
+def test_values_quantized_on_a_second_stream_give_the_same_cache(name, p):
+    """The key and the value quantizer write disjoint parts of the cache and workspace: with the values on a
+    second stream beside the keys (selection before both, streams joined afterwards) the cache holds the
+    same bytes as with everything on one stream, and decodes to the same output."""
+    import paper_2503_16257_b200 as P
+    wl = CONFIGS[name]
+    T, B, L = 1100, 2, 3
+    in_dt = P.VIDKV_F16 if wl.dtype == "fp16" else P.VIDKV_BF16
+    cfg = P.VidKVConfig(B=B, L=L, max_prefill_tokens=T, max_new_tokens=2, p_ratio=p, in_dtype=in_dt, out_dtype=P.VIDKV_F32)
+    KV = [make_layer_kv(wl, layer, "cuda", T=T, B=B) for layer in range(L)]
+    side = torch.cuda.Stream()
+    images, outs = [], []
+    for two_streams in (False, True):
+        c = P.VidKVCache(cfg, device="cuda")
+        if p > 0:
+            c.select_tokens(make_saliency(wl, "cuda", l_v=960, B=B), 0, 960, T)
+        main = torch.cuda.current_stream()
+        side.wait_stream(main)
+        for layer in range(L):
+            c.quantize_keys(layer, KV[layer][0])
+            if two_streams:
+                with torch.cuda.stream(side):
+                    c.quantize_values(layer, KV[layer][1])
+            else:
+                c.quantize_values(layer, KV[layer][1])
+        main.wait_stream(side)
+        q, k, v = [torch.stack(x) for x in zip(*[make_step_inputs(wl, layer, 0, "cuda", T=T, B=B) for layer in range(L)])]
+        out = torch.empty((L, B, cfg.H_q, 128), dtype=torch.float32, device="cuda")
+        c.decode_attention(0, L, q, k, v, out)
+        torch.cuda.synchronize()
+        assert c.status() == 0
+        images.append(c.cache.cpu().numpy())
+        outs.append(out.cpu().numpy())
+    assert np.array_equal(images[0], images[1])
+    assert np.array_equal(outs[0], outs[1])
