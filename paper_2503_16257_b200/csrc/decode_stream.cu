@@ -195,27 +195,26 @@ __device__ __forceinline__ void score_group_general(const uint8_t* kg, const Key
   const int w1 = kf.n2 >> 3, nw1 = (kD - kf.n2) >> 3;
 #pragma unroll 1
   for (int b = 0; b < n1b; ++b) {
-    uint32_t hi[4], lo[4];
+    // the stored scale takes the sign of the code bit and goes to the tensor core as it is; the other
+    // operand is the transformed query as hi + lo (Eq. 5) or the query itself (plain mode, exact in one piece)
+    uint32_t ah[4], al[4];
     const uint4 sv = *reinterpret_cast<const uint4*>(kg + kf.off_s1 + 64 * b + 16 * r);
     const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
     if (kf.plain) {
       const uint4 zv = *reinterpret_cast<const uint4*>(kg + ((hd & 1) ? kf.off_s1 : kf.off_z1) + 64 * b + 16 * r);
       const uint32_t zw[4] = {zv.x, zv.y, zv.z, zv.w};
-      uint32_t qb[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        qb[j] = __ldg(pp + (w1 + 4 * b + j) * 32);
-        hi[j] = hmul2_u(qb[j], sw[j]);
-        lo[j] = hfms2_u(qb[j], sw[j], hi[j]);
+        ah[j] = __ldg(pp + (w1 + 4 * b + j) * 32);
+        al[j] = 0u;
       }
-      mma_f16(cz1, qb[0], 0u, qb[1], 0u, zw[0], zw[1]);
-      mma_f16(cz1, qb[2], 0u, qb[3], 0u, zw[2], zw[3]);
+      mma_f16(cz1, ah[0], 0u, ah[1], 0u, zw[0], zw[1]);
+      mma_f16(cz1, ah[2], 0u, ah[3], 0u, zw[2], zw[3]);
     } else {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const uint32_t qh = __ldg(pp + (w1 + 4 * b + j) * 32), ql = __ldg(pp + (w1 + nw1 + 4 * b + j) * 32);
-        hi[j] = hmul2_u(qh, sw[j]);
-        lo[j] = hfma2_u(ql, sw[j], hfms2_u(qh, sw[j], hi[j]));
+        ah[j] = __ldg(pp + (w1 + 4 * b + j) * 32);
+        al[j] = __ldg(pp + (w1 + nw1 + 4 * b + j) * 32);
       }
     }
     const uint32_t cw = *reinterpret_cast<const uint32_t*>(kg + kf.off_bits1 + 128 * b + lane * 4);
@@ -224,8 +223,8 @@ __device__ __forceinline__ void score_group_general(const uint8_t* kg, const Key
       const uint32_t X = ((cw >> (8 * nt)) & 0xffu) * 0x02000100u;   // low lane: bit 7 at the sign, high lane: bit 6
 #pragma unroll
       for (int kp = 0; kp < 2; ++kp)
-        mma_f16(acc1[nt], hi[2 * kp], lo[2 * kp], hi[2 * kp + 1], lo[2 * kp + 1], and_xor(X << (4 * kp), m_sign, c_neg1),
-                and_xor(X << (4 * kp + 2), m_sign, c_neg1));
+        mma_f16(acc1[nt], ah[2 * kp], al[2 * kp], ah[2 * kp + 1], al[2 * kp + 1], nand_xor(X << (4 * kp), m_sign, sw[2 * kp]),
+                nand_xor(X << (4 * kp + 2), m_sign, sw[2 * kp + 1]));
     }
   }
   const float f1 = kf.plain ? 0.5f : 1.0f;
